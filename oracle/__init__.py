@@ -1,0 +1,18 @@
+"""TEST INFRASTRUCTURE — fp64 CPU oracle for paged chunked-prefill attention.
+
+Only the tests, ``__graft_entry__.smoke()`` and the CPU-baseline legs of
+``bench.py`` may import this package.  It shares no code with the CUDA
+library and never imports it.
+
+``reference``  : ctypes wrapper around the plain C implementation (wpp_oracle.c).
+``brute``      : separate numpy matrix-form implementation used to pin the C one.
+"""
+from .reference import (  # noqa: F401
+    build,
+    oracle_threads,
+    oracle_append,
+    oracle_attention,
+    oracle_attention_units,
+    merge_partials,
+)
+from .brute import brute_dense, gather_contiguous  # noqa: F401
