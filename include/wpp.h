@@ -1,0 +1,183 @@
+/*
+ * wpp.h — C ABI of the chunked-prefill attention path of one pipeline stage.
+ *
+ * One call processes one *wave*: a ragged batch of request chunks (paper,
+ * Section 4 "Waves and lanes").  For request i the caller states
+ *   prefix_lens[i] = P_i  tokens of the request already in the paged KV cache
+ *                         (the reused cached prefix plus earlier chunks; this is the
+ *                         "starting token" of the chunk span, Section 4.6),
+ *   chunk_lens[i]  = C_i  new tokens in this wave (the span's "length"),
+ *   block_tables[i][j]    physical page holding tokens [j*B, (j+1)*B) of request i
+ *                         (Section 3.2: ceil(n/B) logical blocks, physically
+ *                         non-contiguous, shareable between requests).
+ * T = sum_i C_i; the chunks' rows are concatenated in request order in q, k_new,
+ * v_new and out.  Query head h reads KV head h / (num_q_heads / num_kv_heads)
+ * (grouped-query attention, Section 3.1).
+ *
+ * General rules
+ *   - Every function returns a wpp_status (0 = WPP_OK).  Nothing throws, nothing
+ *     synchronises the device, and nothing allocates device memory unless said so.
+ *   - "host" / "device" on each pointer says where the memory lives.  The caller owns
+ *     every buffer; device buffers are borrowed until the work queued on
+ *     `cuda_stream` (a cudaStream_t passed as void*) has completed.
+ *   - bf16 tensors are passed as void*; inner (head_dim) elements are contiguous and
+ *     every row start and stride must be a multiple of 16 bytes.
+ *   - Problems the host can see are reported before anything is launched.  Problems
+ *     only the device can see (a page id outside [0, num_pages), a bounded wait that
+ *     ran out) set *status_dev (first error wins, never cleared by the library), the
+ *     affected work is skipped, and nothing traps; read it after your own sync.
+ *   - A request appears at most once per wave; successive chunks of a request go in
+ *     successive calls on the same stream (Section 4.6: order is preserved on each
+ *     stage's execution stream).  wpp_kv_append must precede
+ *     wpp_prefill_attention_varlen for the same wave on that stream: attention reads
+ *     the chunk's own K/V from the pages.
+ */
+#ifndef WPP_H_
+#define WPP_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    WPP_OK = 0,
+    WPP_ERR_INVALID_ARG = 1,        /* null pointer, negative size, misaligned pointer or stride */
+    WPP_ERR_UNSUPPORTED = 2,        /* dtype, head_dim, page_size or head ratio outside the supported set */
+    WPP_ERR_BOUNDS = 3,             /* ceil((P_i + C_i) / B) > max_blocks_per_req, or page id out of range */
+    WPP_ERR_POSITION_MISMATCH = 4,  /* span start != tokens actually cached (Section 4.6: execution fails) */
+    WPP_ERR_WORKSPACE_TOO_SMALL = 5,
+    WPP_ERR_PLAN_MISMATCH = 6,      /* plan buffer corrupt, too small, or built for another batch description */
+    WPP_ERR_CUDA = 7,               /* CUDA runtime/driver error; see wpp_last_cuda_error */
+    WPP_ERR_TIMEOUT = 8,            /* device side: a bounded barrier wait expired; the tile was abandoned */
+    WPP_ERR_ALIASED_APPEND = 9      /* wpp_validate_batch: two writers, or a writer and a reader, share a slot */
+} wpp_status;
+
+enum { WPP_BF16 = 1 };
+
+/* Opaque per-device context: SM count, shared-memory limit, driver entry points.  Owns host memory only. */
+typedef struct wpp_ctx wpp_ctx;
+
+/* Create a context for CUDA device `cuda_device` (makes no device allocation).  WPP_ERR_CUDA if the device or
+ * driver is unusable (there is no CPU fallback).  *out is host memory owned by the library until wpp_destroy. */
+int wpp_create(wpp_ctx** out, int cuda_device);
+int wpp_destroy(wpp_ctx* ctx);
+const char* wpp_status_string(int status);
+/* Last cudaError_t / CUresult seen by this context (0 if none). */
+int wpp_last_cuda_error(const wpp_ctx* ctx);
+
+/* Description of one wave.  Strides are in ELEMENTS (bf16), inner dim contiguous.
+ * Pools: element (page, kv_head, slot, e) of K lives at
+ *   k_cache + page*kv_page_stride + kv_head*kv_head_stride + slot*kv_token_stride + e,
+ * V likewise in v_cache with the same strides.  A stride of 0 selects the dense default
+ * of the layouts [num_pages][Hkv][B][d] (pools) and [T][H][d] (q, k_new/v_new, out). */
+typedef struct {
+    int32_t num_requests;        /* R >= 0 */
+    int32_t num_q_heads;         /* Hq, a multiple of num_kv_heads */
+    int32_t num_kv_heads;        /* Hkv */
+    int32_t head_dim;            /* d in {64, 128} */
+    int32_t page_size;           /* B in {16, 32, 64, 128} tokens per page */
+    int32_t max_blocks_per_req;  /* row stride of block_tables, in elements */
+    int32_t num_pages;           /* pool size, for bounds checks */
+    int32_t dtype;               /* WPP_BF16 */
+    float sm_scale;              /* 0 selects 1/sqrt(head_dim) */
+    int32_t reserved0;
+    int64_t kv_page_stride, kv_head_stride, kv_token_stride;
+    int64_t q_token_stride, q_head_stride;
+    int64_t kvnew_token_stride, kvnew_head_stride;
+    int64_t o_token_stride, o_head_stride;
+} wpp_batch_desc;
+
+/* Planner knobs; a zero field selects the library default. */
+typedef struct {
+    int32_t tile_m;           /* query rows per work tile: 128 or 256 (default 256: two 128-row halves) */
+    int32_t tile_n;           /* keys per inner step: 128 */
+    int32_t force_kv_splits;  /* >= 2: split every tile's key range into this many parts (when it has that many
+                                 key steps); 1: never split; 0: library decides */
+    int32_t max_ctas;         /* persistent CTAs to plan for (default: SM count of the context, 148 without one) */
+} wpp_plan_opts;
+
+typedef struct {
+    int64_t num_tiles;          /* work tiles in the plan (split parts count separately) */
+    int64_t num_split_tiles;    /* of which write partial results to the workspace */
+    int64_t num_combine_tiles;  /* tiles the combine pass merges (0: no combine pass) */
+    int64_t num_ctas;           /* persistent CTAs the attention kernel will be launched with */
+    int64_t total_new_tokens;   /* T */
+    int64_t key_steps;          /* sum over tiles of 128-row x 128-key steps (work incl. tile quantisation) */
+    int64_t flops;              /* algorithmic: 4 * d * Hq * sum_i (C_i P_i + C_i (C_i + 1) / 2) */
+    size_t workspace_bytes;     /* device scratch wpp_prefill_attention_varlen needs for this plan (may be 0) */
+    size_t plan_bytes;          /* bytes of plan_host actually used; copy that many to the device */
+} wpp_plan_info;
+
+/* Upper bound on the plan size for a wave of this description with `total_new_tokens` rows under these opts
+ * (0 if the description or opts are invalid). */
+size_t wpp_plan_bytes(const wpp_ctx* ctx_or_null, const wpp_batch_desc* desc, int64_t total_new_tokens,
+                      const wpp_plan_opts* opts_or_null);
+
+/* Host-side work split (integer arithmetic only; no CUDA call).  Cuts the wave into work tiles
+ * (request, query-row range, query head, key-step range), decides which tiles are split along the keys,
+ * assigns tiles to persistent CTAs in decreasing-cost order, and sizes the workspace.  Equal-sized chunks
+ * cost different amounts because they attend to different prefix lengths (Section 6), hence cost = key steps.
+ *   prefix_lens_host, chunk_lens_host : host int32 [R].
+ *   cached_lens_host_or_null          : host int32 [R]; tokens each request really has in the cache after
+ *                                       materialisation.  If given and != prefix_lens, returns
+ *                                       WPP_ERR_POSITION_MISMATCH (Section 4.6).
+ *   plan_host / plan_host_bytes       : caller-owned host buffer (pinned if it is to be copied asynchronously);
+ *                                       the caller copies info->plan_bytes bytes of it to the device.
+ * Deterministic: equal inputs give byte-identical plans.  ctx may be NULL (plans for 148 SMs). */
+int wpp_plan_tiles(const wpp_ctx* ctx_or_null, const wpp_batch_desc* desc,
+                   const int32_t* prefix_lens_host, const int32_t* chunk_lens_host,
+                   const int32_t* cached_lens_host_or_null, const wpp_plan_opts* opts_or_null,
+                   void* plan_host, size_t plan_host_bytes, wpp_plan_info* info);
+
+/* Optional host-side check of a wave (host copies of everything): page ids in range, table long enough, no slot
+ * written by two requests, no written slot inside another request's readable range.  block_tables_host is
+ * int32 [R][max_blocks_per_req]. */
+int wpp_validate_batch(const wpp_batch_desc* desc, const int32_t* block_tables_host,
+                       const int32_t* prefix_lens_host, const int32_t* chunk_lens_host);
+
+/* KV append ("prefill fills the cache", Sections 1 and 4.1 steps 3-5): for every new token t of request i,
+ * pos = P_i + t, page = block_tables[i][pos / B], slot = pos % B; copies k_new[q_off_i + t][h][0..d) and
+ * v_new[...] bit for bit to k_cache / v_cache [page][h][slot][0..d).  No other pool byte is written.
+ *   k_new, v_new : device, bf16 [T][Hkv][d] (read).     k_cache, v_cache : device pools (written).
+ *   block_tables : device int32 [R][max_blocks_per_req]; prefix_lens, chunk_lens : device int32 [R].
+ *   plan_dev     : device copy of the plan made for this wave (provides row offsets and T).
+ *   plan_host    : the host plan it was copied from (read during the call only, for launch sizing).
+ *   status_dev   : device int32, sticky first-error word (may be NULL).
+ * One kernel on cuda_stream, 16-byte vector copies.  A page id outside [0, num_pages) sets
+ * *status_dev = WPP_ERR_BOUNDS and that token is skipped. */
+int wpp_kv_append(const wpp_ctx* ctx, const wpp_batch_desc* desc, const void* k_new, const void* v_new,
+                  void* k_cache, void* v_cache, const int32_t* block_tables, const int32_t* prefix_lens,
+                  const int32_t* chunk_lens, const void* plan_host, const void* plan_dev, int32_t* status_dev,
+                  void* cuda_stream);
+
+/* Chunked-prefill attention (Section 4.1 step 5; Section 3.1: token n attends to all n previous positions):
+ * for chunk row t of request i and query head h, with g = h / (Hq/Hkv) and n = P_i + t + 1,
+ *   s_j = sm_scale * <q[q_off_i + t][h], K_j[g]>,  j < n,   K_j = k_cache[block_tables[i][j / B]][g][j % B],
+ *   out[q_off_i + t][h] = sum_j softmax(s)_j V_j[g]   (bf16, round to nearest even),
+ *   lse[q_off_i + t][h] = log sum_j exp(s_j)          (fp32, natural log; optional).
+ * bf16 inputs, fp32 scores/accumulation on tensor cores, probabilities rounded to bf16 before the PV product.
+ * Slots >= P_i + C_i and pages no table references never influence the result, whatever bits they hold.
+ *   q, out        : device bf16 [T][Hq][d];  lse_or_null : device fp32 [T][Hq].
+ *   k_cache, v_cache, block_tables, prefix_lens, chunk_lens : device, read only.
+ *   plan_host / plan_dev : as for wpp_kv_append.
+ *   workspace     : device scratch of >= info.workspace_bytes bytes, 256-byte aligned (NULL allowed when 0);
+ *                   holds split-KV partial results; contents are undefined afterwards.
+ * Launches one persistent kernel, plus one combine kernel iff the plan has split tiles.  Results are
+ * bit-reproducible for a given plan (no atomics on outputs; partials are merged in a fixed order). */
+int wpp_prefill_attention_varlen(const wpp_ctx* ctx, const wpp_batch_desc* desc, const void* q, void* out,
+                                 float* lse_or_null, const void* k_cache, const void* v_cache,
+                                 const int32_t* block_tables, const int32_t* prefix_lens,
+                                 const int32_t* chunk_lens, const void* plan_host, const void* plan_dev,
+                                 void* workspace, size_t workspace_bytes, int32_t* status_dev,
+                                 void* cuda_stream);
+
+/* Number of kernels the library has launched through this context so far (for launch accounting). */
+int64_t wpp_launch_count(const wpp_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* WPP_H_ */

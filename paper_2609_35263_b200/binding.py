@@ -1,0 +1,224 @@
+"""ctypes binding of libwpp.so: argument marshalling only — every step of the path runs in the library.
+
+The functions carry the C names (wpp_plan_tiles, wpp_kv_append, wpp_prefill_attention_varlen).  Tensors are
+torch tensors used as device memory; streams are torch streams.  There is no fallback: if the library cannot be
+loaded, or no sm_100 device is present, the calls raise.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libwpp.so")
+
+WPP_OK = 0
+WPP_BF16 = 1
+STATUS_NAMES = {
+    0: "WPP_OK", 1: "WPP_ERR_INVALID_ARG", 2: "WPP_ERR_UNSUPPORTED", 3: "WPP_ERR_BOUNDS",
+    4: "WPP_ERR_POSITION_MISMATCH", 5: "WPP_ERR_WORKSPACE_TOO_SMALL", 6: "WPP_ERR_PLAN_MISMATCH",
+    7: "WPP_ERR_CUDA", 8: "WPP_ERR_TIMEOUT", 9: "WPP_ERR_ALIASED_APPEND",
+}
+
+
+class WppError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {STATUS_NAMES.get(status, status)}")
+
+
+class BatchDesc(ctypes.Structure):
+    _fields_ = [
+        ("num_requests", ctypes.c_int32), ("num_q_heads", ctypes.c_int32), ("num_kv_heads", ctypes.c_int32),
+        ("head_dim", ctypes.c_int32), ("page_size", ctypes.c_int32), ("max_blocks_per_req", ctypes.c_int32),
+        ("num_pages", ctypes.c_int32), ("dtype", ctypes.c_int32), ("sm_scale", ctypes.c_float),
+        ("reserved0", ctypes.c_int32),
+        ("kv_page_stride", ctypes.c_int64), ("kv_head_stride", ctypes.c_int64), ("kv_token_stride", ctypes.c_int64),
+        ("q_token_stride", ctypes.c_int64), ("q_head_stride", ctypes.c_int64),
+        ("kvnew_token_stride", ctypes.c_int64), ("kvnew_head_stride", ctypes.c_int64),
+        ("o_token_stride", ctypes.c_int64), ("o_head_stride", ctypes.c_int64),
+    ]
+
+
+class PlanOpts(ctypes.Structure):
+    _fields_ = [("tile_m", ctypes.c_int32), ("tile_n", ctypes.c_int32), ("force_kv_splits", ctypes.c_int32),
+                ("max_ctas", ctypes.c_int32)]
+
+
+class PlanInfo(ctypes.Structure):
+    _fields_ = [("num_tiles", ctypes.c_int64), ("num_split_tiles", ctypes.c_int64),
+                ("num_combine_tiles", ctypes.c_int64), ("num_ctas", ctypes.c_int64),
+                ("total_new_tokens", ctypes.c_int64), ("key_steps", ctypes.c_int64), ("flops", ctypes.c_int64),
+                ("workspace_bytes", ctypes.c_size_t), ("plan_bytes", ctypes.c_size_t)]
+
+
+EXPORTS = ["wpp_create", "wpp_destroy", "wpp_status_string", "wpp_last_cuda_error", "wpp_plan_bytes",
+           "wpp_plan_tiles", "wpp_validate_batch", "wpp_kv_append", "wpp_prefill_attention_varlen",
+           "wpp_launch_count"]
+
+_lib = None
+
+
+def load_library() -> ctypes.CDLL:
+    """Load libwpp.so (built in-tree by paper_2609_35263_b200.build); raises if it is missing."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(f"{LIB_PATH} is missing: run `python -m paper_2609_35263_b200.build` "
+                              "(there is no fallback path)")
+        lib = ctypes.CDLL(LIB_PATH)
+        vp, i32p = ctypes.c_void_p, ctypes.c_void_p
+        lib.wpp_create.argtypes = [ctypes.POINTER(vp), ctypes.c_int]
+        lib.wpp_destroy.argtypes = [vp]
+        lib.wpp_status_string.restype = ctypes.c_char_p
+        lib.wpp_status_string.argtypes = [ctypes.c_int]
+        lib.wpp_last_cuda_error.argtypes = [vp]
+        lib.wpp_launch_count.argtypes = [vp]
+        lib.wpp_launch_count.restype = ctypes.c_int64
+        lib.wpp_plan_bytes.restype = ctypes.c_size_t
+        lib.wpp_plan_bytes.argtypes = [vp, ctypes.POINTER(BatchDesc), ctypes.c_int64, ctypes.POINTER(PlanOpts)]
+        lib.wpp_plan_tiles.argtypes = [vp, ctypes.POINTER(BatchDesc), i32p, i32p, i32p, ctypes.POINTER(PlanOpts),
+                                       vp, ctypes.c_size_t, ctypes.POINTER(PlanInfo)]
+        lib.wpp_validate_batch.argtypes = [ctypes.POINTER(BatchDesc), i32p, i32p, i32p]
+        lib.wpp_kv_append.argtypes = [vp, ctypes.POINTER(BatchDesc), vp, vp, vp, vp, i32p, i32p, i32p, vp, vp,
+                                      i32p, vp]
+        lib.wpp_prefill_attention_varlen.argtypes = [vp, ctypes.POINTER(BatchDesc), vp, vp, vp, vp, vp, i32p, i32p,
+                                                     i32p, vp, vp, vp, ctypes.c_size_t, i32p, vp]
+        _lib = lib
+    return _lib
+
+
+def _check(status: int, where: str):
+    if status != WPP_OK:
+        raise WppError(status, where)
+
+
+class Context:
+    """wpp_ctx for one CUDA device."""
+
+    def __init__(self, device: int = 0):
+        lib = load_library()
+        self._h = ctypes.c_void_p()
+        _check(lib.wpp_create(ctypes.byref(self._h), int(device)), "wpp_create")
+        self.device = int(device)
+
+    @property
+    def handle(self):
+        return self._h
+
+    def launch_count(self) -> int:
+        return int(load_library().wpp_launch_count(self._h))
+
+    def last_cuda_error(self) -> int:
+        return int(load_library().wpp_last_cuda_error(self._h))
+
+    def close(self):
+        if self._h:
+            load_library().wpp_destroy(self._h)
+            self._h = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def make_desc(num_requests, num_q_heads, num_kv_heads, head_dim, page_size, max_blocks_per_req, num_pages,
+              sm_scale: float = 0.0, **strides) -> BatchDesc:
+    d = BatchDesc()
+    d.num_requests, d.num_q_heads, d.num_kv_heads = int(num_requests), int(num_q_heads), int(num_kv_heads)
+    d.head_dim, d.page_size = int(head_dim), int(page_size)
+    d.max_blocks_per_req, d.num_pages = int(max_blocks_per_req), int(num_pages)
+    d.dtype = WPP_BF16
+    d.sm_scale = float(sm_scale)
+    for k, v in strides.items():
+        setattr(d, k, int(v))
+    return d
+
+
+def _np_i32(x) -> np.ndarray:
+    return np.ascontiguousarray(np.asarray(x, dtype=np.int32))
+
+
+class Plan:
+    """Host plan buffer (pinned when CUDA is present), its device copy and the planner's summary."""
+
+    def __init__(self, host: torch.Tensor, info: PlanInfo):
+        self.host = host
+        self.info = info
+        self.dev: Optional[torch.Tensor] = None
+
+    @property
+    def plan_bytes(self) -> int:
+        return int(self.info.plan_bytes)
+
+    def to_device(self, device="cuda", non_blocking=True) -> "Plan":
+        self.dev = self.host[: self.plan_bytes].to(device, non_blocking=non_blocking)
+        return self
+
+    def host_bytes(self) -> bytes:
+        return bytes(self.host[: self.plan_bytes].numpy().tobytes())
+
+
+def wpp_plan_tiles(ctx: Optional[Context], desc: BatchDesc, prefix_lens, chunk_lens, cached_lens=None,
+                   opts: Optional[PlanOpts] = None, pin: Optional[bool] = None) -> Plan:
+    """Host-side work split; returns a Plan whose .host buffer must be copied to the device (.to_device())."""
+    lib = load_library()
+    P, C = _np_i32(prefix_lens), _np_i32(chunk_lens)
+    T = int(C.astype(np.int64).sum())
+    h = ctx.handle if ctx is not None else None
+    optp = ctypes.byref(opts) if opts is not None else None
+    nbytes = int(lib.wpp_plan_bytes(h, ctypes.byref(desc), T, optp))
+    if nbytes == 0:
+        # let wpp_plan_tiles report the precise error
+        nbytes = 4096
+    pin = torch.cuda.is_available() if pin is None else pin
+    host = torch.empty(nbytes, dtype=torch.uint8, pin_memory=bool(pin))
+    info = PlanInfo()
+    cached = _np_i32(cached_lens) if cached_lens is not None else None
+    st = lib.wpp_plan_tiles(h, ctypes.byref(desc), P.ctypes.data, C.ctypes.data,
+                            cached.ctypes.data if cached is not None else None, optp,
+                            host.data_ptr(), nbytes, ctypes.byref(info))
+    _check(st, "wpp_plan_tiles")
+    return Plan(host, info)
+
+
+def wpp_validate_batch(desc: BatchDesc, block_tables, prefix_lens, chunk_lens) -> int:
+    bt, P, C = _np_i32(block_tables), _np_i32(prefix_lens), _np_i32(chunk_lens)
+    return int(load_library().wpp_validate_batch(ctypes.byref(desc), bt.ctypes.data, P.ctypes.data, C.ctypes.data))
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream) -> ctypes.c_void_p:
+    s = torch.cuda.current_stream() if stream is None else stream
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def wpp_kv_append(ctx: Context, desc: BatchDesc, k_new, v_new, k_cache, v_cache, block_tables, prefix_lens,
+                  chunk_lens, plan: Plan, status=None, stream=None) -> None:
+    """Queue the KV append of one wave on `stream` (device tensors; int32 metadata on the device)."""
+    st = load_library().wpp_kv_append(ctx.handle, ctypes.byref(desc), _ptr(k_new), _ptr(v_new), _ptr(k_cache),
+                                      _ptr(v_cache), _ptr(block_tables), _ptr(prefix_lens), _ptr(chunk_lens),
+                                      ctypes.c_void_p(plan.host.data_ptr()), _ptr(plan.dev), _ptr(status),
+                                      _stream(stream))
+    _check(st, "wpp_kv_append")
+
+
+def wpp_prefill_attention_varlen(ctx: Context, desc: BatchDesc, q, out, lse, k_cache, v_cache, block_tables,
+                                 prefix_lens, chunk_lens, plan: Plan, workspace=None, status=None,
+                                 stream=None) -> None:
+    """Queue chunked-prefill attention of one wave on `stream`; results land in `out` (and `lse` if given)."""
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    st = load_library().wpp_prefill_attention_varlen(
+        ctx.handle, ctypes.byref(desc), _ptr(q), _ptr(out), _ptr(lse), _ptr(k_cache), _ptr(v_cache),
+        _ptr(block_tables), _ptr(prefix_lens), _ptr(chunk_lens), ctypes.c_void_p(plan.host.data_ptr()),
+        _ptr(plan.dev), _ptr(workspace), ws_bytes, _ptr(status), _stream(stream))
+    _check(st, "wpp_prefill_attention_varlen")

@@ -1,0 +1,212 @@
+// C-ABI entry points that touch CUDA: context, tensor-map construction, argument checks and launches.
+// There is no CPU fallback: without a usable device wpp_create fails and nothing else can be called.
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include "../../include/wpp.h"
+#include "wpp_device.h"
+#include "wpp_host.h"
+#include "wpp_plan_format.h"
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+struct wpp_ctx {
+    int device;
+    int sm_count;
+    int smem_optin;
+    int last_cuda_error;
+    int64_t launches;
+    EncodeTiledFn encode_tiled;
+};
+
+extern "C" int wpp_ctx_sm_count(const wpp_ctx* ctx) { return ctx ? ctx->sm_count : 148; }
+
+static int cuda_fail(const wpp_ctx* ctx, int err) {
+    if (ctx) const_cast<wpp_ctx*>(ctx)->last_cuda_error = err;
+    return WPP_ERR_CUDA;
+}
+
+extern "C" int wpp_create(wpp_ctx** out, int cuda_device) {
+    if (!out) return WPP_ERR_INVALID_ARG;
+    *out = nullptr;
+    int n = 0;
+    cudaError_t e = cudaGetDeviceCount(&n);
+    if (e != cudaSuccess || cuda_device < 0 || cuda_device >= n) return WPP_ERR_CUDA;
+    cudaDeviceProp prop;
+    if ((e = cudaGetDeviceProperties(&prop, cuda_device)) != cudaSuccess) return WPP_ERR_CUDA;
+    if (prop.major != 10) return WPP_ERR_UNSUPPORTED;   // the kernels are built for sm_100a only
+    wpp_ctx* c = static_cast<wpp_ctx*>(calloc(1, sizeof(wpp_ctx)));
+    if (!c) return WPP_ERR_INVALID_ARG;
+    c->device = cuda_device;
+    c->sm_count = prop.multiProcessorCount;
+    c->smem_optin = (int)prop.sharedMemPerBlockOptin;
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+    if (e != cudaSuccess || qres != cudaDriverEntryPointSuccess || !fn) {
+        free(c);
+        return WPP_ERR_CUDA;
+    }
+    c->encode_tiled = reinterpret_cast<EncodeTiledFn>(fn);
+    *out = c;
+    return WPP_OK;
+}
+
+extern "C" int wpp_destroy(wpp_ctx* ctx) {
+    free(ctx);
+    return WPP_OK;
+}
+
+extern "C" int wpp_last_cuda_error(const wpp_ctx* ctx) { return ctx ? ctx->last_cuda_error : 0; }
+extern "C" int64_t wpp_launch_count(const wpp_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+
+// bf16 tensor map with 128-byte swizzle; dims/strides innermost first, strides in bytes for dims 1..rank-1
+static int make_map(const wpp_ctx* ctx, CUtensorMap* m, const void* base, int rank, const uint64_t* dims,
+                    const uint64_t* strides_bytes, const uint32_t* box) {
+    cuuint64_t gd[4];
+    cuuint64_t gs[3];
+    cuuint32_t bx[4], es[4];
+    for (int i = 0; i < rank; ++i) { gd[i] = dims[i]; bx[i] = box[i]; es[i] = 1; }
+    for (int i = 0; i < rank - 1; ++i) gs[i] = strides_bytes[i];
+    CUresult r = ctx->encode_tiled(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void*>(base), gd,
+                                   gs, bx, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                   CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return cuda_fail(ctx, (int)r);
+    return WPP_OK;
+}
+
+extern "C" int wpp_kv_append(const wpp_ctx* ctx, const wpp_batch_desc* desc, const void* k_new, const void* v_new,
+                             void* k_cache, void* v_cache, const int32_t* block_tables, const int32_t* prefix_lens,
+                             const int32_t* chunk_lens, const void* plan_host, const void* plan_dev,
+                             int32_t* status_dev, void* cuda_stream) {
+    if (!ctx) return WPP_ERR_INVALID_ARG;
+    wpp_batch_desc d;
+    int rc = wpp_resolve_desc(desc, &d);
+    if (rc != WPP_OK) return rc;
+    const WppPlanHeader* hd = nullptr;
+    if ((rc = wpp_check_plan(plan_host, &d, &hd)) != WPP_OK) return rc;
+    if (hd->total_new_tokens == 0) return WPP_OK;
+    if (!k_new || !v_new || !k_cache || !v_cache || !block_tables || !prefix_lens || !chunk_lens || !plan_dev)
+        return WPP_ERR_INVALID_ARG;
+    if (!aligned16(k_new) || !aligned16(v_new) || !aligned16(k_cache) || !aligned16(v_cache) || !aligned16(plan_dev))
+        return WPP_ERR_INVALID_ARG;
+    wpp::AppendParams p;
+    memset(&p, 0, sizeof(p));
+    p.plan = plan_dev;
+    p.k_new = static_cast<const uint4*>(k_new);
+    p.v_new = static_cast<const uint4*>(v_new);
+    p.k_cache = static_cast<uint4*>(k_cache);
+    p.v_cache = static_cast<uint4*>(v_cache);
+    p.block_tables = block_tables;
+    p.prefix_lens = prefix_lens;
+    p.status = status_dev;
+    p.kvnew_token_stride = d.kvnew_token_stride / 8;
+    p.kvnew_head_stride = d.kvnew_head_stride / 8;
+    p.kv_page_stride = d.kv_page_stride / 8;
+    p.kv_head_stride = d.kv_head_stride / 8;
+    p.kv_token_stride = d.kv_token_stride / 8;
+    p.num_requests = d.num_requests;
+    p.num_kv_heads = d.num_kv_heads;
+    p.vec_per_row = d.head_dim / 8;
+    p.page_size = d.page_size;
+    p.max_blocks = d.max_blocks_per_req;
+    p.num_pages = d.num_pages;
+    p.total_new_tokens = hd->total_new_tokens;
+    int e = wpp_launch_append(&p, ctx->sm_count, cuda_stream);
+    if (e != 0) return cuda_fail(ctx, e);
+    const_cast<wpp_ctx*>(ctx)->launches += 1;
+    return WPP_OK;
+}
+
+extern "C" int wpp_prefill_attention_varlen(const wpp_ctx* ctx, const wpp_batch_desc* desc, const void* q, void* out,
+                                            float* lse_or_null, const void* k_cache, const void* v_cache,
+                                            const int32_t* block_tables, const int32_t* prefix_lens,
+                                            const int32_t* chunk_lens, const void* plan_host, const void* plan_dev,
+                                            void* workspace, size_t workspace_bytes, int32_t* status_dev,
+                                            void* cuda_stream) {
+    if (!ctx) return WPP_ERR_INVALID_ARG;
+    wpp_batch_desc d;
+    int rc = wpp_resolve_desc(desc, &d);
+    if (rc != WPP_OK) return rc;
+    const WppPlanHeader* hd = nullptr;
+    if ((rc = wpp_check_plan(plan_host, &d, &hd)) != WPP_OK) return rc;
+    if (hd->tile_m > WPP_MAX_TILE_M) return WPP_ERR_PLAN_MISMATCH;
+    if (hd->total_new_tokens == 0 || hd->num_units == 0) return WPP_OK;
+    if (!q || !out || !k_cache || !v_cache || !block_tables || !prefix_lens || !chunk_lens || !plan_dev)
+        return WPP_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(out) || !aligned16(k_cache) || !aligned16(v_cache) || !aligned16(plan_dev))
+        return WPP_ERR_INVALID_ARG;
+    if (hd->workspace_bytes > 0) {
+        if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255) != 0) return WPP_ERR_INVALID_ARG;
+        if (workspace_bytes < hd->workspace_bytes) return WPP_ERR_WORKSPACE_TOO_SMALL;
+    }
+    if (d.num_pages == 0) return WPP_ERR_INVALID_ARG;
+
+    CUtensorMap tq, tk, tv;
+    {
+        const uint64_t dims[3] = {(uint64_t)d.head_dim, (uint64_t)d.num_q_heads, (uint64_t)hd->total_new_tokens};
+        const uint64_t strides[2] = {(uint64_t)d.q_head_stride * 2, (uint64_t)d.q_token_stride * 2};
+        const uint32_t box[3] = {64, 1, 128};
+        if ((rc = make_map(ctx, &tq, q, 3, dims, strides, box)) != WPP_OK) return rc;
+    }
+    {
+        const uint64_t dims[4] = {(uint64_t)d.head_dim, (uint64_t)d.page_size, (uint64_t)d.num_kv_heads,
+                                  (uint64_t)d.num_pages};
+        const uint64_t strides[3] = {(uint64_t)d.kv_token_stride * 2, (uint64_t)d.kv_head_stride * 2,
+                                     (uint64_t)d.kv_page_stride * 2};
+        const uint32_t box[4] = {64, (uint32_t)d.page_size, 1, 1};
+        if ((rc = make_map(ctx, &tk, k_cache, 4, dims, strides, box)) != WPP_OK) return rc;
+        if ((rc = make_map(ctx, &tv, v_cache, 4, dims, strides, box)) != WPP_OK) return rc;
+    }
+
+    wpp::AttnParams p;
+    memset(&p, 0, sizeof(p));
+    p.plan = plan_dev;
+    p.block_tables = block_tables;
+    p.prefix_lens = prefix_lens;
+    p.chunk_lens = chunk_lens;
+    p.out = static_cast<__nv_bfloat16*>(out);
+    p.lse = lse_or_null;
+    p.ws_o = static_cast<float*>(workspace);
+    p.ws_lse = p.ws_o ? p.ws_o + (size_t)hd->num_split_slots * hd->tile_m * d.head_dim : nullptr;
+    p.status = status_dev;
+    p.o_token_stride = d.o_token_stride;
+    p.o_head_stride = d.o_head_stride;
+    p.num_q_heads = d.num_q_heads;
+    p.group = d.num_q_heads / d.num_kv_heads;
+    p.page_size = d.page_size;
+    p.max_blocks = d.max_blocks_per_req;
+    p.num_pages = d.num_pages;
+    const double scale = d.sm_scale > 0.f ? (double)d.sm_scale : 1.0 / sqrt((double)d.head_dim);
+    p.scale_log2 = (float)(scale * 1.4426950408889634);
+
+    int e = wpp_launch_attention(d.head_dim, &tq, &tk, &tv, &p, hd->num_ctas, cuda_stream);
+    if (e != 0) return cuda_fail(ctx, e);
+    const_cast<wpp_ctx*>(ctx)->launches += 1;
+    if (hd->num_combine > 0) {
+        wpp::CombineParams c;
+        memset(&c, 0, sizeof(c));
+        c.plan = plan_dev;
+        c.ws_o = p.ws_o;
+        c.ws_lse = p.ws_lse;
+        c.out = p.out;
+        c.lse = lse_or_null;
+        c.o_token_stride = d.o_token_stride;
+        c.o_head_stride = d.o_head_stride;
+        c.num_q_heads = d.num_q_heads;
+        c.head_dim = d.head_dim;
+        c.tile_m = hd->tile_m;
+        e = wpp_launch_combine(&c, hd->num_combine, cuda_stream);
+        if (e != 0) return cuda_fail(ctx, e);
+        const_cast<wpp_ctx*>(ctx)->launches += 1;
+    }
+    return WPP_OK;
+}

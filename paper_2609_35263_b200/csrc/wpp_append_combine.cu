@@ -1,0 +1,96 @@
+// KV append (bit-exact 16-byte vector copies into the reserved pages) and the split-KV combine pass.
+#include <cuda_runtime.h>
+#include <math.h>
+#include <stdint.h>
+
+#include "wpp_device.h"
+#include "wpp_plan_format.h"
+
+namespace wpp {
+
+// One thread moves one 16-byte vector of K and the matching vector of V.  A vector index decomposes as
+// (token, kv head, vector within the head row); the request is found by bisection in the row offsets.
+__global__ void __launch_bounds__(256) wpp_append_kernel(const AppendParams p) {
+    const char* plan = static_cast<const char*>(p.plan);
+    const WppPlanHeader* hd = reinterpret_cast<const WppPlanHeader*>(plan);
+    const int32_t* q_offsets = reinterpret_cast<const int32_t*>(plan + hd->off_q_offsets);
+    const int64_t per_token = (int64_t)p.num_kv_heads * p.vec_per_row;
+    const int64_t total = p.total_new_tokens * per_token;
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t v = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; v < total; v += stride) {
+        const int64_t tok = v / per_token;
+        const int rem = (int)(v - tok * per_token);
+        const int h = rem / p.vec_per_row, c = rem - h * p.vec_per_row;
+        int lo = 0, hi = p.num_requests;          // largest i with q_offsets[i] <= tok
+        while (hi - lo > 1) {
+            const int mid = (lo + hi) >> 1;
+            if (q_offsets[mid] <= tok) lo = mid; else hi = mid;
+        }
+        const int pos = p.prefix_lens[lo] + (int)(tok - q_offsets[lo]);
+        const int blk = pos / p.page_size, slot = pos - blk * p.page_size;
+        const int page = (blk < p.max_blocks) ? p.block_tables[(int64_t)lo * p.max_blocks + blk] : -1;
+        if (page < 0 || page >= p.num_pages) {
+            if (p.status) atomicCAS(p.status, 0, WPP_ERR_BOUNDS);
+            continue;
+        }
+        const int64_t src = tok * p.kvnew_token_stride + h * p.kvnew_head_stride + c;
+        const int64_t dst = page * p.kv_page_stride + h * p.kv_head_stride + slot * p.kv_token_stride + c;
+        const uint4 kv = p.k_new[src];
+        const uint4 vv = p.v_new[src];
+        p.k_cache[dst] = kv;
+        p.v_cache[dst] = vv;
+    }
+}
+
+// One block per split tile; one warp per row, lanes across head_dim.  Partials are merged in increasing split
+// order with weights exp2(lse_s - max lse), so the result does not depend on scheduling.
+__global__ void __launch_bounds__(256) wpp_combine_kernel(const CombineParams p) {
+    const char* plan = static_cast<const char*>(p.plan);
+    const WppPlanHeader* hd = reinterpret_cast<const WppPlanHeader*>(plan);
+    const int32_t* q_offsets = reinterpret_cast<const int32_t*>(plan + hd->off_q_offsets);
+    const WppCombine cu = reinterpret_cast<const WppCombine*>(plan + hd->off_combine)[blockIdx.x];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int D = p.head_dim;
+    for (int r = warp; r < cu.num_rows; r += 8) {
+        float m = -INFINITY;
+        for (int s = 0; s < cu.num_splits; ++s)
+            m = fmaxf(m, p.ws_lse[(int64_t)(cu.slot0 + s) * p.tile_m + r]);
+        const int64_t tok = (int64_t)q_offsets[cu.request] + cu.q_row0 + r;
+        __nv_bfloat16* dst = p.out + tok * p.o_token_stride + (int64_t)cu.q_head * p.o_head_stride;
+        float wsum = 0.f;
+        float acc[4] = {0.f, 0.f, 0.f, 0.f};
+        if (m > -INFINITY) {
+            for (int s = 0; s < cu.num_splits; ++s) {
+                const int64_t row = (int64_t)(cu.slot0 + s) * p.tile_m + r;
+                const float l = p.ws_lse[row];
+                if (l == -INFINITY) continue;       // that part saw no key of this row; its O row is not defined
+                const float w = exp2f(l - m);
+                wsum += w;
+                for (int e = lane, k = 0; e < D; e += 32, ++k) acc[k] += w * p.ws_o[row * D + e];
+            }
+        }
+        const float inv = wsum > 0.f ? 1.f / wsum : 0.f;
+        for (int e = lane, k = 0; e < D; e += 32, ++k) dst[e] = __float2bfloat16_rn(acc[k] * inv);
+        if (p.lse && lane == 0)
+            p.lse[tok * p.num_q_heads + cu.q_head] =
+                wsum > 0.f ? (m + log2f(wsum)) * 0.6931471805599453f : -INFINITY;
+    }
+}
+
+}  // namespace wpp
+
+extern "C" int wpp_launch_append(const wpp::AppendParams* p, int num_sms, void* stream) {
+    const int64_t total = p->total_new_tokens * p->num_kv_heads * p->vec_per_row;
+    if (total == 0) return 0;
+    int64_t blocks = (total + 255) / 256;
+    const int64_t cap = (int64_t)num_sms * 16;
+    if (blocks > cap) blocks = cap;
+    wpp::wpp_append_kernel<<<(unsigned)blocks, 256, 0, (cudaStream_t)stream>>>(*p);
+    return (int)cudaGetLastError();
+}
+
+extern "C" int wpp_launch_combine(const wpp::CombineParams* p, int num_combine, void* stream) {
+    if (num_combine == 0) return 0;
+    wpp::wpp_combine_kernel<<<(unsigned)num_combine, 256, 0, (cudaStream_t)stream>>>(*p);
+    return (int)cudaGetLastError();
+}

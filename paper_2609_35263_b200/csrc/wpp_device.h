@@ -1,0 +1,58 @@
+// Kernel parameter blocks and launch entry points shared by the launch code and the kernel files.
+#pragma once
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+
+#include "../../include/wpp.h"
+
+namespace wpp {
+
+struct AttnParams {
+    const void* plan;                // device copy of the plan
+    const int32_t* block_tables;     // [R][max_blocks]
+    const int32_t* prefix_lens;      // [R]
+    const int32_t* chunk_lens;       // [R]
+    __nv_bfloat16* out;              // [T][Hq][d]
+    float* lse;                      // [T][Hq] or null
+    float* ws_o;                     // split partials: [slots][tile_m][d]
+    float* ws_lse;                   // [slots][tile_m], log2 units
+    int32_t* status;                 // sticky device status word or null
+    int64_t o_token_stride, o_head_stride;
+    int32_t num_q_heads, group, page_size, max_blocks, num_pages;
+    float scale_log2;                // sm_scale * log2(e)
+};
+
+struct AppendParams {
+    const void* plan;
+    const uint4* k_new;
+    const uint4* v_new;
+    uint4* k_cache;
+    uint4* v_cache;
+    const int32_t* block_tables;
+    const int32_t* prefix_lens;
+    int32_t* status;
+    int64_t kvnew_token_stride, kvnew_head_stride;       // in 16-byte units
+    int64_t kv_page_stride, kv_head_stride, kv_token_stride;
+    int32_t num_requests, num_kv_heads, vec_per_row, page_size, max_blocks, num_pages;
+    int64_t total_new_tokens;
+};
+
+struct CombineParams {
+    const void* plan;
+    const float* ws_o;
+    const float* ws_lse;
+    __nv_bfloat16* out;
+    float* lse;
+    int64_t o_token_stride, o_head_stride;
+    int32_t num_q_heads, head_dim, tile_m;
+};
+
+}  // namespace wpp
+
+extern "C" {
+int wpp_launch_attention(int head_dim, const CUtensorMap* tq, const CUtensorMap* tk, const CUtensorMap* tv,
+                         const wpp::AttnParams* p, int num_ctas, void* stream);
+int wpp_launch_append(const wpp::AppendParams* p, int num_sms, void* stream);
+int wpp_launch_combine(const wpp::CombineParams* p, int num_combine, void* stream);
+}

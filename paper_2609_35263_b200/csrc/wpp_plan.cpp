@@ -1,0 +1,328 @@
+// Host side of the library that needs no CUDA: argument checks, the work split (wpp_plan_tiles)
+// and the optional aliasing check (wpp_validate_batch).  Integer arithmetic only.
+#include <algorithm>
+#include <cstring>
+#include <queue>
+#include <unordered_map>
+#include <vector>
+
+#include "../../include/wpp.h"
+#include "wpp_host.h"
+#include "wpp_plan_format.h"
+
+const char* wpp_status_string(int s) {
+    switch (s) {
+        case WPP_OK: return "WPP_OK";
+        case WPP_ERR_INVALID_ARG: return "WPP_ERR_INVALID_ARG";
+        case WPP_ERR_UNSUPPORTED: return "WPP_ERR_UNSUPPORTED";
+        case WPP_ERR_BOUNDS: return "WPP_ERR_BOUNDS";
+        case WPP_ERR_POSITION_MISMATCH: return "WPP_ERR_POSITION_MISMATCH";
+        case WPP_ERR_WORKSPACE_TOO_SMALL: return "WPP_ERR_WORKSPACE_TOO_SMALL";
+        case WPP_ERR_PLAN_MISMATCH: return "WPP_ERR_PLAN_MISMATCH";
+        case WPP_ERR_CUDA: return "WPP_ERR_CUDA";
+        case WPP_ERR_TIMEOUT: return "WPP_ERR_TIMEOUT";
+        case WPP_ERR_ALIASED_APPEND: return "WPP_ERR_ALIASED_APPEND";
+        default: return "WPP_ERR_UNKNOWN";
+    }
+}
+
+// Fill in default strides and check what the host can check about a description.
+int wpp_resolve_desc(const wpp_batch_desc* in, wpp_batch_desc* d) {
+    if (!in) return WPP_ERR_INVALID_ARG;
+    *d = *in;
+    if (d->num_requests < 0 || d->num_q_heads <= 0 || d->num_kv_heads <= 0 || d->max_blocks_per_req < 0 ||
+        d->num_pages < 0 || d->head_dim <= 0 || d->page_size <= 0 || !(d->sm_scale >= 0.0f))
+        return WPP_ERR_INVALID_ARG;
+    if (d->dtype != WPP_BF16) return WPP_ERR_UNSUPPORTED;
+    if (d->head_dim != 64 && d->head_dim != 128) return WPP_ERR_UNSUPPORTED;
+    if (d->page_size != 16 && d->page_size != 32 && d->page_size != 64 && d->page_size != 128)
+        return WPP_ERR_UNSUPPORTED;
+    if (d->num_q_heads % d->num_kv_heads != 0) return WPP_ERR_UNSUPPORTED;
+    const int64_t dd = d->head_dim;
+    if (!d->kv_token_stride) d->kv_token_stride = dd;
+    if (!d->kv_head_stride) d->kv_head_stride = d->kv_token_stride * d->page_size;
+    if (!d->kv_page_stride) d->kv_page_stride = d->kv_head_stride * d->num_kv_heads;
+    if (!d->q_head_stride) d->q_head_stride = dd;
+    if (!d->q_token_stride) d->q_token_stride = d->q_head_stride * d->num_q_heads;
+    if (!d->kvnew_head_stride) d->kvnew_head_stride = dd;
+    if (!d->kvnew_token_stride) d->kvnew_token_stride = d->kvnew_head_stride * d->num_kv_heads;
+    if (!d->o_head_stride) d->o_head_stride = dd;
+    if (!d->o_token_stride) d->o_token_stride = d->o_head_stride * d->num_q_heads;
+    const int64_t strides[] = {d->kv_page_stride, d->kv_head_stride, d->kv_token_stride, d->q_token_stride,
+                               d->q_head_stride, d->kvnew_token_stride, d->kvnew_head_stride,
+                               d->o_token_stride, d->o_head_stride};
+    for (int64_t s : strides)
+        if (s < dd || (s % 8) != 0) return WPP_ERR_INVALID_ARG;  // 8 bf16 = 16 bytes
+    return WPP_OK;
+}
+
+static uint64_t fnv1a(uint64_t h, const void* p, size_t n) {
+    const unsigned char* b = static_cast<const unsigned char*>(p);
+    for (size_t i = 0; i < n; ++i) { h ^= b[i]; h *= 0x100000001b3ull; }
+    return h;
+}
+
+// Hash of everything a plan depends on except the lengths (those are covered by q_offsets checks).
+uint64_t wpp_desc_hash(const wpp_batch_desc* d) {
+    uint64_t h = 0xcbf29ce484222325ull;
+    const int32_t ints[] = {d->num_requests, d->num_q_heads, d->num_kv_heads, d->head_dim, d->page_size,
+                            d->max_blocks_per_req, d->num_pages, d->dtype};
+    h = fnv1a(h, ints, sizeof(ints));
+    const int64_t strides[] = {d->kv_page_stride, d->kv_head_stride, d->kv_token_stride, d->q_token_stride,
+                               d->q_head_stride, d->kvnew_token_stride, d->kvnew_head_stride,
+                               d->o_token_stride, d->o_head_stride};
+    return fnv1a(h, strides, sizeof(strides));
+}
+
+static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+static int resolve_opts(const wpp_ctx* ctx, const wpp_plan_opts* in, wpp_plan_opts* o) {
+    wpp_plan_opts z = {0, 0, 0, 0};
+    *o = in ? *in : z;
+    if (!o->tile_m) o->tile_m = WPP_DEFAULT_TILE_M;
+    if (!o->tile_n) o->tile_n = WPP_TILE_N;
+    if (!o->max_ctas) o->max_ctas = ctx ? wpp_ctx_sm_count(ctx) : 148;
+    if (o->tile_m != 128 && o->tile_m != 256) return WPP_ERR_UNSUPPORTED;
+    if (o->tile_m > WPP_MAX_TILE_M) return WPP_ERR_UNSUPPORTED;
+    if (o->tile_n != WPP_TILE_N) return WPP_ERR_UNSUPPORTED;
+    if (o->force_kv_splits < 0 || o->force_kv_splits > 64 || o->max_ctas < 1 || o->max_ctas > 4096)
+        return WPP_ERR_INVALID_ARG;
+    return WPP_OK;
+}
+
+static size_t plan_bytes_bound(const wpp_batch_desc* d, const wpp_plan_opts* o, int64_t T) {
+    const int64_t q_tiles = T / o->tile_m + d->num_requests;
+    const int64_t base = q_tiles * d->num_q_heads;
+    const int64_t units = o->force_kv_splits >= 2 ? base * o->force_kv_splits : base + 2 * (int64_t)o->max_ctas;
+    size_t n = sizeof(WppPlanHeader);
+    n += align_up(sizeof(int32_t) * (size_t)(d->num_requests + 1), 16);
+    n += align_up(sizeof(int32_t) * (size_t)(o->max_ctas + 1), 16);
+    n += sizeof(WppUnit) * (size_t)units;
+    n += sizeof(WppCombine) * (size_t)base;
+    return align_up(n, 256);
+}
+
+size_t wpp_plan_bytes(const wpp_ctx* ctx, const wpp_batch_desc* desc, int64_t total_new_tokens,
+                      const wpp_plan_opts* opts_or_null) {
+    wpp_batch_desc d;
+    wpp_plan_opts o;
+    if (wpp_resolve_desc(desc, &d) != WPP_OK || total_new_tokens < 0) return 0;
+    if (resolve_opts(ctx, opts_or_null, &o) != WPP_OK) return 0;
+    return plan_bytes_bound(&d, &o, total_new_tokens);
+}
+
+int wpp_plan_tiles(const wpp_ctx* ctx, const wpp_batch_desc* desc, const int32_t* prefix_lens,
+                   const int32_t* chunk_lens, const int32_t* cached_lens, const wpp_plan_opts* opts_in,
+                   void* plan_host, size_t plan_host_bytes, wpp_plan_info* info) {
+    wpp_batch_desc d;
+    wpp_plan_opts o;
+    int rc = wpp_resolve_desc(desc, &d);
+    if (rc != WPP_OK) return rc;
+    rc = resolve_opts(ctx, opts_in, &o);
+    if (rc != WPP_OK) return rc;
+    const int R = d.num_requests;
+    if (!plan_host || !info || (R > 0 && (!prefix_lens || !chunk_lens))) return WPP_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(plan_host) & 15) != 0) return WPP_ERR_INVALID_ARG;
+    const int B = d.page_size, Hq = d.num_q_heads;
+
+    int64_t T = 0, pairs = 0;
+    for (int i = 0; i < R; ++i) {
+        const int64_t P = prefix_lens[i], C = chunk_lens[i];
+        if (P < 0 || C < 0) return WPP_ERR_INVALID_ARG;
+        if (P + C > (int64_t)0x7fffffff - 4 * WPP_TILE_N) return WPP_ERR_INVALID_ARG;
+        if (cached_lens && cached_lens[i] != prefix_lens[i]) return WPP_ERR_POSITION_MISMATCH;
+        if (C > 0 && (P + C + B - 1) / B > d.max_blocks_per_req) return WPP_ERR_BOUNDS;
+        T += C;
+        pairs += C * P + C * (C + 1) / 2;
+    }
+    if (T > 0x7fffffff) return WPP_ERR_INVALID_ARG;
+    if (plan_host_bytes < plan_bytes_bound(&d, &o, T)) return WPP_ERR_PLAN_MISMATCH;
+
+    // ---- base tiles: (request, query-row tile, query head), natural order keeps the heads of one
+    //      KV group and the row tiles of one request next to each other (they share K/V in L2).
+    struct Base { int32_t request, q_row0, num_rows, q_head, steps; int64_t cost; };
+    std::vector<Base> base;
+    const int TM = o.tile_m;
+    auto steps_for = [](int64_t last_visible_plus1) { return (int32_t)((last_visible_plus1 + WPP_TILE_N - 1) / WPP_TILE_N); };
+    for (int i = 0; i < R; ++i) {
+        const int64_t P = prefix_lens[i], C = chunk_lens[i];
+        for (int64_t r0 = 0; r0 < C; r0 += TM) {
+            const int32_t rows = (int32_t)std::min<int64_t>(TM, C - r0);
+            const int32_t steps = steps_for(P + r0 + rows);
+            for (int h = 0; h < Hq; ++h) base.push_back({i, (int32_t)r0, rows, h, steps, 0});
+        }
+    }
+    const int64_t n_base = (int64_t)base.size();
+
+    // cost of key steps [a, b) of a tile = 128x128 steps over its (up to two) 128-row halves
+    auto cost_of = [&](const Base& t, int32_t a, int32_t b) -> int32_t {
+        const int64_t P = prefix_lens[t.request];
+        int32_t c = 0;
+        for (int32_t r = 0; r < t.num_rows; r += WPP_HALF_M) {
+            const int32_t rows = std::min(WPP_HALF_M, t.num_rows - r);
+            const int32_t end = std::min(b, steps_for(P + t.q_row0 + r + rows));
+            c += std::max(0, end - a);
+        }
+        return c;
+    };
+
+    // ---- split decision
+    int32_t want_parts = 1;
+    if (o.force_kv_splits >= 2) want_parts = o.force_kv_splits;
+    else if (o.force_kv_splits == 0 && n_base > 0 && n_base < o.max_ctas)
+        want_parts = (int32_t)((o.max_ctas + n_base - 1) / n_base);
+
+    std::vector<WppUnit> units;
+    std::vector<WppCombine> combines;
+    units.reserve((size_t)n_base);
+    int32_t slots = 0;
+    int64_t key_steps = 0, n_split_units = 0;
+    for (const Base& t : base) {
+        int32_t parts = 1;
+        if (want_parts > 1) {
+            const int32_t cap = o.force_kv_splits >= 2 ? t.steps : t.steps / 2;  // auto: >= 2 steps per part
+            parts = std::max(1, std::min(want_parts, cap));
+        }
+        if (parts == 1) {
+            const int32_t c = cost_of(t, 0, t.steps);
+            units.push_back({t.request, t.q_row0, t.num_rows, t.q_head, 0, t.steps, -1, c});
+            key_steps += c;
+        } else {
+            combines.push_back({t.request, t.q_row0, t.num_rows, t.q_head, slots, parts, 0, 0});
+            for (int32_t p = 0; p < parts; ++p) {
+                const int32_t a = (int32_t)((int64_t)t.steps * p / parts);
+                const int32_t b = (int32_t)((int64_t)t.steps * (p + 1) / parts);
+                const int32_t c = cost_of(t, a, b);
+                units.push_back({t.request, t.q_row0, t.num_rows, t.q_head, a, b, slots + p, c});
+                key_steps += c;
+                ++n_split_units;
+            }
+            slots += parts;
+        }
+    }
+    const int64_t n_units = (int64_t)units.size();
+    if (n_units > 0x7fffffff) return WPP_ERR_INVALID_ARG;
+
+    // ---- longest-processing-time assignment to persistent CTAs; stable sort keeps neighbours adjacent
+    const int num_ctas = (int)std::max<int64_t>(1, std::min<int64_t>(o.max_ctas, n_units));
+    std::vector<int32_t> order((size_t)n_units);
+    for (int64_t u = 0; u < n_units; ++u) order[(size_t)u] = (int32_t)u;
+    std::stable_sort(order.begin(), order.end(),
+                     [&](int32_t a, int32_t b) { return units[(size_t)a].cost > units[(size_t)b].cost; });
+    typedef std::pair<int64_t, int32_t> Load;  // (accumulated cost, cta)
+    std::priority_queue<Load, std::vector<Load>, std::greater<Load>> heap;
+    for (int c = 0; c < num_ctas; ++c) heap.push({0, c});
+    std::vector<std::vector<int32_t>> lists((size_t)num_ctas);
+    for (int32_t u : order) {
+        Load l = heap.top();
+        heap.pop();
+        lists[(size_t)l.second].push_back(u);
+        l.first += std::max(1, units[(size_t)u].cost);
+        heap.push(l);
+    }
+
+    // ---- serialise
+    WppPlanHeader hd;
+    std::memset(&hd, 0, sizeof(hd));
+    hd.magic = WPP_PLAN_MAGIC;
+    hd.version = WPP_PLAN_VERSION;
+    hd.desc_hash = wpp_desc_hash(&d);
+    hd.num_requests = R;
+    hd.num_ctas = num_ctas;
+    hd.num_units = (int32_t)n_units;
+    hd.num_combine = (int32_t)combines.size();
+    hd.num_split_slots = slots;
+    hd.tile_m = TM;
+    hd.tile_n = WPP_TILE_N;
+    hd.head_dim = d.head_dim;
+    hd.total_new_tokens = T;
+    hd.key_steps = key_steps;
+    hd.flops = 4 * (int64_t)d.head_dim * Hq * pairs;
+    hd.workspace_bytes = slots ? align_up((size_t)slots * TM * (d.head_dim + 1) * sizeof(float), 256) : 0;
+    size_t off = sizeof(WppPlanHeader);
+    hd.off_q_offsets = (uint32_t)off;
+    off += align_up(sizeof(int32_t) * (size_t)(R + 1), 16);
+    hd.off_cta_begin = (uint32_t)off;
+    off += align_up(sizeof(int32_t) * (size_t)(num_ctas + 1), 16);
+    hd.off_units = (uint32_t)off;
+    off += sizeof(WppUnit) * (size_t)n_units;
+    hd.off_combine = (uint32_t)off;
+    off += sizeof(WppCombine) * combines.size();
+    hd.plan_bytes = align_up(off, 16);
+    if (hd.plan_bytes > plan_host_bytes) return WPP_ERR_PLAN_MISMATCH;
+
+    char* p = static_cast<char*>(plan_host);
+    std::memset(p, 0, hd.plan_bytes);
+    std::memcpy(p, &hd, sizeof(hd));
+    int32_t* qo = reinterpret_cast<int32_t*>(p + hd.off_q_offsets);
+    qo[0] = 0;
+    for (int i = 0; i < R; ++i) qo[i + 1] = qo[i] + chunk_lens[i];
+    int32_t* cb = reinterpret_cast<int32_t*>(p + hd.off_cta_begin);
+    WppUnit* us = reinterpret_cast<WppUnit*>(p + hd.off_units);
+    int32_t k = 0;
+    for (int c = 0; c < num_ctas; ++c) {
+        cb[c] = k;
+        for (int32_t u : lists[(size_t)c]) us[k++] = units[(size_t)u];
+    }
+    cb[num_ctas] = k;
+    if (!combines.empty())
+        std::memcpy(p + hd.off_combine, combines.data(), sizeof(WppCombine) * combines.size());
+
+    info->num_tiles = n_units;
+    info->num_split_tiles = n_split_units;
+    info->num_combine_tiles = (int64_t)combines.size();
+    info->num_ctas = num_ctas;
+    info->total_new_tokens = T;
+    info->key_steps = key_steps;
+    info->flops = hd.flops;
+    info->workspace_bytes = hd.workspace_bytes;
+    info->plan_bytes = hd.plan_bytes;
+    return WPP_OK;
+}
+
+// Check a host plan against a description; returns the header on success.
+int wpp_check_plan(const void* plan_host, const wpp_batch_desc* resolved, const WppPlanHeader** out) {
+    if (!plan_host) return WPP_ERR_INVALID_ARG;
+    const WppPlanHeader* h = static_cast<const WppPlanHeader*>(plan_host);
+    if (h->magic != WPP_PLAN_MAGIC || h->version != WPP_PLAN_VERSION) return WPP_ERR_PLAN_MISMATCH;
+    if (h->desc_hash != wpp_desc_hash(resolved) || h->num_requests != resolved->num_requests ||
+        h->head_dim != resolved->head_dim)
+        return WPP_ERR_PLAN_MISMATCH;
+    *out = h;
+    return WPP_OK;
+}
+
+int wpp_validate_batch(const wpp_batch_desc* desc, const int32_t* bt, const int32_t* prefix_lens,
+                       const int32_t* chunk_lens) {
+    wpp_batch_desc d;
+    int rc = wpp_resolve_desc(desc, &d);
+    if (rc != WPP_OK) return rc;
+    const int R = d.num_requests, B = d.page_size;
+    if (R > 0 && (!bt || !prefix_lens || !chunk_lens)) return WPP_ERR_INVALID_ARG;
+    // written slot -> writer; read ranges per page -> max readable slots by a non-writer
+    std::unordered_map<int64_t, int32_t> writer;   // page*B+slot -> request
+    for (int i = 0; i < R; ++i) {
+        const int64_t P = prefix_lens[i], C = chunk_lens[i];
+        if (P < 0 || C < 0) return WPP_ERR_INVALID_ARG;
+        const int64_t n = P + C;
+        if (C > 0 && (n + B - 1) / B > d.max_blocks_per_req) return WPP_ERR_BOUNDS;
+        if (C == 0) continue;
+        for (int64_t j = 0; j < (n + B - 1) / B; ++j) {
+            const int32_t page = bt[(int64_t)i * d.max_blocks_per_req + j];
+            if (page < 0 || page >= d.num_pages) return WPP_ERR_BOUNDS;
+        }
+        for (int64_t pos = P; pos < n; ++pos) {
+            const int64_t key = (int64_t)bt[(int64_t)i * d.max_blocks_per_req + pos / B] * B + pos % B;
+            if (!writer.emplace(key, i).second) return WPP_ERR_ALIASED_APPEND;
+        }
+    }
+    for (int i = 0; i < R; ++i) {
+        if (chunk_lens[i] == 0) continue;
+        const int64_t P = prefix_lens[i];
+        for (int64_t pos = 0; pos < P; ++pos) {
+            const int64_t key = (int64_t)bt[(int64_t)i * d.max_blocks_per_req + pos / B] * B + pos % B;
+            if (writer.count(key)) return WPP_ERR_ALIASED_APPEND;   // someone writes what this request reads
+        }
+    }
+    return WPP_OK;
+}

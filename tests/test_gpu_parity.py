@@ -1,0 +1,178 @@
+"""GPU parity: the CUDA path through the C ABI against the fp64 oracle, element by element."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2609_35263_b200 as wpp
+import wpp_workloads as W
+from tests.helpers import bits, cpu_inputs, f64, from_bits, run_oracle
+from tests import gpu_harness as H
+
+pytestmark = pytest.mark.gpu
+
+
+def _full_parity(w, opts=None, inp=None, sm_scale=0.0):
+    inp = inp or cpu_inputs(w)
+    kp, vp, ref, ref_lse = run_oracle(w, inp, sm_scale=sm_scale or None)
+    res = H.run_wave(w, H.device_inputs(w, inp), opts=opts, sm_scale=sm_scale)
+    assert res["status"] == 0
+    # append and page indexing: bit exact over the whole pools
+    assert np.array_equal(bits(res["k_pool"]), kp), "K pool differs"
+    assert np.array_equal(bits(res["v_pool"]), vp), "V pool differs"
+    e = H.assert_close(f64(res["out"]), ref, w.name)
+    lse = res["lse"].double().cpu().numpy()
+    assert np.isfinite(lse).all() and np.abs(lse - ref_lse).max() < 2e-2, np.abs(lse - ref_lse).max()
+    return res, e
+
+
+def test_cfg1_single_request():
+    res, e = _full_parity(W.cfg1())
+    print("cfg1", e)
+
+
+@pytest.mark.parametrize("P,C,Hq,Hkv,d,B", [
+    ([0], [1], 2, 1, 64, 16),                    # one key: output is V[0] exactly
+    ([0], [128], 4, 2, 128, 64),                 # pure causal, exactly one tile
+    ([0], [129], 2, 2, 128, 64),                 # one row spills into a second tile
+    ([37], [200], 4, 1, 128, 16),                # prefix ends mid page and mid key step
+    ([300, 0, 1000, 64], [17, 260, 3, 128], 8, 2, 128, 64),
+    ([5, 130, 257], [400, 1, 127], 4, 4, 64, 32),
+    ([1024], [512], 2, 1, 128, 128),
+    ([100, 0], [0, 70], 2, 1, 64, 16),           # an empty chunk in the wave
+])
+def test_ragged_small(P, C, Hq, Hkv, d, B):
+    w = W.custom_workload(P, C, Hq, Hkv, d, B, seed=7, spare_pages=5)
+    _full_parity(w)
+
+
+def test_single_key_is_bit_exact():
+    w = W.custom_workload([0], [1], 4, 2, 128, 64, seed=8)
+    inp = cpu_inputs(w)
+    res = H.run_wave(w, H.device_inputs(w, inp))
+    v0 = inp["v_new"][0]                                     # [Hkv, d]
+    out = res["out"].cpu()
+    for h in range(4):
+        assert torch.equal(out[0, h].view(torch.int16), v0[h // 2].view(torch.int16))
+
+
+@pytest.mark.parametrize("splits", [2, 3, 7])
+def test_forced_kv_splits_and_combine(splits):
+    w = W.custom_workload([900, 0, 130], [300, 500, 64], 4, 2, 128, 64, seed=9)
+    opts = wpp.PlanOpts(0, 0, splits, 0)
+    res, _ = _full_parity(w, opts=opts)
+    assert res["plan"].info.num_combine_tiles > 0 and res["plan"].info.workspace_bytes > 0
+
+
+def test_explicit_scale():
+    w = W.custom_workload([70], [150], 2, 1, 128, 64, seed=10)
+    _full_parity(w, sm_scale=0.05)
+
+
+def test_empty_wave_is_a_no_op():
+    w = W.custom_workload([10, 20], [0, 0], 2, 1, 64, 16, seed=11)
+    res = H.run_wave(w, H.device_inputs(w))
+    assert res["status"] == 0 and res["out"].numel() == 0
+
+
+def test_results_are_bit_reproducible():
+    w = W.custom_workload([500, 77], [260, 300], 8, 2, 128, 64, seed=12)
+    inp = cpu_inputs(w)
+    a = H.run_wave(w, H.device_inputs(w, inp), opts=wpp.PlanOpts(0, 0, 3, 0))
+    b = H.run_wave(w, H.device_inputs(w, inp), opts=wpp.PlanOpts(0, 0, 3, 0))
+    assert torch.equal(a["out"].view(torch.int16), b["out"].view(torch.int16))
+    assert torch.equal(a["lse"], b["lse"])
+
+
+def test_stale_slots_unused_pages_and_scratch_poison_do_not_matter():
+    """NaN bit patterns everywhere the method must not look: slots past the sequence end, unreferenced pages."""
+    w = W.custom_workload([90, 3, 0], [40, 200, 5], 4, 2, 128, 64, seed=13, spare_pages=6)
+    inp = cpu_inputs(w)
+    kp, vp = bits(inp["k_pool"]).copy(), bits(inp["v_pool"]).copy()
+    live = np.zeros((w.num_pages, w.page_size), dtype=bool)
+    for i in range(w.num_requests):
+        for pos in range(int(w.prefix_lens[i])):
+            live[w.block_tables[i, pos // w.page_size], pos % w.page_size] = True
+    dead = np.broadcast_to(~live[:, None, :, None], kp.shape)
+    kp[dead] = 0x7FC0
+    vp[dead] = 0xFFFF
+    inp = dict(inp, k_pool=from_bits(kp), v_pool=from_bits(vp))
+    _full_parity(w, inp=inp)
+    _full_parity(w, inp=inp, opts=wpp.PlanOpts(0, 0, 2, 0))
+
+
+def test_page_permutation_gives_identical_bits():
+    w = W.custom_workload([200, 0], [130, 260], 4, 2, 128, 64, seed=14, spare_pages=4)
+    inp = cpu_inputs(w)
+    a = H.run_wave(w, H.device_inputs(w, inp))
+    perm = np.random.default_rng(15).permutation(w.num_pages)
+    kp = torch.empty_like(inp["k_pool"]); vp = torch.empty_like(inp["v_pool"])
+    kp[perm] = inp["k_pool"]; vp[perm] = inp["v_pool"]
+    w2 = W.custom_workload([200, 0], [130, 260], 4, 2, 128, 64, seed=14, spare_pages=4)
+    w2.block_tables = np.where(w.block_tables >= 0, perm[np.maximum(w.block_tables, 0)], -1).astype(np.int32)
+    b = H.run_wave(w2, H.device_inputs(w2, dict(inp, k_pool=kp, v_pool=vp)))
+    assert torch.equal(a["out"].view(torch.int16), b["out"].view(torch.int16))
+
+
+def test_successive_chunks_on_one_stream_equal_one_shot():
+    """Chunks of one request in successive calls (order kept by the stream) give the rows of one call."""
+    n, Hq, Hkv, d, B = 700, 4, 2, 128, 64
+    w_all = W.custom_workload([0], [n], Hq, Hkv, d, B, seed=16)
+    inp = cpu_inputs(w_all)
+    _, _, ref, _ = run_oracle(w_all, inp)
+    dev = H.device_inputs(w_all, inp)
+    outs, start = [], 0
+    for c in (130, 1, 300, 269):
+        w = W.custom_workload([start], [c], Hq, Hkv, d, B, seed=16)
+        w.block_tables = np.full((1, w_all.max_blocks_per_req), -1, dtype=np.int32)
+        w.block_tables[0, :] = w_all.block_tables[0]
+        w.num_pages = w_all.num_pages
+        part = dict(q=dev["q"][start:start + c], k_new=dev["k_new"][start:start + c],
+                    v_new=dev["v_new"][start:start + c], k_pool=dev["k_pool"], v_pool=dev["v_pool"])
+        res = H.run_wave(w, part)
+        assert res["status"] == 0
+        outs.append(f64(res["out"]))
+        start += c
+    H.assert_close(np.concatenate(outs), ref, "successive chunks")
+
+
+def test_bad_page_id_sets_status_without_trapping():
+    w = W.custom_workload([64], [64], 2, 1, 128, 64, seed=17)
+    w.block_tables = w.block_tables.copy()
+    w.block_tables[0, 1] = w.num_pages + 5
+    res = H.run_wave(w, H.device_inputs(w))
+    assert res["status"] == 3          # WPP_ERR_BOUNDS
+    # the context is still usable
+    w2 = W.custom_workload([64], [64], 2, 1, 128, 64, seed=17)
+    _full_parity(w2)
+
+
+def test_cfg2_sampled_rows():
+    """Ragged batch of 16: the oracle checks a seeded sample of (request, row, head) plus boundary rows."""
+    w = W.cfg2()
+    inp = cpu_inputs(w)
+    kp, vp = oracle.oracle_append(inp["k_new"], inp["v_new"], inp["k_pool"], inp["v_pool"], w.block_tables,
+                                  w.prefix_lens, w.chunk_lens)
+    res = H.run_wave(w, H.device_inputs(w, inp))
+    assert res["status"] == 0
+    assert np.array_equal(bits(res["k_pool"]), kp) and np.array_equal(bits(res["v_pool"]), vp)
+    rng = np.random.default_rng(202)
+    units = []
+    for i in range(w.num_requests):
+        C = int(w.chunk_lens[i])
+        for t in sorted({0, 1, 63, 64, 127, 128, C // 2, C - 2, C - 1}):
+            if 0 <= t < C:
+                units += [(i, t, h) for h in (0, 7, 31)]
+    for _ in range(600):
+        i = int(rng.integers(w.num_requests))
+        units.append((i, int(rng.integers(w.chunk_lens[i])), int(rng.integers(w.num_q_heads))))
+    units = np.array(units, dtype=np.int32)
+    ref, ref_lse = oracle.oracle_attention_units(inp["q"], kp, vp, w.block_tables, w.prefix_lens, w.chunk_lens, units)
+    off = w.q_offsets
+    rows = torch.from_numpy(off[units[:, 0]] + units[:, 1]).cuda()
+    heads = torch.from_numpy(units[:, 2].astype(np.int64)).cuda()
+    got = f64(res["out"][rows, heads])
+    print("cfg2", H.assert_close(got, ref, "cfg2 sample"))
+    got_lse = res["lse"][rows, heads].double().cpu().numpy()
+    assert np.abs(got_lse - ref_lse).max() < 2e-2
+    assert not torch.isnan(res["out"].float()).any()
