@@ -1,0 +1,378 @@
+#!/usr/bin/env python
+"""Benchmark of the chunked-prefill attention hot path (plan -> KV append -> paged attention).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config cfg3] [--impl reference]
+
+One step = one wave through the whole path: wpp_plan_tiles on the host, the plan's H2D copy, wpp_kv_append
+and wpp_prefill_attention_varlen, all through the C ABI.  Default workload: the concurrency-128 high-reuse
+configuration (80 % of 128 requests share a 16384-token prefix).  Prints ONE JSON line on rank 0.
+
+  value      new (query) tokens per second with every input resident in HBM
+  e2e        the same through host buffers: per step H2D of q/k_new/v_new/metadata from pinned memory and D2H of out
+  roofline   attention kernel: algorithmic FLOPs (4 d Hq sum(C P + C(C+1)/2)) / CUDA-event time vs measured bf16 peak
+  cpu_baseline  the fp64 oracle on this machine's host cores on a bounded seeded sample, extrapolated by visible pairs
+
+`--impl reference` times the oracle alone (the only reference there is: the paper ships no code).
+Multi-GPU: the path does not shard (one stage, one GPU); N > 1 runs N independent replicas ("weak").
+"""
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "prefill-attention tokens/s at concurrency 128, high prefix reuse"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        try:
+            d = json.load(open(path))
+            return d, "measured"
+        except Exception:
+            pass
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+def build_workload(name):
+    import wpp_workloads as W
+    if name in W.CONFIG_BUILDERS:
+        return W.CONFIG_BUILDERS[name]()
+    if name.startswith("cfg3_r"):         # cfg3_r16: the first 16 requests' worth of the same draw (for profiling)
+        return W.cfg3(num_requests=int(name[6:]))
+    if name.startswith("cfg5_"):          # cfg5_C1024_P4096
+        parts = dict((p[0], int(p[1:])) for p in name.split("_")[1:])
+        return W.cfg5_cell(parts["C"], parts["P"])
+    raise SystemExit(f"unknown config {name}")
+
+
+class ClockSampler:
+    """nvidia-smi clocks / throttle reasons sampled every 200 ms while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.proc = None
+        self.gpu_index = gpu_index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.gpu_index), f"--query-gpu={self.FIELDS}",
+                 "--format=csv,noheader,nounits", "-lms", "200"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.25)
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except Exception:
+            self.proc.kill()
+            out = ""
+        sm, mx, pw, reasons = [], [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.strip().splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1])); pw.append(float(f[2]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "power_w_max": max(pw) if pw else None, "samples": len(sm), "reasons": sorted(reasons)}
+
+
+class OracleSampler:
+    """Times the fp64 oracle on seeded samples of (request, row, head) units; extrapolates by visible pairs."""
+
+    def __init__(self, w, dev_available):
+        import torch
+        import oracle
+        self.oracle, self.w = oracle, w
+        dev = "cuda" if dev_available else "cpu"
+        # inputs straight from the generators (never from the CUDA path), moved to the host
+        self.q = w.q(dev).cpu()
+        k_new, v_new = w.k_new(dev).cpu(), w.v_new(dev).cpu()
+        k_pool, v_pool = w.k_pool(dev).cpu(), w.v_pool(dev).cpu()
+        if dev_available:
+            torch.cuda.empty_cache()
+        self.kp, self.vp = oracle.oracle_append(k_new, v_new, k_pool, v_pool, w.block_tables, w.prefix_lens,
+                                                w.chunk_lens)
+        self.rng = np.random.default_rng(12345)
+        self.P = w.prefix_lens.astype(np.int64)
+        self.C = w.chunk_lens.astype(np.int64)
+        self.live = np.nonzero(self.C > 0)[0]
+        self.total_pairs = w.visible_pairs * w.num_q_heads
+        self.rate = None          # visible pairs per second, from a probe
+        self.mean_pairs = None
+
+    def draw(self, n):
+        i = self.live[self.rng.integers(0, self.live.size, size=n)]
+        t = (self.rng.random(n) * self.C[i]).astype(np.int64)
+        h = self.rng.integers(0, self.w.num_q_heads, size=n)
+        return np.stack([i, t, h], axis=1).astype(np.int32)
+
+    def run(self, units):
+        w = self.w
+        t0 = time.perf_counter()
+        self.oracle.oracle_attention_units(self.q, self.kp, self.vp, w.block_tables, w.prefix_lens, w.chunk_lens,
+                                           units)
+        dt = time.perf_counter() - t0
+        return dt, int((self.P[units[:, 0]] + units[:, 1] + 1).sum())
+
+    def sample(self, seconds_target):
+        if self.rate is None:
+            probe = self.draw(256)
+            dt, pairs = self.run(probe)
+            self.rate, self.mean_pairs = pairs / max(dt, 1e-6), pairs / probe.shape[0]
+        n = int(max(256, min(2_000_000, seconds_target * self.rate / self.mean_pairs)))
+        dt, pairs = self.run(self.draw(n))
+        t_full = dt * self.total_pairs / pairs
+        return {"value": self.w.total_new_tokens / t_full, "unit": "tokens/s",
+                "cores": self.oracle.oracle_threads(), "kind": "oracle",
+                "sample": f"{n} seeded (request,row,head) units = {pairs:.3e} of {self.total_pairs:.3e} visible "
+                          f"pairs, {dt:.1f} s of fp64 CPU work, extrapolated by visible-pair count",
+                "sample_seconds": dt}
+
+
+def run_reference(args):
+    """Reference arm: the oracle as it stands on the host cores; each step is a bounded sample of the workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import torch
+    w = build_workload(args.config)
+    smp = OracleSampler(w, torch.cuda.is_available())
+    per_step = max(1.0, min(15.0, 90.0 / max(1, args.steps + args.warmup)))
+    vals, last = [], None
+    for s in range(args.warmup + args.steps):
+        last = smp.sample(per_step)
+        if s >= args.warmup:
+            vals.append(last["value"])
+    v = float(np.mean(vals))
+    line = {"impl": "reference", "metric": METRIC, "value": v, "unit": "tokens/s", "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * w.total_new_tokens / v,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": w.name, "note": "fp64 CPU oracle, one bounded seeded sample per step; "
+                       "ms_per_step is the extrapolated time of a full wave"},
+            "cpu_baseline": {"value": v, "unit": "tokens/s", "cores": last["cores"], "kind": "oracle",
+                             "sample": last["sample"]},
+            "e2e": {"value": v, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--config", default="cfg3")
+    ap.add_argument("--impl", default="native", choices=["native", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--force-kv-splits", type=int, default=0)
+    ap.add_argument("--cpu-seconds", type=float, default=15.0)
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "native" else args.warmup
+
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    import torch
+    import paper_2609_35263_b200 as wpp
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback for the product path")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+
+    peaks, peak_kind = load_peaks()
+    w = build_workload(args.config)
+    ctx = wpp.Context(local_rank)
+    desc = wpp.make_desc(w.num_requests, w.num_q_heads, w.num_kv_heads, w.head_dim, w.page_size,
+                         w.max_blocks_per_req, w.num_pages)
+    opts = wpp.PlanOpts(0, 0, args.force_kv_splits, 0)
+    T = w.total_new_tokens
+
+    # ---- resident state and inputs on the device
+    q, k_new, v_new = w.q(dev), w.k_new(dev), w.v_new(dev)
+    k_pool, v_pool = w.k_pool(dev), w.v_pool(dev)
+    bt_h = torch.from_numpy(w.block_tables).pin_memory()
+    P_h = torch.from_numpy(w.prefix_lens).pin_memory()
+    C_h = torch.from_numpy(w.chunk_lens).pin_memory()
+    bt, P, C = bt_h.to(dev), P_h.to(dev), C_h.to(dev)
+    out = torch.empty(T, w.num_q_heads, w.head_dim, dtype=torch.bfloat16, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+
+    plan_bytes = wpp.wpp_plan_tiles(ctx, desc, w.prefix_lens, w.chunk_lens, opts=opts).info
+    ring = 3
+    plan_host = [torch.empty(int(plan_bytes.plan_bytes) + 4096, dtype=torch.uint8).pin_memory() for _ in range(ring)]
+    plan_dev = [torch.empty(int(plan_bytes.plan_bytes) + 4096, dtype=torch.uint8, device=dev) for _ in range(ring)]
+    plan_free = [torch.cuda.Event() for _ in range(ring)]
+    ws = torch.empty(max(256, int(plan_bytes.workspace_bytes)), dtype=torch.uint8, device=dev)
+    stream = torch.cuda.current_stream()
+
+    def one_step(i, attn_events=None, qd=q, knd=k_new, vnd=v_new, btd=bt, Pd=P, Cd=C):
+        s = i % ring
+        plan_free[s].synchronize()                       # the copy that last used this buffer has run
+        plan = wpp.wpp_plan_tiles(ctx, desc, w.prefix_lens, w.chunk_lens, opts=opts, out=plan_host[s])
+        plan.to_device(out=plan_dev[s])
+        plan_free[s].record(stream)
+        wpp.wpp_kv_append(ctx, desc, knd, vnd, k_pool, v_pool, btd, Pd, Cd, plan, status=status)
+        if attn_events is not None:
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+        wpp.wpp_prefill_attention_varlen(ctx, desc, qd, out, None, k_pool, v_pool, btd, Pd, Cd, plan,
+                                         workspace=ws, status=status)
+        if attn_events is not None:
+            b.record(stream)
+            attn_events.append((a, b))
+        return plan
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            torch.distributed.barrier()
+        torch.cuda.synchronize()
+
+    def max_over_ranks(x):
+        if world == 1:
+            return x
+        t = torch.tensor([x], dtype=torch.float64, device=dev)
+        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+        return float(t.item())
+
+    # ---- device-resident timing
+    for i in range(args.warmup):
+        plan = one_step(i)
+    barrier()
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    launches0 = ctx.launch_count()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    attn_events = []
+    ev0.record(stream)
+    for i in range(args.steps):
+        plan = one_step(args.warmup + i, attn_events)
+    ev1.record(stream)
+    barrier()
+    launches = ctx.launch_count() - launches0
+    clocks = sampler.stop()
+    ms_step = max_over_ranks(ev0.elapsed_time(ev1) / args.steps)
+    attn_ms = statistics.mean(a.elapsed_time(b) for a, b in attn_events)
+    if int(status.item()) != 0:
+        raise SystemExit(f"device status {int(status.item())} after the timed region")
+    info = plan.info
+    flops = float(info.flops)
+    tokens_per_s = world * T / (ms_step * 1e-3)
+
+    roof_peak = float(peaks.get("bf16_tflops", FALLBACK_PEAKS["bf16_tflops"]))
+    roof_sus = float(peaks.get("bf16_tflops_sustained", FALLBACK_PEAKS["bf16_tflops_sustained"]))
+    achieved = flops / (attn_ms * 1e-3) / 1e12
+    # the bound is the slower of FLOPs at the tensor peak and compulsory bytes at HBM bandwidth
+    kv_bytes = w.unique_kv_pages() * w.num_kv_heads * w.page_size * w.head_dim * 2 * 2
+    qo_bytes = 2 * T * w.num_q_heads * w.head_dim * 2
+    t_flops = flops / (roof_peak * 1e12)
+    t_bytes = (kv_bytes + qo_bytes) / (float(peaks.get("hbm_gbs", FALLBACK_PEAKS["hbm_gbs"])) * 1e9)
+    traffic = None
+    tpath = os.path.join(ROOT, "profiles", "attention_traffic.json")
+    if os.path.exists(tpath):
+        try:
+            tj = json.load(open(tpath))
+            traffic = tj["dram_bytes_per_key_step"] * float(info.key_steps)
+        except Exception:
+            traffic = None
+    roofline = {"bound": "tensor" if t_flops >= t_bytes else "hbm", "kernel": "wpp_attn_kernel",
+                "achieved": achieved, "peak": roof_peak, "unit": "TFLOP/s", "frac": achieved / roof_peak,
+                "peak_source": f"of {peak_kind} (burst bf16 matmul)", "frac_of_sustained": achieved / roof_sus,
+                "traffic": traffic, "flops_per_launch": flops, "kernel_ms": attn_ms,
+                "roofline_ms": max(t_flops, t_bytes) * 1e3, "frac_of_roofline_time": max(t_flops, t_bytes) * 1e3 / attn_ms}
+
+    # ---- end to end through host buffers
+    e2e = None
+    if not args.no_e2e:
+        qh, knh, vnh = [torch.empty(x.shape, dtype=x.dtype).pin_memory() for x in (q, k_new, v_new)]
+        qh.copy_(q); knh.copy_(k_new); vnh.copy_(v_new)
+        out_h = torch.empty(out.shape, dtype=out.dtype).pin_memory()
+        qd2, knd2, vnd2 = torch.empty_like(q), torch.empty_like(k_new), torch.empty_like(v_new)
+        bt2, P2, C2 = torch.empty_like(bt), torch.empty_like(P), torch.empty_like(C)
+        h2d = sum(x.numel() * x.element_size() for x in (qh, knh, vnh, bt_h, P_h, C_h)) + int(info.plan_bytes)
+        d2h = out_h.numel() * out_h.element_size()
+
+        def e2e_step(i):
+            qd2.copy_(qh, non_blocking=True); knd2.copy_(knh, non_blocking=True); vnd2.copy_(vnh, non_blocking=True)
+            bt2.copy_(bt_h, non_blocking=True); P2.copy_(P_h, non_blocking=True); C2.copy_(C_h, non_blocking=True)
+            one_step(i, None, qd2, knd2, vnd2, bt2, P2, C2)
+            out_h.copy_(out, non_blocking=True)
+
+        e2e_steps = max(1, min(args.steps, 5))
+        e2e_step(0)
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for i in range(e2e_steps):
+            e2e_step(1 + i)
+        e1.record(stream)
+        barrier()
+        e2e_ms = max_over_ranks(e0.elapsed_time(e1) / e2e_steps)
+        e2e = {"value": world * T / (e2e_ms * 1e-3), "unit": "tokens/s", "h2d_bytes_per_step": int(h2d),
+               "d2h_bytes_per_step": int(d2h), "ms_per_step": e2e_ms, "steps": e2e_steps}
+        del qh, knh, vnh, out_h, qd2, knd2, vnd2
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        del q, k_new, v_new, k_pool, v_pool, out
+        torch.cuda.empty_cache()
+        cpu = OracleSampler(w, True).sample(args.cpu_seconds)
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": tokens_per_s, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": w.name, "requests": w.num_requests, "new_tokens": T,
+                       "served_tokens": int((w.prefix_lens.astype(np.int64) + w.chunk_lens).sum()),
+                       "q_heads": w.num_q_heads, "kv_heads": w.num_kv_heads, "head_dim": w.head_dim,
+                       "page_size": w.page_size, "parallelism": "replicas only" if world > 1 else "single GPU",
+                       "l2": f"inputs larger than L2: Q+O {qo_bytes / 1e9:.2f} GB + unique KV {kv_bytes / 1e9:.2f} GB touched "
+                             "per step vs 126 MB of L2; no explicit flush",
+                       "step": "wpp_plan_tiles + plan H2D + wpp_kv_append + wpp_prefill_attention_varlen",
+                       "tiles": int(info.num_tiles), "ctas": int(info.num_ctas), "key_steps": int(info.key_steps)},
+            "tflops": flops / (ms_step * 1e-3) / 1e12 * world,
+            "served_tokens_per_s": world * float((w.prefix_lens.astype(np.int64) + w.chunk_lens).sum()) / (ms_step * 1e-3),
+            "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline, "cpu_baseline": cpu,
+        }
+        print(json.dumps(line))
+    if world > 1:
+        torch.distributed.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -157,8 +157,13 @@ class Plan:
     def plan_bytes(self) -> int:
         return int(self.info.plan_bytes)
 
-    def to_device(self, device="cuda", non_blocking=True) -> "Plan":
-        self.dev = self.host[: self.plan_bytes].to(device, non_blocking=non_blocking)
+    def to_device(self, device="cuda", non_blocking=True, out: Optional[torch.Tensor] = None) -> "Plan":
+        """Copy the used part of the host plan to the device (into `out` if given) on the current stream."""
+        if out is not None:
+            out[: self.plan_bytes].copy_(self.host[: self.plan_bytes], non_blocking=non_blocking)
+            self.dev = out
+        else:
+            self.dev = self.host[: self.plan_bytes].to(device, non_blocking=non_blocking)
         return self
 
     def host_bytes(self) -> bytes:
@@ -166,8 +171,11 @@ class Plan:
 
 
 def wpp_plan_tiles(ctx: Optional[Context], desc: BatchDesc, prefix_lens, chunk_lens, cached_lens=None,
-                   opts: Optional[PlanOpts] = None, pin: Optional[bool] = None) -> Plan:
-    """Host-side work split; returns a Plan whose .host buffer must be copied to the device (.to_device())."""
+                   opts: Optional[PlanOpts] = None, pin: Optional[bool] = None,
+                   out: Optional[torch.Tensor] = None) -> Plan:
+    """Host-side work split; returns a Plan whose .host buffer must be copied to the device (.to_device()).
+
+    `out` may be a reusable host uint8 tensor (pinned for asynchronous copies) of at least wpp_plan_bytes bytes."""
     lib = load_library()
     P, C = _np_i32(prefix_lens), _np_i32(chunk_lens)
     T = int(C.astype(np.int64).sum())
@@ -177,8 +185,11 @@ def wpp_plan_tiles(ctx: Optional[Context], desc: BatchDesc, prefix_lens, chunk_l
     if nbytes == 0:
         # let wpp_plan_tiles report the precise error
         nbytes = 4096
-    pin = torch.cuda.is_available() if pin is None else pin
-    host = torch.empty(nbytes, dtype=torch.uint8, pin_memory=bool(pin))
+    if out is not None and out.numel() >= nbytes and out.dtype == torch.uint8 and out.device.type == "cpu":
+        host, nbytes = out, out.numel()
+    else:
+        pin = torch.cuda.is_available() if pin is None else pin
+        host = torch.empty(nbytes, dtype=torch.uint8, pin_memory=bool(pin))
     info = PlanInfo()
     cached = _np_i32(cached_lens) if cached_lens is not None else None
     st = lib.wpp_plan_tiles(h, ctypes.byref(desc), P.ctypes.data, C.ctypes.data,
