@@ -176,7 +176,7 @@ extern "C" int wpp_prefill_attention_varlen(const wpp_ctx* ctx, const wpp_batch_
     p.out = static_cast<__nv_bfloat16*>(out);
     p.lse = lse_or_null;
     p.ws_o = static_cast<float*>(workspace);
-    p.ws_lse = p.ws_o ? p.ws_o + (size_t)hd->num_split_slots * hd->tile_m * d.head_dim : nullptr;
+    p.ws_lse = p.ws_o ? p.ws_o + (size_t)hd->num_split_slots * 2 * WPP_HALF_M * d.head_dim : nullptr;
     p.status = status_dev;
     p.o_token_stride = d.o_token_stride;
     p.o_head_stride = d.o_head_stride;

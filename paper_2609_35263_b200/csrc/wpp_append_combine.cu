@@ -42,7 +42,7 @@ __global__ void __launch_bounds__(256) wpp_append_kernel(const AppendParams p) {
     }
 }
 
-// One block per split tile; one warp per row, lanes across head_dim.  Partials are merged in increasing split
+// One block per split half tile; one warp per row, lanes across head_dim.  Partials are merged in increasing split
 // order with weights exp2(lse_s - max lse), so the result does not depend on scheduling.
 __global__ void __launch_bounds__(256) wpp_combine_kernel(const CombineParams p) {
     const char* plan = static_cast<const char*>(p.plan);
@@ -51,17 +51,17 @@ __global__ void __launch_bounds__(256) wpp_combine_kernel(const CombineParams p)
     const WppCombine cu = reinterpret_cast<const WppCombine*>(plan + hd->off_combine)[blockIdx.x];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int D = p.head_dim;
-    for (int r = warp; r < cu.num_rows; r += 8) {
+    for (int r = warp; r < cu.rows; r += 8) {
         float m = -INFINITY;
         for (int s = 0; s < cu.num_splits; ++s)
-            m = fmaxf(m, p.ws_lse[(int64_t)(cu.slot0 + s) * p.tile_m + r]);
-        const int64_t tok = (int64_t)q_offsets[cu.request] + cu.q_row0 + r;
-        __nv_bfloat16* dst = p.out + tok * p.o_token_stride + (int64_t)cu.q_head * p.o_head_stride;
+            m = fmaxf(m, p.ws_lse[((int64_t)(cu.slot0 + s) * 2 + cu.half) * 128 + r]);
+        const int64_t tok = (int64_t)q_offsets[cu.request] + cu.row0 + r;
+        __nv_bfloat16* dst = p.out + tok * p.o_token_stride + (int64_t)cu.head * p.o_head_stride;
         float wsum = 0.f;
         float acc[4] = {0.f, 0.f, 0.f, 0.f};
         if (m > -INFINITY) {
             for (int s = 0; s < cu.num_splits; ++s) {
-                const int64_t row = (int64_t)(cu.slot0 + s) * p.tile_m + r;
+                const int64_t row = ((int64_t)(cu.slot0 + s) * 2 + cu.half) * 128 + r;
                 const float l = p.ws_lse[row];
                 if (l == -INFINITY) continue;       // that part saw no key of this row; its O row is not defined
                 const float w = exp2f(l - m);
@@ -72,7 +72,7 @@ __global__ void __launch_bounds__(256) wpp_combine_kernel(const CombineParams p)
         const float inv = wsum > 0.f ? 1.f / wsum : 0.f;
         for (int e = lane, k = 0; e < D; e += 32, ++k) dst[e] = __float2bfloat16_rn(acc[k] * inv);
         if (p.lse && lane == 0)
-            p.lse[tok * p.num_q_heads + cu.q_head] =
+            p.lse[tok * p.num_q_heads + cu.head] =
                 wsum > 0.f ? (m + log2f(wsum)) * 0.6931471805599453f : -INFINITY;
     }
 }

@@ -15,8 +15,8 @@ struct AttnParams {
     const int32_t* chunk_lens;       // [R]
     __nv_bfloat16* out;              // [T][Hq][d]
     float* lse;                      // [T][Hq] or null
-    float* ws_o;                     // split partials: [slots][tile_m][d]
-    float* ws_lse;                   // [slots][tile_m], log2 units
+    float* ws_o;                     // split partials: [slots][2][128][d]
+    float* ws_lse;                   // [slots][2][128], log2 units
     int32_t* status;                 // sticky device status word or null
     int64_t o_token_stride, o_head_stride;
     int32_t num_q_heads, group, page_size, max_blocks, num_pages;

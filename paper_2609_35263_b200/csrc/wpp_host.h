@@ -5,8 +5,8 @@
 #include "../../include/wpp.h"
 #include "wpp_plan_format.h"
 
-#define WPP_DEFAULT_TILE_M 128
-#define WPP_MAX_TILE_M 128
+#define WPP_DEFAULT_TILE_M 256
+#define WPP_MAX_TILE_M 256
 
 #ifdef __cplusplus
 extern "C" {

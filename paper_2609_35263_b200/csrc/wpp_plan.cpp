@@ -91,14 +91,14 @@ static int resolve_opts(const wpp_ctx* ctx, const wpp_plan_opts* in, wpp_plan_op
 }
 
 static size_t plan_bytes_bound(const wpp_batch_desc* d, const wpp_plan_opts* o, int64_t T) {
-    const int64_t q_tiles = T / o->tile_m + d->num_requests;
+    const int64_t q_tiles = T / WPP_HALF_M + d->num_requests;   // worst case: the planner falls back to 128-row tiles
     const int64_t base = q_tiles * d->num_q_heads;
     const int64_t units = o->force_kv_splits >= 2 ? base * o->force_kv_splits : base + 2 * (int64_t)o->max_ctas;
     size_t n = sizeof(WppPlanHeader);
     n += align_up(sizeof(int32_t) * (size_t)(d->num_requests + 1), 16);
     n += align_up(sizeof(int32_t) * (size_t)(o->max_ctas + 1), 16);
     n += sizeof(WppUnit) * (size_t)units;
-    n += sizeof(WppCombine) * (size_t)base;
+    n += sizeof(WppCombine) * (size_t)base * 2;
     return align_up(n, 256);
 }
 
@@ -120,6 +120,7 @@ int wpp_plan_tiles(const wpp_ctx* ctx, const wpp_batch_desc* desc, const int32_t
     if (rc != WPP_OK) return rc;
     rc = resolve_opts(ctx, opts_in, &o);
     if (rc != WPP_OK) return rc;
+    const bool auto_tile_m = !(opts_in && opts_in->tile_m);
     const int R = d.num_requests;
     if (!plan_host || !info || (R > 0 && (!prefix_lens || !chunk_lens))) return WPP_ERR_INVALID_ARG;
     if ((reinterpret_cast<uintptr_t>(plan_host) & 15) != 0) return WPP_ERR_INVALID_ARG;
@@ -138,31 +139,45 @@ int wpp_plan_tiles(const wpp_ctx* ctx, const wpp_batch_desc* desc, const int32_t
     if (T > 0x7fffffff) return WPP_ERR_INVALID_ARG;
     if (plan_host_bytes < plan_bytes_bound(&d, &o, T)) return WPP_ERR_PLAN_MISMATCH;
 
-    // ---- base tiles: (request, query-row tile, query head), natural order keeps the heads of one
-    //      KV group and the row tiles of one request next to each other (they share K/V in L2).
-    struct Base { int32_t request, q_row0, num_rows, q_head, steps; int64_t cost; };
-    std::vector<Base> base;
-    const int TM = o.tile_m;
+    // ---- base tiles in natural order (request, row block, head): the heads of one KV group and the row
+    //      blocks of one request stay next to each other, so tiles that run at the same time share K/V in L2.
+    struct Base { int32_t request, row0[2], rows[2], head[2], steps; };
+    const int G = Hq / d.num_kv_heads;
     auto steps_for = [](int64_t last_visible_plus1) { return (int32_t)((last_visible_plus1 + WPP_TILE_N - 1) / WPP_TILE_N); };
-    for (int i = 0; i < R; ++i) {
-        const int64_t P = prefix_lens[i], C = chunk_lens[i];
-        for (int64_t r0 = 0; r0 < C; r0 += TM) {
-            const int32_t rows = (int32_t)std::min<int64_t>(TM, C - r0);
-            const int32_t steps = steps_for(P + r0 + rows);
-            for (int h = 0; h < Hq; ++h) base.push_back({i, (int32_t)r0, rows, h, steps, 0});
+    auto build_base = [&](int tile_m, std::vector<Base>& base) {
+        base.clear();
+        for (int i = 0; i < R; ++i) {
+            const int64_t P = prefix_lens[i], C = chunk_lens[i];
+            for (int64_t r0 = 0; r0 < C; r0 += tile_m) {
+                const int32_t rows = (int32_t)std::min<int64_t>(tile_m, C - r0);
+                if (tile_m == 256 && rows <= WPP_HALF_M && G % 2 == 0) {
+                    // short tail: pair two heads of one KV group over the same rows
+                    for (int h = 0; h < Hq; h += 2)
+                        base.push_back({i, {(int32_t)r0, (int32_t)r0}, {rows, rows}, {h, h + 1}, steps_for(P + r0 + rows)});
+                } else {
+                    const int32_t ra = std::min(rows, WPP_HALF_M), rb = rows - ra;
+                    for (int h = 0; h < Hq; ++h)
+                        base.push_back({i, {(int32_t)r0, (int32_t)r0 + WPP_HALF_M}, {ra, rb}, {h, h}, steps_for(P + r0 + rows)});
+                }
+            }
         }
+    };
+    std::vector<Base> base;
+    int TM = o.tile_m;
+    build_base(TM, base);
+    if (auto_tile_m && TM == 256 && (int64_t)base.size() < o.max_ctas) {   // few tiles: prefer more, smaller ones
+        TM = 128;
+        build_base(TM, base);
     }
     const int64_t n_base = (int64_t)base.size();
 
-    // cost of key steps [a, b) of a tile = 128x128 steps over its (up to two) 128-row halves
+    // cost of key steps [a, b) of a tile = 128x128 steps over its halves, each cut at its own causal end
+    auto half_end = [&](const Base& t, int h) -> int32_t {
+        return t.rows[h] > 0 ? steps_for((int64_t)prefix_lens[t.request] + t.row0[h] + t.rows[h]) : 0;
+    };
     auto cost_of = [&](const Base& t, int32_t a, int32_t b) -> int32_t {
-        const int64_t P = prefix_lens[t.request];
         int32_t c = 0;
-        for (int32_t r = 0; r < t.num_rows; r += WPP_HALF_M) {
-            const int32_t rows = std::min(WPP_HALF_M, t.num_rows - r);
-            const int32_t end = std::min(b, steps_for(P + t.q_row0 + r + rows));
-            c += std::max(0, end - a);
-        }
+        for (int h = 0; h < 2; ++h) c += std::max(0, std::min(b, half_end(t, h)) - a);
         return c;
     };
 
@@ -183,18 +198,24 @@ int wpp_plan_tiles(const wpp_ctx* ctx, const wpp_batch_desc* desc, const int32_t
             const int32_t cap = o.force_kv_splits >= 2 ? t.steps : t.steps / 2;  // auto: >= 2 steps per part
             parts = std::max(1, std::min(want_parts, cap));
         }
+        WppUnit u;
+        std::memset(&u, 0, sizeof(u));
+        u.request = t.request;
+        for (int h = 0; h < 2; ++h) { u.row0[h] = t.row0[h]; u.rows[h] = t.rows[h]; u.head[h] = t.head[h]; }
         if (parts == 1) {
-            const int32_t c = cost_of(t, 0, t.steps);
-            units.push_back({t.request, t.q_row0, t.num_rows, t.q_head, 0, t.steps, -1, c});
-            key_steps += c;
+            u.kv_begin = 0; u.kv_end = t.steps; u.split_slot = -1; u.cost = cost_of(t, 0, t.steps);
+            units.push_back(u);
+            key_steps += u.cost;
         } else {
-            combines.push_back({t.request, t.q_row0, t.num_rows, t.q_head, slots, parts, 0, 0});
+            for (int h = 0; h < 2; ++h)
+                if (t.rows[h] > 0) combines.push_back({t.request, t.row0[h], t.rows[h], t.head[h], slots, parts, h, 0});
             for (int32_t p = 0; p < parts; ++p) {
-                const int32_t a = (int32_t)((int64_t)t.steps * p / parts);
-                const int32_t b = (int32_t)((int64_t)t.steps * (p + 1) / parts);
-                const int32_t c = cost_of(t, a, b);
-                units.push_back({t.request, t.q_row0, t.num_rows, t.q_head, a, b, slots + p, c});
-                key_steps += c;
+                u.kv_begin = (int32_t)((int64_t)t.steps * p / parts);
+                u.kv_end = (int32_t)((int64_t)t.steps * (p + 1) / parts);
+                u.split_slot = slots + p;
+                u.cost = cost_of(t, u.kv_begin, u.kv_end);
+                units.push_back(u);
+                key_steps += u.cost;
                 ++n_split_units;
             }
             slots += parts;
@@ -238,7 +259,7 @@ int wpp_plan_tiles(const wpp_ctx* ctx, const wpp_batch_desc* desc, const int32_t
     hd.total_new_tokens = T;
     hd.key_steps = key_steps;
     hd.flops = 4 * (int64_t)d.head_dim * Hq * pairs;
-    hd.workspace_bytes = slots ? align_up((size_t)slots * TM * (d.head_dim + 1) * sizeof(float), 256) : 0;
+    hd.workspace_bytes = slots ? align_up((size_t)slots * 2 * WPP_HALF_M * (d.head_dim + 1) * sizeof(float), 256) : 0;
     size_t off = sizeof(WppPlanHeader);
     hd.off_q_offsets = (uint32_t)off;
     off += align_up(sizeof(int32_t) * (size_t)(R + 1), 16);

@@ -4,7 +4,7 @@
 #include <stdint.h>
 
 #define WPP_PLAN_MAGIC 0x31505057u /* "WPP1" */
-#define WPP_PLAN_VERSION 2u
+#define WPP_PLAN_VERSION 3u
 #define WPP_TILE_N 128             /* keys per step */
 #define WPP_HALF_M 128             /* query rows per tensor-core tile (one TMEM lane per row) */
 
@@ -12,7 +12,7 @@ struct WppPlanHeader {
     uint32_t magic, version;
     uint64_t desc_hash;             // hash of the batch description + lengths the plan was made for
     int32_t num_requests, num_ctas, num_units, num_combine;
-    int32_t num_split_slots;        // partial-result slots of tile_m rows each in the workspace
+    int32_t num_split_slots;        // partial-result slots of 2 x 128 rows each in the workspace
     int32_t tile_m, tile_n, head_dim;
     int64_t total_new_tokens, key_steps, flops;
     uint64_t workspace_bytes, plan_bytes;
@@ -23,20 +23,26 @@ struct WppPlanHeader {
     uint32_t pad[8];
 };
 
-// One work tile: rows [q_row0, q_row0+num_rows) of request `request`'s chunk, one query head,
-// key steps [kv_begin, kv_end) of 128 keys each (absolute key index = step*128 + column).
+// One work tile = two 128-row "halves" that share one K/V stream (same request, same KV head).  Each half
+// is rows [row0, row0+rows) of the request's chunk for one query head; rows == 0 marks an unused half.
+// Usually the halves are consecutive row blocks of one head; a short chunk tail pairs two heads of one
+// KV group instead.  The tile covers key steps [kv_begin, kv_end) of 128 keys (absolute key = step*128 +
+// column); each half additionally stops at its own causal end.
 struct WppUnit {
-    int32_t request, q_row0, num_rows, q_head;
-    int32_t kv_begin, kv_end;
+    int32_t request, kv_begin, kv_end;
     int32_t split_slot;             // -1: writes the final output; else partial slot in the workspace
-    int32_t cost;                   // 128x128 steps (both halves), what the CTA assignment balanced
+    int32_t row0[2], rows[2], head[2];
+    int32_t cost;                   // 128x128 steps over both halves, what the CTA assignment balanced
+    int32_t pad;
 };
 
+// One half tile whose key range was split: partial slots [slot0, slot0+num_splits) merged in increasing order.
 struct WppCombine {
-    int32_t request, q_row0, num_rows, q_head;
-    int32_t slot0, num_splits;      // partial slots [slot0, slot0+num_splits), merged in increasing order
-    int32_t pad0, pad1;
+    int32_t request, row0, rows, head;
+    int32_t slot0, num_splits;
+    int32_t half;                   // which half of the slot the rows live in
+    int32_t pad;
 };
 
-// Workspace layout: fp32 O_part[num_split_slots][tile_m][head_dim] followed by fp32 lse_part[num_split_slots][tile_m]
+// Workspace layout: fp32 O_part[num_split_slots][2][128][head_dim] followed by fp32 lse_part[num_split_slots][2][128]
 // (log2 units of the scaled scores; -inf marks a row with no visible key in that part).

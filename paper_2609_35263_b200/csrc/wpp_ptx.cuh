@@ -156,6 +156,16 @@ __host__ __device__ constexpr uint32_t idesc_bf16(uint32_t n, uint32_t a_mn_majo
            ((128u >> 4) << 24);
 }
 
+// Register reallocation between warpgroups (all four warps of a warpgroup execute it together).
+template <int N>
+__device__ __forceinline__ void setmaxnreg_inc() {
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N));
+}
+template <int N>
+__device__ __forceinline__ void setmaxnreg_dec() {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N));
+}
+
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
     uint32_t r;
     asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));

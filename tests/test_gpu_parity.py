@@ -26,9 +26,17 @@ def _full_parity(w, opts=None, inp=None, sm_scale=0.0):
     return res, e
 
 
-def test_cfg1_single_request():
-    res, e = _full_parity(W.cfg1())
+@pytest.mark.parametrize("tile_m", [0, 128, 256])
+def test_cfg1_single_request(tile_m):
+    res, e = _full_parity(W.cfg1(), opts=wpp.PlanOpts(tile_m, 0, 0, 0))
     print("cfg1", e)
+
+
+def test_odd_group_size_leaves_single_halves():
+    """Three query heads per KV head: short tails cannot be paired, so tiles with one unused half appear."""
+    w = W.custom_workload([40, 300], [70, 130], 3, 1, 128, 64, seed=18)
+    _full_parity(w, opts=wpp.PlanOpts(256, 0, 0, 0))
+    _full_parity(w, opts=wpp.PlanOpts(256, 0, 2, 0))
 
 
 @pytest.mark.parametrize("P,C,Hq,Hkv,d,B", [
@@ -41,9 +49,10 @@ def test_cfg1_single_request():
     ([1024], [512], 2, 1, 128, 128),
     ([100, 0], [0, 70], 2, 1, 64, 16),           # an empty chunk in the wave
 ])
-def test_ragged_small(P, C, Hq, Hkv, d, B):
+@pytest.mark.parametrize("tile_m", [128, 256])
+def test_ragged_small(P, C, Hq, Hkv, d, B, tile_m):
     w = W.custom_workload(P, C, Hq, Hkv, d, B, seed=7, spare_pages=5)
-    _full_parity(w)
+    _full_parity(w, opts=wpp.PlanOpts(tile_m, 0, 0, 0))
 
 
 def test_single_key_is_bit_exact():
@@ -56,10 +65,11 @@ def test_single_key_is_bit_exact():
         assert torch.equal(out[0, h].view(torch.int16), v0[h // 2].view(torch.int16))
 
 
+@pytest.mark.parametrize("tile_m", [128, 256])
 @pytest.mark.parametrize("splits", [2, 3, 7])
-def test_forced_kv_splits_and_combine(splits):
+def test_forced_kv_splits_and_combine(splits, tile_m):
     w = W.custom_workload([900, 0, 130], [300, 500, 64], 4, 2, 128, 64, seed=9)
-    opts = wpp.PlanOpts(0, 0, splits, 0)
+    opts = wpp.PlanOpts(tile_m, 0, splits, 0)
     res, _ = _full_parity(w, opts=opts)
     assert res["plan"].info.num_combine_tiles > 0 and res["plan"].info.workspace_bytes > 0
 
@@ -78,8 +88,8 @@ def test_empty_wave_is_a_no_op():
 def test_results_are_bit_reproducible():
     w = W.custom_workload([500, 77], [260, 300], 8, 2, 128, 64, seed=12)
     inp = cpu_inputs(w)
-    a = H.run_wave(w, H.device_inputs(w, inp), opts=wpp.PlanOpts(0, 0, 3, 0))
-    b = H.run_wave(w, H.device_inputs(w, inp), opts=wpp.PlanOpts(0, 0, 3, 0))
+    a = H.run_wave(w, H.device_inputs(w, inp), opts=wpp.PlanOpts(256, 0, 3, 0))
+    b = H.run_wave(w, H.device_inputs(w, inp), opts=wpp.PlanOpts(256, 0, 3, 0))
     assert torch.equal(a["out"].view(torch.int16), b["out"].view(torch.int16))
     assert torch.equal(a["lse"], b["lse"])
 
