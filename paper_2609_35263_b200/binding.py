@@ -14,7 +14,7 @@ import numpy as np
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libwpp.so")
+LIB_PATH = os.environ.get("WPP_LIB_PATH") or os.path.join(_HERE, "libwpp.so")   # override: a differently built library
 
 WPP_OK = 0
 WPP_BF16 = 1

@@ -7,10 +7,12 @@
 //   warps 4-7   softmax of half B
 //   warps 8-11  correction: rescales the O accumulators in TMEM when a running maximum moved, and runs the
 //               epilogue (O / l -> bf16 -> global, or fp32 partials for split tiles)
-//   warp 12     tensor-core issuer: S = Q K^T and O += P V with tcgen05.mma (fp32 accumulators in TMEM; P is
-//               read from TMEM where the softmax warps wrote it as packed bf16 over S; V is an MN-major operand)
+//   warp 12     tensor-core issuer (one thread): S = Q K^T and O += P V with tcgen05.mma (fp32 accumulators in
+//               TMEM; P is read from TMEM where the softmax warps wrote it as packed bf16 over S; V is an MN-major
+//               operand).  It alternates A and B, which keeps the two halves in anti-phase.
 //   warp 13     producer: reads the block table and issues TMA tile loads (Q once per tile; per key step one box
-//               per (page, 64-wide half of head_dim) for K and for V, 128-byte swizzle, 4-deep ring)
+//               per (page, 64-wide half of head_dim) for K and for V, 128-byte swizzle).  V(j) and K(j+1) are used
+//               in the same issuer iteration, so they travel as one ring item with one barrier.
 // The two halves ping-pong: while the softmax warps of A work on S_A(j+1), the tensor cores run O_B += P_B V(j)
 // and S_B(j+1).  Rescaling is lazy: the reference maximum of a row only moves when the new maximum exceeds it by
 // more than 2^8, so the correction warps rarely touch O after the first steps.
@@ -34,21 +36,40 @@ constexpr uint32_t kTmemCols = 512;
 __host__ __device__ constexpr uint32_t col_s(int hf) { return 128u * hf; }          // S (and P) of half hf
 __host__ __device__ constexpr uint32_t col_o(int hf) { return 256u + 128u * hf; }   // O of half hf
 constexpr float kRescaleThreshold = 8.0f;     // log2 units
+#ifndef WPP_EMU_PAIRS_OF_4
+#define WPP_EMU_PAIRS_OF_4 0
+#endif
+constexpr int kEmuPairsOf4 = WPP_EMU_PAIRS_OF_4;  // of every 4 score pairs, how many take exp2 on the FMA pipes
 
 template <int D>
 struct Cfg {
     static constexpr int kHalves = D / 64;                 // 64-element (128-byte) swizzled column blocks
     static constexpr int kTileBytes = 128 * D * 2;         // one 128-row Q half, or one K or V step
     static constexpr int kHalfBytes = 128 * 128;           // 128 rows x 128 bytes
-    static constexpr int kStages = 4;                      // K/V ring (K(j), V(j), K(j+1), V(j+1))
+    static constexpr int kItems = (D == 128) ? 2 : 4;      // ring of items {V(j), K(j+1)}
+    static constexpr int kItemBytes = 2 * kTileBytes;      // V part, then K part
     static constexpr int kOffKV = 2 * kTileBytes;
-    static constexpr int kOffBars = kOffKV + kStages * kTileBytes;
-    static constexpr int kNumBars = 2 + 2 * kStages + 6 * 2;
+    static constexpr int kOffBars = kOffKV + kItems * kItemBytes;
+    static constexpr int kNumBars = 2 + 2 * kItems + 5 * 2;
     static constexpr int kOffScale = kOffBars + 8 * kNumBars;          // float alpha[2][128]
     static constexpr int kOffFinal = kOffScale + 2 * 128 * 4;          // float2 (m, l)[2][128]
     static constexpr int kOffMisc = kOffFinal + 2 * 128 * 8;           // tmem ptr, abort flag
     static constexpr int kSmemBytes = kOffMisc + 16 + 1024;            // + alignment slack
 };
+
+// Optional timeline instrumentation for tuning (compiled out unless WPP_TRACE is defined): CTA 0 records the
+// low 32 bits of clock64 at a few points of its first key steps into p.trace[role][step][event].
+#ifdef WPP_TRACE
+#define WPP_TRACE_EVENTS 8
+#define WPP_TRACE_STEPS 64
+#define TRACE(role, step, ev)                                                                              \
+    do {                                                                                                   \
+        if (p.trace && blockIdx.x == 0 && (threadIdx.x & 63) == 0 && (step) < WPP_TRACE_STEPS)            \
+            p.trace[((role) * WPP_TRACE_STEPS + (step)) * WPP_TRACE_EVENTS + (ev)] = (uint32_t)clock64(); \
+    } while (0)
+#else
+#define TRACE(role, step, ev) do { } while (0)
+#endif
 
 struct Ring {
     uint32_t stage, phase;
@@ -88,20 +109,21 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
     const uint32_t sQ = smem_base;                       // two halves, kTileBytes each
-    const uint32_t sKV = smem_base + C::kOffKV;
+    const uint32_t sKV = smem_base + C::kOffKV;          // kItems x {V tile, K tile}
     const uint32_t bars = smem_base + C::kOffBars;
     const uint32_t bQFull = bars, bQEmpty = bars + 8;
-    const uint32_t bKVFull = bars + 16, bKVEmpty = bKVFull + 8 * C::kStages;
-    // per half: s_full, p_full, o_full, corr_ready, corr_done, final_ready.  A thread never arrives twice on one
-    // barrier without a wait in between that implies the earlier phase completed; that is why the end-of-tile
-    // hand-over of (m, l) has a barrier of its own instead of reusing corr_ready.
-    const uint32_t bHalf = bKVEmpty + 8 * C::kStages;
-    auto bSFull = [&](int h) { return bHalf + 48 * h; };
-    auto bPFull = [&](int h) { return bHalf + 48 * h + 8; };
-    auto bOFull = [&](int h) { return bHalf + 48 * h + 16; };
-    auto bCorrReady = [&](int h) { return bHalf + 48 * h + 24; };
-    auto bCorrDone = [&](int h) { return bHalf + 48 * h + 32; };
-    auto bFinalReady = [&](int h) { return bHalf + 48 * h + 40; };
+    const uint32_t bItemFull = bars + 16, bItemEmpty = bItemFull + 8 * C::kItems;
+    // Per half: s_full (S = Q K^T landed; it also proves the previous O += P V landed, the tensor pipe being in
+    // order), p_ready (P written by 128 softmax threads + O fixed up by 128 correction threads), corr_ready
+    // (rescale factors are in smem), final_ready (end-of-tile (m, l) are in smem), o_final (last O += P V landed).
+    // A thread never arrives twice on one barrier without a wait in between that implies the earlier phase
+    // completed; that is why the end-of-tile hand-over has a barrier of its own instead of reusing corr_ready.
+    const uint32_t bHalf = bItemEmpty + 8 * C::kItems;
+    auto bSFull = [&](int h) { return bHalf + 40 * h; };
+    auto bPReady = [&](int h) { return bHalf + 40 * h + 8; };
+    auto bCorrReady = [&](int h) { return bHalf + 40 * h + 16; };
+    auto bFinalReady = [&](int h) { return bHalf + 40 * h + 24; };
+    auto bOFinal = [&](int h) { return bHalf + 40 * h + 32; };
     float* s_alpha = reinterpret_cast<float*>(smem_gen + C::kOffScale);       // [2][128]
     float2* s_final = reinterpret_cast<float2*>(smem_gen + C::kOffFinal);     // [2][128] (m_ref, l)
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_gen + C::kOffMisc);
@@ -112,10 +134,10 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
 
     if (threadIdx.x == 0) {
         mbar_init(bQFull, 1); mbar_init(bQEmpty, 1);
-        for (int s = 0; s < C::kStages; ++s) { mbar_init(bKVFull + 8 * s, 1); mbar_init(bKVEmpty + 8 * s, 1); }
+        for (int s = 0; s < C::kItems; ++s) { mbar_init(bItemFull + 8 * s, 1); mbar_init(bItemEmpty + 8 * s, 1); }
         for (int h = 0; h < 2; ++h) {
-            mbar_init(bSFull(h), 1); mbar_init(bPFull(h), 128); mbar_init(bOFull(h), 1);
-            mbar_init(bCorrReady(h), 128); mbar_init(bCorrDone(h), 128); mbar_init(bFinalReady(h), 128);
+            mbar_init(bSFull(h), 1); mbar_init(bPReady(h), 256); mbar_init(bCorrReady(h), 128);
+            mbar_init(bFinalReady(h), 128); mbar_init(bOFinal(h), 1);
         }
         *abort_flag = 0u;
         fence_barrier_init();
@@ -141,7 +163,7 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     const int B = p.page_size, ppt = 128 / B;   // pages per key step
 
     if (wg == 3) {
-        setmaxnreg_dec<56>();
+        setmaxnreg_dec<80>();
         if (warp == 13) {
             // ================================================================ producer
             Ring ring = {0, 0};
@@ -154,38 +176,42 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 const int n_pages = (v.kv_len + B - 1) / B;
                 const int kvh = un.head[0] / p.group;
                 const int32_t* bt = p.block_tables + (int64_t)un.request * p.max_blocks;
-                // K(j) then V(j) into consecutive ring slots; lane l moves page (j*ppt + l) of the step
-                auto load_step = [&](int j) -> bool {
-                    const int page0 = (v.kv_begin + j) * ppt;
-                    const int cnt = min(ppt, n_pages - page0);
-                    int pid = 0;
-                    if (lane < cnt) {
-                        pid = bt[page0 + lane];
-                        if (pid < 0 || pid >= p.num_pages) {
-                            if (p.status) atomicCAS(p.status, 0, WPP_ERR_BOUNDS);
-                            pid = 0;
-                        }
+                // one ring item: V of step jv (if jv >= 0) and K of step jk (if jk < n_steps); lane l moves
+                // page l of each step
+                auto load_item = [&](int jv, int jk) -> bool {
+                    const bool has_v = jv >= 0, has_k = jk < v.n_steps;
+                    const int page_v = (v.kv_begin + jv) * ppt, page_k = (v.kv_begin + jk) * ppt;
+                    const int cnt_v = has_v ? min(ppt, n_pages - page_v) : 0;
+                    const int cnt_k = has_k ? min(ppt, n_pages - page_k) : 0;
+                    int pid_v = 0, pid_k = 0;
+                    if (lane < cnt_v) pid_v = bt[page_v + lane];
+                    if (lane < cnt_k) pid_k = bt[page_k + lane];
+                    if (pid_v < 0 || pid_v >= p.num_pages || pid_k < 0 || pid_k >= p.num_pages) {
+                        if (p.status) atomicCAS(p.status, 0, WPP_ERR_BOUNDS);
+                        pid_v = (pid_v < 0 || pid_v >= p.num_pages) ? 0 : pid_v;
+                        pid_k = (pid_k < 0 || pid_k >= p.num_pages) ? 0 : pid_k;
                     }
-                    const uint32_t bytes = (uint32_t)cnt * B * D * 2;
+                    const bool ok = mbar_wait(bItemEmpty + 8 * ring.stage, ring.phase ^ 1u, abort_flag);
+                    if (!__all_sync(0xffffffffu, ok)) return false;
+                    const uint32_t full = bItemFull + 8 * ring.stage;
+                    if (lane == 0) mbar_arrive_expect_tx(full, (uint32_t)(cnt_v + cnt_k) * B * D * 2);
+                    __syncwarp();
+                    const uint32_t dst = sKV + ring.stage * C::kItemBytes + lane * B * 128;
+                    if (lane < cnt_v) {
 #pragma unroll
-                    for (int kv = 0; kv < 2; ++kv) {
-                        const bool ok = mbar_wait(bKVEmpty + 8 * ring.stage, ring.phase ^ 1u, abort_flag);
-                        if (!__all_sync(0xffffffffu, ok)) return false;
-                        const uint32_t full = bKVFull + 8 * ring.stage;
-                        if (lane == 0) mbar_arrive_expect_tx(full, bytes);
-                        __syncwarp();
-                        if (lane < cnt) {
-                            const uint32_t dst = sKV + ring.stage * C::kTileBytes + lane * B * 128;
-#pragma unroll
-                            for (int h = 0; h < C::kHalves; ++h)
-                                tma_load_4d(dst + h * C::kHalfBytes, kv == 0 ? &tm_k : &tm_v, full, h * 64, 0, kvh, pid);
-                        }
-                        ring.advance(C::kStages);
+                        for (int h = 0; h < C::kHalves; ++h)
+                            tma_load_4d(dst + h * C::kHalfBytes, &tm_v, full, h * 64, 0, kvh, pid_v);
                     }
+                    if (lane < cnt_k) {
+#pragma unroll
+                        for (int h = 0; h < C::kHalves; ++h)
+                            tma_load_4d(dst + C::kTileBytes + h * C::kHalfBytes, &tm_k, full, h * 64, 0, kvh, pid_k);
+                    }
+                    ring.advance(C::kItems);
                     return true;
                 };
-                // the first step's K/V only needs ring slots, which free up before the previous tile's Q does
-                if (!load_step(0)) { dead = true; break; }
+                // K(0) only needs a ring slot, which frees up before the previous tile's Q does
+                if (!load_item(-1, 0)) { dead = true; break; }
                 const bool ok = mbar_wait(bQEmpty, q_phase ^ 1u, abort_flag);
                 if (!__all_sync(0xffffffffu, ok)) { dead = true; break; }
                 q_phase ^= 1u;
@@ -202,111 +228,93 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     }
                 }
                 __syncwarp();
-                for (int j = 1; j < v.n_steps; ++j)
-                    if (!load_step(j)) { dead = true; break; }
+                for (int j = 0; j < v.n_steps; ++j)
+                    if (!load_item(j, j + 1)) { dead = true; break; }
             }
-        } else if (warp == 12) {
-            // ================================================================ tensor-core issuer
+        } else if (warp == 12 && lane == 0) {
+            // ================================================================ tensor-core issuer (one thread)
+            // It alternates the halves (A: O += P V, next S; then B), which keeps their softmax phases apart:
+            // while the softmax warps of A own the special-function units, the tensor pipe works for B.  (Two
+            // independent issuers were measured: the halves then drift into phase, both softmaxes share the
+            // exp units and the dependency chain of each half gets longer.)
             Ring ring = {0, 0};
-            uint32_t q_phase = 0, p_phase[2] = {0, 0}, c_phase[2] = {0, 0};
+            uint32_t q_phase = 0, p_phase[2] = {0, 0};
+            int tstep = 0;
+            (void)tstep;
             constexpr uint32_t idesc_qk = idesc_bf16(128, 0, 0);
             constexpr uint32_t idesc_pv = idesc_bf16(D, 0, 1);
+            const uint64_t k_desc0 = smem_desc_sw128(sKV + C::kTileBytes, 16, 1024);   // + item * (kItemBytes >> 4)
+            const uint64_t v_desc0 = smem_desc_sw128(sKV, C::kHalfBytes, 1024);
             bool dead = false;
-            auto issue_qk = [&](int hf, uint32_t kb) {
-                if (lane == 0) {
-                    const uint32_t qb = sQ + hf * C::kTileBytes;
+            auto issue_qk = [&](int hf, uint32_t item) {     // S = Q K^T over head_dim in chunks of 16
+                const uint64_t qd = smem_desc_sw128(sQ + hf * C::kTileBytes, 16, 1024);
+                const uint64_t kd = k_desc0 + (uint64_t)(item * (C::kItemBytes >> 4));
+                const uint32_t tS = tmem + col_s(hf);
 #pragma unroll
-                    for (int kk = 0; kk < D / 16; ++kk) {
-                        const uint32_t off = (kk >> 2) * C::kHalfBytes + (kk & 3) * 32;
-                        mma_ss(tmem + col_s(hf), smem_desc_sw128(qb + off, 16, 1024), smem_desc_sw128(kb + off, 16, 1024),
-                               idesc_qk, kk > 0);
-                    }
-                    mma_commit(bSFull(hf));
+                for (int kk = 0; kk < D / 16; ++kk) {
+                    const uint64_t off = (uint64_t)(((kk >> 2) * C::kHalfBytes + (kk & 3) * 32) >> 4);
+                    if (kk == 0) mma_ss_overwrite(tS, qd + off, kd + off, idesc_qk);
+                    else mma_ss_accumulate(tS, qd + off, kd + off, idesc_qk);
                 }
-                __syncwarp();
+                mma_commit(bSFull(hf));
             };
             for (int u = u_begin; u < u_end && !dead; ++u) {
                 const WppUnit un = units[u];
                 const UnitView v = view_of(un, p, q_offsets);
                 if (v.n_steps == 0) continue;
-                // K(0)
-                bool ok = mbar_wait(bKVFull + 8 * ring.stage, ring.phase, abort_flag);
-                if (!__all_sync(0xffffffffu, ok)) { dead = true; break; }
-                ok = mbar_wait(bQFull, q_phase, abort_flag);
-                if (!__all_sync(0xffffffffu, ok)) { dead = true; break; }
+                // K(0), Q
+                if (!mbar_wait(bItemFull + 8 * ring.stage, ring.phase, abort_flag)) break;
+                if (!mbar_wait(bQFull, q_phase, abort_flag)) break;
                 q_phase ^= 1u;
                 tc_fence_after();
-                uint32_t k_stage = ring.stage;
-                ring.advance(C::kStages);
-                if (v.n[0] > 0) issue_qk(0, sKV + k_stage * C::kTileBytes);
-                if (v.n[1] > 0) issue_qk(1, sKV + k_stage * C::kTileBytes);
-                if (lane == 0) {
-                    mma_commit(bKVEmpty + 8 * k_stage);
-                    if (v.n_steps == 1) mma_commit(bQEmpty);
-                }
-                __syncwarp();
+                if (v.n[0] > 0) issue_qk(0, ring.stage);
+                if (v.n[1] > 0) issue_qk(1, ring.stage);
+                mma_commit(bItemEmpty + 8 * ring.stage);
+                if (v.n_steps == 1) mma_commit(bQEmpty);
+                ring.advance(C::kItems);
                 for (int j = 0; j < v.n_steps; ++j) {
-                    // V(j)
-                    ok = mbar_wait(bKVFull + 8 * ring.stage, ring.phase, abort_flag);
-                    if (!__all_sync(0xffffffffu, ok)) { dead = true; break; }
-                    const uint32_t v_stage = ring.stage;
-                    ring.advance(C::kStages);
-                    const uint32_t vb = sKV + v_stage * C::kTileBytes;
+                    // item {V(j), K(j+1)}
+                    if (!mbar_wait(bItemFull + 8 * ring.stage, ring.phase, abort_flag)) { dead = true; break; }
+                    const uint32_t item = ring.stage;
                     const int valid = v.kv_len - (v.kv_begin + j) * 128;      // keys of this step that exist
                     if (valid < 128) {
                         // rows past the end of the sequence may hold anything (stale slots, never-loaded pages):
                         // zero them so that 0 * garbage cannot reach O
-                        uint8_t* vg = smem_gen + (vb - smem_base);
-                        const int rows = 128 - valid;
-                        for (int i = lane; i < rows * 8 * C::kHalves; i += 32) {
-                            const int h = i / (rows * 8), rem = i % (rows * 8);
-                            *reinterpret_cast<uint4*>(vg + h * C::kHalfBytes + (valid + rem / 8) * 128 + (rem % 8) * 16) =
-                                make_uint4(0, 0, 0, 0);
-                        }
+                        uint8_t* vg = smem_gen + C::kOffKV + item * C::kItemBytes;
+                        for (int h = 0; h < C::kHalves; ++h)
+                            for (int i = valid * 8; i < 128 * 8; ++i)
+                                *reinterpret_cast<uint4*>(vg + h * C::kHalfBytes + i * 16) = make_uint4(0, 0, 0, 0);
                         fence_proxy_async_smem();
-                        __syncwarp();
                     }
-                    // K(j+1)
-                    const bool more = j + 1 < v.n_steps;
-                    if (more) {
-                        ok = mbar_wait(bKVFull + 8 * ring.stage, ring.phase, abort_flag);
-                        if (!__all_sync(0xffffffffu, ok)) { dead = true; break; }
-                        k_stage = ring.stage;
-                        ring.advance(C::kStages);
-                    }
+                    const uint64_t vd = v_desc0 + (uint64_t)(item * (C::kItemBytes >> 4));
 #pragma unroll
                     for (int hf = 0; hf < 2; ++hf) {
                         if (j >= v.n[hf]) continue;
-                        ok = mbar_wait(bPFull(hf), p_phase[hf], abort_flag);
-                        if (!__all_sync(0xffffffffu, ok)) { dead = true; break; }
+                        TRACE(2, tstep, hf * 4 + 0);
+                        if (!mbar_wait(bPReady(hf), p_phase[hf], abort_flag)) { dead = true; break; }   // P written, O fixed
                         p_phase[hf] ^= 1u;
-                        ok = mbar_wait(bCorrDone(hf), c_phase[hf], abort_flag);
-                        if (!__all_sync(0xffffffffu, ok)) { dead = true; break; }
-                        c_phase[hf] ^= 1u;
+                        TRACE(2, tstep, hf * 4 + 1);
                         tc_fence_after();
-                        if (lane == 0) {
+                        const uint32_t tS = tmem + col_s(hf), tO = tmem + col_o(hf);
+                        if (j > 0) mma_ts_accumulate(tO, tS, vd, idesc_pv); else mma_ts_overwrite(tO, tS, vd, idesc_pv);
 #pragma unroll
-                            for (int kk = 0; kk < 8; ++kk)
-                                mma_ts(tmem + col_o(hf), tmem + col_s(hf) + kk * 8,
-                                       smem_desc_sw128(vb + kk * 2048, C::kHalfBytes, 1024), idesc_pv, (j > 0) || (kk > 0));
-                            mma_commit(bOFull(hf));
-                        }
-                        __syncwarp();
-                        if (j + 1 < v.n[hf]) issue_qk(hf, sKV + k_stage * C::kTileBytes);
+                        for (int kk = 1; kk < 8; ++kk) mma_ts_accumulate(tO, tS + kk * 8, vd + (uint64_t)(kk * 128), idesc_pv);
+                        TRACE(2, tstep, hf * 4 + 2);
+                        if (j + 1 < v.n[hf]) issue_qk(hf, item);      // its commit also covers the O += P V above
+                        else mma_commit(bOFinal(hf));
+                        TRACE(2, tstep, hf * 4 + 3);
                     }
                     if (dead) break;
-                    if (lane == 0) {
-                        mma_commit(bKVEmpty + 8 * v_stage);
-                        if (more) mma_commit(bKVEmpty + 8 * k_stage);
-                        if (j + 2 == v.n_steps) mma_commit(bQEmpty);   // the last S of this tile has been issued
-                    }
-                    __syncwarp();
+                    mma_commit(bItemEmpty + 8 * item);
+                    if (j + 2 == v.n_steps) mma_commit(bQEmpty);       // the last S of this tile has been issued
+                    ring.advance(C::kItems);
+                    ++tstep;
                 }
             }
         }
     } else if (wg == 2) {
         // ================================================================ correction + epilogue
-        setmaxnreg_dec<88>();
+        setmaxnreg_dec<96>();
         const int r = threadIdx.x & 127;
         const uint32_t lane_addr = tmem + ((uint32_t)((warp & 3) * 32) << 16);
         uint32_t cr_phase[2] = {0, 0}, o_phase[2] = {0, 0}, f_phase[2] = {0, 0};
@@ -318,30 +326,27 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
 #pragma unroll
                 for (int hf = 0; hf < 2; ++hf) {
                     if (j >= v.n[hf]) continue;
-                    bool ok = mbar_wait(bCorrReady(hf), cr_phase[hf], abort_flag);
+                    // the softmax threads signal after they saw S(j), which the tensor pipe finished after the
+                    // O += P V of step j-1: O is safe to touch
+                    const bool ok = mbar_wait(bCorrReady(hf), cr_phase[hf], abort_flag);
                     if (!__all_sync(0xffffffffu, ok)) { dead = true; break; }
                     cr_phase[hf] ^= 1u;
                     const float alpha = s_alpha[hf * 128 + r];
-                    if (j > 0) {
-                        ok = mbar_wait(bOFull(hf), o_phase[hf], abort_flag);     // O += P V of step j-1 has landed
-                        if (!__all_sync(0xffffffffu, ok)) { dead = true; break; }
-                        o_phase[hf] ^= 1u;
-                        if (__any_sync(0xffffffffu, alpha != 1.f)) {
-                            tc_fence_after();
+                    if (__any_sync(0xffffffffu, alpha != 1.f)) {
+                        tc_fence_after();
 #pragma unroll
-                            for (int q4 = 0; q4 < D / 32; ++q4) {
-                                float o[32];
-                                tmem_ld32(lane_addr + col_o(hf) + q4 * 32, reinterpret_cast<uint32_t*>(o));
-                                tmem_wait_ld();
+                        for (int q4 = 0; q4 < D / 32; ++q4) {
+                            float o[32];
+                            tmem_ld32(lane_addr + col_o(hf) + q4 * 32, reinterpret_cast<uint32_t*>(o));
+                            tmem_wait_ld();
 #pragma unroll
-                                for (int i = 0; i < 32; ++i) o[i] *= alpha;
-                                tmem_st32(lane_addr + col_o(hf) + q4 * 32, reinterpret_cast<uint32_t*>(o));
-                            }
-                            tmem_wait_st();
-                            tc_fence_before();
+                            for (int i = 0; i < 32; ++i) o[i] *= alpha;
+                            tmem_st32(lane_addr + col_o(hf) + q4 * 32, reinterpret_cast<uint32_t*>(o));
                         }
+                        tmem_wait_st();
+                        tc_fence_before();
                     }
-                    mbar_arrive(bCorrDone(hf));
+                    mbar_arrive(bPReady(hf));
                 }
             }
             if (dead) break;
@@ -360,7 +365,7 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 bool ok = mbar_wait(bFinalReady(hf), f_phase[hf], abort_flag);      // final (m, l) are in smem
                 if (!__all_sync(0xffffffffu, ok)) { dead = true; break; }
                 f_phase[hf] ^= 1u;
-                ok = mbar_wait(bOFull(hf), o_phase[hf], abort_flag);                // last O += P V has landed
+                ok = mbar_wait(bOFinal(hf), o_phase[hf], abort_flag);               // last O += P V has landed
                 if (!__all_sync(0xffffffffu, ok)) { dead = true; break; }
                 o_phase[hf] ^= 1u;
                 tc_fence_after();
@@ -409,13 +414,16 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         }
     } else {
         // ================================================================ softmax (thread = query row of half `hf`)
-        setmaxnreg_inc<184>();
+        setmaxnreg_inc<168>();
         const int hf = wg;
         const int r = threadIdx.x & 127;
         const uint32_t lane_addr = tmem + ((uint32_t)((warp & 3) * 32) << 16);
         const uint32_t colS = col_s(hf);
         uint32_t s_phase = 0;
+        int tstep = 0;      // steps since kernel start (trace index only)
+        (void)tstep;
         const float c = p.scale_log2;
+        const uint64_t c2 = pack2(c, c);
         bool dead = false;
         for (int u = u_begin; u < u_end && !dead; ++u) {
             const WppUnit un = units[u];
@@ -425,31 +433,44 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             const int first_pos = v.P + un.row0[hf];          // last key visible to row 0 of this half
             float m_ref = -INFINITY, l_run = 0.f;
             for (int j = 0; j < n; ++j) {
+                TRACE(hf, tstep, 0);
                 const bool ok = mbar_wait(bSFull(hf), s_phase, abort_flag);
                 if (!__all_sync(0xffffffffu, ok)) { dead = true; break; }
                 s_phase ^= 1u;
                 tc_fence_after();
+                TRACE(hf, tstep, 1);
+#ifdef WPP_EXPERIMENT_NO_SOFTMAX
+                // tuning experiment: how fast is the tile loop when the softmax costs nothing (results are garbage)
+                s_alpha[hf * 128 + r] = 1.f;
+                mbar_arrive(bCorrReady(hf));
+                tc_fence_before();
+                mbar_arrive(bPReady(hf));
+                continue;
+#endif
                 float s[128];
 #pragma unroll
                 for (int q4 = 0; q4 < 4; ++q4) tmem_ld32(lane_addr + colS + q4 * 32, reinterpret_cast<uint32_t*>(s) + q4 * 32);
                 tmem_wait_ld();
+                TRACE(hf, tstep, 2);
                 const int key0 = (v.kv_begin + j) * 128;
                 if (key0 + 127 > first_pos) {               // only steps that touch the diagonal are masked
                     const int limit = first_pos + r - key0;
 #pragma unroll
                     for (int i = 0; i < 128; ++i) s[i] = (i > limit) ? -INFINITY : s[i];
                 }
-                float mx0 = fmaxf(s[0], s[1]), mx1 = fmaxf(s[2], s[3]);
+                float mx[8];
 #pragma unroll
-                for (int i = 4; i < 128; i += 4) {
-                    mx0 = fmaxf(mx0, fmaxf(s[i], s[i + 1]));
-                    mx1 = fmaxf(mx1, fmaxf(s[i + 2], s[i + 3]));
+                for (int k = 0; k < 8; ++k) mx[k] = fmaxf(s[2 * k], s[2 * k + 1]);
+#pragma unroll
+                for (int i = 16; i < 128; i += 16) {
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) mx[k] = fmax3(mx[k], s[i + 2 * k], s[i + 2 * k + 1]);
                 }
-                const float mx = fmaxf(mx0, mx1);
+                const float mxx = fmaxf(fmax3(mx[0], mx[1], mx[2]), fmaxf(fmax3(mx[3], mx[4], mx[5]), fmaxf(mx[6], mx[7])));
                 // lazy rescale: keep the old reference unless the new maximum is far above it
                 float alpha = 1.f;
-                if ((mx - m_ref) * c > kRescaleThreshold || m_ref == -INFINITY) {
-                    const float m_new = fmaxf(m_ref, mx);
+                if ((mxx - m_ref) * c > kRescaleThreshold || m_ref == -INFINITY) {
+                    const float m_new = fmaxf(m_ref, mxx);
                     const float m_safe = (m_new == -INFINITY) ? 0.f : m_new;
                     alpha = fast_exp2((m_ref - m_safe) * c);        // 0 when there was no reference yet
                     m_ref = m_new;
@@ -457,23 +478,45 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 }
                 s_alpha[hf * 128 + r] = (j == 0) ? 1.f : alpha;
                 mbar_arrive(bCorrReady(hf));
+                TRACE(hf, tstep, 3);
                 const float neg_mc = (m_ref == -INFINITY) ? 0.f : -m_ref * c;
-                float sum0 = 0.f, sum1 = 0.f;
-                uint32_t pk[64];
+                const uint64_t nm2 = pack2(neg_mc, neg_mc);
+                // exp, row sum and bf16 packing in two halves of 64 scores; the first half of P is on its way to
+                // TMEM while the second half is computed.  P word w (scores 2w, 2w+1) overwrites S column w, which
+                // was read before.
+                uint64_t sum2a = pack2(0.f, 0.f), sum2b = pack2(0.f, 0.f);
 #pragma unroll
-                for (int i = 0; i < 64; ++i) {
-                    const float a = fast_exp2(fmaf(s[2 * i], c, neg_mc));
-                    const float b = fast_exp2(fmaf(s[2 * i + 1], c, neg_mc));
-                    sum0 += a;
-                    sum1 += b;
-                    pk[i] = pack_bf16x2(a, b);
+                for (int half = 0; half < 2; ++half) {
+                    uint32_t pk[32];
+#pragma unroll
+                    for (int w = 0; w < 32; ++w) {
+                        const int i = half * 32 + w;
+                        const uint64_t x2 = ffma2(pack2(s[2 * i], s[2 * i + 1]), c2, nm2);
+                        float e0, e1;
+                        if ((i & 3) < kEmuPairsOf4) {
+                            exp2_poly2(x2, e0, e1);
+                        } else {
+                            float x0, x1;
+                            unpack2(x2, x0, x1);
+                            e0 = fast_exp2(x0);
+                            e1 = fast_exp2(x1);
+                        }
+                        if (w & 1) sum2b = fadd2(sum2b, pack2(e0, e1)); else sum2a = fadd2(sum2a, pack2(e0, e1));
+                        pk[w] = pack_bf16x2(e0, e1);
+                    }
+                    tmem_st32(lane_addr + colS + half * 32, pk);
                 }
-                l_run += sum0 + sum1;
-                tmem_st32(lane_addr + colS, pk);
-                tmem_st32(lane_addr + colS + 32, pk + 32);
+                TRACE(hf, tstep, 4);
                 tmem_wait_st();
                 tc_fence_before();
-                mbar_arrive(bPFull(hf));
+                mbar_arrive(bPReady(hf));
+                TRACE(hf, tstep, 5);
+                {
+                    float t0, t1;
+                    unpack2(fadd2(sum2a, sum2b), t0, t1);
+                    l_run += t0 + t1;
+                }
+                ++tstep;
             }
             if (dead) break;
             s_final[hf * 128 + r] = make_float2(m_ref, l_run);

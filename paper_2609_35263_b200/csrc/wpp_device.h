@@ -21,6 +21,7 @@ struct AttnParams {
     int64_t o_token_stride, o_head_stride;
     int32_t num_q_heads, group, page_size, max_blocks, num_pages;
     float scale_log2;                // sm_scale * log2(e)
+    uint32_t* trace;                 // tuning builds only (WPP_TRACE): timeline buffer, else null
 };
 
 struct AppendParams {
