@@ -5,8 +5,7 @@
 // 16 warps, specialised by warpgroup:
 //   warps 0-3   softmax of half A: thread r owns query row r (TMEM lane r): row max / row sum need no shuffles
 //   warps 4-7   softmax of half B
-//   warps 8-11  correction: rescales the O accumulators in TMEM when a running maximum moved, and runs the
-//               epilogue (O / l -> bf16 -> global, or fp32 partials for split tiles)
+//   warps 8-11  epilogue: O / l -> bf16 -> global (or fp32 partials for split tiles), overlapping the next tile
 //   warp 12     tensor-core issuer (one thread): S = Q K^T and O += P V with tcgen05.mma (fp32 accumulators in
 //               TMEM; P is read from TMEM where the softmax warps wrote it as packed bf16 over S; V is an MN-major
 //               operand).  It alternates A and B, which keeps the two halves in anti-phase.
@@ -14,8 +13,9 @@
 //               per (page, 64-wide half of head_dim) for K and for V, 128-byte swizzle).  V(j) and K(j+1) are used
 //               in the same issuer iteration, so they travel as one ring item with one barrier.
 // The two halves ping-pong: while the softmax warps of A work on S_A(j+1), the tensor cores run O_B += P_B V(j)
-// and S_B(j+1).  Rescaling is lazy: the reference maximum of a row only moves when the new maximum exceeds it by
-// more than 2^8, so the correction warps rarely touch O after the first steps.
+// and S_B(j+1).  Rescaling is lazy: a row keeps its reference maximum, and does not even compute the maximum of
+// a step, as long as the step's row sum shows that no score rose far above the reference; only then (and on the
+// first step of a tile) the softmax warps take the true maximum and rescale O and l themselves.
 // Tensor memory (512 columns): S_A [0,128)  S_B [128,256)  O_A [256,256+D)  O_B [384,384+D); P aliases the first
 // 64 columns of its S.
 // All mbarrier waits are bounded; on expiry the CTA raises its abort flag, every role drains, TMEM is freed and
@@ -35,7 +35,7 @@ constexpr int kThreads = 512;
 constexpr uint32_t kTmemCols = 512;
 __host__ __device__ constexpr uint32_t col_s(int hf) { return 128u * hf; }          // S (and P) of half hf
 __host__ __device__ constexpr uint32_t col_o(int hf) { return 256u + 128u * hf; }   // O of half hf
-constexpr float kRescaleThreshold = 8.0f;     // log2 units
+constexpr float kFastPathSumLimit = 65536.f;  // row sum of p below which the old reference was safe to keep
 #ifndef WPP_EMU_PAIRS_OF_4
 #define WPP_EMU_PAIRS_OF_4 0
 #endif
@@ -50,9 +50,8 @@ struct Cfg {
     static constexpr int kItemBytes = 2 * kTileBytes;      // V part, then K part
     static constexpr int kOffKV = 2 * kTileBytes;
     static constexpr int kOffBars = kOffKV + kItems * kItemBytes;
-    static constexpr int kNumBars = 2 + 2 * kItems + 5 * 2;
-    static constexpr int kOffScale = kOffBars + 8 * kNumBars;          // float alpha[2][128]
-    static constexpr int kOffFinal = kOffScale + 2 * 128 * 4;          // float2 (m, l)[2][128]
+    static constexpr int kNumBars = 2 + 2 * kItems + 4 * 2;
+    static constexpr int kOffFinal = kOffBars + 8 * kNumBars;          // float2 (m, l)[2][128]
     static constexpr int kOffMisc = kOffFinal + 2 * 128 * 8;           // tmem ptr, abort flag
     static constexpr int kSmemBytes = kOffMisc + 16 + 1024;            // + alignment slack
 };
@@ -64,7 +63,7 @@ struct Cfg {
 #define WPP_TRACE_STEPS 64
 #define TRACE(role, step, ev)                                                                              \
     do {                                                                                                   \
-        if (p.trace && blockIdx.x == 0 && (threadIdx.x & 63) == 0 && (step) < WPP_TRACE_STEPS)            \
+        if (p.trace && blockIdx.x == 0 && (threadIdx.x & 127) == 0 && (step) < WPP_TRACE_STEPS)            \
             p.trace[((role) * WPP_TRACE_STEPS + (step)) * WPP_TRACE_EVENTS + (ev)] = (uint32_t)clock64(); \
     } while (0)
 #else
@@ -114,17 +113,14 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     const uint32_t bQFull = bars, bQEmpty = bars + 8;
     const uint32_t bItemFull = bars + 16, bItemEmpty = bItemFull + 8 * C::kItems;
     // Per half: s_full (S = Q K^T landed; it also proves the previous O += P V landed, the tensor pipe being in
-    // order), p_ready (P written by 128 softmax threads + O fixed up by 128 correction threads), corr_ready
-    // (rescale factors are in smem), final_ready (end-of-tile (m, l) are in smem), o_final (last O += P V landed).
-    // A thread never arrives twice on one barrier without a wait in between that implies the earlier phase
-    // completed; that is why the end-of-tile hand-over has a barrier of its own instead of reusing corr_ready.
+    // order), p_ready (P written, and O rescaled if the row reference moved, by the 128 softmax threads),
+    // final_ready (end-of-tile (m, l) are in smem), o_final (last O += P V landed).  A thread never arrives twice
+    // on one barrier without a wait in between that implies the earlier phase completed.
     const uint32_t bHalf = bItemEmpty + 8 * C::kItems;
-    auto bSFull = [&](int h) { return bHalf + 40 * h; };
-    auto bPReady = [&](int h) { return bHalf + 40 * h + 8; };
-    auto bCorrReady = [&](int h) { return bHalf + 40 * h + 16; };
-    auto bFinalReady = [&](int h) { return bHalf + 40 * h + 24; };
-    auto bOFinal = [&](int h) { return bHalf + 40 * h + 32; };
-    float* s_alpha = reinterpret_cast<float*>(smem_gen + C::kOffScale);       // [2][128]
+    auto bSFull = [&](int h) { return bHalf + 32 * h; };
+    auto bPReady = [&](int h) { return bHalf + 32 * h + 8; };
+    auto bFinalReady = [&](int h) { return bHalf + 32 * h + 16; };
+    auto bOFinal = [&](int h) { return bHalf + 32 * h + 24; };
     float2* s_final = reinterpret_cast<float2*>(smem_gen + C::kOffFinal);     // [2][128] (m_ref, l)
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_gen + C::kOffMisc);
     volatile uint32_t* abort_flag = tmem_slot + 1;
@@ -136,7 +132,7 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         mbar_init(bQFull, 1); mbar_init(bQEmpty, 1);
         for (int s = 0; s < C::kItems; ++s) { mbar_init(bItemFull + 8 * s, 1); mbar_init(bItemEmpty + 8 * s, 1); }
         for (int h = 0; h < 2; ++h) {
-            mbar_init(bSFull(h), 1); mbar_init(bPReady(h), 256); mbar_init(bCorrReady(h), 128);
+            mbar_init(bSFull(h), 1); mbar_init(bPReady(h), 128);
             mbar_init(bFinalReady(h), 128); mbar_init(bOFinal(h), 1);
         }
         *abort_flag = 0u;
@@ -313,43 +309,15 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             }
         }
     } else if (wg == 2) {
-        // ================================================================ correction + epilogue
+        // ================================================================ epilogue (one thread per output row)
         setmaxnreg_dec<96>();
         const int r = threadIdx.x & 127;
         const uint32_t lane_addr = tmem + ((uint32_t)((warp & 3) * 32) << 16);
-        uint32_t cr_phase[2] = {0, 0}, o_phase[2] = {0, 0}, f_phase[2] = {0, 0};
+        uint32_t o_phase[2] = {0, 0}, f_phase[2] = {0, 0};
         bool dead = false;
         for (int u = u_begin; u < u_end && !dead; ++u) {
             const WppUnit un = units[u];
             const UnitView v = view_of(un, p, q_offsets);
-            for (int j = 0; j < v.n_steps && !dead; ++j) {
-#pragma unroll
-                for (int hf = 0; hf < 2; ++hf) {
-                    if (j >= v.n[hf]) continue;
-                    // the softmax threads signal after they saw S(j), which the tensor pipe finished after the
-                    // O += P V of step j-1: O is safe to touch
-                    const bool ok = mbar_wait(bCorrReady(hf), cr_phase[hf], abort_flag);
-                    if (!__all_sync(0xffffffffu, ok)) { dead = true; break; }
-                    cr_phase[hf] ^= 1u;
-                    const float alpha = s_alpha[hf * 128 + r];
-                    if (__any_sync(0xffffffffu, alpha != 1.f)) {
-                        tc_fence_after();
-#pragma unroll
-                        for (int q4 = 0; q4 < D / 32; ++q4) {
-                            float o[32];
-                            tmem_ld32(lane_addr + col_o(hf) + q4 * 32, reinterpret_cast<uint32_t*>(o));
-                            tmem_wait_ld();
-#pragma unroll
-                            for (int i = 0; i < 32; ++i) o[i] *= alpha;
-                            tmem_st32(lane_addr + col_o(hf) + q4 * 32, reinterpret_cast<uint32_t*>(o));
-                        }
-                        tmem_wait_st();
-                        tc_fence_before();
-                    }
-                    mbar_arrive(bPReady(hf));
-                }
-            }
-            if (dead) break;
             // ---- epilogue of both halves
 #pragma unroll
             for (int hf = 0; hf < 2; ++hf) {
@@ -441,56 +409,31 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 TRACE(hf, tstep, 1);
 #ifdef WPP_EXPERIMENT_NO_SOFTMAX
                 // tuning experiment: how fast is the tile loop when the softmax costs nothing (results are garbage)
-                s_alpha[hf * 128 + r] = 1.f;
-                mbar_arrive(bCorrReady(hf));
                 tc_fence_before();
                 mbar_arrive(bPReady(hf));
                 continue;
 #endif
                 float s[128];
-#pragma unroll
-                for (int q4 = 0; q4 < 4; ++q4) tmem_ld32(lane_addr + colS + q4 * 32, reinterpret_cast<uint32_t*>(s) + q4 * 32);
-                tmem_wait_ld();
-                TRACE(hf, tstep, 2);
                 const int key0 = (v.kv_begin + j) * 128;
-                if (key0 + 127 > first_pos) {               // only steps that touch the diagonal are masked
-                    const int limit = first_pos + r - key0;
+                const bool masked = key0 + 127 > first_pos;    // only steps that touch the diagonal are masked
+                const int limit = min(first_pos + r, v.kv_len - 1) - key0;
+                auto load_scores = [&]() {
 #pragma unroll
-                    for (int i = 0; i < 128; ++i) s[i] = (i > limit) ? -INFINITY : s[i];
-                }
-                float mx[8];
+                    for (int q4 = 0; q4 < 4; ++q4)
+                        tmem_ld32(lane_addr + colS + q4 * 32, reinterpret_cast<uint32_t*>(s) + q4 * 32);
+                    tmem_wait_ld();
+                    if (masked) {
 #pragma unroll
-                for (int k = 0; k < 8; ++k) mx[k] = fmaxf(s[2 * k], s[2 * k + 1]);
+                        for (int i = 0; i < 128; ++i) s[i] = (i > limit) ? -INFINITY : s[i];
+                    }
+                };
+                // p = 2^(s*c - m_ref*c) for the whole row: bf16 pairs for the tensor cores, fp32 row sum
+                uint32_t pk[64];
+                auto exp_pass = [&](float neg_mc) -> float {
+                    const uint64_t nm2 = pack2(neg_mc, neg_mc);
+                    uint64_t sum2a = pack2(0.f, 0.f), sum2b = pack2(0.f, 0.f);
 #pragma unroll
-                for (int i = 16; i < 128; i += 16) {
-#pragma unroll
-                    for (int k = 0; k < 8; ++k) mx[k] = fmax3(mx[k], s[i + 2 * k], s[i + 2 * k + 1]);
-                }
-                const float mxx = fmaxf(fmax3(mx[0], mx[1], mx[2]), fmaxf(fmax3(mx[3], mx[4], mx[5]), fmaxf(mx[6], mx[7])));
-                // lazy rescale: keep the old reference unless the new maximum is far above it
-                float alpha = 1.f;
-                if ((mxx - m_ref) * c > kRescaleThreshold || m_ref == -INFINITY) {
-                    const float m_new = fmaxf(m_ref, mxx);
-                    const float m_safe = (m_new == -INFINITY) ? 0.f : m_new;
-                    alpha = fast_exp2((m_ref - m_safe) * c);        // 0 when there was no reference yet
-                    m_ref = m_new;
-                    l_run *= alpha;
-                }
-                s_alpha[hf * 128 + r] = (j == 0) ? 1.f : alpha;
-                mbar_arrive(bCorrReady(hf));
-                TRACE(hf, tstep, 3);
-                const float neg_mc = (m_ref == -INFINITY) ? 0.f : -m_ref * c;
-                const uint64_t nm2 = pack2(neg_mc, neg_mc);
-                // exp, row sum and bf16 packing in two halves of 64 scores; the first half of P is on its way to
-                // TMEM while the second half is computed.  P word w (scores 2w, 2w+1) overwrites S column w, which
-                // was read before.
-                uint64_t sum2a = pack2(0.f, 0.f), sum2b = pack2(0.f, 0.f);
-#pragma unroll
-                for (int half = 0; half < 2; ++half) {
-                    uint32_t pk[32];
-#pragma unroll
-                    for (int w = 0; w < 32; ++w) {
-                        const int i = half * 32 + w;
+                    for (int i = 0; i < 64; ++i) {
                         const uint64_t x2 = ffma2(pack2(s[2 * i], s[2 * i + 1]), c2, nm2);
                         float e0, e1;
                         if ((i & 3) < kEmuPairsOf4) {
@@ -501,21 +444,64 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                             e0 = fast_exp2(x0);
                             e1 = fast_exp2(x1);
                         }
-                        if (w & 1) sum2b = fadd2(sum2b, pack2(e0, e1)); else sum2a = fadd2(sum2a, pack2(e0, e1));
-                        pk[w] = pack_bf16x2(e0, e1);
+                        if (i & 1) sum2b = fadd2(sum2b, pack2(e0, e1)); else sum2a = fadd2(sum2a, pack2(e0, e1));
+                        pk[i] = pack_bf16x2(e0, e1);
                     }
-                    tmem_st32(lane_addr + colS + half * 32, pk);
+                    float t0, t1;
+                    unpack2(fadd2(sum2a, sum2b), t0, t1);
+                    return t0 + t1;
+                };
+                load_scores();
+                TRACE(hf, tstep, 2);
+                // Fast path: keep the row's reference m_ref and skip the row maximum altogether.  The row sum tells
+                // whether that was safe: every p <= row sum, so a sum below 2^16 means no score rose more than 16
+                // (log2 units) above the reference and nothing can overflow.  Otherwise (or when a row has no
+                // reference yet) the warp takes the slow path: true maximum, new reference, O and l rescaled.
+                bool slow = __any_sync(0xffffffffu, m_ref == -INFINITY);
+                float row_sum = 0.f;
+                if (!slow) {
+                    row_sum = exp_pass(-m_ref * c);
+                    slow = __any_sync(0xffffffffu, !(row_sum <= kFastPathSumLimit));
+                    if (slow) load_scores();          // S is still intact in tensor memory
                 }
+                TRACE(hf, tstep, 3);
+                if (slow) {
+                    float mx[8];
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) mx[k] = fmaxf(s[2 * k], s[2 * k + 1]);
+#pragma unroll
+                    for (int i = 16; i < 128; i += 16) {
+#pragma unroll
+                        for (int k = 0; k < 8; ++k) mx[k] = fmax3(mx[k], s[i + 2 * k], s[i + 2 * k + 1]);
+                    }
+                    const float mxx = fmaxf(fmax3(mx[0], mx[1], mx[2]), fmaxf(fmax3(mx[3], mx[4], mx[5]), fmaxf(mx[6], mx[7])));
+                    const float m_new = fmaxf(m_ref, mxx);
+                    const float m_safe = (m_new == -INFINITY) ? 0.f : m_new;
+                    const float alpha = fast_exp2((m_ref - m_safe) * c);       // 0 when there was no reference yet
+                    m_ref = m_new;
+                    l_run *= alpha;
+                    if (j > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
+                        // S(j) has landed, so the O += P V of step j-1 has too: O may be rescaled in place
+#pragma unroll
+                        for (int q4 = 0; q4 < D / 32; ++q4) {
+                            float o[32];
+                            tmem_ld32(lane_addr + col_o(hf) + q4 * 32, reinterpret_cast<uint32_t*>(o));
+                            tmem_wait_ld();
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) o[i] *= alpha;
+                            tmem_st32(lane_addr + col_o(hf) + q4 * 32, reinterpret_cast<uint32_t*>(o));
+                        }
+                    }
+                    row_sum = exp_pass(-m_safe * c);
+                }
+                l_run += row_sum;
                 TRACE(hf, tstep, 4);
+                tmem_st32(lane_addr + colS, pk);
+                tmem_st32(lane_addr + colS + 32, pk + 32);
                 tmem_wait_st();
                 tc_fence_before();
                 mbar_arrive(bPReady(hf));
                 TRACE(hf, tstep, 5);
-                {
-                    float t0, t1;
-                    unpack2(fadd2(sum2a, sum2b), t0, t1);
-                    l_run += t0 + t1;
-                }
                 ++tstep;
             }
             if (dead) break;
