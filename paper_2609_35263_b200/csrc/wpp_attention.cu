@@ -121,7 +121,7 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     auto bPReady = [&](int h) { return bHalf + 32 * h + 8; };
     auto bFinalReady = [&](int h) { return bHalf + 32 * h + 16; };
     auto bOFinal = [&](int h) { return bHalf + 32 * h + 24; };
-    float2* s_final = reinterpret_cast<float2*>(smem_gen + C::kOffFinal);     // [2][128] (m_ref, l)
+    float2* s_final = reinterpret_cast<float2*>(smem_gen + C::kOffFinal);     // [2][128] (reference in log2 units, l)
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_gen + C::kOffMisc);
     volatile uint32_t* abort_flag = tmem_slot + 1;
 
@@ -339,7 +339,7 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 tc_fence_after();
                 const float2 ml = s_final[hf * 128 + r];
                 const float inv_l = (ml.y > 0.f) ? 1.f / ml.y : 0.f;
-                const float lse2 = (ml.y > 0.f) ? (ml.x * p.scale_log2 + log2f(ml.y)) : -INFINITY;
+                const float lse2 = (ml.y > 0.f) ? (ml.x + log2f(ml.y)) : -INFINITY;
                 if (un.split_slot < 0) {
                     __nv_bfloat16* dst = p.out + tok * p.o_token_stride + (int64_t)un.head[hf] * p.o_head_stride;
 #pragma unroll
@@ -399,7 +399,10 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             const int n = v.n[hf];
             if (n == 0) continue;
             const int first_pos = v.P + un.row0[hf];          // last key visible to row 0 of this half
-            float m_ref = -INFINITY, l_run = 0.f;
+            // m_ref: reference of the row (raw score units); nmc = -(m_ref * c) rounded once.  Every p of the row is
+            // 2^(s*c + nmc) with that same nmc, and a change of reference rescales by 2^(nmc_new - nmc_old) of the two
+            // stored numbers, so old and new terms stay consistent even for scores around 1e8.
+            float m_ref = -INFINITY, l_run = 0.f, nmc = 0.f;
             for (int j = 0; j < n; ++j) {
                 TRACE(hf, tstep, 0);
                 const bool ok = mbar_wait(bSFull(hf), s_phase, abort_flag);
@@ -460,7 +463,7 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 bool slow = __any_sync(0xffffffffu, m_ref == -INFINITY);
                 float row_sum = 0.f;
                 if (!slow) {
-                    row_sum = exp_pass(-m_ref * c);
+                    row_sum = exp_pass(nmc);
                     slow = __any_sync(0xffffffffu, !(row_sum <= kFastPathSumLimit));
                     if (slow) load_scores();          // S is still intact in tensor memory
                 }
@@ -477,7 +480,9 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     const float mxx = fmaxf(fmax3(mx[0], mx[1], mx[2]), fmaxf(fmax3(mx[3], mx[4], mx[5]), fmaxf(mx[6], mx[7])));
                     const float m_new = fmaxf(m_ref, mxx);
                     const float m_safe = (m_new == -INFINITY) ? 0.f : m_new;
-                    const float alpha = fast_exp2((m_ref - m_safe) * c);       // 0 when there was no reference yet
+                    const float nmc_new = -m_safe * c;
+                    const float alpha = (m_ref == -INFINITY) ? 0.f : fast_exp2(nmc_new - nmc);
+                    nmc = nmc_new;
                     m_ref = m_new;
                     l_run *= alpha;
                     if (j > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
@@ -492,7 +497,7 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                             tmem_st32(lane_addr + col_o(hf) + q4 * 32, reinterpret_cast<uint32_t*>(o));
                         }
                     }
-                    row_sum = exp_pass(-m_safe * c);
+                    row_sum = exp_pass(nmc);
                 }
                 l_run += row_sum;
                 TRACE(hf, tstep, 4);
@@ -505,7 +510,7 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 ++tstep;
             }
             if (dead) break;
-            s_final[hf * 128 + r] = make_float2(m_ref, l_run);
+            s_final[hf * 128 + r] = make_float2(-nmc, l_run);
             mbar_arrive(bFinalReady(hf));
         }
     }
