@@ -46,7 +46,7 @@ def _load():
                                              ctypes.c_double, p, p]
         lib.wpp_oracle_attention_units.restype = ctypes.c_int
         lib.wpp_oracle_attention_units.argtypes = [p, p, p, p, p, p, i32, i32, i32, i32, i32, i32,
-                                                   ctypes.c_double, p, ctypes.c_int64, p, p]
+                                                   ctypes.c_double, p, ctypes.c_int64, p, p, p]
         _lib = lib
     return _lib
 
@@ -111,8 +111,10 @@ def oracle_attention(q, k_pool, v_pool, block_tables, prefix_lens, chunk_lens, s
     return out, lse
 
 
-def oracle_attention_units(q, k_pool, v_pool, block_tables, prefix_lens, chunk_lens, units, sm_scale=None):
-    """Selected (request, chunk row, query head) triples: returns (out [n, d], lse [n])."""
+def oracle_attention_units(q, k_pool, v_pool, block_tables, prefix_lens, chunk_lens, units, sm_scale=None,
+                           return_top2=False):
+    """Selected (request, chunk row, query head) triples: returns (out [n, d], lse [n]) and, if asked, the
+    largest and second largest score of each row [n, 2] (how well conditioned the row's softmax is)."""
     qb, kp, vp = _bits(q), _bits(k_pool), _bits(v_pool)
     bt, P, C = _i32(block_tables), _i32(prefix_lens), _i32(chunk_lens)
     units = _i32(units).reshape(-1, 3)
@@ -121,12 +123,14 @@ def oracle_attention_units(q, k_pool, v_pool, block_tables, prefix_lens, chunk_l
     n = units.shape[0]
     out = np.empty((n, d), dtype=np.float64)
     lse = np.empty((n,), dtype=np.float64)
+    top2 = np.empty((n, 2), dtype=np.float64) if return_top2 else None
     rc = _load().wpp_oracle_attention_units(_ptr(qb), _ptr(kp), _ptr(vp), _ptr(bt), _ptr(P), _ptr(C),
                                             P.shape[0], Hq, Hkv, d, B, bt.shape[1], _scale(d, sm_scale),
-                                            _ptr(units), n, _ptr(out), _ptr(lse))
+                                            _ptr(units), n, _ptr(out), _ptr(lse),
+                                            _ptr(top2) if return_top2 else None)
     if rc != 0:
         raise ValueError(f"oracle_attention_units failed ({rc})")
-    return out, lse
+    return (out, lse, top2) if return_top2 else (out, lse)
 
 
 def merge_partials(outs, lses):

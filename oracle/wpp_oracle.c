@@ -88,10 +88,10 @@ int wpp_oracle_append(const uint16_t* k_new, const uint16_t* v_new, uint16_t* k_
  * Sums run in increasing j (and increasing e inside the dot product). */
 static void attention_row(const uint16_t* q_row, const uint16_t* k_pool, const uint16_t* v_pool,
                           const int32_t* bt_row, int64_t n, int32_t g, int32_t Hkv, int32_t d, int32_t B,
-                          double scale, double* scores, double* out_row, double* lse_out) {
+                          double scale, double* scores, double* out_row, double* lse_out, double* top2_out) {
     double qd[1024];
     for (int32_t e = 0; e < d; ++e) qd[e] = bf16_to_f64(q_row[e]);
-    double m = -INFINITY;
+    double m = -INFINITY, second = -INFINITY;
     for (int64_t j = 0; j < n; ++j) {
         int64_t page = bt_row[j / B];
         const uint16_t* kr = k_pool + ((page * Hkv + g) * B + (j % B)) * (int64_t)d;
@@ -99,8 +99,10 @@ static void attention_row(const uint16_t* q_row, const uint16_t* k_pool, const u
         for (int32_t e = 0; e < d; ++e) acc += qd[e] * bf16_to_f64(kr[e]);
         double s = scale * acc;
         scores[j] = s;
-        if (s > m) m = s;
+        if (s > m) { second = m; m = s; }
+        else if (s > second) second = s;
     }
+    if (top2_out) { top2_out[0] = m; top2_out[1] = second; }
     double denom = 0.0;
     for (int32_t e = 0; e < d; ++e) out_row[e] = 0.0;
     for (int64_t j = 0; j < n; ++j) {
@@ -114,13 +116,14 @@ static void attention_row(const uint16_t* q_row, const uint16_t* k_pool, const u
     if (lse_out) *lse_out = m + log(denom);
 }
 
-/* O-attn on a list of (request, row, head) units; out [n_units][d], lse [n_units] (may be NULL).
+/* O-attn on a list of (request, row, head) units; out [n_units][d], lse [n_units] (may be NULL), top2 [n_units][2]
+ * (may be NULL): the largest and second largest score of the row, which tell how well conditioned the softmax is.
  * Reads the pools only (after O-append), never k_new/v_new, never a slot >= P_i + t + 1. */
 int wpp_oracle_attention_units(const uint16_t* q, const uint16_t* k_pool, const uint16_t* v_pool,
                                const int32_t* block_tables, const int32_t* prefix_lens,
                                const int32_t* chunk_lens, int32_t R, int32_t Hq, int32_t Hkv, int32_t d,
                                int32_t B, int32_t max_blocks, double scale, const int32_t* units /* [n][3] */,
-                               int64_t n_units, double* out, double* lse) {
+                               int64_t n_units, double* out, double* lse, double* top2 /* [n][2] or NULL */) {
     if (d > 1024 || Hq % Hkv != 0) return -2;
     int32_t G = Hq / Hkv;
     int64_t* off = (int64_t*)malloc(sizeof(int64_t) * (size_t)(R + 1));
@@ -142,7 +145,7 @@ int wpp_oracle_attention_units(const uint16_t* q, const uint16_t* k_pool, const 
             int64_t n = (int64_t)prefix_lens[i] + t + 1;
             const uint16_t* q_row = q + ((off[i] + t) * Hq + h) * (int64_t)d;
             attention_row(q_row, k_pool, v_pool, block_tables + (int64_t)i * max_blocks, n, h / G, Hkv, d, B,
-                          scale, scores, out + u * (int64_t)d, lse ? lse + u : NULL);
+                          scale, scores, out + u * (int64_t)d, lse ? lse + u : NULL, top2 ? top2 + 2 * u : NULL);
         }
         free(scores);
     }
@@ -167,7 +170,7 @@ int wpp_oracle_attention(const uint16_t* q, const uint16_t* k_pool, const uint16
                 ++u;
             }
     int rc = wpp_oracle_attention_units(q, k_pool, v_pool, block_tables, prefix_lens, chunk_lens, R, Hq, Hkv, d,
-                                        B, max_blocks, scale, units, n_units, out, lse);
+                                        B, max_blocks, scale, units, n_units, out, lse, NULL);
     free(units);
     return rc;
 }
