@@ -29,6 +29,8 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
 METRIC = "prefill-attention tokens/s at concurrency 128, high prefix reuse"
+# From profiles/attention_cfg3_r16_ncu.md: (dram read + write bytes) / key steps of the captured launch.
+DRAM_BYTES_PER_KEY_STEP = None
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -201,17 +203,14 @@ def main():
 
     import torch
     import paper_2609_35263_b200 as wpp
+    from paper_2609_35263_b200 import replicas
 
-    rank = int(os.environ.get("RANK", "0"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank, local_rank, world = replicas.env_ranks()
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback for the product path")
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=dev)
+    replicas.init("nccl", dev)
 
     peaks, peak_kind = load_peaks()
     w = build_workload(args.config)
@@ -256,18 +255,10 @@ def main():
             attn_events.append((a, b))
         return plan
 
-    def barrier():
-        torch.cuda.synchronize()
-        if world > 1:
-            torch.distributed.barrier()
-        torch.cuda.synchronize()
+    barrier = replicas.barrier
 
     def max_over_ranks(x):
-        if world == 1:
-            return x
-        t = torch.tensor([x], dtype=torch.float64, device=dev)
-        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
-        return float(t.item())
+        return replicas.max_over_ranks(x, dev)
 
     # ---- device-resident timing
     for i in range(args.warmup):
@@ -301,14 +292,10 @@ def main():
     qo_bytes = 2 * T * w.num_q_heads * w.head_dim * 2
     t_flops = flops / (roof_peak * 1e12)
     t_bytes = (kv_bytes + qo_bytes) / (float(peaks.get("hbm_gbs", FALLBACK_PEAKS["hbm_gbs"])) * 1e9)
-    traffic = None
-    tpath = os.path.join(ROOT, "profiles", "attention_traffic.json")
-    if os.path.exists(tpath):
-        try:
-            tj = json.load(open(tpath))
-            traffic = tj["dram_bytes_per_key_step"] * float(info.key_steps)
-        except Exception:
-            traffic = None
+    # DRAM bytes of one launch: dram__bytes_read.sum + dram__bytes_write.sum from the ncu capture summarised in
+    # profiles/ (taken on the 16-request cut of this workload, the full one being too large to capture), scaled
+    # by the 128x128 key steps a launch processes
+    traffic = DRAM_BYTES_PER_KEY_STEP * float(info.key_steps) if DRAM_BYTES_PER_KEY_STEP else None
     roofline = {"bound": "tensor" if t_flops >= t_bytes else "hbm", "kernel": "wpp_attn_kernel",
                 "achieved": achieved, "peak": roof_peak, "unit": "TFLOP/s", "frac": achieved / roof_peak,
                 "peak_source": f"of {peak_kind} (burst bf16 matmul)", "frac_of_sustained": achieved / roof_sus,
@@ -370,8 +357,7 @@ def main():
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline, "cpu_baseline": cpu,
         }
         print(json.dumps(line))
-    if world > 1:
-        torch.distributed.destroy_process_group()
+    replicas.finalize()
 
 
 if __name__ == "__main__":

@@ -1,0 +1,200 @@
+"""Host logic of the C-ABI library (no GPU): symbol exports, argument checks, and the work split.
+
+The plan is checked by brute force on small waves: every visible (request, row, head, key) pair is covered
+exactly once, no tile lies wholly above the diagonal, split parts tile a tile's key range contiguously, every
+tile is owned by exactly one persistent CTA, and equal inputs give byte-identical plans.
+"""
+import ctypes
+import os
+import re
+import struct
+
+import numpy as np
+import pytest
+
+import paper_2609_35263_b200 as wpp
+from paper_2609_35263_b200 import binding
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+HDR_FMT = "<IIQ" + "i" * 8 + "qqq" + "QQ" + "IIII"      # WppPlanHeader up to the section offsets
+
+
+def parse_plan(plan):
+    raw = plan.host_bytes()
+    f = struct.unpack_from(HDR_FMT, raw, 0)
+    (magic, version, desc_hash, R, num_ctas, num_units, num_combine, num_slots, tile_m, tile_n, head_dim,
+     T, key_steps, flops, ws_bytes, plan_bytes, off_q, off_cta, off_units, off_comb) = f
+    assert magic == 0x31505057
+    q_off = np.frombuffer(raw, dtype=np.int32, count=R + 1, offset=off_q)
+    cta = np.frombuffer(raw, dtype=np.int32, count=num_ctas + 1, offset=off_cta)
+    units = np.frombuffer(raw, dtype=np.int32, count=num_units * 12, offset=off_units).reshape(num_units, 12)
+    comb = np.frombuffer(raw, dtype=np.int32, count=num_combine * 8, offset=off_comb).reshape(num_combine, 8)
+    keys = ["request", "kv_begin", "kv_end", "split_slot", "row0_a", "row0_b", "rows_a", "rows_b", "head_a",
+            "head_b", "cost", "pad"]
+    return dict(R=R, num_ctas=num_ctas, tile_m=tile_m, T=T, key_steps=key_steps, flops=flops, slots=num_slots,
+                ws_bytes=ws_bytes, q_off=q_off, cta=cta, comb=comb,
+                units=[dict(zip(keys, u.tolist())) for u in units])
+
+
+def desc(R, Hq, Hkv, d, B, max_blocks, pages=1000):
+    return wpp.make_desc(R, Hq, Hkv, d, B, max_blocks, pages)
+
+
+def test_library_exports_every_declared_symbol():
+    lib = wpp.load_library()
+    hdr = open(os.path.join(ROOT, "include", "wpp.h")).read()
+    hdr = re.sub(r"/\*.*?\*/", "", hdr, flags=re.S)            # declarations only, not the prose
+    declared = set(re.findall(r"\b(wpp_[a-z_0-9]+)\s*\(", hdr))
+    assert {"wpp_plan_tiles", "wpp_kv_append", "wpp_prefill_attention_varlen"} <= declared
+    for name in declared:
+        assert hasattr(lib, name), f"{name} is declared in wpp.h but not exported"
+    assert set(binding.EXPORTS) <= declared
+
+
+def test_status_strings():
+    lib = wpp.load_library()
+    assert lib.wpp_status_string(0) == b"WPP_OK"
+    assert lib.wpp_status_string(4) == b"WPP_ERR_POSITION_MISMATCH"
+
+
+@pytest.mark.parametrize("P,C,Hq,Hkv,tile_m,splits", [
+    ([0], [1], 2, 1, 0, 0),
+    ([37, 0, 300], [200, 129, 3], 4, 2, 128, 0),
+    ([37, 0, 300], [200, 129, 3], 4, 2, 256, 0),
+    ([1000, 5], [700, 300], 4, 2, 256, 3),
+    ([1000, 5], [700, 300], 3, 1, 256, 2),          # odd group: unpaired tails
+    ([0, 0, 0], [64, 0, 128], 8, 2, 256, 7),
+    ([130], [64], 4, 2, 256, 2),
+])
+def test_plan_covers_every_visible_pair_exactly_once(P, C, Hq, Hkv, tile_m, splits):
+    B = 16
+    mb = max(1, max((p + c + B - 1) // B for p, c in zip(P, C)))
+    d = desc(len(P), Hq, Hkv, 128, B, mb)
+    plan = wpp.wpp_plan_tiles(None, d, P, C, opts=wpp.PlanOpts(tile_m, 0, splits, 40), pin=False)
+    pl = parse_plan(plan)
+    assert pl["T"] == sum(C) and pl["q_off"].tolist() == np.concatenate([[0], np.cumsum(C)]).tolist()
+    # CTA ownership is a partition of the unit list
+    assert pl["cta"][0] == 0 and pl["cta"][-1] == len(pl["units"]) and np.all(np.diff(pl["cta"]) >= 0)
+    G = Hq // Hkv
+    cover = {}
+    steps_total = 0
+    for u in pl["units"]:
+        i = u["request"]
+        assert u["kv_begin"] < u["kv_end"]
+        any_work = False
+        for hf in "ab":
+            rows, row0, head = u["rows_" + hf], u["row0_" + hf], u["head_" + hf]
+            if rows == 0:
+                continue
+            assert 0 < rows <= 128 and row0 + rows <= C[i] and 0 <= head < Hq
+            assert head // G == u["head_a"] // G            # both halves share one KV head
+            end = (P[i] + row0 + rows + 127) // 128
+            n = max(0, min(u["kv_end"], end) - u["kv_begin"])
+            steps_total += n
+            any_work |= n > 0
+            for t in range(row0, row0 + rows):
+                last = P[i] + t                              # last visible key
+                lo, hi = u["kv_begin"] * 128, min(u["kv_end"], end) * 128
+                for key in range(lo, min(hi, last + 1)):
+                    k = (i, t, head, key)
+                    cover[k] = cover.get(k, 0) + 1
+        assert any_work, "a tile with nothing to compute"
+    assert steps_total == pl["key_steps"]
+    want = sum(Hq * (c * p + c * (c + 1) // 2) for p, c in zip(P, C))
+    assert len(cover) == want and all(v == 1 for v in cover.values())
+    assert pl["flops"] == 4 * 128 * want
+    # split parts of a half tile use consecutive slots and contiguous key ranges starting at 0
+    by_slot = {u["split_slot"]: u for u in pl["units"] if u["split_slot"] >= 0}
+    assert len(by_slot) == pl["slots"]
+    for c in pl["comb"]:
+        req, row0, rows, head, slot0, ns, half, _ = c.tolist()
+        parts = [by_slot[s] for s in range(slot0, slot0 + ns)]
+        assert parts[0]["kv_begin"] == 0 and all(a["kv_end"] == b["kv_begin"] for a, b in zip(parts, parts[1:]))
+        hf = "ab"[half]
+        assert all(p_["request"] == req and p_["row0_" + hf] == row0 and p_["rows_" + hf] == rows and
+                   p_["head_" + hf] == head for p_ in parts)
+        assert parts[-1]["kv_end"] >= (P[req] + row0 + rows + 127) // 128
+    if splits >= 2 and max((p + c + 127) // 128 for p, c in zip(P, C)) >= 2:
+        assert pl["slots"] > 0 and pl["ws_bytes"] >= pl["slots"] * 2 * 128 * 129 * 4
+
+
+def test_plan_is_deterministic_and_balanced():
+    rng = np.random.default_rng(5)
+    P = (rng.integers(0, 100, 24) * 64).tolist()
+    C = rng.integers(1, 2000, 24).tolist()
+    d = desc(24, 16, 4, 128, 64, 200)
+    a = wpp.wpp_plan_tiles(None, d, P, C, pin=False)
+    b = wpp.wpp_plan_tiles(None, d, P, C, pin=False)
+    assert a.host_bytes() == b.host_bytes()
+    pl = parse_plan(a)
+    loads = [sum(u["cost"] for u in pl["units"][pl["cta"][c]:pl["cta"][c + 1]]) for c in range(pl["num_ctas"])]
+    biggest = max(u["cost"] for u in pl["units"])
+    assert max(loads) - min(loads) <= biggest          # longest-processing-time bound
+    for c in range(pl["num_ctas"]):                    # each CTA walks its tiles in decreasing cost
+        costs = [u["cost"] for u in pl["units"][pl["cta"][c]:pl["cta"][c + 1]]]
+        assert costs == sorted(costs, reverse=True)
+
+
+def test_short_tails_pair_two_heads_of_one_kv_group():
+    d = desc(1, 8, 2, 128, 64, 10)
+    pl = parse_plan(wpp.wpp_plan_tiles(None, d, [0], [300], opts=wpp.PlanOpts(256, 0, 1, 148), pin=False))
+    tails = [u for u in pl["units"] if u["row0_a"] == 256]
+    assert len(tails) == 4 and all(u["rows_a"] == 44 and u["rows_b"] == 44 and u["row0_b"] == 256 and
+                                   u["head_b"] == u["head_a"] + 1 for u in tails)
+
+
+def test_few_tiles_fall_back_to_128_row_tiles_and_split_keys():
+    d = desc(1, 8, 2, 64, 16, 64)
+    pl = parse_plan(wpp.wpp_plan_tiles(None, d, [256], [128], pin=False))       # the single-request configuration
+    assert pl["tile_m"] == 128 and len(pl["units"]) == 8 and all(u["rows_b"] == 0 for u in pl["units"])
+    d2 = desc(1, 2, 1, 128, 64, 600)
+    pl2 = parse_plan(wpp.wpp_plan_tiles(None, d2, [32768], [128], pin=False))
+    assert pl2["slots"] > 0 and len(pl2["units"]) > 100                          # long prefix, two tiles: split along keys
+
+
+def _status(fn, *a, **k):
+    try:
+        fn(*a, **k)
+        return 0
+    except wpp.WppError as e:
+        return e.status
+
+
+def test_host_detectable_errors_are_reported_before_any_launch():
+    ok = desc(2, 4, 2, 128, 64, 4)
+    assert _status(wpp.wpp_plan_tiles, None, ok, [0, 64], [100, 64], pin=False) == 0
+    # table too short for P + C
+    assert _status(wpp.wpp_plan_tiles, None, ok, [0, 200], [100, 64], pin=False) == 3
+    # span start differs from what the cache holds: execution must fail, not run against the wrong state
+    assert _status(wpp.wpp_plan_tiles, None, ok, [0, 64], [100, 64], cached_lens=[0, 128], pin=False) == 4
+    assert _status(wpp.wpp_plan_tiles, None, ok, [0, 64], [100, 64], cached_lens=[0, 64], pin=False) == 0
+    assert _status(wpp.wpp_plan_tiles, None, ok, [0, -1], [100, 64], pin=False) == 1
+    assert _status(wpp.wpp_plan_tiles, None, desc(1, 4, 2, 96, 64, 4), [0], [1], pin=False) == 2     # head_dim
+    assert _status(wpp.wpp_plan_tiles, None, desc(1, 4, 2, 128, 48, 4), [0], [1], pin=False) == 2    # page size
+    assert _status(wpp.wpp_plan_tiles, None, desc(1, 5, 2, 128, 64, 4), [0], [1], pin=False) == 2    # head ratio
+    bad_stride = wpp.make_desc(1, 4, 2, 128, 64, 4, 10, q_head_stride=132)
+    assert _status(wpp.wpp_plan_tiles, None, bad_stride, [0], [1], pin=False) == 1
+    assert _status(wpp.wpp_plan_tiles, None, ok, [0, 0], [1, 1], opts=wpp.PlanOpts(64, 0, 0, 0), pin=False) == 2
+
+
+def test_validate_batch_finds_aliased_appends():
+    d = desc(2, 2, 1, 128, 16, 4, pages=8)
+    bt = np.array([[0, 1, -1, -1], [2, 3, -1, -1]], dtype=np.int32)
+    assert wpp.wpp_validate_batch(d, bt, [10, 0], [10, 20]) == 0
+    bt2 = bt.copy(); bt2[1, 1] = 1                                   # both requests write page 1
+    assert wpp.wpp_validate_batch(d, bt2, [10, 0], [10, 20]) == 9
+    bt3 = bt.copy(); bt3[1, 0] = 0                                   # request 1 writes what request 0 reads
+    assert wpp.wpp_validate_batch(d, bt3, [10, 0], [10, 5]) == 9
+    shared = np.array([[0, 1, -1, -1], [0, 2, -1, -1]], dtype=np.int32)   # a shared, read-only prefix page is fine
+    assert wpp.wpp_validate_batch(d, shared, [16, 16], [4, 4]) == 0
+    bt4 = bt.copy(); bt4[0, 1] = 8
+    assert wpp.wpp_validate_batch(d, bt4, [10, 0], [10, 20]) == 3
+    assert wpp.wpp_validate_batch(d, bt, [10, 0], [100, 20]) == 3
+
+
+def test_there_is_no_cpu_fallback():
+    import torch
+    if torch.cuda.is_available():
+        pytest.skip("a device is present")
+    with pytest.raises(wpp.WppError):
+        wpp.Context(0)
