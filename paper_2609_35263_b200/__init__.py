@@ -11,5 +11,7 @@ from .binding import (  # noqa: F401
     wpp_kv_append,
     wpp_plan_tiles,
     wpp_prefill_attention_varlen,
+    wpp_prefill_attention_varlen_static,
+    wpp_static_scratch_bytes,
     wpp_validate_batch,
 )

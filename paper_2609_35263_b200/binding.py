@@ -58,7 +58,7 @@ class PlanInfo(ctypes.Structure):
 
 EXPORTS = ["wpp_create", "wpp_destroy", "wpp_status_string", "wpp_last_cuda_error", "wpp_plan_bytes",
            "wpp_plan_tiles", "wpp_validate_batch", "wpp_kv_append", "wpp_prefill_attention_varlen",
-           "wpp_launch_count"]
+           "wpp_launch_count", "wpp_prefill_attention_varlen_static", "wpp_static_scratch_bytes"]
 
 _lib = None
 
@@ -88,6 +88,10 @@ def load_library() -> ctypes.CDLL:
                                       i32p, vp]
         lib.wpp_prefill_attention_varlen.argtypes = [vp, ctypes.POINTER(BatchDesc), vp, vp, vp, vp, vp, i32p, i32p,
                                                      i32p, vp, vp, vp, ctypes.c_size_t, i32p, vp]
+        lib.wpp_prefill_attention_varlen_static.argtypes = [vp, ctypes.POINTER(BatchDesc), vp, vp, vp, vp, vp, i32p,
+                                                            i32p, i32p, vp, vp, i32p, vp]
+        lib.wpp_static_scratch_bytes.restype = ctypes.c_size_t
+        lib.wpp_static_scratch_bytes.argtypes = []
         _lib = lib
     return _lib
 
@@ -233,3 +237,25 @@ def wpp_prefill_attention_varlen(ctx: Context, desc: BatchDesc, q, out, lse, k_c
         _ptr(block_tables), _ptr(prefix_lens), _ptr(chunk_lens), ctypes.c_void_p(plan.host.data_ptr()),
         _ptr(plan.dev), _ptr(workspace), ws_bytes, _ptr(status), _stream(stream))
     _check(st, "wpp_prefill_attention_varlen")
+
+
+def wpp_static_scratch_bytes() -> int:
+    """Size of the scratch array built into the library (used by wpp_prefill_attention_varlen_static)."""
+    return int(load_library().wpp_static_scratch_bytes())
+
+
+def wpp_prefill_attention_varlen_static(ctx: Context, desc: BatchDesc, q, out, lse, k_cache, v_cache, block_tables,
+                                        prefix_lens, chunk_lens, plan: Plan, status=None, stream=None) -> None:
+    """wpp_prefill_attention_varlen without a caller workspace and without any allocation.
+
+    For callers that cannot obtain device memory at call time (a serving process whose KV page pool already owns
+    all free HBM, an execution stream that must not be stalled by cudaMalloc).  Split-KV partials go to a fixed
+    16 MiB array inside the library; plans that need more raise WPP_ERR_WORKSPACE_TOO_SMALL.  All calls on a
+    device share that array, so calls whose kernels could overlap on the GPU must be serialised.  The first call
+    on a device does a one-time address look-up (the context's device must be current) and should come before any
+    stream capture."""
+    st = load_library().wpp_prefill_attention_varlen_static(
+        ctx.handle, ctypes.byref(desc), _ptr(q), _ptr(out), _ptr(lse), _ptr(k_cache), _ptr(v_cache),
+        _ptr(block_tables), _ptr(prefix_lens), _ptr(chunk_lens), ctypes.c_void_p(plan.host.data_ptr()),
+        _ptr(plan.dev), _ptr(status), _stream(stream))
+    _check(st, "wpp_prefill_attention_varlen_static")

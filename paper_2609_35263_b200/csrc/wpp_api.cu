@@ -216,3 +216,46 @@ extern "C" int wpp_prefill_attention_varlen(const wpp_ctx* ctx, const wpp_batch_
     }
     return WPP_OK;
 }
+
+// ---------------------------------------------------------------------------------------------------------------
+// Entry point that allocates nothing: split-KV partials live in a scratch array inside the library image.
+// Some callers of this library cannot call cudaMalloc when a wave is due: the serving process has handed all free
+// device memory to the KV page pool, and an allocation on the execution path would fail or stall the stream.
+#define WPP_STATIC_SCRATCH_BYTES (16u << 20)
+static __device__ __align__(256) unsigned char wpp_static_scratch[WPP_STATIC_SCRATCH_BYTES];
+
+// In host code the array's name is only a handle; its device address is looked up once per device.
+static void* g_static_scratch_ptr[64];
+static bool g_static_scratch_ready[64];
+
+extern "C" size_t wpp_static_scratch_bytes(void) { return (size_t)WPP_STATIC_SCRATCH_BYTES; }
+
+extern "C" int wpp_prefill_attention_varlen_static(const wpp_ctx* ctx, const wpp_batch_desc* desc, const void* q,
+                                                   void* out, float* lse_or_null, const void* k_cache,
+                                                   const void* v_cache, const int32_t* block_tables,
+                                                   const int32_t* prefix_lens, const int32_t* chunk_lens,
+                                                   const void* plan_host, const void* plan_dev, int32_t* status_dev,
+                                                   void* cuda_stream) {
+    if (!ctx || ctx->device < 0 || ctx->device >= 64) return WPP_ERR_INVALID_ARG;
+    wpp_batch_desc d;
+    int rc = wpp_resolve_desc(desc, &d);
+    if (rc != WPP_OK) return rc;
+    const WppPlanHeader* hd = nullptr;
+    if ((rc = wpp_check_plan(plan_host, &d, &hd)) != WPP_OK) return rc;
+    if (hd->workspace_bytes > (uint64_t)WPP_STATIC_SCRATCH_BYTES) return WPP_ERR_WORKSPACE_TOO_SMALL;
+    if (!g_static_scratch_ready[ctx->device]) {
+        // set-up, once per device, with that device current: the symbol resolves to the current device's copy
+        int cur = -1;
+        cudaError_t e = cudaGetDevice(&cur);
+        if (e != cudaSuccess) return cuda_fail(ctx, (int)e);
+        if (cur != ctx->device) return WPP_ERR_INVALID_ARG;
+        void* ptr = nullptr;
+        e = cudaGetSymbolAddress(&ptr, wpp_static_scratch);
+        if (e != cudaSuccess || !ptr) return cuda_fail(ctx, (int)e);
+        g_static_scratch_ptr[ctx->device] = ptr;
+        g_static_scratch_ready[ctx->device] = true;
+    }
+    return wpp_prefill_attention_varlen(ctx, desc, q, out, lse_or_null, k_cache, v_cache, block_tables, prefix_lens,
+                                        chunk_lens, plan_host, plan_dev, g_static_scratch_ptr[ctx->device],
+                                        (size_t)WPP_STATIC_SCRATCH_BYTES, status_dev, cuda_stream);
+}
