@@ -150,12 +150,12 @@ extern "C" int wpp_prefill_attention_varlen(const wpp_ctx* ctx, const wpp_batch_
     }
     if (d.num_pages == 0) return WPP_ERR_INVALID_ARG;
 
-    CUtensorMap tq, tk, tv;
-    {
+    CUtensorMap tq[4], tk, tv;
+    for (int i = 0; i < 4; ++i) {       // boxes of 128, 64, 32, 16 query rows (packed heads take fewer rows per head)
         const uint64_t dims[3] = {(uint64_t)d.head_dim, (uint64_t)d.num_q_heads, (uint64_t)hd->total_new_tokens};
         const uint64_t strides[2] = {(uint64_t)d.q_head_stride * 2, (uint64_t)d.q_token_stride * 2};
-        const uint32_t box[3] = {64, 1, 128};
-        if ((rc = make_map(ctx, &tq, q, 3, dims, strides, box)) != WPP_OK) return rc;
+        const uint32_t box[3] = {64, 1, (uint32_t)(128 >> i)};
+        if ((rc = make_map(ctx, &tq[i], q, 3, dims, strides, box)) != WPP_OK) return rc;
     }
     {
         const uint64_t dims[4] = {(uint64_t)d.head_dim, (uint64_t)d.page_size, (uint64_t)d.num_kv_heads,
@@ -194,7 +194,7 @@ extern "C" int wpp_prefill_attention_varlen(const wpp_ctx* ctx, const wpp_batch_
     }
 #endif
 
-    int e = wpp_launch_attention(d.head_dim, &tq, &tk, &tv, &p, hd->num_ctas, cuda_stream);
+    int e = wpp_launch_attention(d.head_dim, tq, &tk, &tv, &p, hd->num_ctas, cuda_stream);
     if (e != 0) return cuda_fail(ctx, e);
     const_cast<wpp_ctx*>(ctx)->launches += 1;
     if (hd->num_combine > 0) {

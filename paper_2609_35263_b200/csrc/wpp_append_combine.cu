@@ -54,14 +54,14 @@ __global__ void __launch_bounds__(256) wpp_combine_kernel(const CombineParams p)
     for (int r = warp; r < cu.rows; r += 8) {
         float m = -INFINITY;
         for (int s = 0; s < cu.num_splits; ++s)
-            m = fmaxf(m, p.ws_lse[((int64_t)(cu.slot0 + s) * 2 + cu.half) * 128 + r]);
+            m = fmaxf(m, p.ws_lse[((int64_t)(cu.slot0 + s) * 2 + cu.half) * 128 + cu.lane0 + r]);
         const int64_t tok = (int64_t)q_offsets[cu.request] + cu.row0 + r;
         __nv_bfloat16* dst = p.out + tok * p.o_token_stride + (int64_t)cu.head * p.o_head_stride;
         float wsum = 0.f;
         float acc[4] = {0.f, 0.f, 0.f, 0.f};
         if (m > -INFINITY) {
             for (int s = 0; s < cu.num_splits; ++s) {
-                const int64_t row = ((int64_t)(cu.slot0 + s) * 2 + cu.half) * 128 + r;
+                const int64_t row = ((int64_t)(cu.slot0 + s) * 2 + cu.half) * 128 + cu.lane0 + r;
                 const float l = p.ws_lse[row];
                 if (l == -INFINITY) continue;       // that part saw no key of this row; its O row is not defined
                 const float w = exp2f(l - m);

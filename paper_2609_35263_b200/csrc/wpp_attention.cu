@@ -50,7 +50,7 @@ struct Cfg {
     static constexpr int kItemBytes = 2 * kTileBytes;      // V part, then K part
     static constexpr int kOffKV = 2 * kTileBytes;
     static constexpr int kOffBars = kOffKV + kItems * kItemBytes;
-    static constexpr int kNumBars = 2 + 2 * kItems + 4 * 2;
+    static constexpr int kNumBars = 2 + 2 * kItems + 5 * 2;
     static constexpr int kOffFinal = kOffBars + 8 * kNumBars;          // float2 (m, l)[2][128]
     static constexpr int kOffMisc = kOffFinal + 2 * 128 * 8;           // tmem ptr, abort flag
     static constexpr int kSmemBytes = kOffMisc + 16 + 1024;            // + alignment slack
@@ -101,8 +101,10 @@ __device__ __forceinline__ UnitView view_of(const WppUnit& un, const AttnParams&
 
 template <int D>
 __global__ void __launch_bounds__(kThreads, 1)
-wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
-                const __grid_constant__ CUtensorMap tm_v, const AttnParams p) {
+wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_q64,
+                const __grid_constant__ CUtensorMap tm_q32, const __grid_constant__ CUtensorMap tm_q16,
+                const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
+                const AttnParams p) {
     using C = Cfg<D>;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -114,13 +116,15 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     const uint32_t bItemFull = bars + 16, bItemEmpty = bItemFull + 8 * C::kItems;
     // Per half: s_full (S = Q K^T landed; it also proves the previous O += P V landed, the tensor pipe being in
     // order), p_ready (P written, and O rescaled if the row reference moved, by the 128 softmax threads),
-    // final_ready (end-of-tile (m, l) are in smem), o_final (last O += P V landed).  A thread never arrives twice
-    // on one barrier without a wait in between that implies the earlier phase completed.
+    // final_ready (end-of-tile (m, l) are in smem), o_final (last O += P V landed), o_free (the epilogue threads
+    // have read O out, the next tile may overwrite it).  A thread never arrives twice on one barrier without a
+    // wait in between that implies the earlier phase completed.
     const uint32_t bHalf = bItemEmpty + 8 * C::kItems;
-    auto bSFull = [&](int h) { return bHalf + 32 * h; };
-    auto bPReady = [&](int h) { return bHalf + 32 * h + 8; };
-    auto bFinalReady = [&](int h) { return bHalf + 32 * h + 16; };
-    auto bOFinal = [&](int h) { return bHalf + 32 * h + 24; };
+    auto bSFull = [&](int h) { return bHalf + 40 * h; };
+    auto bPReady = [&](int h) { return bHalf + 40 * h + 8; };
+    auto bFinalReady = [&](int h) { return bHalf + 40 * h + 16; };
+    auto bOFinal = [&](int h) { return bHalf + 40 * h + 24; };
+    auto bOFree = [&](int h) { return bHalf + 40 * h + 32; };
     float2* s_final = reinterpret_cast<float2*>(smem_gen + C::kOffFinal);     // [2][128] (reference in log2 units, l)
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_gen + C::kOffMisc);
     volatile uint32_t* abort_flag = tmem_slot + 1;
@@ -133,7 +137,7 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         for (int s = 0; s < C::kItems; ++s) { mbar_init(bItemFull + 8 * s, 1); mbar_init(bItemEmpty + 8 * s, 1); }
         for (int h = 0; h < 2; ++h) {
             mbar_init(bSFull(h), 1); mbar_init(bPReady(h), 128);
-            mbar_init(bFinalReady(h), 128); mbar_init(bOFinal(h), 1);
+            mbar_init(bFinalReady(h), 128); mbar_init(bOFinal(h), 1); mbar_init(bOFree(h), 128);
         }
         *abort_flag = 0u;
         fence_barrier_init();
@@ -144,6 +148,7 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     }
     if (warp == 13 && lane == 0) {
         prefetch_tensormap(&tm_q); prefetch_tensormap(&tm_k); prefetch_tensormap(&tm_v);
+        prefetch_tensormap(&tm_q64); prefetch_tensormap(&tm_q32); prefetch_tensormap(&tm_q16);
     }
     tc_fence_before();
     __syncthreads();
@@ -159,7 +164,7 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     const int B = p.page_size, ppt = 128 / B;   // pages per key step
 
     if (wg == 3) {
-        setmaxnreg_dec<80>();
+        setmaxnreg_dec<96>();
         if (warp == 13) {
             // ================================================================ producer
             Ring ring = {0, 0};
@@ -214,13 +219,18 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 if (lane == 0) {
                     const int nq = (v.n[0] > 0) + (v.n[1] > 0);
                     mbar_arrive_expect_tx(bQFull, nq * C::kTileBytes);
+                    // head k of a half lands in tensor rows [k*rph, (k+1)*rph): one box of rph rows per head
+                    const int rph = 128 / un.pack;
+                    const CUtensorMap* qm = un.pack == 1 ? &tm_q : un.pack == 2 ? &tm_q64 : un.pack == 4 ? &tm_q32 : &tm_q16;
 #pragma unroll
                     for (int hf = 0; hf < 2; ++hf) {
                         if (v.n[hf] == 0) continue;
+                        for (int k = 0; k < un.pack; ++k) {
 #pragma unroll
-                        for (int h = 0; h < C::kHalves; ++h)
-                            tma_load_3d(sQ + hf * C::kTileBytes + h * C::kHalfBytes, &tm_q, bQFull, h * 64, un.head[hf],
-                                        v.q_off + un.row0[hf]);
+                            for (int h = 0; h < C::kHalves; ++h)
+                                tma_load_3d(sQ + hf * C::kTileBytes + h * C::kHalfBytes + k * rph * 128, qm, bQFull, h * 64,
+                                            un.head[hf] + k, v.q_off + un.row0[hf]);
+                        }
                     }
                 }
                 __syncwarp();
@@ -234,7 +244,7 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             // independent issuers were measured: the halves then drift into phase, both softmaxes share the
             // exp units and the dependency chain of each half gets longer.)
             Ring ring = {0, 0};
-            uint32_t q_phase = 0, p_phase[2] = {0, 0};
+            uint32_t q_phase = 0, p_phase[2] = {0, 0}, of_phase[2] = {0, 0};
             int tstep = 0;
             (void)tstep;
             constexpr uint32_t idesc_qk = idesc_bf16(128, 0, 0);
@@ -290,6 +300,11 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                         if (!mbar_wait(bPReady(hf), p_phase[hf], abort_flag)) { dead = true; break; }   // P written, O fixed
                         p_phase[hf] ^= 1u;
                         TRACE(2, tstep, hf * 4 + 1);
+                        if (j == 0) {
+                            // the first product of a tile overwrites O: the previous tile's epilogue must have read it
+                            if (!mbar_wait(bOFree(hf), of_phase[hf] ^ 1u, abort_flag)) { dead = true; break; }
+                            of_phase[hf] ^= 1u;
+                        }
                         tc_fence_after();
                         const uint32_t tS = tmem + col_s(hf), tO = tmem + col_o(hf);
                         if (j > 0) mma_ts_accumulate(tO, tS, vd, idesc_pv); else mma_ts_overwrite(tO, tS, vd, idesc_pv);
@@ -310,7 +325,7 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         }
     } else if (wg == 2) {
         // ================================================================ epilogue (one thread per output row)
-        setmaxnreg_dec<96>();
+        setmaxnreg_dec<80>();
         const int r = threadIdx.x & 127;
         const uint32_t lane_addr = tmem + ((uint32_t)((warp & 3) * 32) << 16);
         uint32_t o_phase[2] = {0, 0}, f_phase[2] = {0, 0};
@@ -322,8 +337,10 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
 #pragma unroll
             for (int hf = 0; hf < 2; ++hf) {
                 if (un.rows[hf] == 0) continue;
-                const bool row_ok = r < un.rows[hf];
-                const int64_t tok = (int64_t)v.q_off + un.row0[hf] + r;
+                const int rph = 128 / un.pack, rr = r & (rph - 1);       // row inside its head's block
+                const int head = un.head[hf] + r / rph;
+                const bool row_ok = rr < un.rows[hf];
+                const int64_t tok = (int64_t)v.q_off + un.row0[hf] + rr;
                 const int64_t prow = ((int64_t)un.split_slot * 2 + hf) * 128 + r;
                 if (v.n[hf] == 0) {
                     // a split part that lies wholly above this half's diagonal: no key is visible
@@ -341,7 +358,7 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 const float inv_l = (ml.y > 0.f) ? 1.f / ml.y : 0.f;
                 const float lse2 = (ml.y > 0.f) ? (ml.x + log2f(ml.y)) : -INFINITY;
                 if (un.split_slot < 0) {
-                    __nv_bfloat16* dst = p.out + tok * p.o_token_stride + (int64_t)un.head[hf] * p.o_head_stride;
+                    __nv_bfloat16* dst = p.out + tok * p.o_token_stride + (int64_t)head * p.o_head_stride;
 #pragma unroll
                     for (int q4 = 0; q4 < D / 32; ++q4) {
                         float o[32];
@@ -359,7 +376,7 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                             }
                         }
                     }
-                    if (p.lse && row_ok) p.lse[tok * p.num_q_heads + un.head[hf]] = lse2 * 0.6931471805599453f;
+                    if (p.lse && row_ok) p.lse[tok * p.num_q_heads + head] = lse2 * 0.6931471805599453f;
                 } else {
                     float* dst = p.ws_o + prow * D;
 #pragma unroll
@@ -378,6 +395,7 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     if (row_ok) p.ws_lse[prow] = lse2;
                 }
                 tc_fence_before();
+                mbar_arrive(bOFree(hf));
             }
         }
     } else {
@@ -399,6 +417,9 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             const int n = v.n[hf];
             if (n == 0) continue;
             const int first_pos = v.P + un.row0[hf];          // last key visible to row 0 of this half
+            // last key this thread's row may see: its own position (rows of packed heads repeat every 128/pack
+            // tensor rows), never past the end of the sequence
+            const int row_last = min(first_pos + (r & (128 / un.pack - 1)), v.kv_len - 1);
             // m_ref: reference of the row (raw score units); nmc = -(m_ref * c) rounded once.  Every p of the row is
             // 2^(s*c + nmc) with that same nmc, and a change of reference rescales by 2^(nmc_new - nmc_old) of the two
             // stored numbers, so old and new terms stay consistent even for scores around 1e8.
@@ -419,7 +440,7 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 float s[128];
                 const int key0 = (v.kv_begin + j) * 128;
                 const bool masked = key0 + 127 > first_pos;    // only steps that touch the diagonal are masked
-                const int limit = min(first_pos + r, v.kv_len - 1) - key0;
+                const int limit = row_last - key0;
                 auto load_scores = [&]() {
 #pragma unroll
                     for (int q4 = 0; q4 < 4; ++q4)
@@ -530,7 +551,7 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
 }
 
 template <int D>
-static cudaError_t launch(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const AttnParams& p,
+static cudaError_t launch(const CUtensorMap* tq, const CUtensorMap& tk, const CUtensorMap& tv, const AttnParams& p,
                           int num_ctas, cudaStream_t stream) {
     static bool attr_set[64] = {};
     int dev = 0;
@@ -541,15 +562,16 @@ static cudaError_t launch(const CUtensorMap& tq, const CUtensorMap& tk, const CU
         if (e != cudaSuccess) return e;
         attr_set[dev] = true;
     }
-    wpp_attn_kernel<D><<<num_ctas, kThreads, Cfg<D>::kSmemBytes, stream>>>(tq, tk, tv, p);
+    wpp_attn_kernel<D><<<num_ctas, kThreads, Cfg<D>::kSmemBytes, stream>>>(tq[0], tq[1], tq[2], tq[3], tk, tv, p);
     return cudaGetLastError();
 }
 
 }  // namespace wpp
 
+// tq: four maps of q with boxes of 128, 64, 32 and 16 rows
 extern "C" int wpp_launch_attention(int head_dim, const CUtensorMap* tq, const CUtensorMap* tk, const CUtensorMap* tv,
                                     const wpp::AttnParams* p, int num_ctas, void* stream) {
-    if (head_dim == 128) return (int)wpp::launch<128>(*tq, *tk, *tv, *p, num_ctas, (cudaStream_t)stream);
-    if (head_dim == 64) return (int)wpp::launch<64>(*tq, *tk, *tv, *p, num_ctas, (cudaStream_t)stream);
+    if (head_dim == 128) return (int)wpp::launch<128>(tq, *tk, *tv, *p, num_ctas, (cudaStream_t)stream);
+    if (head_dim == 64) return (int)wpp::launch<64>(tq, *tk, *tv, *p, num_ctas, (cudaStream_t)stream);
     return (int)cudaErrorInvalidValue;
 }

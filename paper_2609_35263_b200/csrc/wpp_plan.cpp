@@ -141,7 +141,7 @@ int wpp_plan_tiles(const wpp_ctx* ctx, const wpp_batch_desc* desc, const int32_t
 
     // ---- base tiles in natural order (request, row block, head): the heads of one KV group and the row
     //      blocks of one request stay next to each other, so tiles that run at the same time share K/V in L2.
-    struct Base { int32_t request, row0[2], rows[2], head[2], steps; };
+    struct Base { int32_t request, row0[2], rows[2], head[2], steps, pack; };
     const int G = Hq / d.num_kv_heads;
     auto steps_for = [](int64_t last_visible_plus1) { return (int32_t)((last_visible_plus1 + WPP_TILE_N - 1) / WPP_TILE_N); };
     auto build_base = [&](int tile_m, std::vector<Base>& base) {
@@ -150,14 +150,23 @@ int wpp_plan_tiles(const wpp_ctx* ctx, const wpp_batch_desc* desc, const int32_t
             const int64_t P = prefix_lens[i], C = chunk_lens[i];
             for (int64_t r0 = 0; r0 < C; r0 += tile_m) {
                 const int32_t rows = (int32_t)std::min<int64_t>(tile_m, C - r0);
-                if (tile_m == 256 && rows <= WPP_HALF_M && G % 2 == 0) {
-                    // short tail: pair two heads of one KV group over the same rows
-                    for (int h = 0; h < Hq; h += 2)
-                        base.push_back({i, {(int32_t)r0, (int32_t)r0}, {rows, rows}, {h, h + 1}, steps_for(P + r0 + rows)});
+                if (rows <= WPP_HALF_M) {
+                    // short block: each half takes `pack` heads of one KV group over the same rows (pack is the
+                    // largest power of two that divides the group size and leaves 128/pack >= rows tensor rows
+                    // per head); with 256-row tiles the second half takes the next heads of the group
+                    int pack = 1;
+                    while (pack < 8 && G % (2 * pack) == 0 && WPP_HALF_M / (2 * pack) >= rows) pack *= 2;
+                    const int per_tile = (tile_m == 256 && G % (2 * pack) == 0) ? 2 * pack : pack;
+                    for (int h = 0; h < Hq; h += per_tile) {
+                        const int32_t rows_b = per_tile == 2 * pack ? rows : 0;
+                        base.push_back({i, {(int32_t)r0, (int32_t)r0}, {rows, rows_b}, {h, h + pack},
+                                        steps_for(P + r0 + rows), pack});
+                    }
                 } else {
-                    const int32_t ra = std::min(rows, WPP_HALF_M), rb = rows - ra;
+                    const int32_t ra = WPP_HALF_M, rb = rows - ra;
                     for (int h = 0; h < Hq; ++h)
-                        base.push_back({i, {(int32_t)r0, (int32_t)r0 + WPP_HALF_M}, {ra, rb}, {h, h}, steps_for(P + r0 + rows)});
+                        base.push_back({i, {(int32_t)r0, (int32_t)r0 + WPP_HALF_M}, {ra, rb}, {h, h},
+                                        steps_for(P + r0 + rows), 1});
                 }
             }
         }
@@ -202,13 +211,16 @@ int wpp_plan_tiles(const wpp_ctx* ctx, const wpp_batch_desc* desc, const int32_t
         std::memset(&u, 0, sizeof(u));
         u.request = t.request;
         for (int h = 0; h < 2; ++h) { u.row0[h] = t.row0[h]; u.rows[h] = t.rows[h]; u.head[h] = t.head[h]; }
+        u.pack = t.pack;
         if (parts == 1) {
             u.kv_begin = 0; u.kv_end = t.steps; u.split_slot = -1; u.cost = cost_of(t, 0, t.steps);
             units.push_back(u);
             key_steps += u.cost;
         } else {
             for (int h = 0; h < 2; ++h)
-                if (t.rows[h] > 0) combines.push_back({t.request, t.row0[h], t.rows[h], t.head[h], slots, parts, h, 0});
+                for (int k = 0; k < t.pack && t.rows[h] > 0; ++k)
+                    combines.push_back({t.request, t.row0[h], t.rows[h], t.head[h] + k, slots, parts, h,
+                                        k * (WPP_HALF_M / t.pack)});
             for (int32_t p = 0; p < parts; ++p) {
                 u.kv_begin = (int32_t)((int64_t)t.steps * p / parts);
                 u.kv_end = (int32_t)((int64_t)t.steps * (p + 1) / parts);

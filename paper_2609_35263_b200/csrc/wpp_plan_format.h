@@ -4,7 +4,7 @@
 #include <stdint.h>
 
 #define WPP_PLAN_MAGIC 0x31505057u /* "WPP1" */
-#define WPP_PLAN_VERSION 3u
+#define WPP_PLAN_VERSION 4u
 #define WPP_TILE_N 128             /* keys per step */
 #define WPP_HALF_M 128             /* query rows per tensor-core tile (one TMEM lane per row) */
 
@@ -24,16 +24,19 @@ struct WppPlanHeader {
 };
 
 // One work tile = two 128-row "halves" that share one K/V stream (same request, same KV head).  Each half
-// is rows [row0, row0+rows) of the request's chunk for one query head; rows == 0 marks an unused half.
-// Usually the halves are consecutive row blocks of one head; a short chunk tail pairs two heads of one
-// KV group instead.  The tile covers key steps [kv_begin, kv_end) of 128 keys (absolute key = step*128 +
-// column); each half additionally stops at its own causal end.
+// is rows [row0, row0+rows) of the request's chunk for `pack` consecutive query heads of that KV group
+// (head, head+1, ...): head k of the half sits in tensor rows [k*128/pack, k*128/pack + rows).  pack is 1
+// for row blocks longer than 64 rows; shorter blocks pack 2, 4 or 8 heads so that the 128-row MMA tile is not
+// mostly padding.  rows == 0 marks an unused half.  Usually the halves are consecutive row blocks of one
+// head; a short block gives the second half the next heads of the group instead.  The tile covers key steps
+// [kv_begin, kv_end) of 128 keys (absolute key = step*128 + column); each half additionally stops at its own
+// causal end.
 struct WppUnit {
     int32_t request, kv_begin, kv_end;
     int32_t split_slot;             // -1: writes the final output; else partial slot in the workspace
     int32_t row0[2], rows[2], head[2];
     int32_t cost;                   // 128x128 steps over both halves, what the CTA assignment balanced
-    int32_t pad;
+    int32_t pack;                   // query heads per half: 1, 2, 4 or 8
 };
 
 // One half tile whose key range was split: partial slots [slot0, slot0+num_splits) merged in increasing order.
@@ -41,7 +44,7 @@ struct WppCombine {
     int32_t request, row0, rows, head;
     int32_t slot0, num_splits;
     int32_t half;                   // which half of the slot the rows live in
-    int32_t pad;
+    int32_t lane0;                  // first tensor row of this head inside the half (packed heads)
 };
 
 // Workspace layout: fp32 O_part[num_split_slots][2][128][head_dim] followed by fp32 lse_part[num_split_slots][2][128]

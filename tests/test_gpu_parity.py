@@ -55,6 +55,29 @@ def test_ragged_small(P, C, Hq, Hkv, d, B, tile_m):
     _full_parity(w, opts=wpp.PlanOpts(tile_m, 0, 0, 0))
 
 
+@pytest.mark.parametrize("C,Hq,Hkv,d,B", [
+    ([1, 7, 16], 16, 2, 128, 64),        # eight heads of a KV group packed into one 128-row half
+    ([17, 32, 3], 8, 2, 128, 64),        # four heads per half
+    ([33, 64, 40], 8, 1, 128, 16),       # two heads per half, second half takes the next two
+    ([64, 5], 8, 2, 64, 16),
+    ([20, 50], 6, 1, 128, 64),           # group of six: packs of two
+])
+@pytest.mark.parametrize("splits", [0, 2])
+def test_short_chunks_pack_heads(C, Hq, Hkv, d, B, splits):
+    P = [300, 0, 129][:len(C)]
+    w = W.custom_workload(P, C, Hq, Hkv, d, B, seed=19, spare_pages=4)
+    res, _ = _full_parity(w, opts=wpp.PlanOpts(256, 0, splits, 0))
+    _full_parity(w, opts=wpp.PlanOpts(128, 0, splits, 0))
+
+
+@pytest.mark.parametrize("tile_m,splits,ctas", [(256, 2, 3), (128, 3, 2), (256, 1, 1), (128, 1, 5)])
+def test_many_tiles_per_cta_back_to_back(tile_m, splits, ctas):
+    """Few persistent CTAs walk long tile lists: a tile's first product must not overwrite the accumulator
+    while the previous tile's epilogue (slow for fp32 partials) is still reading it."""
+    w = W.custom_workload([700, 0, 260, 64], [200, 300, 64, 129], 8, 2, 128, 64, seed=23, spare_pages=4)
+    _full_parity(w, opts=wpp.PlanOpts(tile_m, 0, splits, ctas))
+
+
 def test_single_key_is_bit_exact():
     w = W.custom_workload([0], [1], 4, 2, 128, 64, seed=8)
     inp = cpu_inputs(w)

@@ -30,7 +30,7 @@ def parse_plan(plan):
     units = np.frombuffer(raw, dtype=np.int32, count=num_units * 12, offset=off_units).reshape(num_units, 12)
     comb = np.frombuffer(raw, dtype=np.int32, count=num_combine * 8, offset=off_comb).reshape(num_combine, 8)
     keys = ["request", "kv_begin", "kv_end", "split_slot", "row0_a", "row0_b", "rows_a", "rows_b", "head_a",
-            "head_b", "cost", "pad"]
+            "head_b", "cost", "pack"]
     return dict(R=R, num_ctas=num_ctas, tile_m=tile_m, T=T, key_steps=key_steps, flops=flops, slots=num_slots,
                 ws_bytes=ws_bytes, q_off=q_off, cta=cta, comb=comb,
                 units=[dict(zip(keys, u.tolist())) for u in units])
@@ -65,6 +65,8 @@ def test_status_strings():
     ([1000, 5], [700, 300], 3, 1, 256, 2),          # odd group: unpaired tails
     ([0, 0, 0], [64, 0, 128], 8, 2, 256, 7),
     ([130], [64], 4, 2, 256, 2),
+    ([300, 5, 0], [16, 33, 7], 16, 2, 256, 2),      # short chunks: 8, 2 and 8 heads packed per half
+    ([300, 5], [16, 64], 8, 1, 128, 0),
 ])
 def test_plan_covers_every_visible_pair_exactly_once(P, C, Hq, Hkv, tile_m, splits):
     B = 16
@@ -86,18 +88,21 @@ def test_plan_covers_every_visible_pair_exactly_once(P, C, Hq, Hkv, tile_m, spli
             rows, row0, head = u["rows_" + hf], u["row0_" + hf], u["head_" + hf]
             if rows == 0:
                 continue
-            assert 0 < rows <= 128 and row0 + rows <= C[i] and 0 <= head < Hq
-            assert head // G == u["head_a"] // G            # both halves share one KV head
+            pack = u["pack"]
+            assert pack in (1, 2, 4, 8) and 0 < rows <= 128 // pack and row0 + rows <= C[i]
+            assert 0 <= head and head + pack <= Hq
+            assert head // G == (head + pack - 1) // G == u["head_a"] // G      # one KV head per tile
             end = (P[i] + row0 + rows + 127) // 128
             n = max(0, min(u["kv_end"], end) - u["kv_begin"])
             steps_total += n
             any_work |= n > 0
-            for t in range(row0, row0 + rows):
-                last = P[i] + t                              # last visible key
-                lo, hi = u["kv_begin"] * 128, min(u["kv_end"], end) * 128
-                for key in range(lo, min(hi, last + 1)):
-                    k = (i, t, head, key)
-                    cover[k] = cover.get(k, 0) + 1
+            for hd_ in range(head, head + pack):
+                for t in range(row0, row0 + rows):
+                    last = P[i] + t                              # last visible key
+                    lo, hi = u["kv_begin"] * 128, min(u["kv_end"], end) * 128
+                    for key in range(lo, min(hi, last + 1)):
+                        k = (i, t, hd_, key)
+                        cover[k] = cover.get(k, 0) + 1
         assert any_work, "a tile with nothing to compute"
     assert steps_total == pl["key_steps"]
     want = sum(Hq * (c * p + c * (c + 1) // 2) for p, c in zip(P, C))
@@ -107,12 +112,13 @@ def test_plan_covers_every_visible_pair_exactly_once(P, C, Hq, Hkv, tile_m, spli
     by_slot = {u["split_slot"]: u for u in pl["units"] if u["split_slot"] >= 0}
     assert len(by_slot) == pl["slots"]
     for c in pl["comb"]:
-        req, row0, rows, head, slot0, ns, half, _ = c.tolist()
+        req, row0, rows, head, slot0, ns, half, lane0 = c.tolist()
         parts = [by_slot[s] for s in range(slot0, slot0 + ns)]
         assert parts[0]["kv_begin"] == 0 and all(a["kv_end"] == b["kv_begin"] for a, b in zip(parts, parts[1:]))
         hf = "ab"[half]
         assert all(p_["request"] == req and p_["row0_" + hf] == row0 and p_["rows_" + hf] == rows and
-                   p_["head_" + hf] == head for p_ in parts)
+                   p_["head_" + hf] + lane0 // (128 // p_["pack"]) == head and lane0 % (128 // p_["pack"]) == 0
+                   for p_ in parts)
         assert parts[-1]["kv_end"] >= (P[req] + row0 + rows + 127) // 128
     if splits >= 2 and max((p + c + 127) // 128 for p, c in zip(P, C)) >= 2:
         assert pl["slots"] > 0 and pl["ws_bytes"] >= pl["slots"] * 2 * 128 * 129 * 4
@@ -135,12 +141,20 @@ def test_plan_is_deterministic_and_balanced():
         assert costs == sorted(costs, reverse=True)
 
 
-def test_short_tails_pair_two_heads_of_one_kv_group():
-    d = desc(1, 8, 2, 128, 64, 10)
+def test_short_row_blocks_pack_heads_of_one_kv_group():
+    d = desc(1, 8, 2, 128, 64, 10)                  # G = 4
     pl = parse_plan(wpp.wpp_plan_tiles(None, d, [0], [300], opts=wpp.PlanOpts(256, 0, 1, 148), pin=False))
-    tails = [u for u in pl["units"] if u["row0_a"] == 256]
-    assert len(tails) == 4 and all(u["rows_a"] == 44 and u["rows_b"] == 44 and u["row0_b"] == 256 and
-                                   u["head_b"] == u["head_a"] + 1 for u in tails)
+    tails = [u for u in pl["units"] if u["row0_a"] == 256]          # 44 rows: two heads per half, four per tile
+    assert len(tails) == 2 and all(u["pack"] == 2 and u["rows_a"] == 44 and u["rows_b"] == 44 and
+                                   u["row0_b"] == 256 and u["head_b"] == u["head_a"] + 2 for u in tails)
+    full = [u for u in pl["units"] if u["row0_a"] == 0]
+    assert len(full) == 8 and all(u["pack"] == 1 and u["rows_b"] == 128 and u["row0_b"] == 128 for u in full)
+    d8 = desc(1, 16, 2, 128, 64, 10)                # G = 8, a 10-row chunk: all 8 heads of a group in one half
+    pl8 = parse_plan(wpp.wpp_plan_tiles(None, d8, [70], [10], opts=wpp.PlanOpts(256, 0, 1, 148), pin=False))
+    assert [(u["pack"], u["head_a"], u["rows_b"]) for u in pl8["units"]] == [(8, 0, 0), (8, 8, 0)]
+    d100 = desc(1, 8, 2, 128, 64, 10)               # 100 rows do not fit twice into 128: one head per half
+    pl100 = parse_plan(wpp.wpp_plan_tiles(None, d100, [0], [100], opts=wpp.PlanOpts(256, 0, 1, 148), pin=False))
+    assert all(u["pack"] == 1 and u["head_b"] == u["head_a"] + 1 for u in pl100["units"]) and len(pl100["units"]) == 4
 
 
 def test_few_tiles_fall_back_to_128_row_tiles_and_split_keys():
