@@ -405,7 +405,7 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         const int r = threadIdx.x & 127;
         const uint32_t lane_addr = tmem + ((uint32_t)((warp & 3) * 32) << 16);
         const uint32_t colS = col_s(hf);
-        uint32_t s_phase = 0;
+        uint32_t s_phase = 0, fin_phase = 0;
         int tstep = 0;      // steps since kernel start (trace index only)
         (void)tstep;
         const float c = p.scale_log2;
@@ -531,6 +531,13 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 ++tstep;
             }
             if (dead) break;
+            {
+                // the end-of-tile slot (and its barrier) may only be reused once the epilogue threads have consumed
+                // the previous tile's values; for tiles of a single key step nothing else orders the two
+                const bool ok = mbar_wait(bOFree(hf), fin_phase ^ 1u, abort_flag);
+                if (!__all_sync(0xffffffffu, ok)) break;
+                fin_phase ^= 1u;
+            }
             s_final[hf * 128 + r] = make_float2(-nmc, l_run);
             mbar_arrive(bFinalReady(hf));
         }

@@ -78,6 +78,20 @@ def test_many_tiles_per_cta_back_to_back(tile_m, splits, ctas):
     _full_parity(w, opts=wpp.PlanOpts(tile_m, 0, splits, ctas))
 
 
+@pytest.mark.parametrize("ctas", [1, 2, 7])
+def test_single_step_tiles_back_to_back(ctas):
+    """Tiles of one key step, many per CTA: the softmax warps could finish tile k+1 before the epilogue has
+    consumed tile k's end-of-tile values; the hand-over must hold them back (repeated to catch a race)."""
+    w = W.custom_workload([0, 0, 10, 0, 60, 0], [64, 128, 100, 33, 68, 1], 16, 2, 128, 64, seed=24, spare_pages=4)
+    inp = cpu_inputs(w)
+    _, _, ref, _ = run_oracle(w, inp)
+    first = None
+    for rep in range(6):
+        res = H.run_wave(w, H.device_inputs(w, inp), opts=wpp.PlanOpts(256 if rep % 2 else 128, 0, 1, ctas))
+        assert res["status"] == 0
+        H.assert_close(f64(res["out"]), ref, f"single-step tiles, {ctas} CTAs, repeat {rep}")
+
+
 def test_single_key_is_bit_exact():
     w = W.custom_workload([0], [1], 4, 2, 128, 64, seed=8)
     inp = cpu_inputs(w)
