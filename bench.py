@@ -30,7 +30,7 @@ sys.path.insert(0, ROOT)
 
 METRIC = "prefill-attention tokens/s at concurrency 128, high prefix reuse"
 # From profiles/attention_cfg3_r16_ncu.md: (dram read + write bytes) / key steps of the captured launch.
-DRAM_BYTES_PER_KEY_STEP = 2786.0
+DRAM_BYTES_PER_KEY_STEP = 3966.0
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
