@@ -29,8 +29,10 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
 METRIC = "prefill-attention tokens/s at concurrency 128, high prefix reuse"
-# From profiles/attention_cfg3_r16_ncu.md: (dram read + write bytes) / key steps of the captured launch.
-DRAM_BYTES_PER_KEY_STEP = 3966.0
+# From profiles/attention_cfg3_dram.md: dram__bytes_read.sum + dram__bytes_write.sum of one attention launch on the
+# full concurrency-128 workload (a one-pass ncu capture) / its 18,943,680 key steps.  Exact for that workload;
+# for other --config values the product with their key steps is only an estimate.
+DRAM_BYTES_PER_KEY_STEP = 1177.7
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -194,6 +196,7 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--force-kv-splits", type=int, default=0)
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
+    ap.add_argument("--plan-order", type=int, default=0, help="0: stream order (default), 1: longest tile first")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "native" else args.warmup
 
@@ -217,7 +220,7 @@ def main():
     ctx = wpp.Context(local_rank)
     desc = wpp.make_desc(w.num_requests, w.num_q_heads, w.num_kv_heads, w.head_dim, w.page_size,
                          w.max_blocks_per_req, w.num_pages)
-    opts = wpp.PlanOpts(0, 0, args.force_kv_splits, 0)
+    opts = wpp.PlanOpts(0, 0, args.force_kv_splits, 0, args.plan_order)
     T = w.total_new_tokens
 
     # ---- resident state and inputs on the device
@@ -292,9 +295,8 @@ def main():
     qo_bytes = 2 * T * w.num_q_heads * w.head_dim * 2
     t_flops = flops / (roof_peak * 1e12)
     t_bytes = (kv_bytes + qo_bytes) / (float(peaks.get("hbm_gbs", FALLBACK_PEAKS["hbm_gbs"])) * 1e9)
-    # DRAM bytes of one launch: dram__bytes_read.sum + dram__bytes_write.sum from the ncu capture summarised in
-    # profiles/ (taken on the 16-request cut of this workload, the full one being too large to capture), scaled
-    # by the 128x128 key steps a launch processes
+    # DRAM bytes of one launch: dram__bytes_read.sum + dram__bytes_write.sum from the one-pass ncu capture
+    # summarised in profiles/, per 128x128 key step, times the key steps this launch processes
     traffic = DRAM_BYTES_PER_KEY_STEP * float(info.key_steps) if DRAM_BYTES_PER_KEY_STEP else None
     roofline = {"bound": "tensor" if t_flops >= t_bytes else "hbm", "kernel": "wpp_attn_kernel",
                 "achieved": achieved, "peak": roof_peak, "unit": "TFLOP/s", "frac": achieved / roof_peak,

@@ -97,6 +97,9 @@ typedef struct {
     int32_t force_kv_splits;  /* >= 2: split every tile's key range into this many parts (when it has that many
                                  key steps); 1: never split; 0: library decides */
     int32_t max_ctas;         /* persistent CTAs to plan for (default: SM count of the context, 148 without one) */
+    int32_t order;            /* 0: stream order - tiles that read the same (request, KV head) pages run at the same
+                                 time, so the pages are fetched from DRAM once and shared through L2; 1: longest
+                                 tile first */
 } wpp_plan_opts;
 
 typedef struct {
@@ -118,7 +121,7 @@ size_t wpp_plan_bytes(const wpp_ctx* ctx_or_null, const wpp_batch_desc* desc, in
 
 /* Host-side work split (integer arithmetic only; no CUDA call).  Cuts the wave into work tiles
  * (request, query-row range, query head, key-step range), decides which tiles are split along the keys,
- * assigns tiles to persistent CTAs in decreasing-cost order, and sizes the workspace.  Equal-sized chunks
+ * orders them (opts->order) and list-schedules them onto persistent CTAs, and sizes the workspace.  Equal-sized chunks
  * cost different amounts because they attend to different prefix lengths (Section 6), hence cost = key steps.
  *   prefix_lens_host, chunk_lens_host : host int32 [R].
  *   cached_lens_host_or_null          : host int32 [R]; tokens each request really has in the cache after

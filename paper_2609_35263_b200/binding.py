@@ -46,7 +46,7 @@ class BatchDesc(ctypes.Structure):
 
 class PlanOpts(ctypes.Structure):
     _fields_ = [("tile_m", ctypes.c_int32), ("tile_n", ctypes.c_int32), ("force_kv_splits", ctypes.c_int32),
-                ("max_ctas", ctypes.c_int32)]
+                ("max_ctas", ctypes.c_int32), ("order", ctypes.c_int32)]
 
 
 class PlanInfo(ctypes.Structure):

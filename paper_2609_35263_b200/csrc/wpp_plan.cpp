@@ -77,7 +77,7 @@ uint64_t wpp_desc_hash(const wpp_batch_desc* d) {
 static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 static int resolve_opts(const wpp_ctx* ctx, const wpp_plan_opts* in, wpp_plan_opts* o) {
-    wpp_plan_opts z = {0, 0, 0, 0};
+    wpp_plan_opts z = {0, 0, 0, 0, 0};
     *o = in ? *in : z;
     if (!o->tile_m) o->tile_m = WPP_DEFAULT_TILE_M;
     if (!o->tile_n) o->tile_n = WPP_TILE_N;
@@ -85,7 +85,8 @@ static int resolve_opts(const wpp_ctx* ctx, const wpp_plan_opts* in, wpp_plan_op
     if (o->tile_m != 128 && o->tile_m != 256) return WPP_ERR_UNSUPPORTED;
     if (o->tile_m > WPP_MAX_TILE_M) return WPP_ERR_UNSUPPORTED;
     if (o->tile_n != WPP_TILE_N) return WPP_ERR_UNSUPPORTED;
-    if (o->force_kv_splits < 0 || o->force_kv_splits > 64 || o->max_ctas < 1 || o->max_ctas > 4096)
+    if (o->force_kv_splits < 0 || o->force_kv_splits > 64 || o->max_ctas < 1 || o->max_ctas > 4096 ||
+        o->order < 0 || o->order > 1)
         return WPP_ERR_INVALID_ARG;
     return WPP_OK;
 }
@@ -236,12 +237,38 @@ int wpp_plan_tiles(const wpp_ctx* ctx, const wpp_batch_desc* desc, const int32_t
     const int64_t n_units = (int64_t)units.size();
     if (n_units > 0x7fffffff) return WPP_ERR_INVALID_ARG;
 
-    // ---- longest-processing-time assignment to persistent CTAs; stable sort keeps neighbours adjacent
+    // ---- order of execution, then list scheduling onto persistent CTAs (each tile goes to the CTA that is
+    //      free first, so tiles adjacent in the order run at the same time on different SMs).
+    //      order 0 (default), "stream order": KV head major, then requests (longest first), then row blocks and
+    //      heads.  All tiles that read one (request, KV head) stream start together and walk its pages in step,
+    //      so a page comes from DRAM once and is then hit in L2 by the other tiles; a prefix shared by many
+    //      requests stays L2-resident while its KV head is being worked on.
+    //      order 1: longest tile first (best balance, no regard for which tiles run together).
     const int num_ctas = (int)std::max<int64_t>(1, std::min<int64_t>(o.max_ctas, n_units));
     std::vector<int32_t> order((size_t)n_units);
     for (int64_t u = 0; u < n_units; ++u) order[(size_t)u] = (int32_t)u;
-    std::stable_sort(order.begin(), order.end(),
-                     [&](int32_t a, int32_t b) { return units[(size_t)a].cost > units[(size_t)b].cost; });
+    if (o.order == 1) {
+        std::stable_sort(order.begin(), order.end(),
+                         [&](int32_t a, int32_t b) { return units[(size_t)a].cost > units[(size_t)b].cost; });
+    } else {
+        std::vector<int64_t> req_cost((size_t)std::max(R, 1), 0);
+        for (const WppUnit& u : units) req_cost[(size_t)u.request] += u.cost;
+        std::vector<int32_t> req_rank((size_t)std::max(R, 1));
+        {
+            std::vector<int32_t> by_cost((size_t)R);
+            for (int i = 0; i < R; ++i) by_cost[(size_t)i] = i;
+            std::stable_sort(by_cost.begin(), by_cost.end(),
+                             [&](int32_t a, int32_t b) { return req_cost[(size_t)a] > req_cost[(size_t)b]; });
+            for (int i = 0; i < R; ++i) req_rank[(size_t)by_cost[(size_t)i]] = i;
+        }
+        std::stable_sort(order.begin(), order.end(), [&](int32_t a, int32_t b) {
+            const WppUnit& ua = units[(size_t)a];
+            const WppUnit& ub = units[(size_t)b];
+            const int ka = ua.head[0] / G, kb = ub.head[0] / G;
+            if (ka != kb) return ka < kb;
+            return req_rank[(size_t)ua.request] < req_rank[(size_t)ub.request];
+        });
+    }
     typedef std::pair<int64_t, int32_t> Load;  // (accumulated cost, cta)
     std::priority_queue<Load, std::vector<Load>, std::greater<Load>> heap;
     for (int c = 0; c < num_ctas; ++c) heap.push({0, c});

@@ -129,16 +129,32 @@ def test_plan_is_deterministic_and_balanced():
     P = (rng.integers(0, 100, 24) * 64).tolist()
     C = rng.integers(1, 2000, 24).tolist()
     d = desc(24, 16, 4, 128, 64, 200)
-    a = wpp.wpp_plan_tiles(None, d, P, C, pin=False)
-    b = wpp.wpp_plan_tiles(None, d, P, C, pin=False)
-    assert a.host_bytes() == b.host_bytes()
-    pl = parse_plan(a)
-    loads = [sum(u["cost"] for u in pl["units"][pl["cta"][c]:pl["cta"][c + 1]]) for c in range(pl["num_ctas"])]
-    biggest = max(u["cost"] for u in pl["units"])
-    assert max(loads) - min(loads) <= biggest          # longest-processing-time bound
-    for c in range(pl["num_ctas"]):                    # each CTA walks its tiles in decreasing cost
-        costs = [u["cost"] for u in pl["units"][pl["cta"][c]:pl["cta"][c + 1]]]
-        assert costs == sorted(costs, reverse=True)
+    for order in (0, 1):
+        opts = wpp.PlanOpts(0, 0, 0, 0, order)
+        a = wpp.wpp_plan_tiles(None, d, P, C, opts=opts, pin=False)
+        b = wpp.wpp_plan_tiles(None, d, P, C, opts=opts, pin=False)
+        assert a.host_bytes() == b.host_bytes()
+        pl = parse_plan(a)
+        loads = [sum(u["cost"] for u in pl["units"][pl["cta"][c]:pl["cta"][c + 1]]) for c in range(pl["num_ctas"])]
+        biggest = max(u["cost"] for u in pl["units"])
+        assert max(loads) - min(loads) <= biggest          # list scheduling: nobody idles longer than one tile
+        for c in range(pl["num_ctas"]):
+            mine = pl["units"][pl["cta"][c]:pl["cta"][c + 1]]
+            if order == 1:                                 # longest first: each CTA walks decreasing costs
+                costs = [u["cost"] for u in mine]
+                assert costs == sorted(costs, reverse=True)
+            else:                                          # stream order: KV heads never go backwards on a CTA
+                kv = [u["head_a"] // 4 for u in mine]
+                assert kv == sorted(kv)
+
+
+def test_stream_order_runs_the_tiles_of_one_kv_stream_together():
+    d = desc(3, 16, 4, 128, 64, 200)
+    pl = parse_plan(wpp.wpp_plan_tiles(None, d, [4096, 0, 8192], [1024, 512, 256], opts=wpp.PlanOpts(256, 0, 1, 8),
+                                       pin=False))
+    # the first tile of every CTA belongs to KV head 0 of the costliest request (request 0: 4 row blocks x 4 heads)
+    firsts = [pl["units"][pl["cta"][c]] for c in range(pl["num_ctas"])]
+    assert all(u["request"] == 0 and u["head_a"] // 4 == 0 for u in firsts)
 
 
 def test_short_row_blocks_pack_heads_of_one_kv_group():
