@@ -307,37 +307,78 @@ def main():
     # ---- end to end through host buffers
     e2e = None
     if not args.no_e2e:
-        qh, knh, vnh = [torch.empty(x.shape, dtype=x.dtype).pin_memory() for x in (q, k_new, v_new)]
-        qh.copy_(q); knh.copy_(k_new); vnh.copy_(v_new)
-        out_h = torch.empty(out.shape, dtype=out.dtype).pin_memory()
-        qd2, knd2, vnd2 = torch.empty_like(q), torch.empty_like(k_new), torch.empty_like(v_new)
-        bt2, P2, C2 = torch.empty_like(bt), torch.empty_like(P), torch.empty_like(C)
-        h2d = sum(x.numel() * x.element_size() for x in (qh, knh, vnh, bt_h, P_h, C_h)) + int(info.plan_bytes)
-        d2h = out_h.numel() * out_h.element_size()
+        # Host buffers in, host buffer out, every step: q / k_new / v_new / block tables / lengths come from pinned
+        # host memory and `out` goes back to pinned host memory.  The C ABI takes the stream to work on, so a
+        # caller pipelines the three phases on three streams with two sets of device buffers: while wave i runs,
+        # wave i+1's inputs are on their way in and wave i-1's output on its way out.
+        hb = dict(q=q, k_new=k_new, v_new=v_new)
+        host_in = {k: torch.empty(v.shape, dtype=v.dtype).pin_memory() for k, v in hb.items()}
+        for k in hb:
+            host_in[k].copy_(hb[k])
+        out_h = [torch.empty(out.shape, dtype=out.dtype).pin_memory() for _ in range(2)]
+        dev_in = [{k: torch.empty_like(v) for k, v in hb.items()} for _ in range(2)]
+        dev_meta = [(torch.empty_like(bt), torch.empty_like(P), torch.empty_like(C)) for _ in range(2)]
+        dev_out = [out, torch.empty_like(out)]
+        h2d = sum(x.numel() * x.element_size() for x in list(host_in.values()) + [bt_h, P_h, C_h]) + int(info.plan_bytes)
+        d2h = out.numel() * out.element_size()
+        s_in, s_run, s_out = torch.cuda.Stream(), torch.cuda.Stream(), torch.cuda.Stream()
+        in_done = [torch.cuda.Event() for _ in range(2)]
+        run_done = [torch.cuda.Event() for _ in range(2)]
+        out_done = [torch.cuda.Event() for _ in range(2)]
 
         def e2e_step(i):
-            qd2.copy_(qh, non_blocking=True); knd2.copy_(knh, non_blocking=True); vnd2.copy_(vnh, non_blocking=True)
-            bt2.copy_(bt_h, non_blocking=True); P2.copy_(P_h, non_blocking=True); C2.copy_(C_h, non_blocking=True)
-            one_step(i, None, qd2, knd2, vnd2, bt2, P2, C2)
-            out_h.copy_(out, non_blocking=True)
+            b2 = i % 2
+            with torch.cuda.stream(s_in):
+                s_in.wait_event(run_done[b2])            # wave i-2 no longer reads this input set
+                for k in hb:
+                    dev_in[b2][k].copy_(host_in[k], non_blocking=True)
+                for dst, src in zip(dev_meta[b2], (bt_h, P_h, C_h)):
+                    dst.copy_(src, non_blocking=True)
+                in_done[b2].record(s_in)
+            with torch.cuda.stream(s_run):
+                s_run.wait_event(in_done[b2])
+                s_run.wait_event(out_done[b2])           # wave i-2's output has left this output buffer
+                sl = i % ring
+                plan_free[sl].synchronize()
+                plan = wpp.wpp_plan_tiles(ctx, desc, w.prefix_lens, w.chunk_lens, opts=opts, out=plan_host[sl])
+                plan.to_device(out=plan_dev[sl])
+                plan_free[sl].record(s_run)
+                btd, Pd, Cd = dev_meta[b2]
+                wpp.wpp_kv_append(ctx, desc, dev_in[b2]["k_new"], dev_in[b2]["v_new"], k_pool, v_pool, btd, Pd, Cd,
+                                  plan, status=status, stream=s_run)
+                wpp.wpp_prefill_attention_varlen(ctx, desc, dev_in[b2]["q"], dev_out[b2], None, k_pool, v_pool, btd,
+                                                 Pd, Cd, plan, workspace=ws, status=status, stream=s_run)
+                run_done[b2].record(s_run)
+            with torch.cuda.stream(s_out):
+                s_out.wait_event(run_done[b2])
+                out_h[b2].copy_(dev_out[b2], non_blocking=True)
+                out_done[b2].record(s_out)
 
-        e2e_steps = max(1, min(args.steps, 5))
-        e2e_step(0)
+        e2e_steps = max(2, min(args.steps, 6))
+        for i in range(2):
+            e2e_step(i)
         barrier()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record(stream)
+        e0.record(s_in)
         for i in range(e2e_steps):
-            e2e_step(1 + i)
-        e1.record(stream)
+            e2e_step(2 + i)
+        s_out.wait_stream(s_run)
+        s_out.wait_stream(s_in)
+        e1.record(s_out)
         barrier()
         e2e_ms = max_over_ranks(e0.elapsed_time(e1) / e2e_steps)
+        if int(status.item()) != 0:
+            raise SystemExit(f"device status {int(status.item())} after the end-to-end region")
         e2e = {"value": world * T / (e2e_ms * 1e-3), "unit": "tokens/s", "h2d_bytes_per_step": int(h2d),
-               "d2h_bytes_per_step": int(d2h), "ms_per_step": e2e_ms, "steps": e2e_steps}
-        del qh, knh, vnh, out_h, qd2, knd2, vnd2
+               "d2h_bytes_per_step": int(d2h), "ms_per_step": e2e_ms, "steps": e2e_steps,
+               "how": "pinned host buffers; H2D, the C-ABI calls and D2H on three streams, two device buffer sets"}
+        del host_in, out_h, dev_in, dev_out
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         del q, k_new, v_new, k_pool, v_pool, out
+        if not args.no_e2e:
+            del hb
         torch.cuda.empty_cache()
         cpu = OracleSampler(w, True).sample(args.cpu_seconds)
 
