@@ -200,6 +200,13 @@ int wpp_prefill_attention_varlen_static(const wpp_ctx* ctx, const wpp_batch_desc
 /* Size in bytes of the built-in scratch array used by wpp_prefill_attention_varlen_static. */
 size_t wpp_static_scratch_bytes(void);
 
+/* Self-test of the bounded waits the kernels rely on (no counterpart in the paper): launches one warp that waits,
+ * for at most limit_cycles SM clocks (1 .. 2^30), on a barrier nothing ever arrives on.  The wait gives up, the
+ * kernel ends normally, *status_dev becomes WPP_ERR_TIMEOUT (if it was 0) and *waited_cycles_dev (device int64,
+ * may be NULL) receives how long the warp waited.  Nothing hangs or traps; the context stays usable. */
+int wpp_selftest_bounded_wait(const wpp_ctx* ctx, int64_t limit_cycles, int32_t* status_dev,
+                              int64_t* waited_cycles_dev, void* cuda_stream);
+
 /* Number of kernels the library has launched through this context so far (for launch accounting). */
 int64_t wpp_launch_count(const wpp_ctx* ctx);
 

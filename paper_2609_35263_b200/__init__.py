@@ -12,6 +12,7 @@ from .binding import (  # noqa: F401
     wpp_plan_tiles,
     wpp_prefill_attention_varlen,
     wpp_prefill_attention_varlen_static,
+    wpp_selftest_bounded_wait,
     wpp_static_scratch_bytes,
     wpp_validate_batch,
 )

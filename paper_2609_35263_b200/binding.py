@@ -58,7 +58,8 @@ class PlanInfo(ctypes.Structure):
 
 EXPORTS = ["wpp_create", "wpp_destroy", "wpp_status_string", "wpp_last_cuda_error", "wpp_plan_bytes",
            "wpp_plan_tiles", "wpp_validate_batch", "wpp_kv_append", "wpp_prefill_attention_varlen",
-           "wpp_launch_count", "wpp_prefill_attention_varlen_static", "wpp_static_scratch_bytes"]
+           "wpp_launch_count", "wpp_prefill_attention_varlen_static", "wpp_static_scratch_bytes",
+           "wpp_selftest_bounded_wait"]
 
 _lib = None
 
@@ -90,6 +91,7 @@ def load_library() -> ctypes.CDLL:
                                                      i32p, vp, vp, vp, ctypes.c_size_t, i32p, vp]
         lib.wpp_prefill_attention_varlen_static.argtypes = [vp, ctypes.POINTER(BatchDesc), vp, vp, vp, vp, vp, i32p,
                                                             i32p, i32p, vp, vp, i32p, vp]
+        lib.wpp_selftest_bounded_wait.argtypes = [vp, ctypes.c_int64, i32p, vp, vp]
         lib.wpp_static_scratch_bytes.restype = ctypes.c_size_t
         lib.wpp_static_scratch_bytes.argtypes = []
         _lib = lib
@@ -259,3 +261,10 @@ def wpp_prefill_attention_varlen_static(ctx: Context, desc: BatchDesc, q, out, l
         _ptr(block_tables), _ptr(prefix_lens), _ptr(chunk_lens), ctypes.c_void_p(plan.host.data_ptr()),
         _ptr(plan.dev), _ptr(status), _stream(stream))
     _check(st, "wpp_prefill_attention_varlen_static")
+
+
+def wpp_selftest_bounded_wait(ctx: Context, limit_cycles: int, status, waited_cycles=None, stream=None) -> None:
+    """Launch the bounded-wait self-test: a warp waits at most `limit_cycles` on a barrier nothing arrives on."""
+    st = load_library().wpp_selftest_bounded_wait(ctx.handle, int(limit_cycles), _ptr(status), _ptr(waited_cycles),
+                                                  _stream(stream))
+    _check(st, "wpp_selftest_bounded_wait")

@@ -66,6 +66,16 @@ extern "C" int wpp_destroy(wpp_ctx* ctx) {
 extern "C" int wpp_last_cuda_error(const wpp_ctx* ctx) { return ctx ? ctx->last_cuda_error : 0; }
 extern "C" int64_t wpp_launch_count(const wpp_ctx* ctx) { return ctx ? ctx->launches : 0; }
 
+extern "C" int wpp_selftest_bounded_wait(const wpp_ctx* ctx, int64_t limit_cycles, int32_t* status_dev,
+                                         int64_t* waited_cycles_dev, void* cuda_stream) {
+    if (!ctx || !status_dev || limit_cycles < 1 || limit_cycles > (1ll << 30)) return WPP_ERR_INVALID_ARG;
+    int e = wpp_launch_selftest_wait((long long)limit_cycles, status_dev,
+                                     reinterpret_cast<long long*>(waited_cycles_dev), cuda_stream);
+    if (e != 0) return cuda_fail(ctx, e);
+    const_cast<wpp_ctx*>(ctx)->launches += 1;
+    return WPP_OK;
+}
+
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
 
 // bf16 tensor map with 128-byte swizzle; dims/strides innermost first, strides in bytes for dims 1..rank-1

@@ -5,6 +5,7 @@
 
 #include "wpp_device.h"
 #include "wpp_plan_format.h"
+#include "wpp_ptx.cuh"
 
 namespace wpp {
 
@@ -77,7 +78,35 @@ __global__ void __launch_bounds__(256) wpp_combine_kernel(const CombineParams p)
     }
 }
 
+// Self-test of the bounded wait every kernel of the library relies on: one warp waits, with a short limit, on
+// a barrier that nothing ever arrives on.  The wait must give up, raise the abort flag and let the kernel end
+// normally with WPP_ERR_TIMEOUT in the status word - it never hangs and never traps.
+__global__ void wpp_selftest_wait_kernel(long long limit_cycles, int32_t* status, long long* waited_cycles) {
+    __shared__ uint64_t bar;
+    __shared__ uint32_t abort_flag;
+    const uint32_t b = smem_u32(&bar);
+    if (threadIdx.x == 0) {
+        mbar_init(b, 1);
+        abort_flag = 0u;
+        fence_barrier_init();
+    }
+    __syncthreads();
+    const long long t0 = clock64();
+    const bool ok = mbar_wait_limit(b, 0, &abort_flag, limit_cycles);
+    const long long t1 = clock64();
+    if (!__all_sync(0xffffffffu, ok) && threadIdx.x == 0) {
+        if (status) atomicCAS(status, 0, WPP_ERR_TIMEOUT);
+        if (waited_cycles) *waited_cycles = t1 - t0;
+    }
+}
+
 }  // namespace wpp
+
+extern "C" int wpp_launch_selftest_wait(long long limit_cycles, int32_t* status, long long* waited_cycles,
+                                        void* stream) {
+    wpp::wpp_selftest_wait_kernel<<<1, 32, 0, (cudaStream_t)stream>>>(limit_cycles, status, waited_cycles);
+    return (int)cudaGetLastError();
+}
 
 extern "C" int wpp_launch_append(const wpp::AppendParams* p, int num_sms, void* stream) {
     const int64_t total = p->total_new_tokens * p->num_kv_heads * p->vec_per_row;

@@ -43,7 +43,8 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
 #ifndef WPP_WAIT_LIMIT
 #define WPP_WAIT_LIMIT (1ll << 30)
 #endif
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag) {
+__device__ __forceinline__ bool mbar_wait_limit(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
+                                                long long limit_cycles) {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     uint32_t n = 0;
@@ -51,12 +52,15 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
         if (mbar_try_wait(bar, parity)) return true;
         if ((++n & 31u) == 0u) {
             if (*abort_flag) return false;
-            if (clock64() - t0 > WPP_WAIT_LIMIT) {
+            if (clock64() - t0 > limit_cycles) {
                 *abort_flag = 1u;
                 return false;
             }
         }
     }
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag) {
+    return mbar_wait_limit(bar, parity, abort_flag, WPP_WAIT_LIMIT);
 }
 
 // generic-proxy writes to shared memory -> visible to the async proxy (TMA, tensor cores)

@@ -183,6 +183,20 @@ def test_successive_chunks_on_one_stream_equal_one_shot():
     H.assert_close(np.concatenate(outs), ref, "successive chunks")
 
 
+def test_a_wait_that_runs_out_reports_timeout_and_leaves_the_context_usable():
+    """Every device-side wait is bounded: a barrier nothing arrives on makes the wait give up after its limit,
+    the kernel ends normally and the status word says WPP_ERR_TIMEOUT (no hang, no trap)."""
+    c = H.ctx()
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    waited = torch.zeros(1, dtype=torch.int64, device="cuda")
+    limit = 2_000_000                                    # about a millisecond of SM clocks
+    wpp.wpp_selftest_bounded_wait(c, limit, status, waited)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 8                       # WPP_ERR_TIMEOUT
+    assert limit < int(waited.item()) < 50 * limit
+    _full_parity(W.custom_workload([64], [64], 2, 1, 128, 64, seed=17))      # the context still works
+
+
 def test_bad_page_id_sets_status_without_trapping():
     w = W.custom_workload([64], [64], 2, 1, 128, 64, seed=17)
     w.block_tables = w.block_tables.copy()
