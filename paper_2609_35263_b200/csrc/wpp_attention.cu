@@ -278,9 +278,10 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 mma_commit(bItemEmpty + 8 * ring.stage);
                 if (v.n_steps == 1) mma_commit(bQEmpty);
                 ring.advance(C::kItems);
+                bool have_item = false;      // the item of the coming iteration has already been waited for
                 for (int j = 0; j < v.n_steps; ++j) {
                     // item {V(j), K(j+1)}
-                    if (!mbar_wait(bItemFull + 8 * ring.stage, ring.phase, abort_flag)) { dead = true; break; }
+                    if (!have_item && !mbar_wait(bItemFull + 8 * ring.stage, ring.phase, abort_flag)) { dead = true; break; }
                     const uint32_t item = ring.stage;
                     const int valid = v.kv_len - (v.kv_begin + j) * 128;      // keys of this step that exist
                     if (valid < 128) {
@@ -314,6 +315,17 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                         if (j + 1 < v.n[hf]) issue_qk(hf, item);      // its commit also covers the O += P V above
                         else mma_commit(bOFinal(hf));
                         TRACE(2, tstep, hf * 4 + 3);
+                        if (hf == 0) {
+                            // look at the next item now, while the tensor pipe still has half A's work queued,
+                            // instead of at the top of the next iteration when it has run dry
+                            have_item = false;
+                            if (j + 1 < v.n_steps) {
+                                Ring nxt = ring;
+                                nxt.advance(C::kItems);
+                                if (!mbar_wait(bItemFull + 8 * nxt.stage, nxt.phase, abort_flag)) { dead = true; break; }
+                                have_item = true;
+                            }
+                        }
                     }
                     if (dead) break;
                     mma_commit(bItemEmpty + 8 * item);
