@@ -6,9 +6,10 @@
 //   warps 0-3   softmax of half A: thread r owns query row r (TMEM lane r): row max / row sum need no shuffles
 //   warps 4-7   softmax of half B
 //   warps 8-11  epilogue: O / l -> bf16 -> global (or fp32 partials for split tiles), overlapping the next tile
-//   warp 12     tensor-core issuer (one thread): S = Q K^T and O += P V with tcgen05.mma (fp32 accumulators in
-//               TMEM; P is read from TMEM where the softmax warps wrote it as packed bf16 over S; V is an MN-major
-//               operand).  It alternates A and B, which keeps the two halves in anti-phase.
+//   warps 12,14 tensor-core issuers, one thread per half: S = Q K^T and O += P V with tcgen05.mma (fp32 accumulators
+//               in TMEM; P is read from TMEM where the softmax warps wrote it as packed bf16 over S; V is an
+//               MN-major operand).  They issue strictly in turns (A, B, A, ...), which keeps the halves in anti-phase
+//               while one half's barrier waits never hold up the other half's MMAs.
 //   warp 13     producer: reads the block table and issues TMA tile loads (Q once per tile; per key step one box
 //               per (page, 64-wide half of head_dim) for K and for V, 128-byte swizzle).  V(j) and K(j+1) are used
 //               in the same issuer iteration, so they travel as one ring item with one barrier.
@@ -128,18 +129,20 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     float2* s_final = reinterpret_cast<float2*>(smem_gen + C::kOffFinal);     // [2][128] (reference in log2 units, l)
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_gen + C::kOffMisc);
     volatile uint32_t* abort_flag = tmem_slot + 1;
+    volatile uint32_t* turn = tmem_slot + 2;             // which half's issuer may issue next
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int wg = warp >> 2;
 
     if (threadIdx.x == 0) {
-        mbar_init(bQFull, 1); mbar_init(bQEmpty, 1);
-        for (int s = 0; s < C::kItems; ++s) { mbar_init(bItemFull + 8 * s, 1); mbar_init(bItemEmpty + 8 * s, 1); }
+        mbar_init(bQFull, 1); mbar_init(bQEmpty, 2);
+        for (int s = 0; s < C::kItems; ++s) { mbar_init(bItemFull + 8 * s, 1); mbar_init(bItemEmpty + 8 * s, 2); }
         for (int h = 0; h < 2; ++h) {
             mbar_init(bSFull(h), 1); mbar_init(bPReady(h), 128);
             mbar_init(bFinalReady(h), 128); mbar_init(bOFinal(h), 1); mbar_init(bOFree(h), 128);
         }
         *abort_flag = 0u;
+        *turn = 0u;
         fence_barrier_init();
     }
     if (warp == 12) {
@@ -237,99 +240,106 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 for (int j = 0; j < v.n_steps; ++j)
                     if (!load_item(j, j + 1)) { dead = true; break; }
             }
-        } else if (warp == 12 && lane == 0) {
-            // ================================================================ tensor-core issuer (one thread)
-            // It alternates the halves (A: O += P V, next S; then B), which keeps their softmax phases apart:
-            // while the softmax warps of A own the special-function units, the tensor pipe works for B.  (Two
-            // independent issuers were measured: the halves then drift into phase, both softmaxes share the
-            // exp units and the dependency chain of each half gets longer.)
+        } else if ((warp == 12 || warp == 14) && lane == 0) {
+            // ================================================================ tensor-core issuers (one thread per half)
+            // Each half has its own issuing thread, so one half's barrier waits and bookkeeping never hold up the
+            // other half's MMAs.  A turn word makes them issue strictly in turns (A, B, A, B, ...): that keeps the
+            // two halves in anti-phase - while the softmax warps of A own the exp units, the tensor pipe works for
+            // B - which two free-running issuers lose (measured).  Both walk the same item ring; an item and the Q
+            // buffer are released by both (barrier count 2), and a release is only signalled after the item's
+            // "full" barrier was seen, so neither issuer can run a whole ring turn ahead of the other.
+            const int hf = (warp == 12) ? 0 : 1;
             Ring ring = {0, 0};
-            uint32_t q_phase = 0, p_phase[2] = {0, 0}, of_phase[2] = {0, 0};
+            uint32_t q_phase = 0, p_phase = 0, of_phase = 0;
             int tstep = 0;
             (void)tstep;
             constexpr uint32_t idesc_qk = idesc_bf16(128, 0, 0);
             constexpr uint32_t idesc_pv = idesc_bf16(D, 0, 1);
+            const uint64_t q_desc = smem_desc_sw128(sQ + hf * C::kTileBytes, 16, 1024);
             const uint64_t k_desc0 = smem_desc_sw128(sKV + C::kTileBytes, 16, 1024);   // + item * (kItemBytes >> 4)
             const uint64_t v_desc0 = smem_desc_sw128(sKV, C::kHalfBytes, 1024);
+            const uint32_t tS = tmem + col_s(hf), tO = tmem + col_o(hf);
             bool dead = false;
-            auto issue_qk = [&](int hf, uint32_t item) {     // S = Q K^T over head_dim in chunks of 16
-                const uint64_t qd = smem_desc_sw128(sQ + hf * C::kTileBytes, 16, 1024);
+            auto issue_qk = [&](uint32_t item) {     // S = Q K^T over head_dim in chunks of 16
                 const uint64_t kd = k_desc0 + (uint64_t)(item * (C::kItemBytes >> 4));
-                const uint32_t tS = tmem + col_s(hf);
 #pragma unroll
                 for (int kk = 0; kk < D / 16; ++kk) {
                     const uint64_t off = (uint64_t)(((kk >> 2) * C::kHalfBytes + (kk & 3) * 32) >> 4);
-                    if (kk == 0) mma_ss_overwrite(tS, qd + off, kd + off, idesc_qk);
-                    else mma_ss_accumulate(tS, qd + off, kd + off, idesc_qk);
+                    if (kk == 0) mma_ss_overwrite(tS, q_desc + off, kd + off, idesc_qk);
+                    else mma_ss_accumulate(tS, q_desc + off, kd + off, idesc_qk);
                 }
                 mma_commit(bSFull(hf));
+            };
+            // bounded spin on the turn word (shared memory, written by the other issuer)
+            auto take_turn = [&]() -> bool {
+                if (*turn == (uint32_t)hf) return true;
+                const long long t0 = clock64();
+                uint32_t n = 0;
+                while (*turn != (uint32_t)hf) {
+                    if ((++n & 255u) == 0u) {
+                        if (*abort_flag) return false;
+                        if (clock64() - t0 > WPP_WAIT_LIMIT) { *abort_flag = 1u; return false; }
+                    }
+                }
+                return true;
+            };
+            auto pass_turn = [&]() {
+                __threadfence_block();
+                *turn = (uint32_t)(hf ^ 1);
             };
             for (int u = u_begin; u < u_end && !dead; ++u) {
                 const WppUnit un = units[u];
                 const UnitView v = view_of(un, p, q_offsets);
                 if (v.n_steps == 0) continue;
+                const int n = v.n[hf];
                 // K(0), Q
                 if (!mbar_wait(bItemFull + 8 * ring.stage, ring.phase, abort_flag)) break;
                 if (!mbar_wait(bQFull, q_phase, abort_flag)) break;
                 q_phase ^= 1u;
                 tc_fence_after();
-                if (v.n[0] > 0) issue_qk(0, ring.stage);
-                if (v.n[1] > 0) issue_qk(1, ring.stage);
+                if (!take_turn()) break;
+                if (n > 0) issue_qk(ring.stage);
+                pass_turn();
                 mma_commit(bItemEmpty + 8 * ring.stage);
-                if (v.n_steps == 1) mma_commit(bQEmpty);
+                if (n <= 1) mma_commit(bQEmpty);              // this half issues no further S for this tile
                 ring.advance(C::kItems);
-                bool have_item = false;      // the item of the coming iteration has already been waited for
                 for (int j = 0; j < v.n_steps; ++j) {
                     // item {V(j), K(j+1)}
-                    if (!have_item && !mbar_wait(bItemFull + 8 * ring.stage, ring.phase, abort_flag)) { dead = true; break; }
+                    if (!mbar_wait(bItemFull + 8 * ring.stage, ring.phase, abort_flag)) { dead = true; break; }
                     const uint32_t item = ring.stage;
-                    const int valid = v.kv_len - (v.kv_begin + j) * 128;      // keys of this step that exist
-                    if (valid < 128) {
-                        // rows past the end of the sequence may hold anything (stale slots, never-loaded pages):
-                        // zero them so that 0 * garbage cannot reach O
-                        uint8_t* vg = smem_gen + C::kOffKV + item * C::kItemBytes;
-                        for (int h = 0; h < C::kHalves; ++h)
-                            for (int i = valid * 8; i < 128 * 8; ++i)
-                                *reinterpret_cast<uint4*>(vg + h * C::kHalfBytes + i * 16) = make_uint4(0, 0, 0, 0);
-                        fence_proxy_async_smem();
-                    }
-                    const uint64_t vd = v_desc0 + (uint64_t)(item * (C::kItemBytes >> 4));
-#pragma unroll
-                    for (int hf = 0; hf < 2; ++hf) {
-                        if (j >= v.n[hf]) continue;
-                        TRACE(2, tstep, hf * 4 + 0);
-                        if (!mbar_wait(bPReady(hf), p_phase[hf], abort_flag)) { dead = true; break; }   // P written, O fixed
-                        p_phase[hf] ^= 1u;
-                        TRACE(2, tstep, hf * 4 + 1);
+                    const bool active = j < n;
+                    if (active) {
+                        const int valid = v.kv_len - (v.kv_begin + j) * 128;      // keys of this step that exist
+                        if (valid < 128) {
+                            // rows past the end of the sequence may hold anything (stale slots, never-loaded
+                            // pages): zero them so that 0 * garbage cannot reach O (both issuers write the same zeros)
+                            uint8_t* vg = smem_gen + C::kOffKV + item * C::kItemBytes;
+                            for (int h = 0; h < C::kHalves; ++h)
+                                for (int i = valid * 8; i < 128 * 8; ++i)
+                                    *reinterpret_cast<uint4*>(vg + h * C::kHalfBytes + i * 16) = make_uint4(0, 0, 0, 0);
+                            fence_proxy_async_smem();
+                        }
+                        if (!mbar_wait(bPReady(hf), p_phase, abort_flag)) { dead = true; break; }   // P written, O fixed
+                        p_phase ^= 1u;
                         if (j == 0) {
                             // the first product of a tile overwrites O: the previous tile's epilogue must have read it
-                            if (!mbar_wait(bOFree(hf), of_phase[hf] ^ 1u, abort_flag)) { dead = true; break; }
-                            of_phase[hf] ^= 1u;
+                            if (!mbar_wait(bOFree(hf), of_phase ^ 1u, abort_flag)) { dead = true; break; }
+                            of_phase ^= 1u;
                         }
                         tc_fence_after();
-                        const uint32_t tS = tmem + col_s(hf), tO = tmem + col_o(hf);
+                    }
+                    if (!take_turn()) { dead = true; break; }
+                    if (active) {
+                        const uint64_t vd = v_desc0 + (uint64_t)(item * (C::kItemBytes >> 4));
                         if (j > 0) mma_ts_accumulate(tO, tS, vd, idesc_pv); else mma_ts_overwrite(tO, tS, vd, idesc_pv);
 #pragma unroll
                         for (int kk = 1; kk < 8; ++kk) mma_ts_accumulate(tO, tS + kk * 8, vd + (uint64_t)(kk * 128), idesc_pv);
-                        TRACE(2, tstep, hf * 4 + 2);
-                        if (j + 1 < v.n[hf]) issue_qk(hf, item);      // its commit also covers the O += P V above
+                        if (j + 1 < n) issue_qk(item);            // its commit also covers the O += P V above
                         else mma_commit(bOFinal(hf));
-                        TRACE(2, tstep, hf * 4 + 3);
-                        if (hf == 0) {
-                            // look at the next item now, while the tensor pipe still has half A's work queued,
-                            // instead of at the top of the next iteration when it has run dry
-                            have_item = false;
-                            if (j + 1 < v.n_steps) {
-                                Ring nxt = ring;
-                                nxt.advance(C::kItems);
-                                if (!mbar_wait(bItemFull + 8 * nxt.stage, nxt.phase, abort_flag)) { dead = true; break; }
-                                have_item = true;
-                            }
-                        }
                     }
-                    if (dead) break;
+                    pass_turn();
                     mma_commit(bItemEmpty + 8 * item);
-                    if (j + 2 == v.n_steps) mma_commit(bQEmpty);       // the last S of this tile has been issued
+                    if (j + 2 == n) mma_commit(bQEmpty);           // the last S of this half has been issued
                     ring.advance(C::kItems);
                     ++tstep;
                 }
