@@ -197,7 +197,7 @@ extern "C" int wpp_prefill_attention_varlen(const wpp_ctx* ctx, const wpp_batch_
     p.num_pages = d.num_pages;
     const double scale = d.sm_scale > 0.f ? (double)d.sm_scale : 1.0 / sqrt((double)d.head_dim);
     p.scale_log2 = (float)(scale * 1.4426950408889634);
-#ifdef WPP_TRACE
+#if defined(WPP_TRACE) || defined(WPP_STATS)
     {   // tuning builds: the address of a device timeline buffer comes through the environment
         const char* t = getenv("WPP_TRACE_PTR");
         p.trace = t ? reinterpret_cast<uint32_t*>(strtoull(t, nullptr, 0)) : nullptr;

@@ -6,19 +6,23 @@
 //   warps 0-3   softmax of half A: thread r owns query row r (TMEM lane r): row max / row sum need no shuffles
 //   warps 4-7   softmax of half B
 //   warps 8-11  epilogue: O / l -> bf16 -> global (or fp32 partials for split tiles), overlapping the next tile
-//   warps 12,14 tensor-core issuers, one thread per half: S = Q K^T and O += P V with tcgen05.mma (fp32 accumulators
-//               in TMEM; P is read from TMEM where the softmax warps wrote it as packed bf16 over S; V is an
-//               MN-major operand).  They issue strictly in turns (A, B, A, ...), which keeps the halves in anti-phase
-//               while one half's barrier waits never hold up the other half's MMAs.
+//   warp 12     issuer of S = Q K^T (one thread), warp 14 issuer of O += P V (one thread): tcgen05.mma with fp32
+//               accumulators in TMEM; P is read from TMEM where the softmax warps wrote it as packed bf16; V is an
+//               MN-major operand.  Two threads, because the queue of the tensor pipe is only a few MMAs deep: the
+//               barrier waits and bookkeeping of one thread hide behind the MMAs the other one is issuing.
 //   warp 13     producer: reads the block table and issues TMA tile loads (Q once per tile; per key step one box
-//               per (page, 64-wide half of head_dim) for K and for V, 128-byte swizzle).  V(j) and K(j+1) are used
-//               in the same issuer iteration, so they travel as one ring item with one barrier.
-// The two halves ping-pong: while the softmax warps of A work on S_A(j+1), the tensor cores run O_B += P_B V(j)
-// and S_B(j+1).  Rescaling is lazy: a row keeps its reference maximum, and does not even compute the maximum of
-// a step, as long as the step's row sum shows that no score rose far above the reference; only then (and on the
-// first step of a tile) the softmax warps take the true maximum and rescale O and l themselves.
-// Tensor memory (512 columns): S_A [0,128)  S_B [128,256)  O_A [256,256+D)  O_B [384,384+D); P aliases the first
-// 64 columns of its S.
+//               per (page, 64-wide half of head_dim) for K and for V, 128-byte swizzle) into a ring of K tiles
+//               and a ring of V tiles
+// Tensor memory (512 columns) has no room for two S tiles and two P tiles next to the two O accumulators, so the
+// two halves share ONE landing buffer for S: a softmax warpgroup copies its S into registers as soon as it lands
+// and hands the buffer back (s_free) before it starts on the exponentials, and each half has a P buffer of its own.
+// That takes S = Q K^T off the softmax -> O += P V chain of its half: while the softmax warps of A work on step j,
+// the tensor pipe already produces S_B(j) and S_A(j+1) and runs the other half's O += P V, so the exponentials of
+// both halves and the MMAs all overlap.  The order on the tensor pipe is not fixed: every S is issued when the
+// landing buffer is free, every product when its P is ready.
+// Rescaling is lazy: a row keeps its reference maximum as long as the step's maximum stays within 2^16 of it;
+// only then (and on the first step of a tile) the softmax warps move the reference and rescale O and l.
+// Tensor memory: S [0,128)  P_A [128,192)  P_B [192,256)  O_A [256,256+D)  O_B [384,384+D).
 // All mbarrier waits are bounded; on expiry the CTA raises its abort flag, every role drains, TMEM is freed and
 // WPP_ERR_TIMEOUT is written to the status word.
 #include <cuda.h>
@@ -34,9 +38,19 @@ namespace wpp {
 
 constexpr int kThreads = 512;
 constexpr uint32_t kTmemCols = 512;
-__host__ __device__ constexpr uint32_t col_s(int hf) { return 128u * hf; }          // S (and P) of half hf
+constexpr uint32_t kColS = 0;                                                        // landing buffer of S
+__host__ __device__ constexpr uint32_t col_p(int hf) { return 128u + 64u * hf; }    // P of half hf (packed bf16)
 __host__ __device__ constexpr uint32_t col_o(int hf) { return 256u + 128u * hf; }   // O of half hf
-constexpr float kFastPathSumLimit = 65536.f;  // row sum of p below which the old reference was safe to keep
+// registers per thread after the warpgroups re-split the register file (8 x kRegsSoftmax + 4 x kRegsEpilogue +
+// 4 x kRegsUtil <= 2048 per thread slot of 32 lanes, i.e. 65536 in all)
+#ifndef WPP_REGS_SOFTMAX
+#define WPP_REGS_SOFTMAX 176
+#define WPP_REGS_EPILOGUE 64
+#define WPP_REGS_UTIL 96
+#endif
+constexpr int kRegsSoftmax = WPP_REGS_SOFTMAX, kRegsEpilogue = WPP_REGS_EPILOGUE, kRegsUtil = WPP_REGS_UTIL;
+static_assert(8 * kRegsSoftmax + 4 * kRegsEpilogue + 4 * kRegsUtil <= 2048, "register file exceeded");
+constexpr float kRefSlack = 16.f;   // a row keeps its reference while its scores stay below reference + 16 (log2)
 #ifndef WPP_EMU_PAIRS_OF_4
 #define WPP_EMU_PAIRS_OF_4 0
 #endif
@@ -47,28 +61,43 @@ struct Cfg {
     static constexpr int kHalves = D / 64;                 // 64-element (128-byte) swizzled column blocks
     static constexpr int kTileBytes = 128 * D * 2;         // one 128-row Q half, or one K or V step
     static constexpr int kHalfBytes = 128 * 128;           // 128 rows x 128 bytes
-    static constexpr int kItems = (D == 128) ? 2 : 4;      // ring of items {V(j), K(j+1)}
-    static constexpr int kItemBytes = 2 * kTileBytes;      // V part, then K part
+    static constexpr int kSlots = (D == 128) ? 5 : 8;      // ring of K / V tiles (4 if the base is badly aligned)
     static constexpr int kOffKV = 2 * kTileBytes;
-    static constexpr int kOffBars = kOffKV + kItems * kItemBytes;
-    static constexpr int kNumBars = 2 + 2 * kItems + 5 * 2;
+    static constexpr int kOffBars = kOffKV + kSlots * kTileBytes;
+    static constexpr int kNumBars = 2 + 2 * kSlots + 1 + 6 * 2;
     static constexpr int kOffFinal = kOffBars + 8 * kNumBars;          // float2 (m, l)[2][128]
     static constexpr int kOffMisc = kOffFinal + 2 * 128 * 8;           // tmem ptr, abort flag
-    static constexpr int kSmemBytes = kOffMisc + 16 + 1024;            // + alignment slack
+    static constexpr int kUsedBytes = kOffMisc + 16;
+    static constexpr int kMaxSmem = 232448;                            // 227 KB: the most a CTA can have
+    static constexpr int kSmemBytes = (kUsedBytes + 1024 < kMaxSmem) ? kUsedBytes + 1024 : kMaxSmem;
 };
 
-// Optional timeline instrumentation for tuning (compiled out unless WPP_TRACE is defined): CTA 0 records the
-// low 32 bits of clock64 at a few points of its first key steps into p.trace[role][step][event].
-#ifdef WPP_TRACE
-#define WPP_TRACE_EVENTS 8
-#define WPP_TRACE_STEPS 64
-#define TRACE(role, step, ev)                                                                              \
-    do {                                                                                                   \
-        if (p.trace && blockIdx.x == 0 && (threadIdx.x & 127) == 0 && (step) < WPP_TRACE_STEPS)            \
-            p.trace[((role) * WPP_TRACE_STEPS + (step)) * WPP_TRACE_EVENTS + (ev)] = (uint32_t)clock64(); \
+// Optional wait accounting for tuning (compiled out unless WPP_STATS is defined): one thread of each role adds
+// the clocks it spent in each kind of wait to p.trace, read as unsigned long long [role][8].
+#ifdef WPP_STATS
+#define STAT_DECL()                                                                                        \
+    uint32_t stat0_ = 0, stat1_ = 0, stat2_ = 0, stat3_ = 0, stat4_ = 0, stat5_ = 0, stat6_ = 0;           \
+    const long long stat_begin_ = clock64()
+#define STAT_T0() const uint32_t st0_ = (uint32_t)clock64()
+#define STAT_ADD(k) stat##k##_ += (uint32_t)clock64() - st0_
+#define STAT_INC(k) stat##k##_ += 1u
+#define STAT_FLUSH(role, leader)                                                                          \
+    do {                                                                                                  \
+        if (p.trace && (leader)) {                                                                        \
+            unsigned long long* t_ = reinterpret_cast<unsigned long long*>(p.trace) + (role) * 8;         \
+            atomicAdd(t_ + 0, (unsigned long long)stat0_); atomicAdd(t_ + 1, (unsigned long long)stat1_); \
+            atomicAdd(t_ + 2, (unsigned long long)stat2_); atomicAdd(t_ + 3, (unsigned long long)stat3_); \
+            atomicAdd(t_ + 4, (unsigned long long)stat4_); atomicAdd(t_ + 5, (unsigned long long)stat5_); \
+            atomicAdd(t_ + 6, (unsigned long long)stat6_);                                                \
+            atomicAdd(t_ + 7, (unsigned long long)(clock64() - stat_begin_));                             \
+        }                                                                                                 \
     } while (0)
 #else
-#define TRACE(role, step, ev) do { } while (0)
+#define STAT_DECL() do { } while (0)
+#define STAT_T0() do { } while (0)
+#define STAT_ADD(k) do { } while (0)
+#define STAT_INC(k) do { } while (0)
+#define STAT_FLUSH(role, leader) do { } while (0)
 #endif
 
 struct Ring {
@@ -110,39 +139,44 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
+    // the tile ring gives up one slot when the 1024-byte alignment of the base costs more than the spare bytes
+    const uint32_t n_slots =
+        (smem_base - smem_u32(smem_raw)) + (uint32_t)C::kUsedBytes <= (uint32_t)C::kSmemBytes ? C::kSlots : C::kSlots - 1;
     const uint32_t sQ = smem_base;                       // two halves, kTileBytes each
-    const uint32_t sKV = smem_base + C::kOffKV;          // kItems x {V tile, K tile}
+    const uint32_t sKV = smem_base + C::kOffKV;          // kSlots tiles (K or V)
     const uint32_t bars = smem_base + C::kOffBars;
     const uint32_t bQFull = bars, bQEmpty = bars + 8;
-    const uint32_t bItemFull = bars + 16, bItemEmpty = bItemFull + 8 * C::kItems;
-    // Per half: s_full (S = Q K^T landed; it also proves the previous O += P V landed, the tensor pipe being in
-    // order), p_ready (P written, and O rescaled if the row reference moved, by the 128 softmax threads),
-    // final_ready (end-of-tile (m, l) are in smem), o_final (last O += P V landed), o_free (the epilogue threads
-    // have read O out, the next tile may overwrite it).  A thread never arrives twice on one barrier without a
-    // wait in between that implies the earlier phase completed.
-    const uint32_t bHalf = bItemEmpty + 8 * C::kItems;
-    auto bSFull = [&](int h) { return bHalf + 40 * h; };
-    auto bPReady = [&](int h) { return bHalf + 40 * h + 8; };
-    auto bFinalReady = [&](int h) { return bHalf + 40 * h + 16; };
-    auto bOFinal = [&](int h) { return bHalf + 40 * h + 24; };
-    auto bOFree = [&](int h) { return bHalf + 40 * h + 32; };
+    const uint32_t bSlotFull = bars + 16, bSlotEmpty = bSlotFull + 8 * C::kSlots;
+    // s_free: the half that owned the landing buffer has copied its S into registers.
+    // Per half: s_full (S = Q K^T landed), p_ready (P written, and O rescaled if the row reference moved, by the
+    // 128 softmax threads), p_free (O += P V landed: P may be overwritten, O may be rescaled), final_ready
+    // (end-of-tile (m, l) are in smem), o_final (last O += P V landed), o_free (the epilogue threads have read O
+    // out, the next tile may overwrite it).  A thread never arrives twice on one barrier without a wait in
+    // between that implies the earlier phase completed.
+    const uint32_t bSFree = bSlotEmpty + 8 * C::kSlots;
+    const uint32_t bHalf = bSFree + 8;
+    auto bSFull = [&](int h) { return bHalf + 48 * h; };
+    auto bPReady = [&](int h) { return bHalf + 48 * h + 8; };
+    auto bPFree = [&](int h) { return bHalf + 48 * h + 16; };
+    auto bFinalReady = [&](int h) { return bHalf + 48 * h + 24; };
+    auto bOFinal = [&](int h) { return bHalf + 48 * h + 32; };
+    auto bOFree = [&](int h) { return bHalf + 48 * h + 40; };
     float2* s_final = reinterpret_cast<float2*>(smem_gen + C::kOffFinal);     // [2][128] (reference in log2 units, l)
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_gen + C::kOffMisc);
     volatile uint32_t* abort_flag = tmem_slot + 1;
-    volatile uint32_t* turn = tmem_slot + 2;             // which half's issuer may issue next
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int wg = warp >> 2;
 
     if (threadIdx.x == 0) {
-        mbar_init(bQFull, 1); mbar_init(bQEmpty, 2);
-        for (int s = 0; s < C::kItems; ++s) { mbar_init(bItemFull + 8 * s, 1); mbar_init(bItemEmpty + 8 * s, 2); }
+        mbar_init(bQFull, 1); mbar_init(bQEmpty, 1);
+        for (int s = 0; s < C::kSlots; ++s) { mbar_init(bSlotFull + 8 * s, 1); mbar_init(bSlotEmpty + 8 * s, 1); }
+        mbar_init(bSFree, 128);
         for (int h = 0; h < 2; ++h) {
-            mbar_init(bSFull(h), 1); mbar_init(bPReady(h), 128);
+            mbar_init(bSFull(h), 1); mbar_init(bPReady(h), 128); mbar_init(bPFree(h), 1);
             mbar_init(bFinalReady(h), 128); mbar_init(bOFinal(h), 1); mbar_init(bOFree(h), 128);
         }
         *abort_flag = 0u;
-        *turn = 0u;
         fence_barrier_init();
     }
     if (warp == 12) {
@@ -167,12 +201,17 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     const int B = p.page_size, ppt = 128 / B;   // pages per key step
 
     if (wg == 3) {
-        setmaxnreg_dec<96>();
+        setmaxnreg_dec<kRegsUtil>();
+        // The K tiles and the V tiles have a ring each (slots [n_v, n_slots) and [0, n_v) of the tile area), so
+        // that the thread issuing S = Q K^T and the thread issuing O += P V walk their own ring.
+        const uint32_t n_v = C::kSlots / 2, n_k = n_slots - n_v;
         if (warp == 13) {
             // ================================================================ producer
-            Ring ring = {0, 0};
+            // Tiles are requested in the order the issuers first touch them: K(0), K(1), V(0), K(2), V(1), ...
+            Ring ring_k = {0, 0}, ring_v = {0, 0};
             uint32_t q_phase = 0;
             bool dead = false;
+            STAT_DECL();
             for (int u = u_begin; u < u_end && !dead; ++u) {
                 const WppUnit un = units[u];
                 const UnitView v = view_of(un, p, q_offsets);
@@ -180,43 +219,38 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 const int n_pages = (v.kv_len + B - 1) / B;
                 const int kvh = un.head[0] / p.group;
                 const int32_t* bt = p.block_tables + (int64_t)un.request * p.max_blocks;
-                // one ring item: V of step jv (if jv >= 0) and K of step jk (if jk < n_steps); lane l moves
-                // page l of each step
-                auto load_item = [&](int jv, int jk) -> bool {
-                    const bool has_v = jv >= 0, has_k = jk < v.n_steps;
-                    const int page_v = (v.kv_begin + jv) * ppt, page_k = (v.kv_begin + jk) * ppt;
-                    const int cnt_v = has_v ? min(ppt, n_pages - page_v) : 0;
-                    const int cnt_k = has_k ? min(ppt, n_pages - page_k) : 0;
-                    int pid_v = 0, pid_k = 0;
-                    if (lane < cnt_v) pid_v = bt[page_v + lane];
-                    if (lane < cnt_k) pid_k = bt[page_k + lane];
-                    if (pid_v < 0 || pid_v >= p.num_pages || pid_k < 0 || pid_k >= p.num_pages) {
+                // one ring slot: the K or the V tile of key step j; lane l moves page l of the step
+                auto load_tile = [&](const CUtensorMap* tm, int j, Ring& ring, uint32_t slot0, uint32_t n_ring) -> bool {
+                    const int page0 = (v.kv_begin + j) * ppt;
+                    const int cnt = min(ppt, n_pages - page0);
+                    int pid = 0;
+                    if (lane < cnt) pid = bt[page0 + lane];
+                    if (pid < 0 || pid >= p.num_pages) {
                         if (p.status) atomicCAS(p.status, 0, WPP_ERR_BOUNDS);
-                        pid_v = (pid_v < 0 || pid_v >= p.num_pages) ? 0 : pid_v;
-                        pid_k = (pid_k < 0 || pid_k >= p.num_pages) ? 0 : pid_k;
+                        pid = 0;
                     }
-                    const bool ok = mbar_wait(bItemEmpty + 8 * ring.stage, ring.phase ^ 1u, abort_flag);
+                    const uint32_t slot = slot0 + ring.stage;
+                    STAT_T0();
+                    const bool ok = mbar_wait(bSlotEmpty + 8 * slot, ring.phase ^ 1u, abort_flag);
+                    STAT_ADD(0);
                     if (!__all_sync(0xffffffffu, ok)) return false;
-                    const uint32_t full = bItemFull + 8 * ring.stage;
-                    if (lane == 0) mbar_arrive_expect_tx(full, (uint32_t)(cnt_v + cnt_k) * B * D * 2);
+                    const uint32_t full = bSlotFull + 8 * slot;
+                    if (lane == 0) mbar_arrive_expect_tx(full, (uint32_t)cnt * B * D * 2);
                     __syncwarp();
-                    const uint32_t dst = sKV + ring.stage * C::kItemBytes + lane * B * 128;
-                    if (lane < cnt_v) {
+                    const uint32_t dst = sKV + slot * C::kTileBytes + lane * B * 128;
+                    if (lane < cnt) {
 #pragma unroll
                         for (int h = 0; h < C::kHalves; ++h)
-                            tma_load_4d(dst + h * C::kHalfBytes, &tm_v, full, h * 64, 0, kvh, pid_v);
+                            tma_load_4d(dst + h * C::kHalfBytes, tm, full, h * 64, 0, kvh, pid);
                     }
-                    if (lane < cnt_k) {
-#pragma unroll
-                        for (int h = 0; h < C::kHalves; ++h)
-                            tma_load_4d(dst + C::kTileBytes + h * C::kHalfBytes, &tm_k, full, h * 64, 0, kvh, pid_k);
-                    }
-                    ring.advance(C::kItems);
+                    ring.advance(n_ring);
                     return true;
                 };
                 // K(0) only needs a ring slot, which frees up before the previous tile's Q does
-                if (!load_item(-1, 0)) { dead = true; break; }
+                if (!load_tile(&tm_k, 0, ring_k, n_v, n_k)) { dead = true; break; }
+                STAT_T0();
                 const bool ok = mbar_wait(bQEmpty, q_phase ^ 1u, abort_flag);
+                STAT_ADD(1);
                 if (!__all_sync(0xffffffffu, ok)) { dead = true; break; }
                 q_phase ^= 1u;
                 if (lane == 0) {
@@ -237,117 +271,142 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     }
                 }
                 __syncwarp();
-                for (int j = 0; j < v.n_steps; ++j)
-                    if (!load_item(j, j + 1)) { dead = true; break; }
+                for (int k = 0; k <= v.n_steps && !dead; ++k) {
+                    if (k >= 1 && !load_tile(&tm_v, k - 1, ring_v, 0, n_v)) dead = true;
+                    if (!dead && k + 1 < v.n_steps && !load_tile(&tm_k, k + 1, ring_k, n_v, n_k)) dead = true;
+                }
             }
-        } else if ((warp == 12 || warp == 14) && lane == 0) {
-            // ================================================================ tensor-core issuers (one thread per half)
-            // Each half has its own issuing thread, so one half's barrier waits and bookkeeping never hold up the
-            // other half's MMAs.  A turn word makes them issue strictly in turns (A, B, A, B, ...): that keeps the
-            // two halves in anti-phase - while the softmax warps of A own the exp units, the tensor pipe works for
-            // B - which two free-running issuers lose (measured).  Both walk the same item ring; an item and the Q
-            // buffer are released by both (barrier count 2), and a release is only signalled after the item's
-            // "full" barrier was seen, so neither issuer can run a whole ring turn ahead of the other.
-            const int hf = (warp == 12) ? 0 : 1;
+            STAT_FLUSH(4, lane == 0);
+        } else if (warp == 12 && lane == 0) {
+            // ================================================================ issuer of S = Q K^T (one thread)
+            // S_A(0), S_B(0), S_A(1), S_B(1), ...: each S goes into the landing buffer as soon as the previous one
+            // has been copied out of it (s_free).
             Ring ring = {0, 0};
-            uint32_t q_phase = 0, p_phase = 0, of_phase = 0;
-            int tstep = 0;
-            (void)tstep;
+            uint32_t q_phase = 0, sfree_phase = 0;
             constexpr uint32_t idesc_qk = idesc_bf16(128, 0, 0);
-            constexpr uint32_t idesc_pv = idesc_bf16(D, 0, 1);
-            const uint64_t q_desc = smem_desc_sw128(sQ + hf * C::kTileBytes, 16, 1024);
-            const uint64_t k_desc0 = smem_desc_sw128(sKV + C::kTileBytes, 16, 1024);   // + item * (kItemBytes >> 4)
-            const uint64_t v_desc0 = smem_desc_sw128(sKV, C::kHalfBytes, 1024);
-            const uint32_t tS = tmem + col_s(hf), tO = tmem + col_o(hf);
+            const uint64_t q_desc0 = smem_desc_sw128(sQ, 16, 1024);                    // + hf * (kTileBytes >> 4)
+            const uint64_t k_desc0 = smem_desc_sw128(sKV + n_v * C::kTileBytes, 16, 1024);   // + stage * (kTileBytes >> 4)
+            const uint32_t tS = tmem + kColS;
             bool dead = false;
-            auto issue_qk = [&](uint32_t item) {     // S = Q K^T over head_dim in chunks of 16
-                const uint64_t kd = k_desc0 + (uint64_t)(item * (C::kItemBytes >> 4));
-#pragma unroll
-                for (int kk = 0; kk < D / 16; ++kk) {
-                    const uint64_t off = (uint64_t)(((kk >> 2) * C::kHalfBytes + (kk & 3) * 32) >> 4);
-                    if (kk == 0) mma_ss_overwrite(tS, q_desc + off, kd + off, idesc_qk);
-                    else mma_ss_accumulate(tS, q_desc + off, kd + off, idesc_qk);
-                }
-                mma_commit(bSFull(hf));
-            };
-            // bounded spin on the turn word (shared memory, written by the other issuer)
-            auto take_turn = [&]() -> bool {
-                if (*turn == (uint32_t)hf) return true;
-                const long long t0 = clock64();
-                uint32_t n = 0;
-                while (*turn != (uint32_t)hf) {
-                    if ((++n & 255u) == 0u) {
-                        if (*abort_flag) return false;
-                        if (clock64() - t0 > WPP_WAIT_LIMIT) { *abort_flag = 1u; return false; }
-                    }
-                }
-                return true;
-            };
-            auto pass_turn = [&]() {
-                __threadfence_block();
-                *turn = (uint32_t)(hf ^ 1);
-            };
+            STAT_DECL();
             for (int u = u_begin; u < u_end && !dead; ++u) {
                 const WppUnit un = units[u];
                 const UnitView v = view_of(un, p, q_offsets);
                 if (v.n_steps == 0) continue;
-                const int n = v.n[hf];
-                // K(0), Q
-                if (!mbar_wait(bItemFull + 8 * ring.stage, ring.phase, abort_flag)) break;
-                if (!mbar_wait(bQFull, q_phase, abort_flag)) break;
+                {
+                    STAT_T0();
+                    const bool ok = mbar_wait(bQFull, q_phase, abort_flag);
+                    STAT_ADD(4);
+                    if (!ok) break;
+                }
                 q_phase ^= 1u;
-                tc_fence_after();
-                if (!take_turn()) break;
-                if (n > 0) issue_qk(ring.stage);
-                pass_turn();
-                mma_commit(bItemEmpty + 8 * ring.stage);
-                if (n <= 1) mma_commit(bQEmpty);              // this half issues no further S for this tile
-                ring.advance(C::kItems);
-                for (int j = 0; j < v.n_steps; ++j) {
-                    // item {V(j), K(j+1)}
-                    if (!mbar_wait(bItemFull + 8 * ring.stage, ring.phase, abort_flag)) { dead = true; break; }
-                    const uint32_t item = ring.stage;
-                    const bool active = j < n;
-                    if (active) {
-                        const int valid = v.kv_len - (v.kv_begin + j) * 128;      // keys of this step that exist
-                        if (valid < 128) {
-                            // rows past the end of the sequence may hold anything (stale slots, never-loaded
-                            // pages): zero them so that 0 * garbage cannot reach O (both issuers write the same zeros)
-                            uint8_t* vg = smem_gen + C::kOffKV + item * C::kItemBytes;
-                            for (int h = 0; h < C::kHalves; ++h)
-                                for (int i = valid * 8; i < 128 * 8; ++i)
-                                    *reinterpret_cast<uint4*>(vg + h * C::kHalfBytes + i * 16) = make_uint4(0, 0, 0, 0);
-                            fence_proxy_async_smem();
+                for (int k = 0; k < v.n_steps; ++k) {
+                    {
+                        STAT_T0();
+                        const bool ok = mbar_wait(bSlotFull + 8 * (n_v + ring.stage), ring.phase, abort_flag);   // K(k)
+                        STAT_ADD(0);
+                        if (!ok) { dead = true; break; }
+                    }
+                    const uint64_t kd = k_desc0 + (uint64_t)(ring.stage * (C::kTileBytes >> 4));
+#pragma unroll
+                    for (int hf = 0; hf < 2; ++hf) {
+                        if (k >= v.n[hf]) continue;
+                        {
+                            STAT_T0();
+                            const bool ok = mbar_wait(bSFree, sfree_phase ^ 1u, abort_flag);
+                            STAT_ADD(2);
+                            if (!ok) { dead = true; break; }
                         }
-                        if (!mbar_wait(bPReady(hf), p_phase, abort_flag)) { dead = true; break; }   // P written, O fixed
-                        p_phase ^= 1u;
-                        if (j == 0) {
+                        sfree_phase ^= 1u;
+                        tc_fence_after();
+                        const uint64_t qd = q_desc0 + (uint64_t)(hf * (C::kTileBytes >> 4));
+                        STAT_T0();
+#pragma unroll
+                        for (int kk = 0; kk < D / 16; ++kk) {
+                            const uint64_t off = (uint64_t)(((kk >> 2) * C::kHalfBytes + (kk & 3) * 32) >> 4);
+                            if (kk == 0) mma_ss_overwrite(tS, qd + off, kd + off, idesc_qk);
+                            else mma_ss_accumulate(tS, qd + off, kd + off, idesc_qk);
+                        }
+                        mma_commit(bSFull(hf));
+                        STAT_ADD(6);
+                    }
+                    if (dead) break;
+                    mma_commit(bSlotEmpty + 8 * (n_v + ring.stage));                  // K(k) has been read
+                    ring.advance(n_k);
+                }
+                if (!dead) mma_commit(bQEmpty);           // every S of the tile has been issued: Q may be replaced
+            }
+            STAT_FLUSH(0, true);
+        } else if (warp == 14 && lane == 0) {
+            // ================================================================ issuer of O += P V (one thread)
+            // O_A += P_A V(0), O_B += P_B V(0), O_A += P_A V(1), ...: each product waits for its P.
+            Ring ring = {0, 0};
+            uint32_t p_phase[2] = {0, 0}, of_phase[2] = {0, 0};
+            constexpr uint32_t idesc_pv = idesc_bf16(D, 0, 1);
+            const uint64_t v_desc0 = smem_desc_sw128(sKV, C::kHalfBytes, 1024);       // + stage * (kTileBytes >> 4)
+            bool dead = false;
+            STAT_DECL();
+            for (int u = u_begin; u < u_end && !dead; ++u) {
+                const WppUnit un = units[u];
+                const UnitView v = view_of(un, p, q_offsets);
+                if (v.n_steps == 0) continue;
+                for (int k = 0; k < v.n_steps; ++k) {
+                    {
+                        STAT_T0();
+                        const bool ok = mbar_wait(bSlotFull + 8 * ring.stage, ring.phase, abort_flag);           // V(k)
+                        STAT_ADD(0);
+                        if (!ok) { dead = true; break; }
+                    }
+                    const int valid = v.kv_len - (v.kv_begin + k) * 128;      // keys of this step that exist
+                    if (valid < 128) {
+                        // rows past the end of the sequence may hold anything (stale slots, never-loaded
+                        // pages): zero them so that 0 * garbage cannot reach O
+                        uint8_t* vg = smem_gen + C::kOffKV + ring.stage * C::kTileBytes;
+                        for (int h = 0; h < C::kHalves; ++h)
+                            for (int i = valid * 8; i < 128 * 8; ++i)
+                                *reinterpret_cast<uint4*>(vg + h * C::kHalfBytes + i * 16) = make_uint4(0, 0, 0, 0);
+                        fence_proxy_async_smem();
+                    }
+                    const uint64_t vd = v_desc0 + (uint64_t)(ring.stage * (C::kTileBytes >> 4));
+#pragma unroll
+                    for (int hf = 0; hf < 2; ++hf) {
+                        const int n = v.n[hf];
+                        if (k >= n) continue;
+                        {
+                            STAT_T0();
+                            const bool ok = mbar_wait(bPReady(hf), p_phase[hf], abort_flag);     // P written, O fixed
+                            STAT_ADD(1);
+                            if (!ok) { dead = true; break; }
+                        }
+                        p_phase[hf] ^= 1u;
+                        if (k == 0) {
                             // the first product of a tile overwrites O: the previous tile's epilogue must have read it
-                            if (!mbar_wait(bOFree(hf), of_phase ^ 1u, abort_flag)) { dead = true; break; }
-                            of_phase ^= 1u;
+                            STAT_T0();
+                            const bool ok = mbar_wait(bOFree(hf), of_phase[hf] ^ 1u, abort_flag);
+                            STAT_ADD(3);
+                            if (!ok) { dead = true; break; }
+                            of_phase[hf] ^= 1u;
                         }
                         tc_fence_after();
-                    }
-                    if (!take_turn()) { dead = true; break; }
-                    if (active) {
-                        const uint64_t vd = v_desc0 + (uint64_t)(item * (C::kItemBytes >> 4));
-                        if (j > 0) mma_ts_accumulate(tO, tS, vd, idesc_pv); else mma_ts_overwrite(tO, tS, vd, idesc_pv);
+                        const uint32_t tP = tmem + col_p(hf), tO = tmem + col_o(hf);
+                        STAT_T0();
+                        if (k > 0) mma_ts_accumulate(tO, tP, vd, idesc_pv); else mma_ts_overwrite(tO, tP, vd, idesc_pv);
 #pragma unroll
-                        for (int kk = 1; kk < 8; ++kk) mma_ts_accumulate(tO, tS + kk * 8, vd + (uint64_t)(kk * 128), idesc_pv);
-                        if (j + 1 < n) issue_qk(item);            // its commit also covers the O += P V above
-                        else mma_commit(bOFinal(hf));
+                        for (int kk = 1; kk < 8; ++kk) mma_ts_accumulate(tO, tP + kk * 8, vd + (uint64_t)(kk * 128), idesc_pv);
+                        mma_commit(bPFree(hf));
+                        if (k + 1 == n) mma_commit(bOFinal(hf));
+                        STAT_ADD(5);
                     }
-                    pass_turn();
-                    mma_commit(bItemEmpty + 8 * item);
-                    if (j + 2 == n) mma_commit(bQEmpty);           // the last S of this half has been issued
-                    ring.advance(C::kItems);
-                    ++tstep;
+                    if (dead) break;
+                    mma_commit(bSlotEmpty + 8 * ring.stage);                          // V(k) has been read
+                    ring.advance(n_v);
                 }
             }
+            STAT_FLUSH(1, true);
         }
     } else if (wg == 2) {
         // ================================================================ epilogue (one thread per output row)
-        setmaxnreg_dec<80>();
+        setmaxnreg_dec<kRegsEpilogue>();
         const int r = threadIdx.x & 127;
         const uint32_t lane_addr = tmem + ((uint32_t)((warp & 3) * 32) << 16);
         uint32_t o_phase[2] = {0, 0}, f_phase[2] = {0, 0};
@@ -422,17 +481,15 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         }
     } else {
         // ================================================================ softmax (thread = query row of half `hf`)
-        setmaxnreg_inc<168>();
+        setmaxnreg_inc<kRegsSoftmax>();
         const int hf = wg;
         const int r = threadIdx.x & 127;
         const uint32_t lane_addr = tmem + ((uint32_t)((warp & 3) * 32) << 16);
-        const uint32_t colS = col_s(hf);
-        uint32_t s_phase = 0, fin_phase = 0;
-        int tstep = 0;      // steps since kernel start (trace index only)
-        (void)tstep;
+        uint32_t s_phase = 0, fin_phase = 0, pf_phase = 0;
         const float c = p.scale_log2;
         const uint64_t c2 = pack2(c, c);
         bool dead = false;
+        STAT_DECL();
         for (int u = u_begin; u < u_end && !dead; ++u) {
             const WppUnit un = units[u];
             const UnitView v = view_of(un, p, q_offsets);
@@ -447,36 +504,104 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             // stored numbers, so old and new terms stay consistent even for scores around 1e8.
             float m_ref = -INFINITY, l_run = 0.f, nmc = 0.f;
             for (int j = 0; j < n; ++j) {
-                TRACE(hf, tstep, 0);
-                const bool ok = mbar_wait(bSFull(hf), s_phase, abort_flag);
-                if (!__all_sync(0xffffffffu, ok)) { dead = true; break; }
+                {
+                    STAT_T0();
+                    const bool ok = mbar_wait(bSFull(hf), s_phase, abort_flag);
+                    STAT_ADD(0);
+                    STAT_INC(2);
+                    if (!__all_sync(0xffffffffu, ok)) { dead = true; break; }
+                }
                 s_phase ^= 1u;
                 tc_fence_after();
-                TRACE(hf, tstep, 1);
+#ifdef WPP_STATS
+                const uint32_t sta_ = (uint32_t)clock64();
+#endif
+                // copy S out of the landing buffer and hand the buffer back at once
+                float s[128];
+#pragma unroll
+                for (int q4 = 0; q4 < 4; ++q4)
+                    tmem_ld32(lane_addr + kColS + q4 * 32, reinterpret_cast<uint32_t*>(s) + q4 * 32);
+                tmem_wait_ld();
+                tc_fence_before();
+                mbar_arrive(bSFree);
+#ifdef WPP_STATS
+                const uint32_t stb_ = (uint32_t)clock64();
+                stat4_ += stb_ - sta_;
+#endif
 #ifdef WPP_EXPERIMENT_NO_SOFTMAX
                 // tuning experiment: how fast is the tile loop when the softmax costs nothing (results are garbage)
+                {
+                    const bool okp = mbar_wait(bPFree(hf), pf_phase ^ 1u, abort_flag);
+                    if (!__all_sync(0xffffffffu, okp)) { dead = true; break; }
+                    pf_phase ^= 1u;
+                }
                 tc_fence_before();
                 mbar_arrive(bPReady(hf));
                 continue;
 #endif
-                float s[128];
                 const int key0 = (v.kv_begin + j) * 128;
-                const bool masked = key0 + 127 > first_pos;    // only steps that touch the diagonal are masked
-                const int limit = row_last - key0;
-                auto load_scores = [&]() {
+                if (key0 + 127 > first_pos) {                 // only steps that touch the diagonal are masked
+                    const int limit = row_last - key0;
 #pragma unroll
-                    for (int q4 = 0; q4 < 4; ++q4)
-                        tmem_ld32(lane_addr + colS + q4 * 32, reinterpret_cast<uint32_t*>(s) + q4 * 32);
-                    tmem_wait_ld();
-                    if (masked) {
+                    for (int i = 0; i < 128; ++i) s[i] = (i > limit) ? -INFINITY : s[i];
+                }
+                // row maximum of the step: it only decides whether the reference has to move
+                float mx[8];
 #pragma unroll
-                        for (int i = 0; i < 128; ++i) s[i] = (i > limit) ? -INFINITY : s[i];
+                for (int k = 0; k < 8; ++k) mx[k] = fmaxf(s[2 * k], s[2 * k + 1]);
+#pragma unroll
+                for (int i = 16; i < 128; i += 16) {
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) mx[k] = fmax3(mx[k], s[i + 2 * k], s[i + 2 * k + 1]);
+                }
+                const float mxx = fmaxf(fmax3(mx[0], mx[1], mx[2]), fmaxf(fmax3(mx[3], mx[4], mx[5]), fmaxf(mx[6], mx[7])));
+                // Has the previous O += P V of this half been seen to land?  Until then its P may not be replaced
+                // and O may not be rescaled.  (It may belong to the previous tile: the two issuing threads run
+                // independently.  The first wait of the kernel passes at once.)
+                bool waited = false;
+                // The row keeps its reference while 2^(s*c + nmc) <= 2^16 for every score of the step: nothing can
+                // overflow and small terms keep 8 bits below that.  Otherwise (or when the row has no reference
+                // yet) the warp moves its references to the running maxima and rescales O and l.
+                const bool move = (m_ref == -INFINITY) || !(fmaf(mxx, c, nmc) <= kRefSlack);
+                if (__any_sync(0xffffffffu, move)) {
+                    const float m_new = fmaxf(m_ref, mxx);
+                    const float m_safe = (m_new == -INFINITY) ? 0.f : m_new;
+                    const float nmc_new = -m_safe * c;
+                    const float alpha = (m_ref == -INFINITY) ? 0.f : fast_exp2(nmc_new - nmc);
+                    nmc = nmc_new;
+                    m_ref = m_new;
+                    l_run *= alpha;
+                    if (j > 0) {
+                        // O may only be touched once the O += P V of step j-1 has landed
+                        const bool okp = mbar_wait(bPFree(hf), pf_phase ^ 1u, abort_flag);
+                        if (!__all_sync(0xffffffffu, okp)) { dead = true; break; }
+                        pf_phase ^= 1u;
+                        waited = true;
+                        tc_fence_after();
+                        if (__any_sync(0xffffffffu, alpha != 1.f)) {
+                            // eight columns at a time: the 128 scores of the step stay in registers meanwhile
+#pragma unroll 1
+                            for (int q8 = 0; q8 < D / 8; ++q8) {
+                                float o[8];
+                                tmem_ld8(lane_addr + col_o(hf) + q8 * 8, reinterpret_cast<uint32_t*>(o));
+                                tmem_wait_ld();
+#pragma unroll
+                                for (int i = 0; i < 8; ++i) o[i] *= alpha;
+                                tmem_st8(lane_addr + col_o(hf) + q8 * 8, reinterpret_cast<uint32_t*>(o));
+                            }
+                        }
                     }
-                };
-                // p = 2^(s*c - m_ref*c) for the whole row: bf16 pairs for the tensor cores, fp32 row sum
-                uint32_t pk[64];
-                auto exp_pass = [&](float neg_mc) -> float {
-                    const uint64_t nm2 = pack2(neg_mc, neg_mc);
+                }
+#ifdef WPP_STATS
+                const uint32_t stm_ = (uint32_t)clock64();
+                stat3_ += stm_ - stb_;
+#endif
+                // p = 2^(s*c - m_ref*c) for the whole row: bf16 pairs for the tensor cores, fp32 row sum.  The packed
+                // pair i takes the place of score i, which pair i/2 has consumed: the row never needs more than its
+                // 128 registers.
+                uint32_t* pk = reinterpret_cast<uint32_t*>(s);
+                {
+                    const uint64_t nm2 = pack2(nmc, nmc);
                     uint64_t sum2a = pack2(0.f, 0.f), sum2b = pack2(0.f, 0.f);
 #pragma unroll
                     for (int i = 0; i < 64; ++i) {
@@ -501,62 +626,29 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     }
                     float t0, t1;
                     unpack2(fadd2(sum2a, sum2b), t0, t1);
-                    return t0 + t1;
-                };
-                load_scores();
-                TRACE(hf, tstep, 2);
-                // Fast path: keep the row's reference m_ref and skip the row maximum altogether.  The row sum tells
-                // whether that was safe: every p <= row sum, so a sum below 2^16 means no score rose more than 16
-                // (log2 units) above the reference and nothing can overflow.  Otherwise (or when a row has no
-                // reference yet) the warp takes the slow path: true maximum, new reference, O and l rescaled.
-                bool slow = __any_sync(0xffffffffu, m_ref == -INFINITY);
-                float row_sum = 0.f;
-                if (!slow) {
-                    row_sum = exp_pass(nmc);
-                    slow = __any_sync(0xffffffffu, !(row_sum <= kFastPathSumLimit));
-                    if (slow) load_scores();          // S is still intact in tensor memory
+                    l_run += t0 + t1;
                 }
-                TRACE(hf, tstep, 3);
-                if (slow) {
-                    float mx[8];
-#pragma unroll
-                    for (int k = 0; k < 8; ++k) mx[k] = fmaxf(s[2 * k], s[2 * k + 1]);
-#pragma unroll
-                    for (int i = 16; i < 128; i += 16) {
-#pragma unroll
-                        for (int k = 0; k < 8; ++k) mx[k] = fmax3(mx[k], s[i + 2 * k], s[i + 2 * k + 1]);
-                    }
-                    const float mxx = fmaxf(fmax3(mx[0], mx[1], mx[2]), fmaxf(fmax3(mx[3], mx[4], mx[5]), fmaxf(mx[6], mx[7])));
-                    const float m_new = fmaxf(m_ref, mxx);
-                    const float m_safe = (m_new == -INFINITY) ? 0.f : m_new;
-                    const float nmc_new = -m_safe * c;
-                    const float alpha = (m_ref == -INFINITY) ? 0.f : fast_exp2(nmc_new - nmc);
-                    nmc = nmc_new;
-                    m_ref = m_new;
-                    l_run *= alpha;
-                    if (j > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
-                        // S(j) has landed, so the O += P V of step j-1 has too: O may be rescaled in place
-#pragma unroll
-                        for (int q4 = 0; q4 < D / 32; ++q4) {
-                            float o[32];
-                            tmem_ld32(lane_addr + col_o(hf) + q4 * 32, reinterpret_cast<uint32_t*>(o));
-                            tmem_wait_ld();
-#pragma unroll
-                            for (int i = 0; i < 32; ++i) o[i] *= alpha;
-                            tmem_st32(lane_addr + col_o(hf) + q4 * 32, reinterpret_cast<uint32_t*>(o));
-                        }
-                    }
-                    row_sum = exp_pass(nmc);
+#ifdef WPP_STATS
+                const uint32_t stc_ = (uint32_t)clock64();
+                stat5_ += stc_ - stm_;
+#endif
+                if (!waited) {
+                    // P(j-1) must have been consumed before P(j) replaces it
+                    STAT_T0();
+                    const bool okp = mbar_wait(bPFree(hf), pf_phase ^ 1u, abort_flag);
+                    STAT_ADD(1);
+                    if (!__all_sync(0xffffffffu, okp)) { dead = true; break; }
+                    pf_phase ^= 1u;
+                    tc_fence_after();
                 }
-                l_run += row_sum;
-                TRACE(hf, tstep, 4);
-                tmem_st32(lane_addr + colS, pk);
-                tmem_st32(lane_addr + colS + 32, pk + 32);
+                tmem_st32(lane_addr + col_p(hf), pk);
+                tmem_st32(lane_addr + col_p(hf) + 32, pk + 32);
                 tmem_wait_st();
                 tc_fence_before();
                 mbar_arrive(bPReady(hf));
-                TRACE(hf, tstep, 5);
-                ++tstep;
+#ifdef WPP_STATS
+                stat6_ += (uint32_t)clock64() - stc_;
+#endif
             }
             if (dead) break;
             {
@@ -569,6 +661,7 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             s_final[hf * 128 + r] = make_float2(-nmc, l_run);
             mbar_arrive(bFinalReady(hf));
         }
+        STAT_FLUSH(2 + hf, r == 0);
     }
 
     // ---- teardown: every loop above is bounded, so every thread gets here
