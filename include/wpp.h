@@ -96,9 +96,10 @@ typedef struct {
     int32_t tile_n;           /* keys per inner step: 128 */
     int32_t force_kv_splits;  /* >= 2: split every tile's key range into this many parts (when it has that many
                                  key steps); 1: never split; 0: library decides */
-    int32_t max_ctas;         /* persistent CTAs to plan for (default: SM count of the context, 148 without one) */
-    int32_t order;            /* 0: stream order - tiles that read the same (request, KV head) pages run at the same
-                                 time, so the pages are fetched from DRAM once and shared through L2; 1: longest
+    int32_t max_ctas;         /* persistent CTAs to launch (default: SM count of the context, 148 without one) */
+    int32_t order;            /* order in which the persistent CTAs take the tiles at run time.  0: stream order -
+                                 tiles that read the same (request, KV head) pages are neighbours and so run at the
+                                 same time: the pages are fetched from DRAM once and shared through L2; 1: longest
                                  tile first */
 } wpp_plan_opts;
 
@@ -110,7 +111,7 @@ typedef struct {
     int64_t total_new_tokens;   /* T */
     int64_t key_steps;          /* sum over tiles of 128-row x 128-key steps (work incl. tile quantisation) */
     int64_t flops;              /* algorithmic: 4 * d * Hq * sum_i (C_i P_i + C_i (C_i + 1) / 2) */
-    size_t workspace_bytes;     /* device scratch wpp_prefill_attention_varlen needs for this plan (may be 0) */
+    size_t workspace_bytes;     /* device scratch wpp_prefill_attention_varlen needs for this plan (never 0) */
     size_t plan_bytes;          /* bytes of plan_host actually used; copy that many to the device */
 } wpp_plan_info;
 
@@ -121,8 +122,9 @@ size_t wpp_plan_bytes(const wpp_ctx* ctx_or_null, const wpp_batch_desc* desc, in
 
 /* Host-side work split (integer arithmetic only; no CUDA call).  Cuts the wave into work tiles
  * (request, query-row range, query head, key-step range), decides which tiles are split along the keys,
- * orders them (opts->order) and list-schedules them onto persistent CTAs, and sizes the workspace.  Equal-sized chunks
- * cost different amounts because they attend to different prefix lengths (Section 6), hence cost = key steps.
+ * orders them (opts->order) and sizes the workspace; the persistent CTAs of the attention kernel take tiles in that
+ * order as they become free.  Equal-sized chunks cost different amounts because they attend to different prefix
+ * lengths (Section 6), which is why tiles are not preassigned to CTAs.
  *   prefix_lens_host, chunk_lens_host : host int32 [R].
  *   cached_lens_host_or_null          : host int32 [R]; tokens each request really has in the cache after
  *                                       materialisation.  If given and != prefix_lens, returns
@@ -166,10 +168,13 @@ int wpp_kv_append(const wpp_ctx* ctx, const wpp_batch_desc* desc, const void* k_
  *   q, out        : device bf16 [T][Hq][d];  lse_or_null : device fp32 [T][Hq].
  *   k_cache, v_cache, block_tables, prefix_lens, chunk_lens : device, read only.
  *   plan_host / plan_dev : as for wpp_kv_append.
- *   workspace     : device scratch of >= info.workspace_bytes bytes, 256-byte aligned (NULL allowed when 0);
- *                   holds split-KV partial results; contents are undefined afterwards.
- * Launches one persistent kernel, plus one combine kernel iff the plan has split tiles.  Results are
- * bit-reproducible for a given plan (no atomics on outputs; partials are merged in a fixed order). */
+ *   workspace     : device scratch of >= info.workspace_bytes bytes, 256-byte aligned, required: holds the
+ *                   counter the persistent CTAs take their tiles from (zeroed by this call on the stream) and
+ *                   the split-KV partial results; contents are undefined afterwards.  Two calls that may run
+ *                   at the same time need a workspace each.
+ * Enqueues a 256-byte memset and one persistent kernel, plus one combine kernel iff the plan has split tiles.
+ * Results are bit-reproducible for a given plan, whichever CTA takes which tile (no atomics on outputs; partials
+ * are merged in a fixed order). */
 int wpp_prefill_attention_varlen(const wpp_ctx* ctx, const wpp_batch_desc* desc, const void* q, void* out,
                                  float* lse_or_null, const void* k_cache, const void* v_cache,
                                  const int32_t* block_tables, const int32_t* prefix_lens,

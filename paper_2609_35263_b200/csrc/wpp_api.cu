@@ -154,10 +154,9 @@ extern "C" int wpp_prefill_attention_varlen(const wpp_ctx* ctx, const wpp_batch_
         return WPP_ERR_INVALID_ARG;
     if (!aligned16(q) || !aligned16(out) || !aligned16(k_cache) || !aligned16(v_cache) || !aligned16(plan_dev))
         return WPP_ERR_INVALID_ARG;
-    if (hd->workspace_bytes > 0) {
-        if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255) != 0) return WPP_ERR_INVALID_ARG;
-        if (workspace_bytes < hd->workspace_bytes) return WPP_ERR_WORKSPACE_TOO_SMALL;
-    }
+    // the workspace always holds the tile counter, and the split partials behind it when the plan has any
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255) != 0) return WPP_ERR_INVALID_ARG;
+    if (workspace_bytes < hd->workspace_bytes) return WPP_ERR_WORKSPACE_TOO_SMALL;
     if (d.num_pages == 0) return WPP_ERR_INVALID_ARG;
 
     CUtensorMap tq[4], tk, tv;
@@ -185,8 +184,9 @@ extern "C" int wpp_prefill_attention_varlen(const wpp_ctx* ctx, const wpp_batch_
     p.chunk_lens = chunk_lens;
     p.out = static_cast<__nv_bfloat16*>(out);
     p.lse = lse_or_null;
-    p.ws_o = static_cast<float*>(workspace);
-    p.ws_lse = p.ws_o ? p.ws_o + (size_t)hd->num_split_slots * 2 * WPP_HALF_M * d.head_dim : nullptr;
+    p.tile_counter = static_cast<uint32_t*>(workspace);
+    p.ws_o = reinterpret_cast<float*>(static_cast<char*>(workspace) + WPP_WS_HEADER_BYTES);
+    p.ws_lse = p.ws_o + (size_t)hd->num_split_slots * 2 * WPP_HALF_M * d.head_dim;
     p.status = status_dev;
     p.o_token_stride = d.o_token_stride;
     p.o_head_stride = d.o_head_stride;
@@ -204,7 +204,10 @@ extern "C" int wpp_prefill_attention_varlen(const wpp_ctx* ctx, const wpp_batch_
     }
 #endif
 
-    int e = wpp_launch_attention(d.head_dim, tq, &tk, &tv, &p, hd->num_ctas, cuda_stream);
+    // the counter the CTAs take their tiles from starts at zero (a memset node on the caller's stream)
+    int e = (int)cudaMemsetAsync(workspace, 0, WPP_WS_HEADER_BYTES, (cudaStream_t)cuda_stream);
+    if (e != 0) return cuda_fail(ctx, e);
+    e = wpp_launch_attention(d.head_dim, tq, &tk, &tv, &p, hd->num_ctas, cuda_stream);
     if (e != 0) return cuda_fail(ctx, e);
     const_cast<wpp_ctx*>(ctx)->launches += 1;
     if (hd->num_combine > 0) {

@@ -44,17 +44,22 @@ __host__ __device__ constexpr uint32_t col_o(int hf) { return 256u + 128u * hf; 
 // registers per thread after the warpgroups re-split the register file (8 x kRegsSoftmax + 4 x kRegsEpilogue +
 // 4 x kRegsUtil <= 2048 per thread slot of 32 lanes, i.e. 65536 in all)
 #ifndef WPP_REGS_SOFTMAX
-#define WPP_REGS_SOFTMAX 176
-#define WPP_REGS_EPILOGUE 64
-#define WPP_REGS_UTIL 96
+#define WPP_REGS_SOFTMAX 192
+#define WPP_REGS_EPILOGUE 56
+#define WPP_REGS_UTIL 72
 #endif
 constexpr int kRegsSoftmax = WPP_REGS_SOFTMAX, kRegsEpilogue = WPP_REGS_EPILOGUE, kRegsUtil = WPP_REGS_UTIL;
 static_assert(8 * kRegsSoftmax + 4 * kRegsEpilogue + 4 * kRegsUtil <= 2048, "register file exceeded");
-constexpr float kRefSlack = 16.f;   // a row keeps its reference while its scores stay below reference + 16 (log2)
-#ifndef WPP_EMU_PAIRS_OF_4
-#define WPP_EMU_PAIRS_OF_4 0
+// arrivals on s_free and p_ready: every softmax thread (128), or one elected lane per warp after __syncwarp (4)
+#ifndef WPP_ELECT_ARRIVE
+#define WPP_ELECT_ARRIVE 0
 #endif
-constexpr int kEmuPairsOf4 = WPP_EMU_PAIRS_OF_4;  // of every 4 score pairs, how many take exp2 on the FMA pipes
+constexpr uint32_t kSoftmaxArrivals = WPP_ELECT_ARRIVE ? 4 : 128;
+constexpr float kRefSlack = 16.f;   // a row keeps its reference while its scores stay below reference + 16 (log2)
+#ifndef WPP_EXP_BLOCK
+#define WPP_EXP_BLOCK 8
+#endif
+constexpr int kExpBlock = WPP_EXP_BLOCK;   // score pairs whose exponentials are in flight together
 
 template <int D>
 struct Cfg {
@@ -64,10 +69,11 @@ struct Cfg {
     static constexpr int kSlots = (D == 128) ? 5 : 8;      // ring of K / V tiles (4 if the base is badly aligned)
     static constexpr int kOffKV = 2 * kTileBytes;
     static constexpr int kOffBars = kOffKV + kSlots * kTileBytes;
-    static constexpr int kNumBars = 2 + 2 * kSlots + 1 + 6 * 2;
+    static constexpr int kTileQ = 2;                       // tile ids the producer may publish ahead
+    static constexpr int kNumBars = 2 + 2 * kSlots + 1 + 6 * 2 + 2 * kTileQ;
     static constexpr int kOffFinal = kOffBars + 8 * kNumBars;          // float2 (m, l)[2][128]
-    static constexpr int kOffMisc = kOffFinal + 2 * 128 * 8;           // tmem ptr, abort flag
-    static constexpr int kUsedBytes = kOffMisc + 16;
+    static constexpr int kOffMisc = kOffFinal + 2 * 128 * 8;           // tmem ptr, abort flag, tile ids
+    static constexpr int kUsedBytes = kOffMisc + 16 + 4 * kTileQ + 8;
     static constexpr int kMaxSmem = 232448;                            // 227 KB: the most a CTA can have
     static constexpr int kSmemBytes = (kUsedBytes + 1024 < kMaxSmem) ? kUsedBytes + 1024 : kMaxSmem;
 };
@@ -140,8 +146,12 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
     // the tile ring gives up one slot when the 1024-byte alignment of the base costs more than the spare bytes
+#ifdef WPP_FORCE_SMALL_RING
+    const uint32_t n_slots = C::kSlots - 1;              // test builds: always take the fallback
+#else
     const uint32_t n_slots =
         (smem_base - smem_u32(smem_raw)) + (uint32_t)C::kUsedBytes <= (uint32_t)C::kSmemBytes ? C::kSlots : C::kSlots - 1;
+#endif
     const uint32_t sQ = smem_base;                       // two halves, kTileBytes each
     const uint32_t sKV = smem_base + C::kOffKV;          // kSlots tiles (K or V)
     const uint32_t bars = smem_base + C::kOffBars;
@@ -161,9 +171,16 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     auto bFinalReady = [&](int h) { return bHalf + 48 * h + 24; };
     auto bOFinal = [&](int h) { return bHalf + 48 * h + 32; };
     auto bOFree = [&](int h) { return bHalf + 48 * h + 40; };
+    // Work tiles are not preassigned: the producer warp takes the next tile of the planner's order from a counter
+    // in global memory and publishes its index to the other roles through a small queue in shared memory, so the
+    // CTAs of the grid always work on neighbouring tiles of that order (which share K/V pages, see the planner)
+    // however their speeds differ, and the tail balances itself.
+    const uint32_t bTileFull = bHalf + 96, bTileEmpty = bTileFull + 8 * C::kTileQ;
     float2* s_final = reinterpret_cast<float2*>(smem_gen + C::kOffFinal);     // [2][128] (reference in log2 units, l)
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_gen + C::kOffMisc);
     volatile uint32_t* abort_flag = tmem_slot + 1;
+    volatile int32_t* tile_ids = reinterpret_cast<volatile int32_t*>(tmem_slot + 4);      // [kTileQ]
+    constexpr uint32_t kTileConsumers = 2 + 256 + 128;   // two issuing threads, softmax threads, epilogue threads
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int wg = warp >> 2;
@@ -171,11 +188,12 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     if (threadIdx.x == 0) {
         mbar_init(bQFull, 1); mbar_init(bQEmpty, 1);
         for (int s = 0; s < C::kSlots; ++s) { mbar_init(bSlotFull + 8 * s, 1); mbar_init(bSlotEmpty + 8 * s, 1); }
-        mbar_init(bSFree, 128);
+        mbar_init(bSFree, kSoftmaxArrivals);
         for (int h = 0; h < 2; ++h) {
-            mbar_init(bSFull(h), 1); mbar_init(bPReady(h), 128); mbar_init(bPFree(h), 1);
+            mbar_init(bSFull(h), 1); mbar_init(bPReady(h), kSoftmaxArrivals); mbar_init(bPFree(h), 1);
             mbar_init(bFinalReady(h), 128); mbar_init(bOFinal(h), 1); mbar_init(bOFree(h), 128);
         }
+        for (int i = 0; i < C::kTileQ; ++i) { mbar_init(bTileFull + 8 * i, 1); mbar_init(bTileEmpty + 8 * i, kTileConsumers); }
         *abort_flag = 0u;
         fence_barrier_init();
     }
@@ -195,9 +213,17 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     const char* plan = static_cast<const char*>(p.plan);
     const WppPlanHeader* hd = reinterpret_cast<const WppPlanHeader*>(plan);
     const int32_t* q_offsets = reinterpret_cast<const int32_t*>(plan + hd->off_q_offsets);
-    const int32_t* cta_begin = reinterpret_cast<const int32_t*>(plan + hd->off_cta_begin);
     const WppUnit* units = reinterpret_cast<const WppUnit*>(plan + hd->off_units);
-    const int u_begin = cta_begin[blockIdx.x], u_end = cta_begin[blockIdx.x + 1];
+    const int num_units = hd->num_units;
+    // next tile index for a consuming role: -1 = no more tiles, -2 = the wait was abandoned
+    Ring tile_ring = {0, 0};
+    auto next_tile = [&]() -> int {
+        if (!mbar_wait(bTileFull + 8 * tile_ring.stage, tile_ring.phase, abort_flag)) return -2;
+        const int id = tile_ids[tile_ring.stage];
+        mbar_arrive(bTileEmpty + 8 * tile_ring.stage);
+        tile_ring.advance(C::kTileQ);
+        return id;
+    };
     const int B = p.page_size, ppt = 128 / B;   // pages per key step
 
     if (wg == 3) {
@@ -212,7 +238,22 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             uint32_t q_phase = 0;
             bool dead = false;
             STAT_DECL();
-            for (int u = u_begin; u < u_end && !dead; ++u) {
+            while (!dead) {
+                // take the next tile of the planner's order and tell the other roles
+                int u = 0;
+                if (lane == 0) u = (int)atomicAdd(p.tile_counter, 1u);
+                u = __shfl_sync(0xffffffffu, u, 0);
+                if (u >= num_units) u = -1;
+                {
+                    const bool ok = mbar_wait(bTileEmpty + 8 * tile_ring.stage, tile_ring.phase ^ 1u, abort_flag);
+                    if (!__all_sync(0xffffffffu, ok)) break;
+                    if (lane == 0) {
+                        tile_ids[tile_ring.stage] = u;
+                        mbar_arrive(bTileFull + 8 * tile_ring.stage);
+                    }
+                    tile_ring.advance(C::kTileQ);
+                }
+                if (u < 0) break;
                 const WppUnit un = units[u];
                 const UnitView v = view_of(un, p, q_offsets);
                 if (v.n_steps == 0) continue;
@@ -289,7 +330,9 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             const uint32_t tS = tmem + kColS;
             bool dead = false;
             STAT_DECL();
-            for (int u = u_begin; u < u_end && !dead; ++u) {
+            while (!dead) {
+                const int u = next_tile();
+                if (u < 0) break;
                 const WppUnit un = units[u];
                 const UnitView v = view_of(un, p, q_offsets);
                 if (v.n_steps == 0) continue;
@@ -346,7 +389,9 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             const uint64_t v_desc0 = smem_desc_sw128(sKV, C::kHalfBytes, 1024);       // + stage * (kTileBytes >> 4)
             bool dead = false;
             STAT_DECL();
-            for (int u = u_begin; u < u_end && !dead; ++u) {
+            while (!dead) {
+                const int u = next_tile();
+                if (u < 0) break;
                 const WppUnit un = units[u];
                 const UnitView v = view_of(un, p, q_offsets);
                 if (v.n_steps == 0) continue;
@@ -411,7 +456,9 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         const uint32_t lane_addr = tmem + ((uint32_t)((warp & 3) * 32) << 16);
         uint32_t o_phase[2] = {0, 0}, f_phase[2] = {0, 0};
         bool dead = false;
-        for (int u = u_begin; u < u_end && !dead; ++u) {
+        while (!dead) {
+            const int u = next_tile();
+            if (!__all_sync(0xffffffffu, u != -2) || u < 0) break;
             const WppUnit un = units[u];
             const UnitView v = view_of(un, p, q_offsets);
             // ---- epilogue of both halves
@@ -490,7 +537,9 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         const uint64_t c2 = pack2(c, c);
         bool dead = false;
         STAT_DECL();
-        for (int u = u_begin; u < u_end && !dead; ++u) {
+        while (!dead) {
+            const int u = next_tile();
+            if (!__all_sync(0xffffffffu, u != -2) || u < 0) break;
             const WppUnit un = units[u];
             const UnitView v = view_of(un, p, q_offsets);
             const int n = v.n[hf];
@@ -513,7 +562,7 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 }
                 s_phase ^= 1u;
                 tc_fence_after();
-#ifdef WPP_STATS
+#ifdef WPP_STATS_FINE
                 const uint32_t sta_ = (uint32_t)clock64();
 #endif
                 // copy S out of the landing buffer and hand the buffer back at once
@@ -523,8 +572,13 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     tmem_ld32(lane_addr + kColS + q4 * 32, reinterpret_cast<uint32_t*>(s) + q4 * 32);
                 tmem_wait_ld();
                 tc_fence_before();
-                mbar_arrive(bSFree);
-#ifdef WPP_STATS
+                if (WPP_ELECT_ARRIVE) {
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bSFree);
+                } else {
+                    mbar_arrive(bSFree);
+                }
+#ifdef WPP_STATS_FINE
                 const uint32_t stb_ = (uint32_t)clock64();
                 stat4_ += stb_ - sta_;
 #endif
@@ -592,7 +646,7 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                         }
                     }
                 }
-#ifdef WPP_STATS
+#ifdef WPP_STATS_FINE
                 const uint32_t stm_ = (uint32_t)clock64();
                 stat3_ += stm_ - stb_;
 #endif
@@ -603,32 +657,40 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 {
                     const uint64_t nm2 = pack2(nmc, nmc);
                     uint64_t sum2a = pack2(0.f, 0.f), sum2b = pack2(0.f, 0.f);
+                    // in blocks of kExpBlock pairs: all scalings, then all exponentials, then sums and packing, so
+                    // that the special-function unit always has independent work queued
 #pragma unroll
-                    for (int i = 0; i < 64; ++i) {
-                        const uint64_t x2 = ffma2(pack2(s[2 * i], s[2 * i + 1]), c2, nm2);
-                        float e0, e1;
-                        if ((i & 3) < kEmuPairsOf4) {
-                            exp2_poly2(x2, e0, e1);
-                        } else {
+                    for (int i0 = 0; i0 < 64; i0 += kExpBlock) {
+                        uint64_t x2[kExpBlock];
+                        float e[2 * kExpBlock];
+#pragma unroll
+                        for (int k = 0; k < kExpBlock; ++k)
+                            x2[k] = ffma2(pack2(s[2 * (i0 + k)], s[2 * (i0 + k) + 1]), c2, nm2);
+#pragma unroll
+                        for (int k = 0; k < kExpBlock; ++k) {
                             float x0, x1;
-                            unpack2(x2, x0, x1);
+                            unpack2(x2[k], x0, x1);
 #ifdef WPP_EXPERIMENT_CHEAP_EXP
                             // tuning experiment: the same loop without the special-function unit (results are garbage)
-                            e0 = __saturatef(x0 * 0.01f + 0.5f);
-                            e1 = __saturatef(x1 * 0.01f + 0.5f);
+                            e[2 * k] = __saturatef(x0 * 0.01f + 0.5f);
+                            e[2 * k + 1] = __saturatef(x1 * 0.01f + 0.5f);
 #else
-                            e0 = fast_exp2(x0);
-                            e1 = fast_exp2(x1);
+                            e[2 * k] = fast_exp2(x0);
+                            e[2 * k + 1] = fast_exp2(x1);
 #endif
                         }
-                        if (i & 1) sum2b = fadd2(sum2b, pack2(e0, e1)); else sum2a = fadd2(sum2a, pack2(e0, e1));
-                        pk[i] = pack_bf16x2(e0, e1);
+#pragma unroll
+                        for (int k = 0; k < kExpBlock; ++k) {
+                            if (k & 1) sum2b = fadd2(sum2b, pack2(e[2 * k], e[2 * k + 1]));
+                            else sum2a = fadd2(sum2a, pack2(e[2 * k], e[2 * k + 1]));
+                            pk[i0 + k] = pack_bf16x2(e[2 * k], e[2 * k + 1]);
+                        }
                     }
                     float t0, t1;
                     unpack2(fadd2(sum2a, sum2b), t0, t1);
                     l_run += t0 + t1;
                 }
-#ifdef WPP_STATS
+#ifdef WPP_STATS_FINE
                 const uint32_t stc_ = (uint32_t)clock64();
                 stat5_ += stc_ - stm_;
 #endif
@@ -645,8 +707,13 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 tmem_st32(lane_addr + col_p(hf) + 32, pk + 32);
                 tmem_wait_st();
                 tc_fence_before();
-                mbar_arrive(bPReady(hf));
-#ifdef WPP_STATS
+                if (WPP_ELECT_ARRIVE) {
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bPReady(hf));
+                } else {
+                    mbar_arrive(bPReady(hf));
+                }
+#ifdef WPP_STATS_FINE
                 stat6_ += (uint32_t)clock64() - stc_;
 #endif
             }

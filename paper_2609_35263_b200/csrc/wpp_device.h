@@ -18,6 +18,7 @@ struct AttnParams {
     float* ws_o;                     // split partials: [slots][2][128][d]
     float* ws_lse;                   // [slots][2][128], log2 units
     int32_t* status;                 // sticky device status word or null
+    uint32_t* tile_counter;          // zeroed before the launch: index of the next tile nobody has taken yet
     int64_t o_token_stride, o_head_stride;
     int32_t num_q_heads, group, page_size, max_blocks, num_pages;
     float scale_log2;                // sm_scale * log2(e)

@@ -237,8 +237,8 @@ int wpp_plan_tiles(const wpp_ctx* ctx, const wpp_batch_desc* desc, const int32_t
     const int64_t n_units = (int64_t)units.size();
     if (n_units > 0x7fffffff) return WPP_ERR_INVALID_ARG;
 
-    // ---- order of execution, then list scheduling onto persistent CTAs (each tile goes to the CTA that is
-    //      free first, so tiles adjacent in the order run at the same time on different SMs).
+    // ---- order of execution.  The persistent CTAs take tiles in this order at run time (a counter in the
+    //      workspace), so tiles adjacent in the order run at the same time on different SMs.
     //      order 0 (default), "stream order": KV head major, then requests (longest first), then row blocks and
     //      heads.  All tiles that read one (request, KV head) stream start together and walk its pages in step,
     //      so a page comes from DRAM once and is then hit in L2 by the other tiles; a prefix shared by many
@@ -269,18 +269,6 @@ int wpp_plan_tiles(const wpp_ctx* ctx, const wpp_batch_desc* desc, const int32_t
             return req_rank[(size_t)ua.request] < req_rank[(size_t)ub.request];
         });
     }
-    typedef std::pair<int64_t, int32_t> Load;  // (accumulated cost, cta)
-    std::priority_queue<Load, std::vector<Load>, std::greater<Load>> heap;
-    for (int c = 0; c < num_ctas; ++c) heap.push({0, c});
-    std::vector<std::vector<int32_t>> lists((size_t)num_ctas);
-    for (int32_t u : order) {
-        Load l = heap.top();
-        heap.pop();
-        lists[(size_t)l.second].push_back(u);
-        l.first += std::max(1, units[(size_t)u].cost);
-        heap.push(l);
-    }
-
     // ---- serialise
     WppPlanHeader hd;
     std::memset(&hd, 0, sizeof(hd));
@@ -298,12 +286,10 @@ int wpp_plan_tiles(const wpp_ctx* ctx, const wpp_batch_desc* desc, const int32_t
     hd.total_new_tokens = T;
     hd.key_steps = key_steps;
     hd.flops = 4 * (int64_t)d.head_dim * Hq * pairs;
-    hd.workspace_bytes = slots ? align_up((size_t)slots * 2 * WPP_HALF_M * (d.head_dim + 1) * sizeof(float), 256) : 0;
+    hd.workspace_bytes = WPP_WS_HEADER_BYTES + align_up((size_t)slots * 2 * WPP_HALF_M * (d.head_dim + 1) * sizeof(float), 256);
     size_t off = sizeof(WppPlanHeader);
     hd.off_q_offsets = (uint32_t)off;
     off += align_up(sizeof(int32_t) * (size_t)(R + 1), 16);
-    hd.off_cta_begin = (uint32_t)off;
-    off += align_up(sizeof(int32_t) * (size_t)(num_ctas + 1), 16);
     hd.off_units = (uint32_t)off;
     off += sizeof(WppUnit) * (size_t)n_units;
     hd.off_combine = (uint32_t)off;
@@ -317,14 +303,8 @@ int wpp_plan_tiles(const wpp_ctx* ctx, const wpp_batch_desc* desc, const int32_t
     int32_t* qo = reinterpret_cast<int32_t*>(p + hd.off_q_offsets);
     qo[0] = 0;
     for (int i = 0; i < R; ++i) qo[i + 1] = qo[i] + chunk_lens[i];
-    int32_t* cb = reinterpret_cast<int32_t*>(p + hd.off_cta_begin);
     WppUnit* us = reinterpret_cast<WppUnit*>(p + hd.off_units);
-    int32_t k = 0;
-    for (int c = 0; c < num_ctas; ++c) {
-        cb[c] = k;
-        for (int32_t u : lists[(size_t)c]) us[k++] = units[(size_t)u];
-    }
-    cb[num_ctas] = k;
+    for (int64_t k = 0; k < n_units; ++k) us[k] = units[(size_t)order[(size_t)k]];
     if (!combines.empty())
         std::memcpy(p + hd.off_combine, combines.data(), sizeof(WppCombine) * combines.size());
 

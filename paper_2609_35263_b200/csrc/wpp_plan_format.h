@@ -4,8 +4,9 @@
 #include <stdint.h>
 
 #define WPP_PLAN_MAGIC 0x31505057u /* "WPP1" */
-#define WPP_PLAN_VERSION 4u
+#define WPP_PLAN_VERSION 5u
 #define WPP_TILE_N 128             /* keys per step */
+#define WPP_WS_HEADER_BYTES 256
 #define WPP_HALF_M 128             /* query rows per tensor-core tile (one TMEM lane per row) */
 
 struct WppPlanHeader {
@@ -17,8 +18,8 @@ struct WppPlanHeader {
     int64_t total_new_tokens, key_steps, flops;
     uint64_t workspace_bytes, plan_bytes;
     uint32_t off_q_offsets;         // int32 [R+1]   exclusive scan of chunk_lens
-    uint32_t off_cta_begin;         // int32 [num_ctas+1] range of units owned by each persistent CTA
-    uint32_t off_units;             // WppUnit [num_units]
+    uint32_t reserved0;
+    uint32_t off_units;             // WppUnit [num_units] in the order the persistent CTAs take them
     uint32_t off_combine;           // WppCombine [num_combine]
     uint32_t pad[8];
 };
@@ -35,7 +36,7 @@ struct WppUnit {
     int32_t request, kv_begin, kv_end;
     int32_t split_slot;             // -1: writes the final output; else partial slot in the workspace
     int32_t row0[2], rows[2], head[2];
-    int32_t cost;                   // 128x128 steps over both halves, what the CTA assignment balanced
+    int32_t cost;                   // 128x128 steps over both halves
     int32_t pack;                   // query heads per half: 1, 2, 4 or 8
 };
 
@@ -47,5 +48,7 @@ struct WppCombine {
     int32_t lane0;                  // first tensor row of this head inside the half (packed heads)
 };
 
-// Workspace layout: fp32 O_part[num_split_slots][2][128][head_dim] followed by fp32 lse_part[num_split_slots][2][128]
-// (log2 units of the scaled scores; -inf marks a row with no visible key in that part).
+// Workspace layout: WPP_WS_HEADER_BYTES of header (a uint32 counter: the next tile of the order nobody has taken
+// yet; the attention call zeroes it on the stream before the launch), then fp32
+// O_part[num_split_slots][2][128][head_dim] followed by fp32 lse_part[num_split_slots][2][128] (log2 units of the
+// scaled scores; -inf marks a row with no visible key in that part).

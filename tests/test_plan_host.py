@@ -23,16 +23,15 @@ def parse_plan(plan):
     raw = plan.host_bytes()
     f = struct.unpack_from(HDR_FMT, raw, 0)
     (magic, version, desc_hash, R, num_ctas, num_units, num_combine, num_slots, tile_m, tile_n, head_dim,
-     T, key_steps, flops, ws_bytes, plan_bytes, off_q, off_cta, off_units, off_comb) = f
+     T, key_steps, flops, ws_bytes, plan_bytes, off_q, _reserved, off_units, off_comb) = f
     assert magic == 0x31505057
     q_off = np.frombuffer(raw, dtype=np.int32, count=R + 1, offset=off_q)
-    cta = np.frombuffer(raw, dtype=np.int32, count=num_ctas + 1, offset=off_cta)
     units = np.frombuffer(raw, dtype=np.int32, count=num_units * 12, offset=off_units).reshape(num_units, 12)
     comb = np.frombuffer(raw, dtype=np.int32, count=num_combine * 8, offset=off_comb).reshape(num_combine, 8)
     keys = ["request", "kv_begin", "kv_end", "split_slot", "row0_a", "row0_b", "rows_a", "rows_b", "head_a",
             "head_b", "cost", "pack"]
     return dict(R=R, num_ctas=num_ctas, tile_m=tile_m, T=T, key_steps=key_steps, flops=flops, slots=num_slots,
-                ws_bytes=ws_bytes, q_off=q_off, cta=cta, comb=comb,
+                ws_bytes=ws_bytes, q_off=q_off, comb=comb,
                 units=[dict(zip(keys, u.tolist())) for u in units])
 
 
@@ -75,8 +74,7 @@ def test_plan_covers_every_visible_pair_exactly_once(P, C, Hq, Hkv, tile_m, spli
     plan = wpp.wpp_plan_tiles(None, d, P, C, opts=wpp.PlanOpts(tile_m, 0, splits, 40), pin=False)
     pl = parse_plan(plan)
     assert pl["T"] == sum(C) and pl["q_off"].tolist() == np.concatenate([[0], np.cumsum(C)]).tolist()
-    # CTA ownership is a partition of the unit list
-    assert pl["cta"][0] == 0 and pl["cta"][-1] == len(pl["units"]) and np.all(np.diff(pl["cta"]) >= 0)
+    assert 1 <= pl["num_ctas"] <= 40
     G = Hq // Hkv
     cover = {}
     steps_total = 0
@@ -121,10 +119,20 @@ def test_plan_covers_every_visible_pair_exactly_once(P, C, Hq, Hkv, tile_m, spli
                    for p_ in parts)
         assert parts[-1]["kv_end"] >= (P[req] + row0 + rows + 127) // 128
     if splits >= 2 and max((p + c + 127) // 128 for p, c in zip(P, C)) >= 2:
-        assert pl["slots"] > 0 and pl["ws_bytes"] >= pl["slots"] * 2 * 128 * 129 * 4
+        assert pl["slots"] > 0 and pl["ws_bytes"] >= 256 + pl["slots"] * 2 * 128 * 129 * 4
 
 
-def test_plan_is_deterministic_and_balanced():
+def _greedy_finish_times(costs, n_ctas):
+    """Finish time of every CTA when free CTAs take the tiles in list order (what the kernel's counter does)."""
+    import heapq
+    heap = [(0, c) for c in range(n_ctas)]
+    for cost in costs:
+        t, c = heapq.heappop(heap)
+        heapq.heappush(heap, (t + max(1, cost), c))
+    return [t for t, _ in heap]
+
+
+def test_plan_is_deterministic_and_its_order_balances():
     rng = np.random.default_rng(5)
     P = (rng.integers(0, 100, 24) * 64).tolist()
     C = rng.integers(1, 2000, 24).tolist()
@@ -135,25 +143,26 @@ def test_plan_is_deterministic_and_balanced():
         b = wpp.wpp_plan_tiles(None, d, P, C, opts=opts, pin=False)
         assert a.host_bytes() == b.host_bytes()
         pl = parse_plan(a)
-        loads = [sum(u["cost"] for u in pl["units"][pl["cta"][c]:pl["cta"][c + 1]]) for c in range(pl["num_ctas"])]
-        biggest = max(u["cost"] for u in pl["units"])
-        assert max(loads) - min(loads) <= biggest          # list scheduling: nobody idles longer than one tile
-        for c in range(pl["num_ctas"]):
-            mine = pl["units"][pl["cta"][c]:pl["cta"][c + 1]]
-            if order == 1:                                 # longest first: each CTA walks decreasing costs
-                costs = [u["cost"] for u in mine]
-                assert costs == sorted(costs, reverse=True)
-            else:                                          # stream order: KV heads never go backwards on a CTA
-                kv = [u["head_a"] // 4 for u in mine]
-                assert kv == sorted(kv)
+        costs = [u["cost"] for u in pl["units"]]
+        finish = _greedy_finish_times(costs, pl["num_ctas"])
+        assert max(finish) - min(finish) <= max(costs)     # taking tiles in order: nobody idles longer than one tile
+        if order == 1:                                     # longest first
+            assert costs == sorted(costs, reverse=True)
+        else:                                              # stream order: KV head major, a request's tiles together
+            kv = [u["head_a"] // 4 for u in pl["units"]]
+            assert kv == sorted(kv)
+            for g in range(4):
+                reqs = [u["request"] for u in pl["units"] if u["head_a"] // 4 == g]
+                runs = [r for i, r in enumerate(reqs) if i == 0 or reqs[i - 1] != r]
+                assert len(runs) == len(set(runs))         # each request appears as one contiguous run
 
 
 def test_stream_order_runs_the_tiles_of_one_kv_stream_together():
     d = desc(3, 16, 4, 128, 64, 200)
     pl = parse_plan(wpp.wpp_plan_tiles(None, d, [4096, 0, 8192], [1024, 512, 256], opts=wpp.PlanOpts(256, 0, 1, 8),
                                        pin=False))
-    # the first tile of every CTA belongs to KV head 0 of the costliest request (request 0: 4 row blocks x 4 heads)
-    firsts = [pl["units"][pl["cta"][c]] for c in range(pl["num_ctas"])]
+    # the first tiles (one per CTA) belong to KV head 0 of the costliest request (request 0: 4 row blocks x 4 heads)
+    firsts = pl["units"][:pl["num_ctas"]]
     assert all(u["request"] == 0 and u["head_a"] // 4 == 0 for u in firsts)
 
 
