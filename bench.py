@@ -32,7 +32,7 @@ METRIC = "prefill-attention tokens/s at concurrency 128, high prefix reuse"
 # From profiles/attention_cfg3_dram.md: dram__bytes_read.sum + dram__bytes_write.sum of one attention launch on the
 # full concurrency-128 workload (a one-pass ncu capture) / its 18,682,768 key steps.  Exact for that workload;
 # for other --config values the product with their key steps is only an estimate.
-DRAM_BYTES_PER_KEY_STEP = 1041.6
+DRAM_BYTES_PER_KEY_STEP = 628.9
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 

@@ -250,28 +250,4 @@ __device__ __forceinline__ float fmax3(float a, float b, float c) {
     return r;
 }
 
-// 2^x for a pair, on the FMA/ALU pipes instead of the special-function unit: round x to the nearest integer n
-// with the 1.5*2^23 trick, evaluate a cubic for 2^(x-n) on [-0.5, 0.5] (relative error 7.5e-5, far below the
-// bf16 rounding the probabilities get anyway), then add n to the exponent field.  x is clamped at -126.
-__device__ __forceinline__ void exp2_poly2(uint64_t x2, float& e0, float& e1) {
-    float x0, x1;
-    unpack2(x2, x0, x1);
-    x0 = fmaxf(x0, -126.f);
-    x1 = fmaxf(x1, -126.f);
-    const uint64_t xc = pack2(x0, x1);
-    const uint64_t magic = pack2(12582912.f, 12582912.f);
-    const uint64_t t2 = fadd2(xc, magic);                                   // low mantissa bits = n
-    const uint64_t n2 = fadd2(t2, pack2(-12582912.f, -12582912.f));
-    const uint64_t f2 = ffma2(n2, pack2(-1.f, -1.f), xc);
-    uint64_t p2 = ffma2(f2, pack2(0.05517164245247841f, 0.05517164245247841f),
-                        pack2(0.2426111251115799f, 0.2426111251115799f));
-    p2 = ffma2(p2, f2, pack2(0.6932609677314758f, 0.6932609677314758f));
-    p2 = ffma2(p2, f2, pack2(0.9999280571937561f, 0.9999280571937561f));
-    float p0, p1, t0, t1;
-    unpack2(p2, p0, p1);
-    unpack2(t2, t0, t1);
-    e0 = __int_as_float(__float_as_int(p0) + (__float_as_int(t0) << 23));
-    e1 = __int_as_float(__float_as_int(p1) + (__float_as_int(t1) << 23));
-}
-
 }  // namespace wpp
