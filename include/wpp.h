@@ -186,17 +186,18 @@ int wpp_prefill_attention_varlen(const wpp_ctx* ctx, const wpp_batch_desc* desc,
  * get any.  (The paper has no counterpart; this is a convenience of this library.)  A prefill stage usually runs
  * inside a serving process whose cache manager has already claimed every free byte of HBM for KV pages, and on an
  * execution stream that must not stall: there a cudaMalloc at call time either fails or synchronises the whole
- * device.  This entry point therefore allocates nothing, neither directly nor through any library: the split-KV
- * partial results go to a fixed scratch array that is part of the library image
+ * device.  This entry point therefore allocates nothing, neither directly nor through any library: the tile
+ * counter and the split-KV partial results live in a fixed scratch array that is part of the library image
  * (wpp_static_scratch_bytes() bytes, 16 MiB; every GPU that loads the library holds it until the process exits).
  *   - Arguments as for wpp_prefill_attention_varlen, without workspace / workspace_bytes.
  *   - A plan that needs more scratch than the array holds is rejected with WPP_ERR_WORKSPACE_TOO_SMALL before
  *     anything is launched (plan with fewer key splits, or use the caller-workspace entry point).
  *   - The first call on a device looks up the array's device address, with the context's device current
  *     (WPP_ERR_INVALID_ARG otherwise); make that first call before any stream capture begins.
- *   - All calls on a device share the one array and it keeps whatever the last call left in it.  Nothing in it has
- *     to start at zero (every partial row is written before the combine pass reads it), but two calls whose
- *     kernels overlap on the GPU, e.g. on different streams, race on it: serialise them. */
+ *   - All calls on a device share the one array and it keeps whatever the last call left in it.  The call zeroes
+ *     the tile counter itself (a memset node on the stream) and every partial row is written before the combine
+ *     pass reads it, but two calls whose kernels overlap on the GPU, e.g. on different streams, race on it:
+ *     serialise them. */
 int wpp_prefill_attention_varlen_static(const wpp_ctx* ctx, const wpp_batch_desc* desc, const void* q, void* out,
                                         float* lse_or_null, const void* k_cache, const void* v_cache,
                                         const int32_t* block_tables, const int32_t* prefix_lens,
