@@ -66,7 +66,7 @@ struct Cfg {
     static constexpr int kHalves = D / 64;                 // 64-element (128-byte) swizzled column blocks
     static constexpr int kTileBytes = 128 * D * 2;         // one 128-row Q half, or one K or V step
     static constexpr int kHalfBytes = 128 * 128;           // 128 rows x 128 bytes
-    static constexpr int kSlots = (D == 128) ? 5 : 8;      // ring of K / V tiles (4 if the base is badly aligned)
+    static constexpr int kSlots = (D == 128) ? 4 : 8;      // K / V tiles in shared memory: half for K, half for V
     static constexpr int kOffKV = 2 * kTileBytes;
     static constexpr int kOffBars = kOffKV + kSlots * kTileBytes;
     static constexpr int kTileQ = 2;                       // tile ids the producer may publish ahead
@@ -74,8 +74,8 @@ struct Cfg {
     static constexpr int kOffFinal = kOffBars + 8 * kNumBars;          // float2 (m, l)[2][128]
     static constexpr int kOffMisc = kOffFinal + 2 * 128 * 8;           // tmem ptr, abort flag, tile ids
     static constexpr int kUsedBytes = kOffMisc + 16 + 4 * kTileQ + 8;
-    static constexpr int kMaxSmem = 232448;                            // 227 KB: the most a CTA can have
-    static constexpr int kSmemBytes = (kUsedBytes + 1024 < kMaxSmem) ? kUsedBytes + 1024 : kMaxSmem;
+    static constexpr int kSmemBytes = kUsedBytes + 1024;               // + alignment slack (193 KB at D = 128)
+    static_assert(kSmemBytes <= 232448, "more shared memory than a CTA can have");
 };
 
 // Optional wait accounting for tuning (compiled out unless WPP_STATS is defined): one thread of each role adds
@@ -145,13 +145,6 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
-    // the tile ring gives up one slot when the 1024-byte alignment of the base costs more than the spare bytes
-#ifdef WPP_FORCE_SMALL_RING
-    const uint32_t n_slots = C::kSlots - 1;              // test builds: always take the fallback
-#else
-    const uint32_t n_slots =
-        (smem_base - smem_u32(smem_raw)) + (uint32_t)C::kUsedBytes <= (uint32_t)C::kSmemBytes ? C::kSlots : C::kSlots - 1;
-#endif
     const uint32_t sQ = smem_base;                       // two halves, kTileBytes each
     const uint32_t sKV = smem_base + C::kOffKV;          // kSlots tiles (K or V)
     const uint32_t bars = smem_base + C::kOffBars;
@@ -228,9 +221,10 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
 
     if (wg == 3) {
         setmaxnreg_dec<kRegsUtil>();
-        // The K tiles and the V tiles have a ring each (slots [n_v, n_slots) and [0, n_v) of the tile area), so
-        // that the thread issuing S = Q K^T and the thread issuing O += P V walk their own ring.
-        const uint32_t n_v = C::kSlots / 2, n_k = n_slots - n_v;
+        // The K tiles and the V tiles have a ring each (slots [n_v, kSlots) and [0, n_v) of the tile area), so
+        // that the thread issuing S = Q K^T and the thread issuing O += P V walk their own ring.  (A third K
+        // slot, which would still fit, was measured and makes no difference.)
+        const uint32_t n_v = C::kSlots / 2, n_k = C::kSlots - n_v;
         if (warp == 13) {
             // ================================================================ producer
             // Tiles are requested in the order the issuers first touch them: K(0), K(1), V(0), K(2), V(1), ...
