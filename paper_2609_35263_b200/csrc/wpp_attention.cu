@@ -55,6 +55,10 @@ static_assert(8 * kRegsSoftmax + 4 * kRegsEpilogue + 4 * kRegsUtil <= 2048, "reg
 #define WPP_ELECT_ARRIVE 0
 #endif
 constexpr uint32_t kSoftmaxArrivals = WPP_ELECT_ARRIVE ? 4 : 128;
+#ifndef WPP_RESCALE_COLS
+#define WPP_RESCALE_COLS 16
+#endif
+constexpr int kRescaleCols = WPP_RESCALE_COLS;   // columns of O in flight while a moved reference rescales it
 constexpr float kRefSlack = 16.f;   // a row keeps its reference while its scores stay below reference + 16 (log2)
 #ifndef WPP_EXP_BLOCK
 #define WPP_EXP_BLOCK 8
@@ -627,15 +631,19 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                         waited = true;
                         tc_fence_after();
                         if (__any_sync(0xffffffffu, alpha != 1.f)) {
-                            // eight columns at a time: the 128 scores of the step stay in registers meanwhile
+                            // kRescaleCols columns at a time: the 128 scores of the step stay in registers meanwhile
 #pragma unroll 1
-                            for (int q8 = 0; q8 < D / 8; ++q8) {
-                                float o[8];
-                                tmem_ld8(lane_addr + col_o(hf) + q8 * 8, reinterpret_cast<uint32_t*>(o));
+                            for (int q0 = 0; q0 < D; q0 += kRescaleCols) {
+                                float o[kRescaleCols];
+#pragma unroll
+                                for (int c8 = 0; c8 < kRescaleCols; c8 += 8)
+                                    tmem_ld8(lane_addr + col_o(hf) + q0 + c8, reinterpret_cast<uint32_t*>(o) + c8);
                                 tmem_wait_ld();
 #pragma unroll
-                                for (int i = 0; i < 8; ++i) o[i] *= alpha;
-                                tmem_st8(lane_addr + col_o(hf) + q8 * 8, reinterpret_cast<uint32_t*>(o));
+                                for (int i = 0; i < kRescaleCols; ++i) o[i] *= alpha;
+#pragma unroll
+                                for (int c8 = 0; c8 < kRescaleCols; c8 += 8)
+                                    tmem_st8(lane_addr + col_o(hf) + q0 + c8, reinterpret_cast<uint32_t*>(o) + c8);
                             }
                         }
                     }
