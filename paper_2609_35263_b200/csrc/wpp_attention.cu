@@ -1,7 +1,8 @@
 // Persistent chunked-prefill attention kernel for sm_100a.
 //
-// One CTA per SM walks the list of work tiles the host planner gave it.  A work tile is two 128-row query
-// "halves" (A, B) that share one K/V stream, against key steps [kv_begin, kv_end) of 128 keys each.
+// One CTA per SM; the CTAs take the work tiles the host planner cut, in the planner's order, from a counter in
+// global memory as they become free.  A work tile is two 128-row query "halves" (A, B) that share one K/V
+// stream, against key steps [kv_begin, kv_end) of 128 keys each.
 // 16 warps, specialised by warpgroup:
 //   warps 0-3   softmax of half A: thread r owns query row r (TMEM lane r): row max / row sum need no shuffles
 //   warps 4-7   softmax of half B
@@ -10,7 +11,8 @@
 //               accumulators in TMEM; P is read from TMEM where the softmax warps wrote it as packed bf16; V is an
 //               MN-major operand.  Two threads, because the queue of the tensor pipe is only a few MMAs deep: the
 //               barrier waits and bookkeeping of one thread hide behind the MMAs the other one is issuing.
-//   warp 13     producer: reads the block table and issues TMA tile loads (Q once per tile; per key step one box
+//   warp 13     producer: takes the next tile from the counter and tells the other roles (a two-entry queue in
+//               shared memory); reads the block table and issues TMA tile loads (Q once per tile; per key step one box
 //               per (page, 64-wide half of head_dim) for K and for V, 128-byte swizzle) into a ring of K tiles
 //               and a ring of V tiles
 // Tensor memory (512 columns) has no room for two S tiles and two P tiles next to the two O accumulators, so the
