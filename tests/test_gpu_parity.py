@@ -131,6 +131,25 @@ def test_results_are_bit_reproducible():
     assert torch.equal(a["lse"], b["lse"])
 
 
+def test_results_do_not_depend_on_which_cta_takes_which_tile():
+    """Tiles are handed out at run time, so the assignment differs from run to run and with the order option; the
+    tiles themselves (and the fixed combine order) are the same, so every bit of the result must be too."""
+    w = W.custom_workload([1500, 40, 900, 0, 2048, 300], [700, 512, 130, 260, 64, 333], 8, 2, 128, 64, seed=21)
+    inp = cpu_inputs(w)
+    ref = None
+    for order in (0, 1, 0, 1):
+        for splits in (1, 3):
+            r = H.run_wave(w, H.device_inputs(w, inp), opts=wpp.PlanOpts(256, 0, splits, 0, order))
+            assert r["status"] == 0
+            key = (splits,)
+            ref = ref or {}
+            if key not in ref:
+                ref[key] = (r["out"].view(torch.int16).clone(), r["lse"].clone())
+            else:
+                assert torch.equal(ref[key][0], r["out"].view(torch.int16)), (order, splits)
+                assert torch.equal(ref[key][1], r["lse"]), (order, splits)
+
+
 def test_stale_slots_unused_pages_and_scratch_poison_do_not_matter():
     """NaN bit patterns everywhere the method must not look: slots past the sequence end, unreferenced pages."""
     w = W.custom_workload([90, 3, 0], [40, 200, 5], 4, 2, 128, 64, seed=13, spare_pages=6)
