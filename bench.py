@@ -197,6 +197,7 @@ def main():
     ap.add_argument("--force-kv-splits", type=int, default=0)
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
     ap.add_argument("--plan-order", type=int, default=0, help="0: stream order (default), 1: longest tile first")
+    ap.add_argument("--max-ctas", type=int, default=0, help="persistent CTAs to launch (0: one per SM)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "native" else args.warmup
 
@@ -220,7 +221,7 @@ def main():
     ctx = wpp.Context(local_rank)
     desc = wpp.make_desc(w.num_requests, w.num_q_heads, w.num_kv_heads, w.head_dim, w.page_size,
                          w.max_blocks_per_req, w.num_pages)
-    opts = wpp.PlanOpts(0, 0, args.force_kv_splits, 0, args.plan_order)
+    opts = wpp.PlanOpts(0, 0, args.force_kv_splits, args.max_ctas, args.plan_order)
     T = w.total_new_tokens
 
     # ---- resident state and inputs on the device
