@@ -185,6 +185,66 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+def run_waves(args):
+    """Host-only leg for the wave-budget planner (Section 4.5): wpp_plan_waves through the C ABI and the oracle
+    walk the same seeded serving loop (bursty arrivals, one wave per decision, the last R waves in flight); both
+    are timed on the host cores and their decisions compared.  No GPU is touched."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    import paper_2609_35263_b200 as wpp
+    from oracle import waves as O
+    P, F, B, lanes, M, b_min = 4, 2, 64, 64, 16384, 1024
+    cfg = wpp.WaveConfig(P, F, B, lanes, M, b_min)
+    R = 2 * P
+    rng = np.random.default_rng(7)
+    decisions = 20000
+    arrivals = [[int(x) for x in rng.integers(1, 40000, rng.integers(1, 8))] if rng.random() < 0.12 else []
+                for _ in range(decisions)]
+
+    def loop(decide):
+        queue, ring, trace = [], [], []
+        t0 = time.perf_counter()
+        for it in range(decisions):
+            queue += arrivals[it]
+            chunks, budget = decide(queue, [c for wv in ring for c in wv])
+            trace.append((budget, sum(chunks)))
+            ring = (ring + [[c for c in chunks if c]])[-R:]
+            queue = [r - c for r, c in zip(queue, chunks) if r - c > 0]
+        return time.perf_counter() - t0, trace
+
+    st = wpp.WaveState()
+
+    def decide_c(queue, inflight):
+        ch, info = wpp.wpp_plan_waves(cfg, st, queue, inflight)
+        return ch.tolist(), int(info.budget)
+
+    ost = [O.BudgetState()]
+
+    def decide_o(queue, inflight):
+        ost[0], b, ch, _ = O.plan_wave(P, F, M, b_min, B, lanes, queue, inflight, ost[0])
+        return ch, b
+
+    for _ in range(max(0, args.warmup)):
+        st = wpp.WaveState()
+        loop(decide_c)
+    st = wpp.WaveState()
+    t_c, trace_c = loop(decide_c)
+    t_o, trace_o = loop(decide_o)
+    if trace_c != trace_o:
+        raise SystemExit("wpp_plan_waves and the oracle took different decisions")
+    budgets = sorted({b for b, _ in trace_c}, reverse=True)
+    line = {"metric": "wave-planning decisions/s (host, through the binding)", "value": decisions / t_c,
+            "unit": "decisions/s", "n_gpus": 0, "steps": decisions, "warmup": args.warmup,
+            "ms_per_step": 1e3 * t_c / decisions, "higher_is_better": True, "vs_baseline": None, "dtype": "int64",
+            "data": "synthetic", "gpu_launches": 0,
+            "config": {"workload": "seeded serving loop", "P": P, "F": F, "M": M, "b_min": b_min, "B": B,
+                       "max_lanes": lanes, "budgets_used": budgets,
+                       "tokens_scheduled": int(sum(t for _, t in trace_c)), "decisions_identical_to_oracle": True},
+            "cpu_baseline": {"value": decisions / t_o, "unit": "decisions/s", "cores": 1, "kind": "oracle",
+                             "sample": f"the same {decisions} decisions"}}
+    print(json.dumps(line))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -198,9 +258,13 @@ def main():
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
     ap.add_argument("--plan-order", type=int, default=0, help="0: stream order (default), 1: longest tile first")
     ap.add_argument("--max-ctas", type=int, default=0, help="persistent CTAs to launch (0: one per SM)")
+    ap.add_argument("--waves", action="store_true", help="time the wave-budget planner (host only) instead")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "native" else args.warmup
 
+    if args.waves:
+        run_waves(args)
+        return
     if args.impl == "reference":
         run_reference(args)
         return

@@ -216,6 +216,71 @@ int wpp_selftest_bounded_wait(const wpp_ctx* ctx, int64_t limit_cycles, int32_t*
 /* Number of kernels the library has launched through this context so far (for launch accounting). */
 int64_t wpp_launch_count(const wpp_ctx* ctx);
 
+/* ---------------------------------------------------------------------------------------------------------
+ * Wave-budget planner (Section 4.5, "Pipeline Scheduling": Maximum Pipeline Utilization).  Host only, integer
+ * arithmetic only, no CUDA call; it produces the chunk_lens the calls above consume: the step directly upstream of
+ * the attention path.  With P pipeline stages the executor keeps a ring of R = 2P waves and the planner aims at
+ * S = R + (F - 1) P waves of work; it picks the wave budget from the ladder b_0 = M, b_{j+1} = max(b_min,
+ * alignDown_B(b_j / 2)) (Eq. design-budget) by the estimate n(b) = max(W / b, N_{>b/2}) of the waves a budget b
+ * yields, where the pieces are the unscheduled suffixes of admitted requests and their most recent chunks still in
+ * the ring, W their token sum and N_{>b/2} the number of pieces larger than half a wave.
+ * Rules, in the paper's order: the largest budget with n(b) >= S, b_min if none; once a budget supplies R waves the
+ * next smaller one is only taken if the pieces it would newly split (size in (b_{j+1}, b_j]) are at most 12.5 % of
+ * W; a burst asking for a budget two or more ladder steps larger takes effect at once, a one-step increase after
+ * R/2 consecutive decisions asked for it, a decrease (one step) after R consecutive decisions asked for it and
+ * only while the budget in force misses the target by a whole wave (n(b_cur) <= S - 1: the paper names a
+ * hysteresis check without defining it; this is the reading taken).  Packing is first come, first served: a
+ * request that fits takes its whole suffix; one that does not gets the leftover space as a fragment unless the
+ * fragment is smaller than max(b_min, b / 2), in which case packing stops (nobody overtakes it). */
+typedef struct {
+    int32_t num_stages;   /* P >= 1 */
+    int32_t fill_factor;  /* F >= 1 (the paper's matched experiments use 2) */
+    int32_t block_size;   /* B >= 1 */
+    int32_t max_lanes;    /* requests a wave may carry (maximum batch size) >= 1 */
+    int64_t max_budget;   /* M: multiple of B, <= 2^31 - 1 */
+    int64_t min_budget;   /* b_min: multiple of B, B <= b_min <= M */
+} wpp_wave_config;
+
+/* Planner state carried from one decision to the next; start from all zeros (budget M in force). */
+typedef struct {
+    int32_t cur;          /* ladder index of the budget in force (0 = M) */
+    int32_t direction;    /* pending change: -1 towards larger budgets, +1 towards smaller, 0 none */
+    int32_t count;        /* consecutive decisions that asked for the pending change */
+    int32_t reserved;
+} wpp_wave_state;
+
+typedef struct {
+    int64_t budget;       /* budget in force for this wave */
+    int64_t work;         /* W */
+    int64_t wave_tokens;  /* sum of chunk_lens */
+    int32_t target_index; /* ladder index the selection rule asked for, before hysteresis */
+    int32_t budget_index; /* ladder index in force */
+    int32_t lanes;        /* requests in the wave */
+    int32_t defer;        /* 1: a lone request below half capacity; it may wait one iteration for company */
+} wpp_wave_info;
+
+#define WPP_WAVE_RING_BUSY 1         /* flags of wpp_plan_waves */
+#define WPP_WAVE_ADMISSION_PENDING 2
+#define WPP_WAVE_ALREADY_DEFERRED 4
+
+/* The ladder of budgets for cfg: writes min(*count, capacity) entries to ladder_out (may be NULL with capacity 0)
+ * and the ladder's length to *count.  WPP_ERR_INVALID_ARG for an invalid configuration. */
+int wpp_wave_ladder(const wpp_wave_config* cfg, int64_t* ladder_out, int32_t capacity, int32_t* count);
+
+/* One planning decision of rank 0.
+ *   remaining_host : host int64 [num_requests], unscheduled suffix tokens per admitted request in arrival order
+ *                    (0 = finished); inflight_host : host int64 [num_inflight], the most recently committed chunks
+ *                    still in the ring (either may be NULL when its count is 0).
+ *   state          : in/out, see wpp_wave_state.
+ *   flags          : WPP_WAVE_* bits; `defer` is reported only when the ring is busy, admission has further
+ *                    requests pending and this wave has not been deferred before.
+ *   chunk_lens_host: out, host int32 [num_requests]: tokens of each request in this wave (0 = not in it); the
+ *                    caller advances its positions by the spans it actually accepts.
+ * Returns WPP_ERR_INVALID_ARG for null pointers, negative lengths or an invalid configuration or state. */
+int wpp_plan_waves(const wpp_wave_config* cfg, wpp_wave_state* state, const int64_t* remaining_host,
+                   int32_t num_requests, const int64_t* inflight_host, int32_t num_inflight, int32_t flags,
+                   int32_t* chunk_lens_host, wpp_wave_info* info);
+
 #ifdef __cplusplus
 }
 #endif

@@ -56,10 +56,31 @@ class PlanInfo(ctypes.Structure):
                 ("workspace_bytes", ctypes.c_size_t), ("plan_bytes", ctypes.c_size_t)]
 
 
+class WaveConfig(ctypes.Structure):
+    _fields_ = [("num_stages", ctypes.c_int32), ("fill_factor", ctypes.c_int32), ("block_size", ctypes.c_int32),
+                ("max_lanes", ctypes.c_int32), ("max_budget", ctypes.c_int64), ("min_budget", ctypes.c_int64)]
+
+
+class WaveState(ctypes.Structure):
+    _fields_ = [("cur", ctypes.c_int32), ("direction", ctypes.c_int32), ("count", ctypes.c_int32),
+                ("reserved", ctypes.c_int32)]
+
+    def as_tuple(self):
+        return (int(self.cur), int(self.direction), int(self.count))
+
+
+class WaveInfo(ctypes.Structure):
+    _fields_ = [("budget", ctypes.c_int64), ("work", ctypes.c_int64), ("wave_tokens", ctypes.c_int64),
+                ("target_index", ctypes.c_int32), ("budget_index", ctypes.c_int32), ("lanes", ctypes.c_int32),
+                ("defer", ctypes.c_int32)]
+
+
+WAVE_RING_BUSY, WAVE_ADMISSION_PENDING, WAVE_ALREADY_DEFERRED = 1, 2, 4
+
 EXPORTS = ["wpp_create", "wpp_destroy", "wpp_status_string", "wpp_last_cuda_error", "wpp_plan_bytes",
            "wpp_plan_tiles", "wpp_validate_batch", "wpp_kv_append", "wpp_prefill_attention_varlen",
            "wpp_launch_count", "wpp_prefill_attention_varlen_static", "wpp_static_scratch_bytes",
-           "wpp_selftest_bounded_wait"]
+           "wpp_selftest_bounded_wait", "wpp_wave_ladder", "wpp_plan_waves"]
 
 _lib = None
 
@@ -94,6 +115,9 @@ def load_library() -> ctypes.CDLL:
         lib.wpp_selftest_bounded_wait.argtypes = [vp, ctypes.c_int64, i32p, vp, vp]
         lib.wpp_static_scratch_bytes.restype = ctypes.c_size_t
         lib.wpp_static_scratch_bytes.argtypes = []
+        lib.wpp_wave_ladder.argtypes = [ctypes.POINTER(WaveConfig), vp, ctypes.c_int32, ctypes.POINTER(ctypes.c_int32)]
+        lib.wpp_plan_waves.argtypes = [ctypes.POINTER(WaveConfig), ctypes.POINTER(WaveState), vp, ctypes.c_int32, vp,
+                                       ctypes.c_int32, ctypes.c_int32, vp, ctypes.POINTER(WaveInfo)]
         _lib = lib
     return _lib
 
@@ -268,3 +292,28 @@ def wpp_selftest_bounded_wait(ctx: Context, limit_cycles: int, status, waited_cy
     st = load_library().wpp_selftest_bounded_wait(ctx.handle, int(limit_cycles), _ptr(status), _ptr(waited_cycles),
                                                   _stream(stream))
     _check(st, "wpp_selftest_bounded_wait")
+
+
+def wpp_wave_ladder(cfg: WaveConfig):
+    """The budgets the wave planner chooses from, largest first (Eq. design-budget)."""
+    lib = load_library()
+    n = ctypes.c_int32(0)
+    _check(lib.wpp_wave_ladder(ctypes.byref(cfg), None, 0, ctypes.byref(n)), "wpp_wave_ladder")
+    out = np.zeros(n.value, dtype=np.int64)
+    _check(lib.wpp_wave_ladder(ctypes.byref(cfg), out.ctypes.data_as(ctypes.c_void_p), n.value, ctypes.byref(n)),
+           "wpp_wave_ladder")
+    return out.tolist()
+
+
+def wpp_plan_waves(cfg: WaveConfig, state: WaveState, remaining, inflight=(), flags: int = 0):
+    """One planning decision (Section 4.5): updates `state` in place, returns (chunk_lens int32 array, WaveInfo)."""
+    rem = np.ascontiguousarray(np.asarray(remaining, dtype=np.int64))
+    inf = np.ascontiguousarray(np.asarray(inflight, dtype=np.int64))
+    chunks = np.zeros(rem.shape[0], dtype=np.int32)
+    info = WaveInfo()
+    st = load_library().wpp_plan_waves(
+        ctypes.byref(cfg), ctypes.byref(state), rem.ctypes.data_as(ctypes.c_void_p) if rem.size else None,
+        int(rem.size), inf.ctypes.data_as(ctypes.c_void_p) if inf.size else None, int(inf.size), int(flags),
+        chunks.ctypes.data_as(ctypes.c_void_p) if rem.size else None, ctypes.byref(info))
+    _check(st, "wpp_plan_waves")
+    return chunks, info
