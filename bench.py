@@ -393,8 +393,16 @@ def main():
 
         def e2e_step(i):
             b2 = i % 2
+            sl = i % ring
+            # the plan is an input like the others: it is made first and travels on the input stream, ahead of the
+            # large copies (a small copy issued later from the compute stream would queue behind the next wave's
+            # 4.5 GB query copy on the one host-to-device engine and stall the kernels for 100 ms)
+            plan_free[sl].synchronize()                  # the copy that last read this pinned buffer has run
+            plan = wpp.wpp_plan_tiles(ctx, desc, w.prefix_lens, w.chunk_lens, opts=opts, out=plan_host[sl])
             with torch.cuda.stream(s_in):
-                s_in.wait_event(run_done[b2])            # wave i-2 no longer reads this input set
+                s_in.wait_event(run_done[b2])            # wave i-2 (and so wave i-3, which used this plan buffer) is done
+                plan.to_device(out=plan_dev[sl])
+                plan_free[sl].record(s_in)
                 for k in hb:
                     dev_in[b2][k].copy_(host_in[k], non_blocking=True)
                 for dst, src in zip(dev_meta[b2], (bt_h, P_h, C_h)):
@@ -403,11 +411,6 @@ def main():
             with torch.cuda.stream(s_run):
                 s_run.wait_event(in_done[b2])
                 s_run.wait_event(out_done[b2])           # wave i-2's output has left this output buffer
-                sl = i % ring
-                plan_free[sl].synchronize()
-                plan = wpp.wpp_plan_tiles(ctx, desc, w.prefix_lens, w.chunk_lens, opts=opts, out=plan_host[sl])
-                plan.to_device(out=plan_dev[sl])
-                plan_free[sl].record(s_run)
                 btd, Pd, Cd = dev_meta[b2]
                 wpp.wpp_kv_append(ctx, desc, dev_in[b2]["k_new"], dev_in[b2]["v_new"], k_pool, v_pool, btd, Pd, Cd,
                                   plan, status=status, stream=s_run)
