@@ -245,6 +245,100 @@ def run_waves(args):
     print(json.dumps(line))
 
 
+def run_waves_sim(args):
+    """Wave planner and attention path together (Section 4.5 with this library's kernels): a burst of admitted
+    requests is cut into waves by wpp_plan_waves, once with the budget fixed at M and once with the paper's budget
+    ladder; every wave's chunk_lens go through wpp_plan_tiles, wpp_kv_append and wpp_prefill_attention_varlen on
+    the GPU and its time is measured; a P-stage pipeline whose stages each take that time is then simulated
+    (stage s starts wave w when it has finished wave w-1 and stage s-1 has finished wave w).  One GPU stands in
+    for every stage: the stages' attention work is the same, their other layers are not modelled."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    import torch
+    import paper_2609_35263_b200 as wpp
+    import wpp_workloads as W
+    from wpp_workloads.generate import make_workload
+    dev = torch.device("cuda", 0)
+    P_stages, F, B, M, lanes = 4, 2, 64, 16384, 64
+    rng = np.random.default_rng(11)
+    R = 40
+    sharer = rng.random(R) < 0.8
+    cached = np.where(sharer, 16384, rng.integers(0, 129, R) * 64).astype(np.int64)
+    suffix = rng.integers(500, 24001, R).astype(np.int64)
+    w = make_workload("waves_sim", 11, rng, cached, suffix, 64, 8, 128, B, shared_tokens=16384, sharers=sharer)
+    ctx = wpp.Context(0)
+    desc = wpp.make_desc(R, w.num_q_heads, w.num_kv_heads, w.head_dim, B, w.max_blocks_per_req, w.num_pages)
+    k_pool, v_pool = w.k_pool(dev), w.v_pool(dev)
+    bt = torch.from_numpy(w.block_tables).to(dev)
+    g = torch.Generator(device=dev).manual_seed(5)
+    q = torch.randn(M, w.num_q_heads, w.head_dim, device=dev, generator=g).to(torch.bfloat16)
+    kn = torch.randn(M, w.num_kv_heads, w.head_dim, device=dev, generator=g).to(torch.bfloat16)
+    vn = torch.randn(M, w.num_kv_heads, w.head_dim, device=dev, generator=g).to(torch.bfloat16)
+    out = torch.empty_like(q)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    ws = torch.empty(64 << 20, dtype=torch.uint8, device=dev)
+    ring = 2 * P_stages
+
+    def run_policy(b_min, n_req):
+        # the first n_req requests form the burst; the planner starts from an idle system (floor budget in force)
+        cfg = wpp.WaveConfig(P_stages, F, B, lanes, M, b_min)
+        st = wpp.WaveState(len(wpp.wpp_wave_ladder(cfg)) - 1, 0, 0, 0)
+        done = np.zeros(R, dtype=np.int64)
+        done[n_req:] = suffix[n_req:]
+        inflight, times, sizes, budgets = [], [], [], []
+        while True:
+            chunks, info = wpp.wpp_plan_waves(cfg, st, (suffix - done).tolist(), [c for wv in inflight for c in wv])
+            if int(info.wave_tokens) == 0:
+                break
+            Pw = (cached + done).astype(np.int32)
+            Cw = chunks.astype(np.int32)
+            plan = wpp.wpp_plan_tiles(ctx, desc, Pw, Cw)
+            plan.to_device()
+            if int(plan.info.workspace_bytes) > ws.numel():
+                raise SystemExit("workspace too small for the simulation")
+            Pd, Cd = torch.from_numpy(Pw).to(dev), torch.from_numpy(Cw).to(dev)
+            T = int(Cw.sum())
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            wpp.wpp_kv_append(ctx, desc, kn[:T], vn[:T], k_pool, v_pool, bt, Pd, Cd, plan, status=status)
+            wpp.wpp_prefill_attention_varlen(ctx, desc, q[:T], out[:T], None, k_pool, v_pool, bt, Pd, Cd, plan,
+                                             workspace=ws, status=status)
+            b.record()
+            torch.cuda.synchronize()
+            times.append(a.elapsed_time(b))
+            sizes.append(T)
+            budgets.append(int(info.budget))
+            done += chunks
+            inflight = (inflight + [[int(c) for c in chunks if c]])[-ring:]
+        if int(status.item()) != 0:
+            raise SystemExit(f"device status {int(status.item())}")
+        finish = [0.0] * P_stages                       # finish time of the latest wave on each stage
+        for t in times:
+            prev = 0.0
+            for s_ in range(P_stages):
+                start = max(finish[s_], prev)
+                finish[s_] = prev = start + t
+        makespan = finish[-1]
+        return {"waves": len(times), "budgets_used": sorted(set(budgets), reverse=True),
+                "stage_busy_ms": float(sum(times)), "makespan_ms": float(makespan),
+                "fill": float(sum(times) / makespan), "tokens_per_s": float(sum(sizes) / (makespan * 1e-3)),
+                "mean_wave_ms": float(np.mean(times)), "max_wave_ms": float(np.max(times))}
+
+    run_policy(M, R)                                    # warm-up pass (allocator, tensor maps, clocks)
+    bursts = {}
+    for n_req in (R, 12, 4):
+        bursts[f"{n_req} requests, {int(suffix[:n_req].sum())} new tokens"] = {
+            "budget_fixed_at_M": run_policy(M, n_req), "budget_ladder": run_policy(1024, n_req)}
+    big = next(iter(bursts.values()))
+    line = {"metric": "simulated 4-stage pipeline: new tokens/s for one burst of admitted requests",
+            "value": big["budget_ladder"]["tokens_per_s"], "unit": "tokens/s", "n_gpus": 1, "higher_is_better": True,
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": "bursts of 40, 12 and 4 requests, 80 % sharing a 16384-token cached prefix, "
+                                   "suffixes 500-24000", "P": P_stages, "F": F, "M": M, "b_min": 1024, "B": B},
+            "bursts": bursts}
+    print(json.dumps(line))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -259,11 +353,15 @@ def main():
     ap.add_argument("--plan-order", type=int, default=0, help="0: stream order (default), 1: longest tile first")
     ap.add_argument("--max-ctas", type=int, default=0, help="persistent CTAs to launch (0: one per SM)")
     ap.add_argument("--waves", action="store_true", help="time the wave-budget planner (host only) instead")
+    ap.add_argument("--waves-sim", action="store_true", help="wave planner + kernels: simulated pipeline fill")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "native" else args.warmup
 
     if args.waves:
         run_waves(args)
+        return
+    if args.waves_sim:
+        run_waves_sim(args)
         return
     if args.impl == "reference":
         run_reference(args)
