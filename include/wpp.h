@@ -281,6 +281,52 @@ int wpp_plan_waves(const wpp_wave_config* cfg, wpp_wave_state* state, const int6
                    int32_t num_requests, const int64_t* inflight_host, int32_t num_inflight, int32_t flags,
                    int32_t* chunk_lens_host, wpp_wave_info* info);
 
+/* ---------------------------------------------------------------------------------------------------------
+ * Prefix hints (Section 4.3): chained hashes of full token blocks and a counted index probed by galloping and
+ * bisecting.  This is the step that produces prefix_lens: the number of leading blocks of a request whose keys
+ * are in the index, times the block size, is the reuse candidate.
+ *
+ * Eq. design-hash: H_{-1} = 0, H_i = hash(B_i, extraKeys_i, salt, H_{i-1}) over the FULL blocks of a request.  The
+ * paper does not name the hash; this library uses 64-bit arithmetic with mix64 = the splitmix64 finaliser:
+ *   term_k = mix64(((token_k mod 2^32) << 32 | k) xor 0xD6E8FEB86659FD93)   (k = position inside the block)
+ *   digest_i = sum_k term_k (mod 2^64)
+ *   H_i = mix64(H_{i-1} xor mix64(digest_i + extraKeys_i) xor (salt * 0x9E3779B97F4A7C15)). */
+
+/* Chained block hashes of a batch of requests, on the GPU (two small kernels on `cuda_stream`).
+ *   tokens        : device int32 [token_offsets[R]], the requests' token ids back to back.
+ *   token_offsets : device int64 [R+1], start of each request in `tokens`.
+ *   block_offsets : device int64 [R+1], exclusive scan of floor(n_i / block_size): where each request's hashes go.
+ *   extra_keys_or_null : device uint64 [total_blocks] or NULL (all zero).
+ *   hashes_out    : device uint64 [total_blocks]; request i's H_0.. are at hashes_out[block_offsets[i]..].
+ * Partial last blocks are not hashed.  Returns WPP_ERR_INVALID_ARG for null pointers or sizes < 0, WPP_ERR_CUDA for
+ * a launch failure. */
+int wpp_hash_blocks(const wpp_ctx* ctx, const int32_t* tokens, const int64_t* token_offsets,
+                    const int64_t* block_offsets, int32_t num_requests, int32_t block_size, uint64_t salt,
+                    const uint64_t* extra_keys_or_null, uint64_t* hashes_out, int64_t total_blocks,
+                    void* cuda_stream);
+
+/* The same chain for one request on the host (host pointers; hashes_out holds n_tokens / block_size entries). */
+int wpp_hash_blocks_host(const int32_t* tokens, int64_t n_tokens, int32_t block_size, uint64_t salt,
+                         const uint64_t* extra_keys_or_null, uint64_t* hashes_out);
+
+/* Counted index keyed by (cache window, H_i): a key's counter goes up when a block joins the cache tree and down
+ * when it is detached; the entry disappears at zero.  Sharded by hash, one mutex per shard; safe to call from
+ * several host threads. */
+typedef struct wpp_hint_index wpp_hint_index;
+int wpp_hint_index_create(wpp_hint_index** out);
+int wpp_hint_index_destroy(wpp_hint_index* idx);
+int wpp_hint_index_add(wpp_hint_index* idx, int32_t window, const uint64_t* hashes_host, int64_t n);
+int wpp_hint_index_remove(wpp_hint_index* idx, int32_t window, const uint64_t* hashes_host, int64_t n);
+int64_t wpp_hint_index_size(const wpp_hint_index* idx);     /* number of keys; -1 for NULL */
+
+/* Longest cached prefix of a request, in blocks: probes depths 1, 2, 4, ... until the first miss, then bisects
+ * between the last match and that miss (about log2 N probes instead of N; exact when presence is monotone in
+ * depth, which chained keys added prefix by prefix guarantee).  The index may change while the probe runs; the
+ * result is a hint that the caller's authoritative walk confirms.
+ *   hashes_host : host uint64 [n_blocks], H_0 .. of the request;  *matched_blocks and *probes_or_null are outputs. */
+int wpp_hint_probe(const wpp_hint_index* idx, int32_t window, const uint64_t* hashes_host, int64_t n_blocks,
+                   int64_t* matched_blocks, int32_t* probes_or_null);
+
 #ifdef __cplusplus
 }
 #endif

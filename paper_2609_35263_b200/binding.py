@@ -80,7 +80,9 @@ WAVE_RING_BUSY, WAVE_ADMISSION_PENDING, WAVE_ALREADY_DEFERRED = 1, 2, 4
 EXPORTS = ["wpp_create", "wpp_destroy", "wpp_status_string", "wpp_last_cuda_error", "wpp_plan_bytes",
            "wpp_plan_tiles", "wpp_validate_batch", "wpp_kv_append", "wpp_prefill_attention_varlen",
            "wpp_launch_count", "wpp_prefill_attention_varlen_static", "wpp_static_scratch_bytes",
-           "wpp_selftest_bounded_wait", "wpp_wave_ladder", "wpp_plan_waves"]
+           "wpp_selftest_bounded_wait", "wpp_wave_ladder", "wpp_plan_waves",
+           "wpp_hash_blocks", "wpp_hash_blocks_host", "wpp_hint_index_create", "wpp_hint_index_destroy",
+           "wpp_hint_index_add", "wpp_hint_index_remove", "wpp_hint_index_size", "wpp_hint_probe"]
 
 _lib = None
 
@@ -115,6 +117,17 @@ def load_library() -> ctypes.CDLL:
         lib.wpp_selftest_bounded_wait.argtypes = [vp, ctypes.c_int64, i32p, vp, vp]
         lib.wpp_static_scratch_bytes.restype = ctypes.c_size_t
         lib.wpp_static_scratch_bytes.argtypes = []
+        lib.wpp_hash_blocks.argtypes = [vp, vp, vp, vp, ctypes.c_int32, ctypes.c_int32, ctypes.c_uint64, vp, vp,
+                                        ctypes.c_int64, vp]
+        lib.wpp_hash_blocks_host.argtypes = [vp, ctypes.c_int64, ctypes.c_int32, ctypes.c_uint64, vp, vp]
+        lib.wpp_hint_index_create.argtypes = [ctypes.POINTER(vp)]
+        lib.wpp_hint_index_destroy.argtypes = [vp]
+        lib.wpp_hint_index_add.argtypes = [vp, ctypes.c_int32, vp, ctypes.c_int64]
+        lib.wpp_hint_index_remove.argtypes = [vp, ctypes.c_int32, vp, ctypes.c_int64]
+        lib.wpp_hint_index_size.argtypes = [vp]
+        lib.wpp_hint_index_size.restype = ctypes.c_int64
+        lib.wpp_hint_probe.argtypes = [vp, ctypes.c_int32, vp, ctypes.c_int64, ctypes.POINTER(ctypes.c_int64),
+                                       ctypes.POINTER(ctypes.c_int32)]
         lib.wpp_wave_ladder.argtypes = [ctypes.POINTER(WaveConfig), vp, ctypes.c_int32, ctypes.POINTER(ctypes.c_int32)]
         lib.wpp_plan_waves.argtypes = [ctypes.POINTER(WaveConfig), ctypes.POINTER(WaveState), vp, ctypes.c_int32, vp,
                                        ctypes.c_int32, ctypes.c_int32, vp, ctypes.POINTER(WaveInfo)]
@@ -317,3 +330,82 @@ def wpp_plan_waves(cfg: WaveConfig, state: WaveState, remaining, inflight=(), fl
         chunks.ctypes.data_as(ctypes.c_void_p) if rem.size else None, ctypes.byref(info))
     _check(st, "wpp_plan_waves")
     return chunks, info
+
+
+def wpp_hash_blocks(ctx: Context, tokens, token_offsets, block_offsets, block_size: int, salt: int = 0, extra_keys=None,
+                    stream=None, total_blocks: Optional[int] = None, out=None):
+    """Chained hashes of the full token blocks of a batch of requests on the GPU (Eq. design-hash).
+
+    tokens: cuda int32; token_offsets, block_offsets: cuda int64 [R+1]; returns a cuda int64 tensor holding the
+    64-bit hashes' bit patterns, request i's at [block_offsets[i], block_offsets[i+1])."""
+    R = int(token_offsets.numel()) - 1
+    if total_blocks is None:                 # reads the last offset back from the device: pass it to avoid the sync
+        total_blocks = int(block_offsets[-1].item()) if R >= 0 and block_offsets.numel() else 0
+    total = int(total_blocks)
+    if out is None:
+        out = torch.empty(total, dtype=torch.int64, device=tokens.device)
+    st = load_library().wpp_hash_blocks(ctx.handle, _ptr(tokens), _ptr(token_offsets), _ptr(block_offsets), max(R, 0),
+                                        int(block_size), ctypes.c_uint64(int(salt) & (2 ** 64 - 1)), _ptr(extra_keys),
+                                        _ptr(out), total, _stream(stream))
+    _check(st, "wpp_hash_blocks")
+    return out
+
+
+def wpp_hash_blocks_host(tokens, block_size: int, salt: int = 0, extra_keys=None) -> np.ndarray:
+    """The same chain for one request on the host; returns uint64 [len(tokens) // block_size]."""
+    t = np.ascontiguousarray(np.asarray(tokens, dtype=np.int32))
+    out = np.zeros(t.size // int(block_size), dtype=np.uint64)
+    e = None if extra_keys is None else np.ascontiguousarray(np.asarray(extra_keys, dtype=np.uint64))
+    st = load_library().wpp_hash_blocks_host(
+        t.ctypes.data_as(ctypes.c_void_p) if t.size else None, int(t.size), int(block_size),
+        ctypes.c_uint64(int(salt) & (2 ** 64 - 1)), e.ctypes.data_as(ctypes.c_void_p) if e is not None else None,
+        out.ctypes.data_as(ctypes.c_void_p) if out.size else None)
+    _check(st, "wpp_hash_blocks_host")
+    return out
+
+
+class HintIndex:
+    """Counted index keyed by (cache window, chained block hash) with the gallop-and-bisect probe (Section 4.3)."""
+
+    def __init__(self):
+        self.handle = ctypes.c_void_p()
+        _check(load_library().wpp_hint_index_create(ctypes.byref(self.handle)), "wpp_hint_index_create")
+
+    def close(self):
+        if self.handle:
+            load_library().wpp_hint_index_destroy(self.handle)
+            self.handle = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    @staticmethod
+    def _u64(hashes):
+        return np.ascontiguousarray(np.asarray(hashes, dtype=np.uint64))
+
+    def add(self, window: int, hashes) -> None:
+        h = self._u64(hashes)
+        _check(load_library().wpp_hint_index_add(self.handle, int(window),
+                                                 h.ctypes.data_as(ctypes.c_void_p) if h.size else None, int(h.size)),
+               "wpp_hint_index_add")
+
+    def remove(self, window: int, hashes) -> None:
+        h = self._u64(hashes)
+        _check(load_library().wpp_hint_index_remove(self.handle, int(window),
+                                                    h.ctypes.data_as(ctypes.c_void_p) if h.size else None, int(h.size)),
+               "wpp_hint_index_remove")
+
+    def __len__(self) -> int:
+        return int(load_library().wpp_hint_index_size(self.handle))
+
+    def probe(self, window: int, hashes):
+        """(matched blocks, number of probes) for a request's chained hashes H_0 .."""
+        h = self._u64(hashes)
+        m, p = ctypes.c_int64(0), ctypes.c_int32(0)
+        _check(load_library().wpp_hint_probe(self.handle, int(window),
+                                             h.ctypes.data_as(ctypes.c_void_p) if h.size else None, int(h.size),
+                                             ctypes.byref(m), ctypes.byref(p)), "wpp_hint_probe")
+        return int(m.value), int(p.value)
