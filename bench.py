@@ -292,7 +292,7 @@ def run_waves_sim(args):
                 break
             Pw = (cached + done).astype(np.int32)
             Cw = chunks.astype(np.int32)
-            plan = wpp.wpp_plan_tiles(ctx, desc, Pw, Cw)
+            plan = wpp.wpp_plan_tiles(ctx, desc, Pw, Cw, opts=wpp.PlanOpts(0, 0, 0, 0, args.plan_order))
             plan.to_device()
             if int(plan.info.workspace_bytes) > ws.numel():
                 raise SystemExit("workspace too small for the simulation")
