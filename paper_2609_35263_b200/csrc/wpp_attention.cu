@@ -707,8 +707,10 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     pf_phase ^= 1u;
                     tc_fence_after();
                 }
-                tmem_st32(lane_addr + col_p(hf), pk);
-                tmem_st32(lane_addr + col_p(hf) + 32, pk + 32);
+                // eight stores of eight columns rather than two of 32: the narrow form only needs eight consecutive
+                // registers at a time, which leaves the register allocator free in the loop above (+0.7 % measured)
+#pragma unroll
+                for (int c8 = 0; c8 < 64; c8 += 8) tmem_st8(lane_addr + col_p(hf) + c8, pk + c8);
                 tmem_wait_st();
                 tc_fence_before();
                 if (WPP_ELECT_ARRIVE) {
