@@ -6,6 +6,10 @@ library and never imports it.
 
 ``reference``  : ctypes wrapper around the plain C implementation (wpp_oracle.c).
 ``brute``      : separate numpy matrix-form implementation used to pin the C one.
+``waves``      : the wave-budget planner and FCFS packing of Section 4.5 (plain Python); some rules the paper
+                 leaves open are readings: parity unpinned for those (listed in the module).
+``hints``      : chained block hash and gallop/bisect index probe of Section 4.3 (plain Python); the hash function
+                 is a reading: parity unpinned for that choice.
 """
 from .reference import (  # noqa: F401
     build,
