@@ -47,8 +47,8 @@ __host__ __device__ constexpr uint32_t col_o(int hf) { return 256u + 128u * hf; 
 // 4 x kRegsUtil <= 2048 per thread slot of 32 lanes, i.e. 65536 in all)
 #ifndef WPP_REGS_SOFTMAX
 #define WPP_REGS_SOFTMAX 192
-#define WPP_REGS_EPILOGUE 56
-#define WPP_REGS_UTIL 72
+#define WPP_REGS_EPILOGUE 64
+#define WPP_REGS_UTIL 64
 #endif
 constexpr int kRegsSoftmax = WPP_REGS_SOFTMAX, kRegsEpilogue = WPP_REGS_EPILOGUE, kRegsUtil = WPP_REGS_UTIL;
 static_assert(8 * kRegsSoftmax + 4 * kRegsEpilogue + 4 * kRegsUtil <= 2048, "register file exceeded");
