@@ -477,18 +477,22 @@ def main():
     def one_step(i, attn_events=None, qd=q, knd=k_new, vnd=v_new, btd=bt, Pd=P, Cd=C):
         s = i % ring
         plan_free[s].synchronize()                       # the copy that last used this buffer has run
+        t_plan = time.perf_counter()
         plan = wpp.wpp_plan_tiles(ctx, desc, w.prefix_lens, w.chunk_lens, opts=opts, out=plan_host[s])
+        t_plan = time.perf_counter() - t_plan
         plan.to_device(out=plan_dev[s])
         plan_free[s].record(stream)
+        if attn_events is not None:
+            a0, a, b = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+            a0.record(stream)
         wpp.wpp_kv_append(ctx, desc, knd, vnd, k_pool, v_pool, btd, Pd, Cd, plan, status=status)
         if attn_events is not None:
-            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             a.record(stream)
         wpp.wpp_prefill_attention_varlen(ctx, desc, qd, out, None, k_pool, v_pool, btd, Pd, Cd, plan,
                                          workspace=ws, status=status)
         if attn_events is not None:
             b.record(stream)
-            attn_events.append((a, b))
+            attn_events.append((a, b, a0, t_plan))
         return plan
 
     barrier = replicas.barrier
@@ -513,7 +517,12 @@ def main():
     launches = ctx.launch_count() - launches0
     clocks = sampler.stop()
     ms_step = max_over_ranks(ev0.elapsed_time(ev1) / args.steps)
-    attn_ms = statistics.mean(a.elapsed_time(b) for a, b in attn_events)
+    attn_ms = statistics.mean(a.elapsed_time(b) for a, b, _, _ in attn_events)
+    phases = {"plan_host_ms": 1e3 * statistics.mean(t for _, _, _, t in attn_events),
+              "append_ms": statistics.mean(a0.elapsed_time(a) for a, _, a0, _ in attn_events),
+              "attention_ms": attn_ms,
+              "note": "the host plans the next wave while the GPU runs the current one; append and attention are "
+                      "CUDA-event times on the launching stream"}
     if int(status.item()) != 0:
         raise SystemExit(f"device status {int(status.item())} after the timed region")
     info = plan.info
@@ -645,6 +654,7 @@ def main():
             "tflops": flops / (ms_step * 1e-3) / 1e12 * world,
             "served_tokens_per_s": world * float((w.prefix_lens.astype(np.int64) + w.chunk_lens).sum()) / (ms_step * 1e-3),
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline, "cpu_baseline": cpu,
+            "phases": phases,
         }
         print(json.dumps(line))
     replicas.finalize()
