@@ -10,6 +10,8 @@ library and never imports it.
                  leaves open are readings: parity unpinned for those (listed in the module).
 ``hints``      : chained block hash and gallop/bisect index probe of Section 4.3 (plain Python); the hash function
                  is a reading: parity unpinned for that choice.
+``kda``        : the recurrent-state (KDA) update of Section 3.1 token by token in fp64, with the snapshots of
+                 Section 3.2 (plain numpy); pinned by a hand-worked example, closed forms and a library solve.
 """
 from .reference import (  # noqa: F401
     build,
