@@ -327,6 +327,49 @@ int64_t wpp_hint_index_size(const wpp_hint_index* idx);     /* number of keys; -
 int wpp_hint_probe(const wpp_hint_index* idx, int32_t window, const uint64_t* hashes_host, int64_t n_blocks,
                    int64_t* matched_blocks, int32_t* probes_or_null);
 
+/* ---------------------------------------------------------------------------------------------------------
+ * Recurrent-state layer of a chunk (Section 3.1, the simplified KDA update; Section 3.2, snapshots): the other
+ * cache type of a hybrid model's stage.  Per request and head, token by token over the chunk,
+ *     S_t = (I - beta_t k_t k_t^T) Diag(alpha_t) S_{t-1} + beta_t k_t v_t^T,      o_t = S_t^T q_t,
+ * with S (d_k x d_v, fp32) resumed from the state after exactly the reused prefix - a recurrent layer cannot
+ * resume from anything else - and written back at the chunk end and, optionally, at sparse periodic boundaries.
+ * Heads are independent.  No normalisation or scaling of q or k is applied here (the update has none).
+ * Arithmetic: fp32 throughout (inputs widened, fp32 fused multiply-adds in token order), outputs rounded to bf16. */
+typedef struct {
+    int32_t num_requests;   /* R >= 0 */
+    int32_t num_heads;      /* H >= 1: state heads */
+    int32_t d_k;            /* 128 */
+    int32_t d_v;            /* 128 */
+    int32_t num_slots;      /* slots of state_pool, each H * d_k * d_v floats */
+    int32_t snap_interval;  /* > 0: snapshot whenever the tokens folded into S reach a multiple of it; 0: none */
+    int32_t max_snaps;      /* row length of snap_slots (0 when snap_interval is 0) */
+    int32_t reserved;       /* 0 */
+    int64_t total_tokens;   /* T = row_offsets[R] */
+} wpp_kda_desc;
+
+/* One launch on `cuda_stream` for the whole ragged batch; request i owns rows [row_offsets[i], row_offsets[i+1]).
+ *   q, k        : device bf16 [T, H, d_k], dense;  v : device bf16 [T, H, d_v];  all 16-byte aligned.
+ *   alpha       : device fp32 [T, H, d_k] (the per-channel decay Diag(alpha_t));  beta : device fp32 [T, H].
+ *   row_offsets : device int64 [R+1], exclusive scan of the chunk lengths.
+ *   prefix_lens : device int32 [R], tokens already folded into the resumed state (needed for periodic snapshots:
+ *                 boundaries are multiples of snap_interval in sequence positions); may be NULL if snap_interval = 0.
+ *   state_pool  : device fp32 [num_slots, H, d_k, d_v], 16-byte aligned; the library reads and writes slots in
+ *                 place and owns none of it.
+ *   state_in    : device int32 [R]: slot holding S after the reused prefix, or -1 for the zero state.
+ *   state_out   : device int32 [R]: slot that receives the state after the chunk, or -1.  May equal state_in[i];
+ *                 no slot may be written for one request and read or written for another in the same call.
+ *   snap_slots  : device int32 [R, max_snaps] or NULL: slot for the n-th boundary inside the chunk, -1 = skip;
+ *                 boundaries past max_snaps are skipped.
+ *   out         : device bf16 [T, H, d_v].
+ *   status_dev  : device int32 or NULL; a slot id outside [-1, num_slots) sets it to WPP_ERR_BOUNDS (if it was 0)
+ *                 and that request's state is neither read (zero state used) nor written there.
+ * A request with an empty chunk copies state_in to state_out.  Returns WPP_ERR_INVALID_ARG for null or misaligned
+ * pointers or negative sizes, WPP_ERR_UNSUPPORTED for d_k, d_v other than 128, WPP_ERR_CUDA for a launch failure. */
+int wpp_kda_chunk(const wpp_ctx* ctx, const wpp_kda_desc* desc, const void* q, const void* k, const void* v,
+                  const float* alpha, const float* beta, const int64_t* row_offsets, const int32_t* prefix_lens,
+                  float* state_pool, const int32_t* state_in, const int32_t* state_out, const int32_t* snap_slots,
+                  void* out, int32_t* status_dev, void* cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

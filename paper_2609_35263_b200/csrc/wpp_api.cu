@@ -272,3 +272,47 @@ extern "C" int wpp_prefill_attention_varlen_static(const wpp_ctx* ctx, const wpp
                                         chunk_lens, plan_host, plan_dev, g_static_scratch_ptr[ctx->device],
                                         (size_t)WPP_STATIC_SCRATCH_BYTES, status_dev, cuda_stream);
 }
+
+extern "C" int wpp_kda_chunk(const wpp_ctx* ctx, const wpp_kda_desc* desc, const void* q, const void* k, const void* v,
+                             const float* alpha, const float* beta, const int64_t* row_offsets,
+                             const int32_t* prefix_lens, float* state_pool, const int32_t* state_in,
+                             const int32_t* state_out, const int32_t* snap_slots, void* out, int32_t* status_dev,
+                             void* cuda_stream) {
+    if (!ctx || !desc) return WPP_ERR_INVALID_ARG;
+    if (desc->num_requests < 0 || desc->num_heads < 1 || desc->num_slots < 0 || desc->snap_interval < 0 ||
+        desc->max_snaps < 0 || desc->total_tokens < 0 || desc->reserved != 0)
+        return WPP_ERR_INVALID_ARG;
+    if (desc->d_k != 128 || desc->d_v != 128) return WPP_ERR_UNSUPPORTED;
+    if (desc->num_requests > 65535) return WPP_ERR_UNSUPPORTED;      // one grid row per request
+    if (desc->num_requests == 0) return WPP_OK;
+    if (!row_offsets || !state_in || !state_out) return WPP_ERR_INVALID_ARG;
+    if (desc->num_slots > 0 && !state_pool) return WPP_ERR_INVALID_ARG;
+    if (desc->total_tokens > 0 && (!q || !k || !v || !alpha || !beta || !out)) return WPP_ERR_INVALID_ARG;
+    if (desc->snap_interval > 0 && !prefix_lens) return WPP_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(alpha) || !aligned16(out) || !aligned16(state_pool))
+        return WPP_ERR_INVALID_ARG;
+    wpp::KdaParams p;
+    memset(&p, 0, sizeof(p));
+    p.q = static_cast<const __nv_bfloat16*>(q);
+    p.k = static_cast<const __nv_bfloat16*>(k);
+    p.v = static_cast<const __nv_bfloat16*>(v);
+    p.alpha = alpha;
+    p.beta = beta;
+    p.row_offsets = row_offsets;
+    p.prefix_lens = prefix_lens;
+    p.state_pool = state_pool;
+    p.state_in = state_in;
+    p.state_out = state_out;
+    p.snap_slots = desc->max_snaps > 0 ? snap_slots : nullptr;
+    p.out = static_cast<__nv_bfloat16*>(out);
+    p.status = status_dev;
+    p.num_requests = desc->num_requests;
+    p.num_heads = desc->num_heads;
+    p.num_slots = desc->num_slots;
+    p.snap_interval = desc->snap_interval;
+    p.max_snaps = desc->max_snaps;
+    int e = wpp_launch_kda(&p, cuda_stream);
+    if (e != 0) return cuda_fail(ctx, e);
+    const_cast<wpp_ctx*>(ctx)->launches += 1;
+    return WPP_OK;
+}

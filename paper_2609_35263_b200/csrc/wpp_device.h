@@ -50,6 +50,23 @@ struct CombineParams {
     int32_t num_q_heads, head_dim, tile_m;
 };
 
+struct KdaParams {
+    const __nv_bfloat16* q;
+    const __nv_bfloat16* k;
+    const __nv_bfloat16* v;
+    const float* alpha;
+    const float* beta;
+    const int64_t* row_offsets;
+    const int32_t* prefix_lens;
+    float* state_pool;
+    const int32_t* state_in;
+    const int32_t* state_out;
+    const int32_t* snap_slots;
+    __nv_bfloat16* out;
+    int32_t* status;
+    int32_t num_requests, num_heads, num_slots, snap_interval, max_snaps;
+};
+
 }  // namespace wpp
 
 extern "C" {
@@ -57,5 +74,6 @@ int wpp_launch_attention(int head_dim, const CUtensorMap* tq, const CUtensorMap*
                          const wpp::AttnParams* p, int num_ctas, void* stream);
 int wpp_launch_append(const wpp::AppendParams* p, int num_sms, void* stream);
 int wpp_launch_combine(const wpp::CombineParams* p, int num_combine, void* stream);
+int wpp_launch_kda(const wpp::KdaParams* p, void* stream);
 int wpp_launch_selftest_wait(long long limit_cycles, int32_t* status, long long* waited_cycles, void* stream);
 }

@@ -1,0 +1,171 @@
+"""wpp_kda_chunk (CUDA, through the C ABI) against the fp64 oracle of the recurrent-state layer (Section 3.1 update,
+Section 3.2 snapshots), element by element on seeded inputs, plus the properties that hold at any size.
+
+Tolerances: the kernel computes in fp32 (relative error of a step about 1e-7, a few 1e-6 after thousands of
+contracting steps) and rounds outputs to bf16 (relative 2^-9); states stay fp32.
+  outputs : |delta| <= 2^-8 |ref| + 1e-4 max|ref|          states : |delta| <= 1e-4 max|ref|"""
+import numpy as np
+import pytest
+import torch
+
+import paper_2609_35263_b200 as wpp
+import wpp_workloads as W
+from oracle import kda as O
+from tests import gpu_harness as H
+
+pytestmark = pytest.mark.gpu
+
+
+def _oracle(w, t, heads=None):
+    hs = slice(None) if heads is None else heads
+    f = lambda x: x[:, hs].double().numpy()
+    pool = t["state_pool"][:, hs].double().numpy().copy()
+    o = O.kda_chunk(f(t["q"]), f(t["k"]), f(t["v"]), f(t["alpha"]), f(t["beta"]), w.chunk_lens, pool, w.state_in,
+                    w.state_out, w.prefix_lens, w.snap_interval, w.snap_slots)
+    return o, pool
+
+
+def _gpu(w, t, state_in=None, state_out=None):
+    dev = torch.device("cuda")
+    d = {k: v.to(dev) for k, v in t.items()}
+    i32 = lambda a: None if a is None else torch.from_numpy(np.ascontiguousarray(a, dtype=np.int32)).to(dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    out = wpp.wpp_kda_chunk(H.ctx(), d["q"], d["k"], d["v"], d["alpha"], d["beta"],
+                            torch.from_numpy(w.row_offsets).to(dev), d["state_pool"],
+                            i32(w.state_in if state_in is None else state_in),
+                            i32(w.state_out if state_out is None else state_out),
+                            prefix_lens=i32(w.prefix_lens), snap_interval=w.snap_interval,
+                            snap_slots=i32(w.snap_slots), status=status)
+    torch.cuda.synchronize()
+    return out.float().cpu().double().numpy(), d["state_pool"].cpu().double().numpy(), int(status.item())
+
+
+def _close_out(got, ref, what):
+    if ref.size == 0:
+        return
+    bound = 2.0 ** -8 * np.abs(ref) + 1e-4 * np.abs(ref).max()
+    bad = np.abs(got - ref) > bound
+    assert not bad.any(), f"{what}: {bad.sum()} outputs off, worst {np.abs(got - ref).max():.3e}"
+
+
+def _close_state(got, ref, what):
+    assert np.abs(got - ref).max() <= 1e-4 * max(np.abs(ref).max(), 1e-30), f"{what}: {np.abs(got - ref).max():.3e}"
+
+
+@pytest.mark.parametrize("lens,prefix,interval,H_", [
+    ([37, 5, 64, 0, 1, 16, 17, 130], [11, 0, 128, 7, 0, 16, 3, 1000], 16, 2),     # ragged, stage tails, empty chunk
+    ([300], [0], 0, 3),                                                            # one request from the zero state
+    ([15, 16, 17, 31, 32, 33], [1, 2, 3, 4, 5, 6], 7, 1),                          # around the staging size; odd interval
+])
+def test_ragged_batches_match_the_oracle(lens, prefix, interval, H_):
+    w = W.kda_workload("ragged", 11, lens, H_, prefix, snap_interval=interval)
+    t = w.tensors()
+    ref_o, ref_pool = _oracle(w, t)
+    got_o, got_pool, status = _gpu(w, t)
+    assert status == 0
+    _close_out(got_o, ref_o, "outputs")
+    _close_state(got_pool, ref_pool, "state pool")
+    # slots nobody writes keep their bits
+    written = set(int(s) for s in w.state_out if s >= 0)
+    if w.snap_slots is not None:
+        written |= set(int(s) for s in w.snap_slots.ravel() if s >= 0)
+    for s in range(w.num_slots):
+        if s not in written:
+            assert np.array_equal(got_pool[s], t["state_pool"][s].double().numpy())
+
+
+def test_a_long_chain_stays_within_tolerance():
+    w = W.kda_workload("long", 5, [2048], 1, [4096])
+    t = w.tensors()
+    ref_o, ref_pool = _oracle(w, t)
+    got_o, got_pool, status = _gpu(w, t)
+    assert status == 0
+    _close_out(got_o, ref_o, "outputs")
+    _close_state(got_pool, ref_pool, "state pool")
+
+
+def test_splitting_a_chunk_and_resuming_is_bit_identical():
+    """Section 3.2: the state after exactly r tokens is all a recurrent layer needs; the kernel's arithmetic per
+    token does not depend on where a chunk starts, so one call and two resumed calls agree to the bit."""
+    w = W.kda_workload("whole", 3, [100, 64], 2, [5, 0], resume=[True, False])
+    t = w.tensors()
+    whole_o, whole_pool, _ = _gpu(w, t)
+    rows = w.row_offsets
+    parts_o = np.zeros_like(whole_o)
+    pool = t["state_pool"].clone()
+    for (a, b), first in (((37, 20), True), ((63, 44), False)):
+        cut = [37, 20]
+        sel = np.concatenate([np.arange(rows[i] + (0 if first else cut[i]), rows[i] + (cut[i] if first else w.chunk_lens[i]))
+                              for i in range(2)])
+        wp = W.kda_workload("part", 3, [a, b], 2, [5, 0])
+        wp.num_slots = w.num_slots
+        tp = {k: (v[sel].contiguous() if k != "state_pool" else pool) for k, v in t.items()}
+        s_in = w.state_in if first else w.state_out          # the second call resumes from what the first stored
+        o, new_pool, status = _gpu(wp, tp, state_in=s_in, state_out=w.state_out)
+        assert status == 0
+        parts_o[sel] = o
+        pool = torch.from_numpy(new_pool).float()
+    assert np.array_equal(parts_o, whole_o)
+    assert np.array_equal(pool.double().numpy(), whole_pool)
+
+
+def test_in_place_slots_and_pure_decay():
+    # state_out == state_in updates a slot in place; with beta = 0 and alpha = 1 the state must not change at all
+    w = W.kda_workload("inplace", 9, [50, 20], 2, [10, 10])
+    t = w.tensors()
+    t["beta"].zero_()
+    t["alpha"].fill_(1.0)
+    got_o, got_pool, status = _gpu(w, t, state_out=w.state_in)
+    assert status == 0
+    assert np.array_equal(got_pool, t["state_pool"].double().numpy())
+    ref = np.einsum("rhkv,rhk->rhv", t["state_pool"][[0] * 50 + [1] * 20].double().numpy(), t["q"].double().numpy())
+    _close_out(got_o, ref, "o = S0^T q")
+
+
+def test_bad_slot_ids_are_reported_and_skipped():
+    w = W.kda_workload("bad", 2, [20, 20, 20], 1, [4, 4, 4])
+    t = w.tensors()
+    s_in, s_out = w.state_in.copy(), w.state_out.copy()
+    s_in[1], s_out[2] = w.num_slots + 5, -7
+    got_o, got_pool, status = _gpu(w, t, state_in=s_in, state_out=s_out)
+    assert status == 3                                                 # WPP_ERR_BOUNDS
+    w.state_in, w.state_out = np.where(s_in >= w.num_slots, -1, s_in), np.where(s_out < -1, -1, s_out)
+    ref_o, ref_pool = _oracle(w, t)                                    # bad ids behave like -1
+    _close_out(got_o, ref_o, "outputs")
+    _close_state(got_pool, ref_pool, "state pool")
+
+
+def test_argument_errors():
+    dev = torch.device("cuda")
+    z = lambda *s, dt=torch.bfloat16: torch.zeros(*s, dtype=dt, device=dev)
+    ro = torch.tensor([0, 4], dtype=torch.int64, device=dev)
+    slot = torch.zeros(1, dtype=torch.int32, device=dev)
+    pool = z(1, 1, 64, 64, dt=torch.float32)
+    with pytest.raises(wpp.WppError) as e:                            # d_k = d_v = 64 is not built
+        wpp.wpp_kda_chunk(H.ctx(), z(4, 1, 64), z(4, 1, 64), z(4, 1, 64), z(4, 1, 64, dt=torch.float32),
+                          z(4, 1, dt=torch.float32), ro, pool, slot, slot)
+    assert e.value.status == 2
+    pool = z(1, 1, 128, 128, dt=torch.float32)
+    with pytest.raises(wpp.WppError) as e:                            # periodic snapshots need prefix_lens
+        wpp.wpp_kda_chunk(H.ctx(), z(4, 1, 128), z(4, 1, 128), z(4, 1, 128), z(4, 1, 128, dt=torch.float32),
+                          z(4, 1, dt=torch.float32), ro, pool, slot, slot, snap_interval=2,
+                          snap_slots=torch.zeros(1, 2, dtype=torch.int32, device=dev))
+    assert e.value.status == 1
+
+
+def test_full_size_wave_on_sampled_heads():
+    """The benchmark's wave (8 lanes x 2,048 tokens, 32 heads, resumed states): the oracle recomputes three
+    (request, head) chains and all of their outputs and final states are compared."""
+    w = W.kda_wave()
+    t = w.tensors()
+    got_o, got_pool, status = _gpu(w, t)
+    assert status == 0
+    rows = w.row_offsets
+    for req, head in ((0, 0), (3, 17), (7, 31)):
+        sl = slice(rows[req], rows[req + 1])
+        sub = W.kda_workload("one", 0, [int(w.chunk_lens[req])], 1, [int(w.prefix_lens[req])])
+        sub.num_slots, sub.state_in, sub.state_out = w.num_slots, w.state_in[req:req + 1], w.state_out[req:req + 1]
+        ts = {k: (v[sl] if k != "state_pool" else v) for k, v in t.items()}
+        ref_o, ref_pool = _oracle(sub, ts, heads=slice(head, head + 1))
+        _close_out(got_o[sl, head:head + 1], ref_o, f"outputs of request {req} head {head}")
+        _close_state(got_pool[w.state_out[req], head], ref_pool[w.state_out[req], 0], "final state")

@@ -17,4 +17,7 @@ from .generate import (  # noqa: F401
     cfg4,
     cfg5_cell,
     CONFIG_BUILDERS,
+    KdaWorkload,
+    kda_workload,
+    kda_wave,
 )

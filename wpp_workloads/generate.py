@@ -291,3 +291,79 @@ CONFIG_BUILDERS: Dict[str, Callable[[], Workload]] = {
     "cfg4": cfg4,
     "cfg4_alt": lambda: cfg4("alternate"),
 }
+
+
+# ---------------------------------------------------------------------------------------------------------------
+# Inputs of the recurrent-state (KDA) layer.  Only value streams and their pre-processing live here: keys are
+# L2-normalised and queries scaled by d_k^-1/2 *before* the operation, as a model does ahead of the update the
+# paper prints; decays are sigmoid(4 + 2 n) (median 0.98, a few per cent of channels below 0.9) and write
+# strengths sigmoid(n), n standard normal.
+STREAM_KDA_Q, STREAM_KDA_K, STREAM_KDA_V, STREAM_KDA_ALPHA, STREAM_KDA_BETA, STREAM_KDA_STATE = 8, 9, 10, 11, 12, 13
+
+
+@dataclasses.dataclass
+class KdaWorkload:
+    name: str
+    seed: int
+    chunk_lens: np.ndarray        # int64 [R]
+    prefix_lens: np.ndarray       # int32 [R]: tokens already folded into the resumed state
+    num_heads: int
+    d_k: int
+    d_v: int
+    num_slots: int
+    state_in: np.ndarray          # int32 [R]
+    state_out: np.ndarray         # int32 [R]
+    snap_interval: int = 0
+    snap_slots: Optional[np.ndarray] = None      # int32 [R, max_snaps]
+
+    @property
+    def total_tokens(self) -> int:
+        return int(self.chunk_lens.sum())
+
+    @property
+    def row_offsets(self) -> np.ndarray:
+        return np.concatenate([[0], np.cumsum(self.chunk_lens)]).astype(np.int64)
+
+    def tensors(self, device="cpu") -> Dict[str, torch.Tensor]:
+        """q, k, v (bf16), alpha, beta (fp32) and the state pool (fp32); always computed on the CPU so that the
+        bits do not depend on the device, then moved."""
+        T, H, dk, dv = self.total_tokens, self.num_heads, self.d_k, self.d_v
+        n = lambda stream, count: counter_normal_bf16(self.seed, stream, 0, count).float()
+        q = (n(STREAM_KDA_Q, T * H * dk).view(T, H, dk) * dk ** -0.5).to(torch.bfloat16)
+        k = n(STREAM_KDA_K, T * H * dk).view(T, H, dk)
+        k = (k / k.norm(dim=-1, keepdim=True).clamp_min(1e-6)).to(torch.bfloat16)
+        v = n(STREAM_KDA_V, T * H * dv).view(T, H, dv).to(torch.bfloat16)
+        alpha = torch.sigmoid(4.0 + 2.0 * n(STREAM_KDA_ALPHA, T * H * dk)).view(T, H, dk).contiguous()
+        beta = torch.sigmoid(n(STREAM_KDA_BETA, T * H)).view(T, H).contiguous()
+        state = (0.1 * n(STREAM_KDA_STATE, self.num_slots * H * dk * dv)).view(self.num_slots, H, dk, dv).contiguous()
+        out = dict(q=q, k=k, v=v, alpha=alpha, beta=beta, state_pool=state)
+        return {name: t.to(device) for name, t in out.items()}
+
+
+def kda_workload(name, seed, chunk_lens, num_heads, prefix_lens=None, resume=None, snap_interval=0, d_k=128,
+                 d_v=128, spare_slots=2) -> KdaWorkload:
+    """Request i resumes from slot i when resume[i] (default: when its prefix is not empty) and stores its final
+    state in slot R + i; periodic snapshots, if any, go to slots after those, one per boundary inside the chunk."""
+    chunk_lens = np.asarray(chunk_lens, dtype=np.int64)
+    R = int(chunk_lens.size)
+    prefix_lens = np.zeros(R, np.int32) if prefix_lens is None else np.asarray(prefix_lens, dtype=np.int32)
+    resume = (prefix_lens > 0) if resume is None else np.asarray(resume, dtype=bool)
+    state_in = np.where(resume, np.arange(R), -1).astype(np.int32)
+    state_out = (R + np.arange(R)).astype(np.int32)
+    slots, snaps = 2 * R, None
+    if snap_interval > 0:
+        counts = (prefix_lens + chunk_lens) // snap_interval - prefix_lens // snap_interval
+        snaps = np.full((R, max(1, int(counts.max()) if R else 1)), -1, dtype=np.int32)
+        for i in range(R):
+            for j in range(int(counts[i])):
+                snaps[i, j] = slots
+                slots += 1
+    return KdaWorkload(name, seed, chunk_lens, prefix_lens, num_heads, d_k, d_v, slots + spare_slots, state_in,
+                       state_out, snap_interval, snaps)
+
+
+def kda_wave(num_requests: int = 8, chunk: int = 2048, num_heads: int = 32, prefix: int = 65536, seed: int = 7) -> KdaWorkload:
+    """One wave of a hybrid model's recurrent layer at the paper's matched settings: a 16,384-token budget shared
+    by 8 lanes, 32 state heads of 128 x 128, every request resuming from the snapshot of a reused prefix."""
+    return kda_workload(f"kda_wave_{num_requests}x{chunk}", seed, [chunk] * num_requests, num_heads,
+                        [prefix] * num_requests)
