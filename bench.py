@@ -405,6 +405,79 @@ def run_hints(args):
     print(json.dumps(line))
 
 
+def run_kda(args):
+    """The recurrent-state (KDA) layer of one wave (Section 3.1 update, Section 3.2 snapshots): `--kda-lanes`
+    requests of `--kda-chunk` tokens, 32 state heads of 128 x 128, every request resuming from a snapshot and
+    storing one at the chunk end.  Timed with CUDA events over back-to-back launches on inputs larger than L2;
+    the roofline is plain fp32 arithmetic: 7 flop per state element and token (one multiply and three fused
+    multiply-adds) against 148 SMs x 128 lanes x 2 flop x the maximum SM clock."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    import torch
+    import paper_2609_35263_b200 as wpp
+    import wpp_workloads as W
+    from oracle import kda as O
+    dev = torch.device("cuda", 0)
+    ctx = wpp.Context(0)
+    w = W.kda_wave(args.kda_lanes, args.kda_chunk)
+    t = w.tensors()
+    d = {k: v.to(dev) for k, v in t.items()}
+    i32 = lambda a: torch.from_numpy(np.ascontiguousarray(a, dtype=np.int32)).to(dev)
+    ro, s_in, s_out = torch.from_numpy(w.row_offsets).to(dev), i32(w.state_in), i32(w.state_out)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    out = torch.empty((w.total_tokens, w.num_heads, w.d_v), dtype=torch.bfloat16, device=dev)
+    step = lambda: wpp.wpp_kda_chunk(ctx, d["q"], d["k"], d["v"], d["alpha"], d["beta"], ro, d["state_pool"], s_in, s_out,
+                                     out=out, status=status)
+    warm, steps = max(3, args.warmup), max(1, args.steps)
+    for _ in range(warm):
+        step()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(0)
+    sampler.start()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for _ in range(steps):
+        step()
+    b.record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    ms = a.elapsed_time(b) / steps
+    if int(status.item()) != 0:
+        raise SystemExit(f"wpp_kda_chunk reported status {int(status.item())}")
+    # parity on one chain, and the oracle's own speed on it
+    req, head = w.chunk_lens.size - 1, w.num_heads - 1
+    sl = slice(int(w.row_offsets[req]), int(w.row_offsets[req + 1]))
+    f = lambda x: x[sl, head:head + 1].double().numpy()
+    pool = t["state_pool"][:, head:head + 1].double().numpy().copy()
+    t0 = time.perf_counter()
+    ref = O.kda_chunk(f(t["q"]), f(t["k"]), f(t["v"]), f(t["alpha"]), f(t["beta"]), [sl.stop - sl.start], pool,
+                      w.state_in[req:req + 1], w.state_out[req:req + 1])
+    t_cpu = time.perf_counter() - t0
+    got = out[sl, head:head + 1].float().cpu().double().numpy()
+    err = float(np.abs(got - ref).max())
+    if not np.all(np.abs(got - ref) <= 2.0 ** -8 * np.abs(ref) + 1e-4 * np.abs(ref).max()):
+        raise SystemExit(f"wpp_kda_chunk disagrees with the oracle (max |delta| {err:.3e})")
+    T, Hh = w.total_tokens, w.num_heads
+    flops = 7.0 * w.d_k * w.d_v * T * Hh
+    peak = 148 * 128 * 2 * 1965e6 / 1e12
+    nbytes = T * Hh * (2 * w.d_k * 2 + 2 * w.d_v * 2 + 4 * w.d_k + 4) + 2 * w.chunk_lens.size * Hh * w.d_k * w.d_v * 4
+    line = {"metric": "recurrent-state (KDA) layer, new tokens/s through one layer", "value": T / (ms * 1e-3),
+            "unit": "tokens/s", "n_gpus": 1, "steps": steps, "warmup": warm, "ms_per_step": ms, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic", "gpu_launches": steps,
+            "config": {"workload": w.name, "requests": int(w.chunk_lens.size), "chunk": int(w.chunk_lens[0]),
+                       "state_heads": Hh, "d_k": w.d_k, "d_v": w.d_v, "l2": "inputs larger than L2"},
+            "clocks": clocks,
+            "roofline": {"bound": "alu", "kernel": "wpp_kda_chunk_kernel", "achieved": flops / (ms * 1e-3) / 1e12,
+                         "peak": peak, "unit": "TFLOP/s", "frac": flops / (ms * 1e-3) / 1e12 / peak,
+                         "peak_source": "derived: 148 SMs x 128 fp32 lanes x 2 flop x 1965 MHz",
+                         "flop_per_token_head": 7 * w.d_k * w.d_v, "traffic": None,
+                         "hbm_gbs_algorithmic": nbytes / (ms * 1e-3) / 1e9},
+            "cpu_baseline": {"value": (sl.stop - sl.start) / t_cpu / Hh, "unit": "tokens/s", "cores": 1, "kind": "oracle",
+                             "sample": f"one (request, head) chain of {sl.stop - sl.start} tokens, scaled to {Hh} heads"},
+            "parity": {"checked": f"request {req}, head {head}: all outputs against the fp64 oracle", "max_abs_err": err}}
+    print(json.dumps(line))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -421,6 +494,9 @@ def main():
     ap.add_argument("--waves", action="store_true", help="time the wave-budget planner (host only) instead")
     ap.add_argument("--waves-sim", action="store_true", help="wave planner + kernels: simulated pipeline fill")
     ap.add_argument("--hints", action="store_true", help="chained block hashing on the GPU and the hint probe")
+    ap.add_argument("--kda", action="store_true", help="the recurrent-state (KDA) layer of one wave")
+    ap.add_argument("--kda-lanes", type=int, default=8)
+    ap.add_argument("--kda-chunk", type=int, default=2048)
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "native" else args.warmup
 
@@ -432,6 +508,9 @@ def main():
         return
     if args.hints:
         run_hints(args)
+        return
+    if args.kda:
+        run_kda(args)
         return
     if args.impl == "reference":
         run_reference(args)

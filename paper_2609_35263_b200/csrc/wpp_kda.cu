@@ -2,14 +2,19 @@
 //     S_t = (I - beta_t k_t k_t^T) Diag(alpha_t) S_{t-1} + beta_t k_t v_t^T,     o_t = S_t^T q_t,
 // resumed from a snapshot and snapshotted at the chunk end and at periodic boundaries (Section 3.2).
 //
-// The columns of S evolve independently: with s = S[:, j], d = (k*alpha) . s and c = v_j - d,
-//     s <- alpha * s + c * (beta k),        o_j = (q*alpha) . s_old + c * (q . beta k).
+// The columns of S evolve independently: with s = S[:, j],
+//     s' = alpha * s,    c = beta (v_j - k . s'),    s <- s' + c k,    o_j = q . s' + c (q . k).
 // One CTA owns one (request, head).  256 compute threads hold the 128 x 128 fp32 state in registers: a thread has
-// two adjacent columns and a quarter of the rows (64 values, packed in pairs for the two-wide fp32 FMA), so a dot
-// product over d_k is 16 packed FMAs per column and two shuffles.  A ninth warp stages the next 16 tokens while
-// the others work: it widens q, k, v, forms k*alpha, q*alpha, beta*k and q . (beta k) once per token (shared by
-// all 128 columns) and leaves them in shared memory, where the four row quarters read 64 consecutive bytes
-// (no bank conflicts) and the eight column pairs of a warp read the same words (broadcast).
+// four adjacent columns and an eighth of the rows (64 values, packed in pairs for the two-wide fp32 FMA).  The
+// shared vectors alpha, k, q reach the registers of every thread that needs them through shared memory, whose
+// 128 bytes per clock bound this layout: four columns per thread need 12 sixteen-byte loads per token and thread
+// (two columns needed 24 and ran at the shared-memory limit), paid for with an eight-lane reduction per column,
+// done as exchange-and-halve steps (4 shuffles for four columns, 3 more to hand the results round).  A ninth warp stages the next 32 tokens while
+// the others work: it widens q, k, v to fp32, forms q . k once per token (shared by all 128 columns) and leaves
+// them with alpha and beta in shared memory, where the eight row groups read 128 consecutive bytes (no bank
+// conflicts) and the four column groups of a warp read the same words (broadcast).  A thread's operands for the
+// next token are requested while it still works on this one: the shared-memory latency is off the token chain,
+// which is what bounds a recurrence (two warps per scheduler cannot hide it otherwise).
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -21,18 +26,17 @@ namespace wpp {
 namespace {
 
 constexpr int kDK = 128, kDV = 128;
-constexpr int kStageTokens = 16;
+constexpr int kStageTokens = 32;
 constexpr int kComputeWarps = 8;
 constexpr int kThreads = (kComputeWarps + 1) * 32;
 
 struct KdaStage {
-    float ka[kStageTokens][kDK];    // k * alpha
-    float qa[kStageTokens][kDK];    // q * alpha
-    float kb[kStageTokens][kDK];    // beta * k
     float al[kStageTokens][kDK];    // alpha
+    float kk[kStageTokens][kDK];    // k
+    float qq[kStageTokens][kDK];    // q
     float v[kStageTokens][kDV];
-    float qkb[kStageTokens];        // q . (beta k)
-    float pad[kStageTokens];
+    float beta[kStageTokens];
+    float qk[kStageTokens];         // q . k
 };
 
 __device__ __forceinline__ uint64_t pk(float lo, float hi) {
@@ -52,19 +56,6 @@ __device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b) {
     uint64_t r;
     asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
     return r;
-}
-__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
-    uint64_t r;
-    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
-    return r;
-}
-__device__ __forceinline__ float quad_sum(uint64_t a, uint64_t b) {      // lanes of a row-quarter group: xor 1, 2
-    float lo, hi;
-    upk(add2(a, b), lo, hi);
-    float x = lo + hi;
-    x += __shfl_xor_sync(0xffffffffu, x, 1);
-    x += __shfl_xor_sync(0xffffffffu, x, 2);
-    return x;
 }
 __device__ __forceinline__ void widen4(uint2 raw, float (&f)[4]) {
     const __nv_bfloat162 a = *reinterpret_cast<const __nv_bfloat162*>(&raw.x);
@@ -100,27 +91,22 @@ __device__ __forceinline__ void kda_fill(const KdaParams& p, KdaStage* st, int64
         for (int u = 0; u < 4; ++u) {
             const int t = base + u;
             if (t < n) {
-                float q[4], k[4], v[4];
+                float q[4], k[4], v[4], part = 0.f;
                 widen4(rq[u], q);
                 widen4(rk[u], k);
                 widen4(rv[u], v);
-                const float a[4] = {ra[u].x, ra[u].y, ra[u].z, ra[u].w};
-                float ka[4], qa[4], kb[4], part = 0.f;
 #pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    ka[e] = k[e] * a[e];
-                    qa[e] = q[e] * a[e];
-                    kb[e] = rb[u] * k[e];
-                    part = fmaf(q[e], kb[e], part);
-                }
+                for (int e = 0; e < 4; ++e) part = fmaf(q[e], k[e], part);
 #pragma unroll
                 for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
-                *reinterpret_cast<float4*>(&st->ka[t][lane * 4]) = make_float4(ka[0], ka[1], ka[2], ka[3]);
-                *reinterpret_cast<float4*>(&st->qa[t][lane * 4]) = make_float4(qa[0], qa[1], qa[2], qa[3]);
-                *reinterpret_cast<float4*>(&st->kb[t][lane * 4]) = make_float4(kb[0], kb[1], kb[2], kb[3]);
                 *reinterpret_cast<float4*>(&st->al[t][lane * 4]) = ra[u];
+                *reinterpret_cast<float4*>(&st->kk[t][lane * 4]) = make_float4(k[0], k[1], k[2], k[3]);
+                *reinterpret_cast<float4*>(&st->qq[t][lane * 4]) = make_float4(q[0], q[1], q[2], q[3]);
                 *reinterpret_cast<float4*>(&st->v[t][lane * 4]) = make_float4(v[0], v[1], v[2], v[3]);
-                if (lane == 0) st->qkb[t] = part;
+                if (lane == 0) {
+                    st->beta[t] = rb[u];
+                    st->qk[t] = part;
+                }
             }
         }
     }
@@ -156,40 +142,63 @@ __global__ void __launch_bounds__(kThreads, 1) wpp_kda_chunk_kernel(const KdaPar
         return;
     }
 
-    // ---- compute threads: rows 16m + 4r + e (m < 8, e < 4) of columns 2cp and 2cp + 1
-    const int r = lane & 3, cp = warp * 8 + (lane >> 2);
+    // ---- compute threads: rows 32m + 4r + e (m < 4, e < 4; r = lane & 7) of columns 4cq .. 4cq + 3
+    const int r = lane & 7, cq = warp * 4 + (lane >> 3);
+    const bool b0 = lane & 1, b1 = lane & 2;
+    const int my_col = (b0 ? 2 : 0) + (b1 ? 1 : 0);                    // the column whose dot products end on this lane
     const size_t head_floats = (size_t)kDK * kDV;
-    uint64_t sA[8][2], sB[8][2];
+    uint64_t S[4][4][2];                                                // [column][m][row pair]
     if (slot_in >= 0) {
-        const float* src = p.state_pool + ((size_t)slot_in * H + head) * head_floats + 2 * cp;
+        const float* src = p.state_pool + ((size_t)slot_in * H + head) * head_floats + 4 * cq;
 #pragma unroll
-        for (int m = 0; m < 8; ++m) {
-            float2 x[4];
+        for (int m = 0; m < 4; ++m) {
+            float4 x[4];
 #pragma unroll
-            for (int e = 0; e < 4; ++e) x[e] = *reinterpret_cast<const float2*>(src + (size_t)(16 * m + 4 * r + e) * kDV);
-            sA[m][0] = pk(x[0].x, x[1].x);
-            sA[m][1] = pk(x[2].x, x[3].x);
-            sB[m][0] = pk(x[0].y, x[1].y);
-            sB[m][1] = pk(x[2].y, x[3].y);
+            for (int e = 0; e < 4; ++e) x[e] = *reinterpret_cast<const float4*>(src + (size_t)(32 * m + 4 * r + e) * kDV);
+            S[0][m][0] = pk(x[0].x, x[1].x), S[0][m][1] = pk(x[2].x, x[3].x);
+            S[1][m][0] = pk(x[0].y, x[1].y), S[1][m][1] = pk(x[2].y, x[3].y);
+            S[2][m][0] = pk(x[0].z, x[1].z), S[2][m][1] = pk(x[2].z, x[3].z);
+            S[3][m][0] = pk(x[0].w, x[1].w), S[3][m][1] = pk(x[2].w, x[3].w);
         }
     } else {
 #pragma unroll
-        for (int m = 0; m < 8; ++m) sA[m][0] = sA[m][1] = sB[m][0] = sB[m][1] = 0ull;
+        for (int c = 0; c < 4; ++c)
+#pragma unroll
+            for (int m = 0; m < 4; ++m) S[c][m][0] = S[c][m][1] = 0ull;
     }
 
     auto store_state = [&](int slot) {
-        float* dst = p.state_pool + ((size_t)slot * H + head) * head_floats + 2 * cp;
+        float* dst = p.state_pool + ((size_t)slot * H + head) * head_floats + 4 * cq;
 #pragma unroll
-        for (int m = 0; m < 8; ++m) {
-            float a[4], b[4];
-            upk(sA[m][0], a[0], a[1]);
-            upk(sA[m][1], a[2], a[3]);
-            upk(sB[m][0], b[0], b[1]);
-            upk(sB[m][1], b[2], b[3]);
+        for (int m = 0; m < 4; ++m) {
+            float x[4][4];
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                upk(S[c][m][0], x[c][0], x[c][1]);
+                upk(S[c][m][1], x[c][2], x[c][3]);
+            }
 #pragma unroll
             for (int e = 0; e < 4; ++e)
-                *reinterpret_cast<float2*>(dst + (size_t)(16 * m + 4 * r + e) * kDV) = make_float2(a[e], b[e]);
+                *reinterpret_cast<float4*>(dst + (size_t)(32 * m + 4 * r + e) * kDV) =
+                    make_float4(x[0][e], x[1][e], x[2][e], x[3][e]);
         }
+    };
+
+    // Sum over the eight row groups of four per-column partial sums: after two exchange-and-halve steps and one
+    // plain step, every lane holds the complete sum of column `my_col` (4 shuffles instead of 12).
+    auto reduce_scatter = [&](const uint64_t (&acc)[4]) -> float {
+        float x[4];
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            float lo, hi;
+            upk(acc[c], lo, hi);
+            x[c] = lo + hi;
+        }
+        const float y0 = (b0 ? x[2] : x[0]) + __shfl_xor_sync(0xffffffffu, b0 ? x[0] : x[2], 1);
+        const float y1 = (b0 ? x[3] : x[1]) + __shfl_xor_sync(0xffffffffu, b0 ? x[1] : x[3], 1);
+        float z = (b1 ? y1 : y0) + __shfl_xor_sync(0xffffffffu, b1 ? y0 : y1, 2);
+        z += __shfl_xor_sync(0xffffffffu, z, 4);
+        return z;
     };
 
     // periodic snapshots: the next sequence position at which one is due
@@ -201,47 +210,63 @@ __global__ void __launch_bounds__(kThreads, 1) wpp_kda_chunk_kernel(const KdaPar
         next_snap = (pos / interval + 1) * (int64_t)interval;
     }
 
-    __nv_bfloat16* out = p.out + (row0 * H + head) * kDV + 2 * cp;
+    __nv_bfloat16* out = p.out + (row0 * H + head) * kDV + 4 * cq + my_col;
     __syncthreads();                                                    // stage 0 is filled
     for (int s = 0; s < n_stages; ++s) {
         const KdaStage* st = &stages[s & 1];
         const int n = min(kStageTokens, C - s * kStageTokens);
+        // operands of the stage's first token; after that, each token's are requested one token ahead
+        float4 A[4], K[4], Q[4];
+#pragma unroll
+        for (int m = 0; m < 4; ++m) {
+            A[m] = reinterpret_cast<const float4*>(st->al[0])[m * 8 + r];
+            K[m] = reinterpret_cast<const float4*>(st->kk[0])[m * 8 + r];
+            Q[m] = reinterpret_cast<const float4*>(st->qq[0])[m * 8 + r];
+        }
         for (int t = 0; t < n; ++t) {
-            const float4* ka4 = reinterpret_cast<const float4*>(st->ka[t]) + r;
-            const float4* qa4 = reinterpret_cast<const float4*>(st->qa[t]) + r;
-            uint64_t dA0 = 0, dA1 = 0, dB0 = 0, dB1 = 0, eA0 = 0, eA1 = 0, eB0 = 0, eB1 = 0;
+            const int tn = min(t + 1, n - 1);                          // the last token re-reads itself (unused)
+            const float4* al4 = reinterpret_cast<const float4*>(st->al[tn]) + r;
+            const float4* kk4 = reinterpret_cast<const float4*>(st->kk[tn]) + r;
+            const float4* qq4 = reinterpret_cast<const float4*>(st->qq[tn]) + r;
+            const float v_col = st->v[t][4 * cq + my_col];
+            const float beta = st->beta[t], qk = st->qk[t];
+            uint64_t d[4] = {0ull, 0ull, 0ull, 0ull}, e[4] = {0ull, 0ull, 0ull, 0ull};
 #pragma unroll
-            for (int m = 0; m < 8; ++m) {
-                const float4 a = ka4[m * 4], b = qa4[m * 4];
-                const uint64_t a01 = pk(a.x, a.y), a23 = pk(a.z, a.w), b01 = pk(b.x, b.y), b23 = pk(b.z, b.w);
-                dA0 = fma2(a01, sA[m][0], dA0);
-                dA1 = fma2(a23, sA[m][1], dA1);
-                dB0 = fma2(a01, sB[m][0], dB0);
-                dB1 = fma2(a23, sB[m][1], dB1);
-                eA0 = fma2(b01, sA[m][0], eA0);
-                eA1 = fma2(b23, sA[m][1], eA1);
-                eB0 = fma2(b01, sB[m][0], eB0);
-                eB1 = fma2(b23, sB[m][1], eB1);
-            }
-            const float2 vv = *reinterpret_cast<const float2*>(&st->v[t][2 * cp]);
-            const float cA = vv.x - quad_sum(dA0, dA1), cB = vv.y - quad_sum(dB0, dB1);
-            const uint64_t cA2 = pk(cA, cA), cB2 = pk(cB, cB);
-            const float4* kb4 = reinterpret_cast<const float4*>(st->kb[t]) + r;
-            const float4* al4 = reinterpret_cast<const float4*>(st->al[t]) + r;
+            for (int m = 0; m < 4; ++m) {
+                const uint64_t a01 = pk(A[m].x, A[m].y), a23 = pk(A[m].z, A[m].w);
+                const uint64_t k01 = pk(K[m].x, K[m].y), k23 = pk(K[m].z, K[m].w);
+                const uint64_t q01 = pk(Q[m].x, Q[m].y), q23 = pk(Q[m].z, Q[m].w);
 #pragma unroll
-            for (int m = 0; m < 8; ++m) {
-                const float4 kb = kb4[m * 4], al = al4[m * 4];
-                const uint64_t k01 = pk(kb.x, kb.y), k23 = pk(kb.z, kb.w), l01 = pk(al.x, al.y), l23 = pk(al.z, al.w);
-                sA[m][0] = fma2(l01, sA[m][0], mul2(k01, cA2));
-                sA[m][1] = fma2(l23, sA[m][1], mul2(k23, cA2));
-                sB[m][0] = fma2(l01, sB[m][0], mul2(k01, cB2));
-                sB[m][1] = fma2(l23, sB[m][1], mul2(k23, cB2));
+                for (int c = 0; c < 4; ++c) {
+                    S[c][m][0] = mul2(a01, S[c][m][0]);                 // s' = alpha * s
+                    S[c][m][1] = mul2(a23, S[c][m][1]);
+                    d[c] = fma2(k01, S[c][m][0], d[c]);                 // k . s'
+                    d[c] = fma2(k23, S[c][m][1], d[c]);
+                    e[c] = fma2(q01, S[c][m][0], e[c]);                 // q . s'
+                    e[c] = fma2(q23, S[c][m][1], e[c]);
+                }
+                A[m] = al4[m * 8];
+                Q[m] = qq4[m * 8];
             }
-            const float qkb = st->qkb[t];
-            const float oA = fmaf(cA, qkb, quad_sum(eA0, eA1)), oB = fmaf(cB, qkb, quad_sum(eB0, eB1));
-            if (r == 0)
-                *reinterpret_cast<__nv_bfloat162*>(out + (size_t)(s * kStageTokens + t) * H * kDV) =
-                    __floats2bfloat162_rn(oA, oB);
+            // c = beta (v - k . s') for this lane's column, then all four columns' values to every lane
+            const float c_mine = beta * (v_col - reduce_scatter(d));
+            const float c_pair = __shfl_xor_sync(0xffffffffu, c_mine, 2);
+            const float lo = b1 ? c_pair : c_mine, hi = b1 ? c_mine : c_pair;        // columns 2 b0 and 2 b0 + 1
+            const float lo_x = __shfl_xor_sync(0xffffffffu, lo, 1), hi_x = __shfl_xor_sync(0xffffffffu, hi, 1);
+            const float cc[4] = {b0 ? lo_x : lo, b0 ? hi_x : hi, b0 ? lo : lo_x, b0 ? hi : hi_x};
+#pragma unroll
+            for (int m = 0; m < 4; ++m) {
+                const uint64_t k01 = pk(K[m].x, K[m].y), k23 = pk(K[m].z, K[m].w);
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    const uint64_t c2 = pk(cc[c], cc[c]);
+                    S[c][m][0] = fma2(c2, k01, S[c][m][0]);             // s = s' + c k
+                    S[c][m][1] = fma2(c2, k23, S[c][m][1]);
+                }
+                K[m] = kk4[m * 8];
+            }
+            const float o_col = fmaf(c_mine, qk, reduce_scatter(e));
+            if (!(lane & 4)) out[(size_t)(s * kStageTokens + t) * H * kDV] = __float2bfloat16_rn(o_col);
             if (interval > 0) {
                 ++pos;
                 if (pos == next_snap) {
