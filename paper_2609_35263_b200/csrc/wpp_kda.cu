@@ -9,8 +9,8 @@
 // shared vectors alpha, k, q reach the registers of every thread that needs them through shared memory, whose
 // 128 bytes per clock bound this layout: four columns per thread need 12 sixteen-byte loads per token and thread
 // (two columns needed 24 and ran at the shared-memory limit), paid for with an eight-lane reduction per column,
-// done as exchange-and-halve steps (4 shuffles for four columns, 3 more to hand the results round).  A ninth warp stages the next 32 tokens while
-// the others work: it widens q, k, v to fp32, forms q . k once per token (shared by all 128 columns) and leaves
+// done as exchange-and-halve steps (4 shuffles for four columns, 3 more to hand the results round).  A ninth warp
+// stages the next 32 tokens while the others work: it widens q, k, v to fp32, forms q . k once per token (shared by all 128 columns) and leaves
 // them with alpha and beta in shared memory, where the eight row groups read 128 consecutive bytes (no bank
 // conflicts) and the four column groups of a warp read the same words (broadcast).  A thread's operands for the
 // next token are requested while it still works on this one: the shared-memory latency is off the token chain,
@@ -26,8 +26,9 @@ namespace wpp {
 namespace {
 
 constexpr int kDK = 128, kDV = 128;
-constexpr int kStageTokens = 32;
 constexpr int kComputeWarps = 8;
+
+constexpr int kStageTokens = 32;
 constexpr int kThreads = (kComputeWarps + 1) * 32;
 
 struct KdaStage {
@@ -39,23 +40,17 @@ struct KdaStage {
     float qk[kStageTokens];         // q . k
 };
 
-__device__ __forceinline__ uint64_t pk(float lo, float hi) {
-    uint64_t r;
-    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
-    return r;
+// Pairs of fp32 values for the two-wide FMA of sm_100 (scalar FMAs were 25 % slower here).
+__device__ __forceinline__ float2 pk(float lo, float hi) { return make_float2(lo, hi); }
+__device__ __forceinline__ void upk(float2 v, float& lo, float& hi) {
+    lo = v.x;
+    hi = v.y;
 }
-__device__ __forceinline__ void upk(uint64_t v, float& lo, float& hi) {
-    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+__device__ __forceinline__ float2 fma2(float2 a, float2 b, float2 c) {
+    return __ffma2_rn(a, b, c);
 }
-__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
-    uint64_t r;
-    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
-    return r;
-}
-__device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b) {
-    uint64_t r;
-    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
-    return r;
+__device__ __forceinline__ float2 mul2(float2 a, float2 b) {
+    return __fmul2_rn(a, b);
 }
 __device__ __forceinline__ void widen4(uint2 raw, float (&f)[4]) {
     const __nv_bfloat162 a = *reinterpret_cast<const __nv_bfloat162*>(&raw.x);
@@ -66,55 +61,59 @@ __device__ __forceinline__ void widen4(uint2 raw, float (&f)[4]) {
     f[3] = __high2float(b);
 }
 
-// The staging warp: tokens [first, first + n) of the request (rows row0 + first ...), four at a time so that
-// their loads are in flight together.
-__device__ __forceinline__ void kda_fill(const KdaParams& p, KdaStage* st, int64_t row0, int first, int n, int head,
-                                         int lane) {
+// Staging by one warp: n <= 4 tokens starting at absolute row `row` go to slots slot0 .. of the stage; their loads
+// are in flight together.  The warp widens q, k, v and forms q . k (shared by all 128 columns).
+__device__ __forceinline__ void kda_fill4(const KdaParams& p, KdaStage* st, int64_t row, int slot0, int n, int head, int lane) {
     const int H = p.num_heads;
-    for (int base = 0; base < n; base += 4) {
-        uint2 rq[4], rk[4], rv[4];
-        float4 ra[4];
-        float rb[4];
+    uint2 rq[4], rk[4], rv[4];
+    float4 ra[4];
+    float rb[4];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            const int t = base + u;
-            if (t < n) {
-                const int64_t rh = (row0 + first + t) * H + head;
-                rq[u] = *reinterpret_cast<const uint2*>(p.q + rh * kDK + lane * 4);
-                rk[u] = *reinterpret_cast<const uint2*>(p.k + rh * kDK + lane * 4);
-                rv[u] = *reinterpret_cast<const uint2*>(p.v + rh * kDV + lane * 4);
-                ra[u] = *reinterpret_cast<const float4*>(p.alpha + rh * kDK + lane * 4);
-                rb[u] = p.beta[rh];
-            }
+    for (int u = 0; u < 4; ++u) {
+        if (u < n) {
+            const int64_t rh = (row + u) * H + head;
+            rq[u] = *reinterpret_cast<const uint2*>(p.q + rh * kDK + lane * 4);
+            rk[u] = *reinterpret_cast<const uint2*>(p.k + rh * kDK + lane * 4);
+            rv[u] = *reinterpret_cast<const uint2*>(p.v + rh * kDV + lane * 4);
+            ra[u] = *reinterpret_cast<const float4*>(p.alpha + rh * kDK + lane * 4);
+            rb[u] = p.beta[rh];
         }
+    }
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            const int t = base + u;
-            if (t < n) {
-                float q[4], k[4], v[4], part = 0.f;
-                widen4(rq[u], q);
-                widen4(rk[u], k);
-                widen4(rv[u], v);
+    for (int u = 0; u < 4; ++u) {
+        if (u < n) {
+            const int t = slot0 + u;
+            float q[4], k[4], v[4], part = 0.f;
+            widen4(rq[u], q);
+            widen4(rk[u], k);
+            widen4(rv[u], v);
 #pragma unroll
-                for (int e = 0; e < 4; ++e) part = fmaf(q[e], k[e], part);
+            for (int e = 0; e < 4; ++e) part = fmaf(q[e], k[e], part);
 #pragma unroll
-                for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
-                *reinterpret_cast<float4*>(&st->al[t][lane * 4]) = ra[u];
-                *reinterpret_cast<float4*>(&st->kk[t][lane * 4]) = make_float4(k[0], k[1], k[2], k[3]);
-                *reinterpret_cast<float4*>(&st->qq[t][lane * 4]) = make_float4(q[0], q[1], q[2], q[3]);
-                *reinterpret_cast<float4*>(&st->v[t][lane * 4]) = make_float4(v[0], v[1], v[2], v[3]);
-                if (lane == 0) {
-                    st->beta[t] = rb[u];
-                    st->qk[t] = part;
-                }
+            for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
+            *reinterpret_cast<float4*>(&st->al[t][lane * 4]) = ra[u];
+            *reinterpret_cast<float4*>(&st->kk[t][lane * 4]) = make_float4(k[0], k[1], k[2], k[3]);
+            *reinterpret_cast<float4*>(&st->qq[t][lane * 4]) = make_float4(q[0], q[1], q[2], q[3]);
+            *reinterpret_cast<float4*>(&st->v[t][lane * 4]) = make_float4(v[0], v[1], v[2], v[3]);
+            if (lane == 0) {
+                st->beta[t] = rb[u];
+                st->qk[t] = part;
             }
         }
     }
 }
 
+// Stage `s` of the request (tokens s * kStageTokens ...), filled by the staging warp four tokens at a time.
+__device__ __forceinline__ void kda_fill_stage(const KdaParams& p, KdaStage* st, int64_t row0, int C, int s, int head,
+                                               int lane) {
+    const int first = s * kStageTokens, n = min(kStageTokens, C - first);
+    for (int base = 0; base < n; base += 4) kda_fill4(p, st, row0 + first + base, base, min(4, n - base), head, lane);
+}
+
 __global__ void __launch_bounds__(kThreads, 1) wpp_kda_chunk_kernel(const KdaParams p) {
+    using Stage = KdaStage;
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    KdaStage* stages = reinterpret_cast<KdaStage*>(smem_raw);
+    Stage* stages = reinterpret_cast<Stage*>(smem_raw);
 
     const int head = blockIdx.x, req = blockIdx.y, H = p.num_heads;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -131,12 +130,10 @@ __global__ void __launch_bounds__(kThreads, 1) wpp_kda_chunk_kernel(const KdaPar
     }
 
     if (warp == kComputeWarps) {
-        if (n_stages > 0) kda_fill(p, &stages[0], row0, 0, min(kStageTokens, C), head, lane);
+        if (n_stages > 0) kda_fill_stage(p, &stages[0], row0, C, 0, head, lane);
         __syncthreads();
         for (int s = 0; s < n_stages; ++s) {
-            if (s + 1 < n_stages)
-                kda_fill(p, &stages[(s + 1) & 1], row0, (s + 1) * kStageTokens, min(kStageTokens, C - (s + 1) * kStageTokens),
-                         head, lane);
+            if (s + 1 < n_stages) kda_fill_stage(p, &stages[(s + 1) & 1], row0, C, s + 1, head, lane);
             __syncthreads();
         }
         return;
@@ -147,7 +144,7 @@ __global__ void __launch_bounds__(kThreads, 1) wpp_kda_chunk_kernel(const KdaPar
     const bool b0 = lane & 1, b1 = lane & 2;
     const int my_col = (b0 ? 2 : 0) + (b1 ? 1 : 0);                    // the column whose dot products end on this lane
     const size_t head_floats = (size_t)kDK * kDV;
-    uint64_t S[4][4][2];                                                // [column][m][row pair]
+    float2 S[4][4][2];                                                // [column][m][row pair]
     if (slot_in >= 0) {
         const float* src = p.state_pool + ((size_t)slot_in * H + head) * head_floats + 4 * cq;
 #pragma unroll
@@ -164,7 +161,7 @@ __global__ void __launch_bounds__(kThreads, 1) wpp_kda_chunk_kernel(const KdaPar
 #pragma unroll
         for (int c = 0; c < 4; ++c)
 #pragma unroll
-            for (int m = 0; m < 4; ++m) S[c][m][0] = S[c][m][1] = 0ull;
+            for (int m = 0; m < 4; ++m) S[c][m][0] = S[c][m][1] = make_float2(0.f, 0.f);
     }
 
     auto store_state = [&](int slot) {
@@ -186,7 +183,7 @@ __global__ void __launch_bounds__(kThreads, 1) wpp_kda_chunk_kernel(const KdaPar
 
     // Sum over the eight row groups of four per-column partial sums: after two exchange-and-halve steps and one
     // plain step, every lane holds the complete sum of column `my_col` (4 shuffles instead of 12).
-    auto reduce_scatter = [&](const uint64_t (&acc)[4]) -> float {
+    auto reduce_scatter = [&](const float2 (&acc)[4]) -> float {
         float x[4];
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
@@ -213,7 +210,7 @@ __global__ void __launch_bounds__(kThreads, 1) wpp_kda_chunk_kernel(const KdaPar
     __nv_bfloat16* out = p.out + (row0 * H + head) * kDV + 4 * cq + my_col;
     __syncthreads();                                                    // stage 0 is filled
     for (int s = 0; s < n_stages; ++s) {
-        const KdaStage* st = &stages[s & 1];
+        const Stage* st = &stages[s & 1];
         const int n = min(kStageTokens, C - s * kStageTokens);
         // operands of the stage's first token; after that, each token's are requested one token ahead
         float4 A[4], K[4], Q[4];
@@ -230,12 +227,14 @@ __global__ void __launch_bounds__(kThreads, 1) wpp_kda_chunk_kernel(const KdaPar
             const float4* qq4 = reinterpret_cast<const float4*>(st->qq[tn]) + r;
             const float v_col = st->v[t][4 * cq + my_col];
             const float beta = st->beta[t], qk = st->qk[t];
-            uint64_t d[4] = {0ull, 0ull, 0ull, 0ull}, e[4] = {0ull, 0ull, 0ull, 0ull};
+            float2 d[4], e[4];
+#pragma unroll
+            for (int c = 0; c < 4; ++c) d[c] = e[c] = make_float2(0.f, 0.f);
 #pragma unroll
             for (int m = 0; m < 4; ++m) {
-                const uint64_t a01 = pk(A[m].x, A[m].y), a23 = pk(A[m].z, A[m].w);
-                const uint64_t k01 = pk(K[m].x, K[m].y), k23 = pk(K[m].z, K[m].w);
-                const uint64_t q01 = pk(Q[m].x, Q[m].y), q23 = pk(Q[m].z, Q[m].w);
+                const float2 a01 = pk(A[m].x, A[m].y), a23 = pk(A[m].z, A[m].w);
+                const float2 k01 = pk(K[m].x, K[m].y), k23 = pk(K[m].z, K[m].w);
+                const float2 q01 = pk(Q[m].x, Q[m].y), q23 = pk(Q[m].z, Q[m].w);
 #pragma unroll
                 for (int c = 0; c < 4; ++c) {
                     S[c][m][0] = mul2(a01, S[c][m][0]);                 // s' = alpha * s
@@ -256,10 +255,10 @@ __global__ void __launch_bounds__(kThreads, 1) wpp_kda_chunk_kernel(const KdaPar
             const float cc[4] = {b0 ? lo_x : lo, b0 ? hi_x : hi, b0 ? lo : lo_x, b0 ? hi : hi_x};
 #pragma unroll
             for (int m = 0; m < 4; ++m) {
-                const uint64_t k01 = pk(K[m].x, K[m].y), k23 = pk(K[m].z, K[m].w);
+                const float2 k01 = pk(K[m].x, K[m].y), k23 = pk(K[m].z, K[m].w);
 #pragma unroll
                 for (int c = 0; c < 4; ++c) {
-                    const uint64_t c2 = pk(cc[c], cc[c]);
+                    const float2 c2 = pk(cc[c], cc[c]);
                     S[c][m][0] = fma2(c2, k01, S[c][m][0]);             // s = s' + c k
                     S[c][m][1] = fma2(c2, k23, S[c][m][1]);
                 }
