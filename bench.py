@@ -427,7 +427,7 @@ def run_kda(args):
     status = torch.zeros(1, dtype=torch.int32, device=dev)
     out = torch.empty((w.total_tokens, w.num_heads, w.d_v), dtype=torch.bfloat16, device=dev)
     step = lambda: wpp.wpp_kda_chunk(ctx, d["q"], d["k"], d["v"], d["alpha"], d["beta"], ro, d["state_pool"], s_in, s_out,
-                                     out=out, status=status)
+                                     out=out, status=status, layout=args.kda_layout)
     warm, steps = max(3, args.warmup), max(1, args.steps)
     for _ in range(warm):
         step()
@@ -465,7 +465,8 @@ def run_kda(args):
             "unit": "tokens/s", "n_gpus": 1, "steps": steps, "warmup": warm, "ms_per_step": ms, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic", "gpu_launches": steps,
             "config": {"workload": w.name, "requests": int(w.chunk_lens.size), "chunk": int(w.chunk_lens[0]),
-                       "state_heads": Hh, "d_k": w.d_k, "d_v": w.d_v, "l2": "inputs larger than L2"},
+                       "state_heads": Hh, "d_k": w.d_k, "d_v": w.d_v, "layout": args.kda_layout,
+                       "l2": "inputs larger than L2"},
             "clocks": clocks,
             "roofline": {"bound": "alu", "kernel": "wpp_kda_chunk_kernel", "achieved": flops / (ms * 1e-3) / 1e12,
                          "peak": peak, "unit": "TFLOP/s", "frac": flops / (ms * 1e-3) / 1e12 / peak,
@@ -497,6 +498,7 @@ def main():
     ap.add_argument("--kda", action="store_true", help="the recurrent-state (KDA) layer of one wave")
     ap.add_argument("--kda-lanes", type=int, default=8)
     ap.add_argument("--kda-chunk", type=int, default=2048)
+    ap.add_argument("--kda-layout", type=int, default=0, help="0: library chooses, 1: one CTA per (request, head), 2: four")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "native" else args.warmup
 

@@ -343,7 +343,8 @@ typedef struct {
     int32_t num_slots;      /* slots of state_pool, each H * d_k * d_v floats */
     int32_t snap_interval;  /* > 0: snapshot whenever the tokens folded into S reach a multiple of it; 0: none */
     int32_t max_snaps;      /* row length of snap_slots (0 when snap_interval is 0) */
-    int32_t reserved;       /* 0 */
+    int32_t layout;         /* 0: the library chooses; 1: one CTA per (request, head); 2: four CTAs per (request,
+                             * head), 32 columns each - a shorter token chain, chosen when 4 R H <= the SM count */
     int64_t total_tokens;   /* T = row_offsets[R] */
 } wpp_kda_desc;
 

@@ -78,7 +78,7 @@ class WaveInfo(ctypes.Structure):
 class KdaDesc(ctypes.Structure):
     _fields_ = [("num_requests", ctypes.c_int32), ("num_heads", ctypes.c_int32), ("d_k", ctypes.c_int32),
                 ("d_v", ctypes.c_int32), ("num_slots", ctypes.c_int32), ("snap_interval", ctypes.c_int32),
-                ("max_snaps", ctypes.c_int32), ("reserved", ctypes.c_int32), ("total_tokens", ctypes.c_int64)]
+                ("max_snaps", ctypes.c_int32), ("layout", ctypes.c_int32), ("total_tokens", ctypes.c_int64)]
 
 
 WAVE_RING_BUSY, WAVE_ADMISSION_PENDING, WAVE_ALREADY_DEFERRED = 1, 2, 4
@@ -419,20 +419,21 @@ class HintIndex:
 
 
 def wpp_kda_chunk(ctx: Context, q, k, v, alpha, beta, row_offsets, state_pool, state_in, state_out, out=None,
-                  prefix_lens=None, snap_interval: int = 0, snap_slots=None, status=None, stream=None):
+                  prefix_lens=None, snap_interval: int = 0, snap_slots=None, status=None, stream=None, layout: int = 0):
     """Queue the recurrent-state (KDA) layer of one wave on `stream` (Section 3.1 update, Section 3.2 snapshots).
 
     q, k: cuda bf16 [T, H, 128]; v: cuda bf16 [T, H, 128]; alpha: cuda fp32 [T, H, 128]; beta: cuda fp32 [T, H];
     row_offsets: cuda int64 [R+1]; state_pool: cuda fp32 [slots, H, 128, 128] (updated in place); state_in,
     state_out: cuda int32 [R] (-1: zero state / do not store); snap_slots: cuda int32 [R, max_snaps] with
-    prefix_lens (cuda int32 [R]) and snap_interval > 0 for periodic snapshots.  Returns the cuda bf16 output."""
+    prefix_lens (cuda int32 [R]) and snap_interval > 0 for periodic snapshots; layout 0 lets the library choose
+    between one and four CTAs per (request, head).  Returns the cuda bf16 output."""
     T, H, dk = (int(x) for x in q.shape)
     dv = int(v.shape[2])
     R = int(row_offsets.numel()) - 1
     if out is None:
         out = torch.empty((T, H, dv), dtype=torch.bfloat16, device=q.device)
     max_snaps = 0 if snap_slots is None else int(snap_slots.shape[1])
-    desc = KdaDesc(R, H, dk, dv, int(state_pool.shape[0]), int(snap_interval), max_snaps, 0, T)
+    desc = KdaDesc(R, H, dk, dv, int(state_pool.shape[0]), int(snap_interval), max_snaps, int(layout), T)
     st = load_library().wpp_kda_chunk(ctx.handle, ctypes.byref(desc), _ptr(q), _ptr(k), _ptr(v), _ptr(alpha), _ptr(beta),
                                       _ptr(row_offsets), _ptr(prefix_lens), _ptr(state_pool), _ptr(state_in),
                                       _ptr(state_out), _ptr(snap_slots), _ptr(out), _ptr(status), _stream(stream))

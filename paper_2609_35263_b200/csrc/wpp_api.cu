@@ -280,7 +280,7 @@ extern "C" int wpp_kda_chunk(const wpp_ctx* ctx, const wpp_kda_desc* desc, const
                              void* cuda_stream) {
     if (!ctx || !desc) return WPP_ERR_INVALID_ARG;
     if (desc->num_requests < 0 || desc->num_heads < 1 || desc->num_slots < 0 || desc->snap_interval < 0 ||
-        desc->max_snaps < 0 || desc->total_tokens < 0 || desc->reserved != 0)
+        desc->max_snaps < 0 || desc->total_tokens < 0 || desc->layout < 0 || desc->layout > 2)
         return WPP_ERR_INVALID_ARG;
     if (desc->d_k != 128 || desc->d_v != 128) return WPP_ERR_UNSUPPORTED;
     if (desc->num_requests > 65535) return WPP_ERR_UNSUPPORTED;      // one grid row per request
@@ -311,7 +311,7 @@ extern "C" int wpp_kda_chunk(const wpp_ctx* ctx, const wpp_kda_desc* desc, const
     p.num_slots = desc->num_slots;
     p.snap_interval = desc->snap_interval;
     p.max_snaps = desc->max_snaps;
-    int e = wpp_launch_kda(&p, cuda_stream);
+    int e = wpp_launch_kda(&p, ctx->sm_count, desc->layout, cuda_stream);
     if (e != 0) return cuda_fail(ctx, e);
     const_cast<wpp_ctx*>(ctx)->launches += 1;
     return WPP_OK;

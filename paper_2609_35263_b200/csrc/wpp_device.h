@@ -74,6 +74,6 @@ int wpp_launch_attention(int head_dim, const CUtensorMap* tq, const CUtensorMap*
                          const wpp::AttnParams* p, int num_ctas, void* stream);
 int wpp_launch_append(const wpp::AppendParams* p, int num_sms, void* stream);
 int wpp_launch_combine(const wpp::CombineParams* p, int num_combine, void* stream);
-int wpp_launch_kda(const wpp::KdaParams* p, void* stream);
+int wpp_launch_kda(const wpp::KdaParams* p, int num_sms, int layout, void* stream);
 int wpp_launch_selftest_wait(long long limit_cycles, int32_t* status, long long* waited_cycles, void* stream);
 }

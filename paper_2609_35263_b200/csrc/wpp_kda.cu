@@ -110,12 +110,20 @@ __device__ __forceinline__ void kda_fill_stage(const KdaParams& p, KdaStage* st,
     for (int base = 0; base < n; base += 4) kda_fill4(p, st, row0 + first + base, base, min(4, n - base), head, lane);
 }
 
+// kSplit = lanes that share a column's rows.  8: a CTA owns all 128 columns of a (request, head), a thread holds
+// 4 columns x 16 rows - the throughput build.  32: a CTA owns 32 columns (four CTAs per head), a thread holds
+// 4 columns x 4 rows, so a token costs a quarter of the FMAs per thread and two more shuffle steps - the build for
+// waves with too few (request, head) pairs to fill the SMs, where the length of the token chain is all that counts.
+template <int kSplit>
 __global__ void __launch_bounds__(kThreads, 1) wpp_kda_chunk_kernel(const KdaParams p) {
+    constexpr int kM = 32 / kSplit;                      // 16-byte row groups per thread
+    constexpr int kQuadsPerWarp = 32 / kSplit;           // column quads per warp
+    constexpr int kSlices = kDV / (kComputeWarps * kQuadsPerWarp * 4);
     using Stage = KdaStage;
     extern __shared__ __align__(16) unsigned char smem_raw[];
     Stage* stages = reinterpret_cast<Stage*>(smem_raw);
 
-    const int head = blockIdx.x, req = blockIdx.y, H = p.num_heads;
+    const int head = blockIdx.x / kSlices, slice = blockIdx.x % kSlices, req = blockIdx.y, H = p.num_heads;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int64_t row0 = p.row_offsets[req];
     const int C = (int)(p.row_offsets[req + 1] - row0);
@@ -139,19 +147,19 @@ __global__ void __launch_bounds__(kThreads, 1) wpp_kda_chunk_kernel(const KdaPar
         return;
     }
 
-    // ---- compute threads: rows 32m + 4r + e (m < 4, e < 4; r = lane & 7) of columns 4cq .. 4cq + 3
-    const int r = lane & 7, cq = warp * 4 + (lane >> 3);
+    // ---- compute threads: rows 4 kSplit m + 4r + e (m < kM, e < 4; r = lane mod kSplit) of columns 4cq .. 4cq + 3
+    const int r = lane & (kSplit - 1), cq = (slice * kComputeWarps + warp) * kQuadsPerWarp + lane / kSplit;
     const bool b0 = lane & 1, b1 = lane & 2;
     const int my_col = (b0 ? 2 : 0) + (b1 ? 1 : 0);                    // the column whose dot products end on this lane
     const size_t head_floats = (size_t)kDK * kDV;
-    float2 S[4][4][2];                                                // [column][m][row pair]
+    float2 S[4][kM][2];                                                // [column][m][row pair]
     if (slot_in >= 0) {
         const float* src = p.state_pool + ((size_t)slot_in * H + head) * head_floats + 4 * cq;
 #pragma unroll
-        for (int m = 0; m < 4; ++m) {
+        for (int m = 0; m < kM; ++m) {
             float4 x[4];
 #pragma unroll
-            for (int e = 0; e < 4; ++e) x[e] = *reinterpret_cast<const float4*>(src + (size_t)(32 * m + 4 * r + e) * kDV);
+            for (int e = 0; e < 4; ++e) x[e] = *reinterpret_cast<const float4*>(src + (size_t)(4 * kSplit * m + 4 * r + e) * kDV);
             S[0][m][0] = pk(x[0].x, x[1].x), S[0][m][1] = pk(x[2].x, x[3].x);
             S[1][m][0] = pk(x[0].y, x[1].y), S[1][m][1] = pk(x[2].y, x[3].y);
             S[2][m][0] = pk(x[0].z, x[1].z), S[2][m][1] = pk(x[2].z, x[3].z);
@@ -161,13 +169,13 @@ __global__ void __launch_bounds__(kThreads, 1) wpp_kda_chunk_kernel(const KdaPar
 #pragma unroll
         for (int c = 0; c < 4; ++c)
 #pragma unroll
-            for (int m = 0; m < 4; ++m) S[c][m][0] = S[c][m][1] = make_float2(0.f, 0.f);
+            for (int m = 0; m < kM; ++m) S[c][m][0] = S[c][m][1] = make_float2(0.f, 0.f);
     }
 
     auto store_state = [&](int slot) {
         float* dst = p.state_pool + ((size_t)slot * H + head) * head_floats + 4 * cq;
 #pragma unroll
-        for (int m = 0; m < 4; ++m) {
+        for (int m = 0; m < kM; ++m) {
             float x[4][4];
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
@@ -176,7 +184,7 @@ __global__ void __launch_bounds__(kThreads, 1) wpp_kda_chunk_kernel(const KdaPar
             }
 #pragma unroll
             for (int e = 0; e < 4; ++e)
-                *reinterpret_cast<float4*>(dst + (size_t)(32 * m + 4 * r + e) * kDV) =
+                *reinterpret_cast<float4*>(dst + (size_t)(4 * kSplit * m + 4 * r + e) * kDV) =
                     make_float4(x[0][e], x[1][e], x[2][e], x[3][e]);
         }
     };
@@ -195,6 +203,10 @@ __global__ void __launch_bounds__(kThreads, 1) wpp_kda_chunk_kernel(const KdaPar
         const float y1 = (b0 ? x[3] : x[1]) + __shfl_xor_sync(0xffffffffu, b0 ? x[1] : x[3], 1);
         float z = (b1 ? y1 : y0) + __shfl_xor_sync(0xffffffffu, b1 ? y0 : y1, 2);
         z += __shfl_xor_sync(0xffffffffu, z, 4);
+        if (kSplit == 32) {
+            z += __shfl_xor_sync(0xffffffffu, z, 8);
+            z += __shfl_xor_sync(0xffffffffu, z, 16);
+        }
         return z;
     };
 
@@ -213,12 +225,12 @@ __global__ void __launch_bounds__(kThreads, 1) wpp_kda_chunk_kernel(const KdaPar
         const Stage* st = &stages[s & 1];
         const int n = min(kStageTokens, C - s * kStageTokens);
         // operands of the stage's first token; after that, each token's are requested one token ahead
-        float4 A[4], K[4], Q[4];
+        float4 A[kM], K[kM], Q[kM];
 #pragma unroll
-        for (int m = 0; m < 4; ++m) {
-            A[m] = reinterpret_cast<const float4*>(st->al[0])[m * 8 + r];
-            K[m] = reinterpret_cast<const float4*>(st->kk[0])[m * 8 + r];
-            Q[m] = reinterpret_cast<const float4*>(st->qq[0])[m * 8 + r];
+        for (int m = 0; m < kM; ++m) {
+            A[m] = reinterpret_cast<const float4*>(st->al[0])[m * kSplit + r];
+            K[m] = reinterpret_cast<const float4*>(st->kk[0])[m * kSplit + r];
+            Q[m] = reinterpret_cast<const float4*>(st->qq[0])[m * kSplit + r];
         }
         for (int t = 0; t < n; ++t) {
             const int tn = min(t + 1, n - 1);                          // the last token re-reads itself (unused)
@@ -231,7 +243,7 @@ __global__ void __launch_bounds__(kThreads, 1) wpp_kda_chunk_kernel(const KdaPar
 #pragma unroll
             for (int c = 0; c < 4; ++c) d[c] = e[c] = make_float2(0.f, 0.f);
 #pragma unroll
-            for (int m = 0; m < 4; ++m) {
+            for (int m = 0; m < kM; ++m) {
                 const float2 a01 = pk(A[m].x, A[m].y), a23 = pk(A[m].z, A[m].w);
                 const float2 k01 = pk(K[m].x, K[m].y), k23 = pk(K[m].z, K[m].w);
                 const float2 q01 = pk(Q[m].x, Q[m].y), q23 = pk(Q[m].z, Q[m].w);
@@ -244,8 +256,8 @@ __global__ void __launch_bounds__(kThreads, 1) wpp_kda_chunk_kernel(const KdaPar
                     e[c] = fma2(q01, S[c][m][0], e[c]);                 // q . s'
                     e[c] = fma2(q23, S[c][m][1], e[c]);
                 }
-                A[m] = al4[m * 8];
-                Q[m] = qq4[m * 8];
+                A[m] = al4[m * kSplit];
+                Q[m] = qq4[m * kSplit];
             }
             // c = beta (v - k . s') for this lane's column, then all four columns' values to every lane
             const float c_mine = beta * (v_col - reduce_scatter(d));
@@ -254,7 +266,7 @@ __global__ void __launch_bounds__(kThreads, 1) wpp_kda_chunk_kernel(const KdaPar
             const float lo_x = __shfl_xor_sync(0xffffffffu, lo, 1), hi_x = __shfl_xor_sync(0xffffffffu, hi, 1);
             const float cc[4] = {b0 ? lo_x : lo, b0 ? hi_x : hi, b0 ? lo : lo_x, b0 ? hi : hi_x};
 #pragma unroll
-            for (int m = 0; m < 4; ++m) {
+            for (int m = 0; m < kM; ++m) {
                 const float2 k01 = pk(K[m].x, K[m].y), k23 = pk(K[m].z, K[m].w);
 #pragma unroll
                 for (int c = 0; c < 4; ++c) {
@@ -262,10 +274,10 @@ __global__ void __launch_bounds__(kThreads, 1) wpp_kda_chunk_kernel(const KdaPar
                     S[c][m][0] = fma2(c2, k01, S[c][m][0]);             // s = s' + c k
                     S[c][m][1] = fma2(c2, k23, S[c][m][1]);
                 }
-                K[m] = kk4[m * 8];
+                K[m] = kk4[m * kSplit];
             }
             const float o_col = fmaf(c_mine, qk, reduce_scatter(e));
-            if (!(lane & 4)) out[(size_t)(s * kStageTokens + t) * H * kDV] = __float2bfloat16_rn(o_col);
+            if (!(lane & (kSplit - 1) & ~3)) out[(size_t)(s * kStageTokens + t) * H * kDV] = __float2bfloat16_rn(o_col);
             if (interval > 0) {
                 ++pos;
                 if (pos == next_snap) {
@@ -290,17 +302,28 @@ __global__ void __launch_bounds__(kThreads, 1) wpp_kda_chunk_kernel(const KdaPar
 }  // namespace
 }  // namespace wpp
 
-extern "C" int wpp_launch_kda(const wpp::KdaParams* p, void* stream) {
+template <int kSplit>
+static int launch_kda(const wpp::KdaParams* p, void* stream) {
     static bool attr_set[64] = {};
     const int smem = 2 * (int)sizeof(wpp::KdaStage);
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev >= 0 && dev < 64 && !attr_set[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(wpp::wpp_kda_chunk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        cudaError_t e = cudaFuncSetAttribute(wpp::wpp_kda_chunk_kernel<kSplit>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             smem);
         if (e != cudaSuccess) return (int)e;
         attr_set[dev] = true;
     }
-    dim3 grid((unsigned)p->num_heads, (unsigned)p->num_requests);
-    wpp::wpp_kda_chunk_kernel<<<grid, wpp::kThreads, smem, (cudaStream_t)stream>>>(*p);
+    dim3 grid((unsigned)p->num_heads * (kSplit == 32 ? 4 : 1), (unsigned)p->num_requests);
+    wpp::wpp_kda_chunk_kernel<kSplit><<<grid, wpp::kThreads, smem, (cudaStream_t)stream>>>(*p);
     return (int)cudaGetLastError();
+}
+
+// layout: 0 = choose (the column-sliced build when its four CTAs per (request, head) pair still fit the SMs in one
+// round: measured, 1 x 16,384 tokens x 32 heads 5.3 ms against 7.3 ms, but 2 x 8,192 5.3 ms against 3.7 ms),
+// 1 = one CTA per (request, head), 2 = four CTAs per (request, head).
+extern "C" int wpp_launch_kda(const wpp::KdaParams* p, int num_sms, int layout, void* stream) {
+    const long long pairs = (long long)p->num_heads * p->num_requests;
+    const bool sliced = layout == 2 || (layout == 0 && 4 * pairs <= num_sms);
+    return sliced ? launch_kda<32>(p, stream) : launch_kda<8>(p, stream);
 }

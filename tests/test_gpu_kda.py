@@ -25,7 +25,7 @@ def _oracle(w, t, heads=None):
     return o, pool
 
 
-def _gpu(w, t, state_in=None, state_out=None):
+def _gpu(w, t, state_in=None, state_out=None, layout=0):
     dev = torch.device("cuda")
     d = {k: v.to(dev) for k, v in t.items()}
     i32 = lambda a: None if a is None else torch.from_numpy(np.ascontiguousarray(a, dtype=np.int32)).to(dev)
@@ -35,7 +35,7 @@ def _gpu(w, t, state_in=None, state_out=None):
                             i32(w.state_in if state_in is None else state_in),
                             i32(w.state_out if state_out is None else state_out),
                             prefix_lens=i32(w.prefix_lens), snap_interval=w.snap_interval,
-                            snap_slots=i32(w.snap_slots), status=status)
+                            snap_slots=i32(w.snap_slots), status=status, layout=layout)
     torch.cuda.synchronize()
     return out.float().cpu().double().numpy(), d["state_pool"].cpu().double().numpy(), int(status.item())
 
@@ -57,11 +57,12 @@ def _close_state(got, ref, what):
     ([300], [0], 0, 3),                                                            # one request from the zero state
     ([15, 16, 17, 31, 32, 33], [1, 2, 3, 4, 5, 6], 7, 1),                          # around the staging size; odd interval
 ])
-def test_ragged_batches_match_the_oracle(lens, prefix, interval, H_):
+@pytest.mark.parametrize("layout", [1, 2])          # one CTA per (request, head) / four column slices
+def test_ragged_batches_match_the_oracle(lens, prefix, interval, H_, layout):
     w = W.kda_workload("ragged", 11, lens, H_, prefix, snap_interval=interval)
     t = w.tensors()
     ref_o, ref_pool = _oracle(w, t)
-    got_o, got_pool, status = _gpu(w, t)
+    got_o, got_pool, status = _gpu(w, t, layout=layout)
     assert status == 0
     _close_out(got_o, ref_o, "outputs")
     _close_state(got_pool, ref_pool, "state pool")
@@ -74,22 +75,24 @@ def test_ragged_batches_match_the_oracle(lens, prefix, interval, H_):
             assert np.array_equal(got_pool[s], t["state_pool"][s].double().numpy())
 
 
-def test_a_long_chain_stays_within_tolerance():
+@pytest.mark.parametrize("layout", [1, 2])
+def test_a_long_chain_stays_within_tolerance(layout):
     w = W.kda_workload("long", 5, [2048], 1, [4096])
     t = w.tensors()
     ref_o, ref_pool = _oracle(w, t)
-    got_o, got_pool, status = _gpu(w, t)
+    got_o, got_pool, status = _gpu(w, t, layout=layout)
     assert status == 0
     _close_out(got_o, ref_o, "outputs")
     _close_state(got_pool, ref_pool, "state pool")
 
 
-def test_splitting_a_chunk_and_resuming_is_bit_identical():
+@pytest.mark.parametrize("layout", [1, 2])
+def test_splitting_a_chunk_and_resuming_is_bit_identical(layout):
     """Section 3.2: the state after exactly r tokens is all a recurrent layer needs; the kernel's arithmetic per
     token does not depend on where a chunk starts, so one call and two resumed calls agree to the bit."""
     w = W.kda_workload("whole", 3, [100, 64], 2, [5, 0], resume=[True, False])
     t = w.tensors()
-    whole_o, whole_pool, _ = _gpu(w, t)
+    whole_o, whole_pool, _ = _gpu(w, t, layout=layout)
     rows = w.row_offsets
     parts_o = np.zeros_like(whole_o)
     pool = t["state_pool"].clone()
@@ -101,7 +104,7 @@ def test_splitting_a_chunk_and_resuming_is_bit_identical():
         wp.num_slots = w.num_slots
         tp = {k: (v[sel].contiguous() if k != "state_pool" else pool) for k, v in t.items()}
         s_in = w.state_in if first else w.state_out          # the second call resumes from what the first stored
-        o, new_pool, status = _gpu(wp, tp, state_in=s_in, state_out=w.state_out)
+        o, new_pool, status = _gpu(wp, tp, state_in=s_in, state_out=w.state_out, layout=layout)
         assert status == 0
         parts_o[sel] = o
         pool = torch.from_numpy(new_pool).float()
@@ -109,13 +112,14 @@ def test_splitting_a_chunk_and_resuming_is_bit_identical():
     assert np.array_equal(pool.double().numpy(), whole_pool)
 
 
-def test_in_place_slots_and_pure_decay():
+@pytest.mark.parametrize("layout", [1, 2])
+def test_in_place_slots_and_pure_decay(layout):
     # state_out == state_in updates a slot in place; with beta = 0 and alpha = 1 the state must not change at all
     w = W.kda_workload("inplace", 9, [50, 20], 2, [10, 10])
     t = w.tensors()
     t["beta"].zero_()
     t["alpha"].fill_(1.0)
-    got_o, got_pool, status = _gpu(w, t, state_out=w.state_in)
+    got_o, got_pool, status = _gpu(w, t, state_out=w.state_in, layout=layout)
     assert status == 0
     assert np.array_equal(got_pool, t["state_pool"].double().numpy())
     ref = np.einsum("rhkv,rhk->rhv", t["state_pool"][[0] * 50 + [1] * 20].double().numpy(), t["q"].double().numpy())
@@ -146,6 +150,10 @@ def test_argument_errors():
                           z(4, 1, dt=torch.float32), ro, pool, slot, slot)
     assert e.value.status == 2
     pool = z(1, 1, 128, 128, dt=torch.float32)
+    with pytest.raises(wpp.WppError) as e:                            # no such layout
+        wpp.wpp_kda_chunk(H.ctx(), z(4, 1, 128), z(4, 1, 128), z(4, 1, 128), z(4, 1, 128, dt=torch.float32),
+                          z(4, 1, dt=torch.float32), ro, pool, slot, slot, layout=3)
+    assert e.value.status == 1
     with pytest.raises(wpp.WppError) as e:                            # periodic snapshots need prefix_lens
         wpp.wpp_kda_chunk(H.ctx(), z(4, 1, 128), z(4, 1, 128), z(4, 1, 128), z(4, 1, 128, dt=torch.float32),
                           z(4, 1, dt=torch.float32), ro, pool, slot, slot, snap_interval=2,
@@ -153,15 +161,17 @@ def test_argument_errors():
     assert e.value.status == 1
 
 
-def test_full_size_wave_on_sampled_heads():
-    """The benchmark's wave (8 lanes x 2,048 tokens, 32 heads, resumed states): the oracle recomputes three
-    (request, head) chains and all of their outputs and final states are compared."""
-    w = W.kda_wave()
+@pytest.mark.parametrize("lanes,chunk", [(8, 2048), (1, 16384)])
+def test_full_size_wave_on_sampled_heads(lanes, chunk):
+    """The benchmark's waves (8 lanes x 2,048 tokens: one CTA per pair; one lane x 16,384 tokens: the library picks
+    four column slices per pair), 32 heads, resumed states: the oracle recomputes sampled (request, head) chains and
+    all of their outputs and final states are compared."""
+    w = W.kda_wave(lanes, chunk)
     t = w.tensors()
     got_o, got_pool, status = _gpu(w, t)
     assert status == 0
     rows = w.row_offsets
-    for req, head in ((0, 0), (3, 17), (7, 31)):
+    for req, head in (((0, 0), (3, 17), (7, 31)) if lanes == 8 else ((0, 5),)):
         sl = slice(rows[req], rows[req + 1])
         sub = W.kda_workload("one", 0, [int(w.chunk_lens[req])], 1, [int(w.prefix_lens[req])])
         sub.num_slots, sub.state_in, sub.state_out = w.num_slots, w.state_in[req:req + 1], w.state_out[req:req + 1]
