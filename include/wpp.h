@@ -327,6 +327,14 @@ int64_t wpp_hint_index_size(const wpp_hint_index* idx);     /* number of keys; -
 int wpp_hint_probe(const wpp_hint_index* idx, int32_t window, const uint64_t* hashes_host, int64_t n_blocks,
                    int64_t* matched_blocks, int32_t* probes_or_null);
 
+/* Endpoint of a recurrent-state cache (Section 4.3): snapshots exist only at sparse boundaries, so presence is not
+ * monotone in depth and the probe walks backward from the attention-limited endpoint `limit_blocks` until it meets a
+ * depth whose key is in the index under `window` (the recurrent cache's window id); *matched_blocks is that depth,
+ * 0 if there is none.  The reuse candidate of a request is the minimum of its caches' endpoints (and, across
+ * ranks, the all-rank minimum); lowering it may call for another backward scan from the lower endpoint. */
+int wpp_hint_probe_recurrent(const wpp_hint_index* idx, int32_t window, const uint64_t* hashes_host,
+                             int64_t limit_blocks, int64_t* matched_blocks, int32_t* probes_or_null);
+
 /* ---------------------------------------------------------------------------------------------------------
  * Recurrent-state layer of a chunk (Section 3.1, the simplified KDA update; Section 3.2, snapshots): the other
  * cache type of a hybrid model's stage.  Per request and head, token by token over the chunk,

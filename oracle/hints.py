@@ -1,5 +1,5 @@
 """Oracle for the chained block hash and the hint index probe of Section 4.3 (Eq. design-hash and the paragraph on
-galloping and bisecting).
+galloping and bisecting, and the paragraph on the backward scan for recurrent snapshots).
 
 TEST INFRASTRUCTURE ONLY: plain Python integers and a dict; shares no code with the library's implementation
 (`wpp_hash_blocks`, `wpp_hint_*`); only tests import it.
@@ -79,6 +79,24 @@ def longest_prefix_linear(index, window, hashes):
             break
         n += 1
     return n
+
+
+def probe_reverse_scan(index, window, hashes, limit):
+    """Recurrent snapshots are sparse: walk backward from the attention-limited endpoint `limit` to the first depth
+    whose key is present.  Returns (depth, list of probed depths); depth 0 when nothing at or below `limit` is."""
+    probed = []
+    d = min(limit, len(hashes))
+    while d >= 1:
+        probed.append(d)
+        if index.has(window, hashes[d - 1]):
+            break
+        d -= 1
+    return d, probed
+
+
+def reuse_candidate(endpoints):
+    """The minimum of the local caches' endpoints (Section 4.3); the all-rank minimum is taken over these."""
+    return min(endpoints)
 
 
 def probe_gallop_bisect(index, window, hashes):

@@ -88,7 +88,8 @@ EXPORTS = ["wpp_create", "wpp_destroy", "wpp_status_string", "wpp_last_cuda_erro
            "wpp_launch_count", "wpp_prefill_attention_varlen_static", "wpp_static_scratch_bytes",
            "wpp_selftest_bounded_wait", "wpp_wave_ladder", "wpp_plan_waves",
            "wpp_hash_blocks", "wpp_hash_blocks_host", "wpp_hint_index_create", "wpp_hint_index_destroy",
-           "wpp_hint_index_add", "wpp_hint_index_remove", "wpp_hint_index_size", "wpp_hint_probe", "wpp_kda_chunk"]
+           "wpp_hint_index_add", "wpp_hint_index_remove", "wpp_hint_index_size", "wpp_hint_probe",
+           "wpp_hint_probe_recurrent", "wpp_kda_chunk"]
 
 _lib = None
 
@@ -134,6 +135,8 @@ def load_library() -> ctypes.CDLL:
         lib.wpp_hint_index_size.restype = ctypes.c_int64
         lib.wpp_hint_probe.argtypes = [vp, ctypes.c_int32, vp, ctypes.c_int64, ctypes.POINTER(ctypes.c_int64),
                                        ctypes.POINTER(ctypes.c_int32)]
+        lib.wpp_hint_probe_recurrent.argtypes = [vp, ctypes.c_int32, vp, ctypes.c_int64, ctypes.POINTER(ctypes.c_int64),
+                                                 ctypes.POINTER(ctypes.c_int32)]
         lib.wpp_wave_ladder.argtypes = [ctypes.POINTER(WaveConfig), vp, ctypes.c_int32, ctypes.POINTER(ctypes.c_int32)]
         lib.wpp_plan_waves.argtypes = [ctypes.POINTER(WaveConfig), ctypes.POINTER(WaveState), vp, ctypes.c_int32, vp,
                                        ctypes.c_int32, ctypes.c_int32, vp, ctypes.POINTER(WaveInfo)]
@@ -415,6 +418,17 @@ class HintIndex:
         _check(load_library().wpp_hint_probe(self.handle, int(window),
                                              h.ctypes.data_as(ctypes.c_void_p) if h.size else None, int(h.size),
                                              ctypes.byref(m), ctypes.byref(p)), "wpp_hint_probe")
+        return int(m.value), int(p.value)
+
+    def probe_recurrent(self, window: int, hashes, limit_blocks: int):
+        """(endpoint in blocks, number of probes) of a recurrent-state cache: the deepest snapshot boundary at or
+        below `limit_blocks` whose key is in the index, found by scanning backward (Section 4.3)."""
+        h = self._u64(hashes)
+        limit = min(int(limit_blocks), int(h.size))
+        m, p = ctypes.c_int64(0), ctypes.c_int32(0)
+        _check(load_library().wpp_hint_probe_recurrent(self.handle, int(window),
+                                                       h.ctypes.data_as(ctypes.c_void_p) if h.size else None, limit,
+                                                       ctypes.byref(m), ctypes.byref(p)), "wpp_hint_probe_recurrent")
         return int(m.value), int(p.value)
 
 

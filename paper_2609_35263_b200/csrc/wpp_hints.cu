@@ -208,3 +208,17 @@ extern "C" int wpp_hint_probe(const wpp_hint_index* idx, int32_t window, const u
     if (probes_or_null) *probes_or_null = probes;
     return WPP_OK;
 }
+
+extern "C" int wpp_hint_probe_recurrent(const wpp_hint_index* idx, int32_t window, const uint64_t* hashes,
+                                        int64_t limit_blocks, int64_t* matched_blocks, int32_t* probes_or_null) {
+    if (!idx || limit_blocks < 0 || !matched_blocks || (limit_blocks > 0 && !hashes)) return WPP_ERR_INVALID_ARG;
+    int32_t probes = 0;
+    int64_t d = limit_blocks;                   // snapshots are sparse: walk back from the attention-limited endpoint
+    for (; d >= 1; --d) {
+        ++probes;
+        if (idx->has(window, hashes[d - 1])) break;
+    }
+    *matched_blocks = d;
+    if (probes_or_null) *probes_or_null = probes;
+    return WPP_OK;
+}

@@ -83,3 +83,27 @@ def test_probe_equals_the_linear_definition_with_logarithmically_many_probes():
     assert O.probe_gallop_bisect(idx, 0, [5, 6, 7]) == (0, [1])
     idx.add(0, [5, 6, 7, 8, 9])
     assert O.probe_gallop_bisect(idx, 0, [5, 6, 7, 8, 9]) == (5, [1, 2, 4, 5])
+
+
+def test_reverse_scan_finds_the_deepest_snapshot_at_or_below_the_attention_endpoint():
+    # the definition: max depth d <= limit with the key present (brute force over all depths), 0 if none
+    rng = np.random.default_rng(2)
+    for _ in range(300):
+        N = int(rng.integers(0, 120))
+        hashes = [int(x) for x in rng.integers(1, 1 << 62, N)]
+        snaps = sorted(set(int(d) for d in rng.integers(1, N + 1, rng.integers(0, 6)))) if N else []
+        idx = O.HintIndex()
+        idx.add(3, [hashes[d - 1] for d in snaps])
+        idx.add(0, hashes)                                      # the attention window holds every block; must not matter
+        limit = int(rng.integers(0, N + 1))
+        want = max([d for d in snaps if d <= limit], default=0)
+        depth, probed = O.probe_reverse_scan(idx, 3, hashes, limit)
+        assert depth == want
+        assert probed == list(range(limit, max(want, 1) - 1, -1))          # limit, limit-1, ..., down to the hit (or 1)
+    # Section 4.4's example in blocks: snapshots at 64K, 72K, 90K tokens; an attention endpoint of 80K falls back to 72K
+    B, toks = 1024, list(range(96 * 1024))
+    h = O.chained_hashes(toks, B)
+    idx = O.HintIndex()
+    idx.add(1, [h[64 - 1], h[72 - 1], h[90 - 1]])
+    assert O.probe_reverse_scan(idx, 1, h, 80)[0] == 72 and O.probe_reverse_scan(idx, 1, h, 71)[0] == 64
+    assert O.probe_reverse_scan(idx, 1, h, 63)[0] == 0 and O.reuse_candidate([80, 72]) == 72

@@ -62,6 +62,30 @@ def test_index_and_probe_match_the_oracle_on_a_churning_cache():
     idx.close()
 
 
+def test_reverse_scan_matches_the_oracle_and_gives_the_joint_candidate():
+    """Attention blocks are dense, recurrent snapshots sparse: the candidate is the minimum of the two endpoints, the
+    recurrent one found by scanning backward from the attention one (Section 4.3)."""
+    rng = np.random.default_rng(8)
+    ATT, REC = 0, 1
+    for _ in range(200):
+        N = int(rng.integers(0, 150))
+        hashes = np.array([int(x) for x in rng.integers(1, 1 << 62, N)], dtype=np.uint64)
+        cached = int(rng.integers(0, N + 1))
+        snaps = sorted(set(int(d) for d in rng.integers(1, N + 1, rng.integers(0, 5)))) if N else []
+        idx, oidx = wpp.HintIndex(), O.HintIndex()
+        for i in (idx, oidx):
+            i.add(ATT, hashes[:cached].tolist())
+            i.add(REC, [int(hashes[d - 1]) for d in snaps])
+        att, _ = idx.probe(ATT, hashes)
+        assert att == O.probe_gallop_bisect(oidx, ATT, hashes.tolist())[0] == cached
+        rec, probes = idx.probe_recurrent(REC, hashes, att)
+        want, probed = O.probe_reverse_scan(oidx, REC, hashes.tolist(), att)
+        assert (rec, probes) == (want, len(probed))
+        assert O.reuse_candidate([att, rec]) == max([d for d in snaps if d <= cached], default=0)
+    idx = wpp.HintIndex()
+    assert idx.probe_recurrent(REC, [], 0) == (0, 0) and idx.probe_recurrent(REC, [5, 6], 9) == (0, 2)
+
+
 def test_figure_example_through_the_library():
     h = wpp.wpp_hash_blocks_host(np.arange(12 * 16, dtype=np.int32), 16)
     idx = wpp.HintIndex()
