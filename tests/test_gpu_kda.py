@@ -87,7 +87,8 @@ def test_a_long_chain_stays_within_tolerance(layout):
 
 
 @pytest.mark.parametrize("layout", [1, 2])
-def test_splitting_a_chunk_and_resuming_is_bit_identical(layout):
+@pytest.mark.parametrize("cut", [(64, 32), (37, 20)])
+def test_splitting_a_chunk_and_resuming_is_bit_identical(layout, cut):
     """Section 3.2: the state after exactly r tokens is all a recurrent layer needs; the kernel's arithmetic per
     token does not depend on where a chunk starts, so one call and two resumed calls agree to the bit."""
     w = W.kda_workload("whole", 3, [100, 64], 2, [5, 0], resume=[True, False])
@@ -96,11 +97,11 @@ def test_splitting_a_chunk_and_resuming_is_bit_identical(layout):
     rows = w.row_offsets
     parts_o = np.zeros_like(whole_o)
     pool = t["state_pool"].clone()
-    for (a, b), first in (((37, 20), True), ((63, 44), False)):
-        cut = [37, 20]
+    for first in (True, False):
+        lens = [cut[i] if first else int(w.chunk_lens[i]) - cut[i] for i in range(2)]
         sel = np.concatenate([np.arange(rows[i] + (0 if first else cut[i]), rows[i] + (cut[i] if first else w.chunk_lens[i]))
                               for i in range(2)])
-        wp = W.kda_workload("part", 3, [a, b], 2, [5, 0])
+        wp = W.kda_workload("part", 3, lens, 2, [5, 0])
         wp.num_slots = w.num_slots
         tp = {k: (v[sel].contiguous() if k != "state_pool" else pool) for k, v in t.items()}
         s_in = w.state_in if first else w.state_out          # the second call resumes from what the first stored
@@ -110,6 +111,26 @@ def test_splitting_a_chunk_and_resuming_is_bit_identical(layout):
         pool = torch.from_numpy(new_pool).float()
     assert np.array_equal(parts_o, whole_o)
     assert np.array_equal(pool.double().numpy(), whole_pool)
+
+
+@pytest.mark.parametrize("layout", [1, 2])
+def test_tiny_and_zero_decays(layout):
+    """Decays of exactly 0 (a channel forgets everything), of 1e-6 and 1e-20, and runs of small ones."""
+    w = W.kda_workload("decays", 17, [90, 40], 2, [3, 0])
+    t = w.tensors()
+    rng = np.random.default_rng(17)
+    a = t["alpha"].numpy()
+    T = a.shape[0]
+    for val, count in ((0.0, 40), (1e-6, 40), (1e-20, 20), (0.3, 2000)):
+        idx = (rng.integers(0, T, count), rng.integers(0, 2, count), rng.integers(0, 128, count))
+        a[idx] = val
+    a[50:58, 0, 7] = 0.05                                      # eight small decays in a row on one channel
+    a[0, :, :] = 0.0                                           # the first token forgets the resumed state entirely
+    ref_o, ref_pool = _oracle(w, t)
+    got_o, got_pool, status = _gpu(w, t, layout=layout)
+    assert status == 0 and np.isfinite(got_o).all() and np.isfinite(got_pool).all()
+    _close_out(got_o, ref_o, "outputs")
+    _close_state(got_pool, ref_pool, "state pool")
 
 
 @pytest.mark.parametrize("layout", [1, 2])
