@@ -9,7 +9,7 @@ waves; block size B; maximum wave budget M and floor b_min (both multiples of B,
 the not-yet-scheduled suffixes of admitted requests together with their most recently committed chunks that are
 still in the ring; W is their token sum.
 
-Where the paper leaves a rule open, the reading taken here is marked "READING" (the same list is in DESIGN.md);
+Where the paper leaves a rule open, the reading taken here is marked "READING";
 those parts are pinned only by examples constructed from the reading: parity unpinned for them.
 """
 from fractions import Fraction
