@@ -33,6 +33,10 @@ METRIC = "prefill-attention tokens/s at concurrency 128, high prefix reuse"
 # full concurrency-128 workload (a one-pass ncu capture) / its 18,682,768 key steps.  Exact for that workload;
 # for other --config values the product with their key steps is only an estimate.
 DRAM_BYTES_PER_KEY_STEP = 628.9
+# From profiles/kda_wave_8x2048_ncu.md: dram read + write bytes of one wpp_kda_chunk launch on the default wave
+# (8 x 2,048 tokens, 32 heads) / its 524,288 (token, head) pairs; other wave shapes scale with the pairs (the state
+# traffic per request is a small part).
+KDA_DRAM_BYTES_PER_TOKEN_HEAD = 1571.3
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -471,7 +475,7 @@ def run_kda(args):
             "roofline": {"bound": "alu", "kernel": "wpp_kda_chunk_kernel", "achieved": flops / (ms * 1e-3) / 1e12,
                          "peak": peak, "unit": "TFLOP/s", "frac": flops / (ms * 1e-3) / 1e12 / peak,
                          "peak_source": "derived: 148 SMs x 128 fp32 lanes x 2 flop x 1965 MHz",
-                         "flop_per_token_head": 7 * w.d_k * w.d_v, "traffic": None,
+                         "flop_per_token_head": 7 * w.d_k * w.d_v, "traffic": KDA_DRAM_BYTES_PER_TOKEN_HEAD * T * Hh,
                          "hbm_gbs_algorithmic": nbytes / (ms * 1e-3) / 1e9},
             "cpu_baseline": {"value": (sl.stop - sl.start) / t_cpu / Hh, "unit": "tokens/s", "cores": 1, "kind": "oracle",
                              "sample": f"one (request, head) chain of {sl.stop - sl.start} tokens, scaled to {Hh} heads"},
