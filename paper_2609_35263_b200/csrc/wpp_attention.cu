@@ -260,12 +260,15 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 const int n_pages = (v.kv_len + B - 1) / B;
                 const int kvh = un.head[0] / p.group;
                 const int32_t* bt = p.block_tables + (int64_t)un.request * p.max_blocks;
-                // one ring slot: the K or the V tile of key step j; lane l moves page l of the step
+                // one ring slot: the K or the V tile of key step j.  Every 64-column box of every page is issued by a
+                // lane of its own (a thread spends about 400 clocks per TMA instruction, and at the start of a tile
+                // this warp is what everybody waits for): lane l moves column block l % kHalves of page l / kHalves.
                 auto load_tile = [&](const CUtensorMap* tm, int j, Ring& ring, uint32_t slot0, uint32_t n_ring) -> bool {
                     const int page0 = (v.kv_begin + j) * ppt;
                     const int cnt = min(ppt, n_pages - page0);
+                    const int pg = lane / C::kHalves, h = lane % C::kHalves;
                     int pid = 0;
-                    if (lane < cnt) pid = bt[page0 + lane];
+                    if (pg < cnt) pid = bt[page0 + pg];
                     if (pid < 0 || pid >= p.num_pages) {
                         if (p.status) atomicCAS(p.status, 0, WPP_ERR_BOUNDS);
                         pid = 0;
@@ -278,12 +281,8 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     const uint32_t full = bSlotFull + 8 * slot;
                     if (lane == 0) mbar_arrive_expect_tx(full, (uint32_t)cnt * B * D * 2);
                     __syncwarp();
-                    const uint32_t dst = sKV + slot * C::kTileBytes + lane * B * 128;
-                    if (lane < cnt) {
-#pragma unroll
-                        for (int h = 0; h < C::kHalves; ++h)
-                            tma_load_4d(dst + h * C::kHalfBytes, tm, full, h * 64, 0, kvh, pid);
-                    }
+                    if (pg < cnt)
+                        tma_load_4d(sKV + slot * C::kTileBytes + pg * B * 128 + h * C::kHalfBytes, tm, full, h * 64, 0, kvh, pid);
                     ring.advance(n_ring);
                     return true;
                 };
@@ -294,21 +293,21 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 STAT_ADD(1);
                 if (!__all_sync(0xffffffffu, ok)) { dead = true; break; }
                 q_phase ^= 1u;
-                if (lane == 0) {
+                {
                     const int nq = (v.n[0] > 0) + (v.n[1] > 0);
-                    mbar_arrive_expect_tx(bQFull, nq * C::kTileBytes);
-                    // head k of a half lands in tensor rows [k*rph, (k+1)*rph): one box of rph rows per head
+                    if (lane == 0) mbar_arrive_expect_tx(bQFull, nq * C::kTileBytes);
+                    __syncwarp();
+                    // head k of a half lands in tensor rows [k*rph, (k+1)*rph): one box of rph rows per head and
+                    // 64-column block; box b = (half, head, column block) is issued by lane b (at most 2 x 8 x 2)
                     const int rph = 128 / un.pack;
                     const CUtensorMap* qm = un.pack == 1 ? &tm_q : un.pack == 2 ? &tm_q64 : un.pack == 4 ? &tm_q32 : &tm_q16;
-#pragma unroll
-                    for (int hf = 0; hf < 2; ++hf) {
-                        if (v.n[hf] == 0) continue;
-                        for (int k = 0; k < un.pack; ++k) {
-#pragma unroll
-                            for (int h = 0; h < C::kHalves; ++h)
-                                tma_load_3d(sQ + hf * C::kTileBytes + h * C::kHalfBytes + k * rph * 128, qm, bQFull, h * 64,
-                                            un.head[hf] + k, v.q_off + un.row0[hf]);
-                        }
+                    const int per_half = un.pack * C::kHalves;
+                    for (int b = lane; b < 2 * per_half; b += 32) {
+                        const int hf = b / per_half, k = (b % per_half) / C::kHalves, h = b % C::kHalves;
+                        const int n_hf = hf ? v.n[1] : v.n[0];
+                        if (n_hf == 0) continue;
+                        tma_load_3d(sQ + hf * C::kTileBytes + h * C::kHalfBytes + k * rph * 128, qm, bQFull, h * 64,
+                                    (hf ? un.head[1] : un.head[0]) + k, v.q_off + (hf ? un.row0[1] : un.row0[0]));
                     }
                 }
                 __syncwarp();
