@@ -29,13 +29,16 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
 METRIC = "prefill-attention tokens/s at concurrency 128, high prefix reuse"
-# From profiles/attention_cfg3_dram.md: dram__bytes_read.sum + dram__bytes_write.sum of one attention launch on the
-# full concurrency-128 workload (a one-pass ncu capture) / its 18,682,768 key steps.  Exact for that workload;
-# for other --config values the product with their key steps is only an estimate.
+# DRAM traffic is not measured by this script (it would need a profiler): `roofline.traffic` scales a figure from an
+# ncu capture by the work of the launch timed here, and `roofline.traffic_source` says so in the JSON line.
+# Attention: dram__bytes_read.sum + dram__bytes_write.sum of one launch / its 128-row x 128-key steps, captured on the
+# 16-request cut of the concurrency-128 workload (--config cfg3_r16, 1.4 GB resident).
 DRAM_BYTES_PER_KEY_STEP = 628.9
-# From profiles/kda_wave_8x2048_ncu.md: dram read + write bytes of one wpp_kda_chunk launch on the default wave
-# (8 x 2,048 tokens, 32 heads) / its 524,288 (token, head) pairs; other wave shapes scale with the pairs (the state
-# traffic per request is a small part).
+DRAM_SOURCE = ("estimate: 628.9 DRAM bytes per 128x128 key step (dram__bytes_read.sum + dram__bytes_write.sum of one "
+               "wpp_attn_kernel launch, ncu capture on the 16-request cut of this workload) x this launch's key steps; "
+               "not measured in this run")
+# Recurrent layer: dram read + write bytes of one wpp_kda_chunk launch on the default wave (8 x 2,048 tokens, 32 heads)
+# / its 524,288 (token, head) pairs; other wave shapes scale with the pairs (the state traffic per request is small).
 KDA_DRAM_BYTES_PER_TOKEN_HEAD = 1571.3
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
@@ -61,6 +64,69 @@ def build_workload(name):
         parts = dict((p[0], int(p[1:])) for p in name.split("_")[1:])
         return W.cfg5_cell(parts["C"], parts["P"])
     raise SystemExit(f"unknown config {name}")
+
+
+def describe_config(w, world=1):
+    """The workload description both arms print (same keys, so the two lines can be matched)."""
+    return {"workload": w.name, "requests": w.num_requests, "new_tokens": w.total_new_tokens,
+            "served_tokens": int((w.prefix_lens.astype(np.int64) + w.chunk_lens).sum()),
+            "q_heads": w.num_q_heads, "kv_heads": w.num_kv_heads, "head_dim": w.head_dim,
+            "page_size": w.page_size, "parallelism": "replicas only" if world > 1 else "single GPU"}
+
+
+def roofline_times(w, flops, peaks):
+    """(tensor-bound ms, HBM-bound ms) of one attention launch: FLOPs at the bf16 peak, compulsory bytes (Q in, O
+    out, each unique KV page once) at the copy bandwidth."""
+    kv_bytes = w.unique_kv_pages() * w.num_kv_heads * w.page_size * w.head_dim * 2 * 2
+    qo_bytes = 2 * w.total_new_tokens * w.num_q_heads * w.head_dim * 2
+    t_flops = flops / (float(peaks.get("bf16_tflops", FALLBACK_PEAKS["bf16_tflops"])) * 1e12)
+    t_bytes = (kv_bytes + qo_bytes) / (float(peaks.get("hbm_gbs", FALLBACK_PEAKS["hbm_gbs"])) * 1e9)
+    return t_flops * 1e3, t_bytes * 1e3, kv_bytes, qo_bytes
+
+
+def measure_other_config(name, ctx, dev, peaks, steps=3, warmup=3):
+    """One more workload under the same clock: append + attention through the C ABI, CUDA events on the launching
+    stream, L2 flushed between steps when the inputs fit it.  Returns the kernel time, TFLOP/s and the fraction of
+    the roofline time (the slower of FLOPs at the tensor peak and compulsory bytes at HBM bandwidth)."""
+    import torch
+    import paper_2609_35263_b200 as wpp
+    w = build_workload(name)
+    desc = wpp.make_desc(w.num_requests, w.num_q_heads, w.num_kv_heads, w.head_dim, w.page_size,
+                         w.max_blocks_per_req, w.num_pages)
+    q, k_new, v_new, k_pool, v_pool = w.q(dev), w.k_new(dev), w.v_new(dev), w.k_pool(dev), w.v_pool(dev)
+    bt, P, C = (torch.from_numpy(x).to(dev) for x in (w.block_tables, w.prefix_lens, w.chunk_lens))
+    out = torch.empty(w.total_new_tokens, w.num_q_heads, w.head_dim, dtype=torch.bfloat16, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    plan = wpp.wpp_plan_tiles(ctx, desc, w.prefix_lens, w.chunk_lens).to_device()
+    ws = torch.empty(max(256, int(plan.info.workspace_bytes)), dtype=torch.uint8, device=dev)
+    flops = float(plan.info.flops)
+    t_flops, t_bytes, kv_bytes, qo_bytes = roofline_times(w, flops, peaks)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev) if kv_bytes + qo_bytes < 2 * (126 << 20) else None
+    stream = torch.cuda.current_stream()
+    times = []
+    for i in range(warmup + steps):
+        if flush is not None:
+            flush.fill_(i & 0xFF)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        wpp.wpp_kv_append(ctx, desc, k_new, v_new, k_pool, v_pool, bt, P, C, plan, status=status)
+        a.record(stream)
+        wpp.wpp_prefill_attention_varlen(ctx, desc, q, out, None, k_pool, v_pool, bt, P, C, plan, workspace=ws,
+                                         status=status)
+        b.record(stream)
+        if i >= warmup:
+            times.append((a, b))
+    torch.cuda.synchronize()
+    if int(status.item()) != 0:
+        raise SystemExit(f"device status {int(status.item())} on {name}")
+    ms = statistics.mean(a.elapsed_time(b) for a, b in times)
+    return {"workload": w.name, "steps": steps, "new_tokens": w.total_new_tokens, "kernel_ms": ms,
+            "tokens_per_s": w.total_new_tokens / (ms * 1e-3), "tflops": flops / (ms * 1e-3) / 1e12,
+            "bound": "tensor" if t_flops >= t_bytes else "hbm", "roofline_ms": max(t_flops, t_bytes),
+            "frac_of_roofline_time": max(t_flops, t_bytes) / ms,
+            "l2": "flushed between steps" if flush is not None else "inputs larger than L2"}
+
+
+OTHER_CONFIGS = ("cfg2", "cfg4_alt", "cfg5_C256_P0", "cfg5_C1024_P4096", "cfg5_C4096_P32768")
 
 
 class ClockSampler:
@@ -180,8 +246,8 @@ def run_reference(args):
     line = {"impl": "reference", "metric": METRIC, "value": v, "unit": "tokens/s", "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * w.total_new_tokens / v,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": w.name, "note": "fp64 CPU oracle, one bounded seeded sample per step; "
-                       "ms_per_step is the extrapolated time of a full wave"},
+            "config": dict(describe_config(w), note="fp64 CPU oracle, one bounded seeded sample per step; "
+                           "ms_per_step is the extrapolated time of a full wave"),
             "cpu_baseline": {"value": v, "unit": "tokens/s", "cores": last["cores"], "kind": "oracle",
                              "sample": last["sample"]},
             "e2e": {"value": v, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -492,6 +558,8 @@ def main():
     ap.add_argument("--impl", default="native", choices=["native", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-other-configs", action="store_true",
+                    help="skip the short runs of further workloads reported under other_configs")
     ap.add_argument("--force-kv-splits", type=int, default=0)
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
     ap.add_argument("--plan-order", type=int, default=0, help="0: stream order (default), 1: longest tile first")
@@ -630,18 +698,28 @@ def main():
     roof_sus = float(peaks.get("bf16_tflops_sustained", FALLBACK_PEAKS["bf16_tflops_sustained"]))
     achieved = flops / (attn_ms * 1e-3) / 1e12
     # the bound is the slower of FLOPs at the tensor peak and compulsory bytes at HBM bandwidth
-    kv_bytes = w.unique_kv_pages() * w.num_kv_heads * w.page_size * w.head_dim * 2 * 2
-    qo_bytes = 2 * T * w.num_q_heads * w.head_dim * 2
-    t_flops = flops / (roof_peak * 1e12)
-    t_bytes = (kv_bytes + qo_bytes) / (float(peaks.get("hbm_gbs", FALLBACK_PEAKS["hbm_gbs"])) * 1e9)
-    # DRAM bytes of one launch: dram__bytes_read.sum + dram__bytes_write.sum from the one-pass ncu capture
-    # summarised in profiles/, per 128x128 key step, times the key steps this launch processes
-    traffic = DRAM_BYTES_PER_KEY_STEP * float(info.key_steps) if DRAM_BYTES_PER_KEY_STEP else None
+    t_flops, t_bytes, kv_bytes, qo_bytes = roofline_times(w, flops, peaks)
+    traffic = DRAM_BYTES_PER_KEY_STEP * float(info.key_steps)
     roofline = {"bound": "tensor" if t_flops >= t_bytes else "hbm", "kernel": "wpp_attn_kernel",
                 "achieved": achieved, "peak": roof_peak, "unit": "TFLOP/s", "frac": achieved / roof_peak,
                 "peak_source": f"of {peak_kind} (burst bf16 matmul)", "frac_of_sustained": achieved / roof_sus,
-                "traffic": traffic, "flops_per_launch": flops, "kernel_ms": attn_ms,
-                "roofline_ms": max(t_flops, t_bytes) * 1e3, "frac_of_roofline_time": max(t_flops, t_bytes) * 1e3 / attn_ms}
+                "traffic": traffic, "traffic_source": DRAM_SOURCE, "compulsory_bytes": kv_bytes + qo_bytes,
+                "flops_per_launch": flops, "kernel_ms": attn_ms,
+                "roofline_ms": max(t_flops, t_bytes), "frac_of_roofline_time": max(t_flops, t_bytes) / attn_ms}
+
+    # the append alone, back to back (the per-step bracket above includes the gap to the previous kernel)
+    n_app = 20
+    a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a0.record(stream)
+    for _ in range(n_app):
+        wpp.wpp_kv_append(ctx, desc, k_new, v_new, k_pool, v_pool, bt, P, C, plan, status=status)
+    a1.record(stream)
+    a1.synchronize()
+    app_ms = a0.elapsed_time(a1) / n_app
+    app_bytes = 2 * 2 * T * w.num_kv_heads * w.head_dim * 2           # K and V, read and written
+    hbm = float(peaks.get("hbm_gbs", FALLBACK_PEAKS["hbm_gbs"]))
+    phases["append_back_to_back"] = {"launches": n_app, "ms": app_ms, "gb_per_s": app_bytes / (app_ms * 1e-3) / 1e9,
+                                     "frac_of_hbm_copy_peak": app_bytes / (app_ms * 1e-3) / 1e9 / hbm}
 
     # ---- end to end through host buffers
     e2e = None
@@ -727,12 +805,18 @@ def main():
                       "timed from wave 1's output on the host to the last wave's output on the host"}
         del host_in, out_h, dev_in, dev_out
 
+    del q, k_new, v_new, k_pool, v_pool, out
+    if not args.no_e2e:
+        del hb
+    torch.cuda.empty_cache()
+    others = None
+    if rank == 0 and world == 1 and not args.no_other_configs and args.config == "cfg3":
+        others = []
+        for name in OTHER_CONFIGS:
+            others.append(measure_other_config(name, ctx, dev, peaks))
+            torch.cuda.empty_cache()
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        del q, k_new, v_new, k_pool, v_pool, out
-        if not args.no_e2e:
-            del hb
-        torch.cuda.empty_cache()
         cpu = OracleSampler(w, True).sample(args.cpu_seconds)
 
     if rank == 0:
@@ -740,20 +824,17 @@ def main():
             "metric": METRIC, "value": tokens_per_s, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": w.name, "requests": w.num_requests, "new_tokens": T,
-                       "served_tokens": int((w.prefix_lens.astype(np.int64) + w.chunk_lens).sum()),
-                       "q_heads": w.num_q_heads, "kv_heads": w.num_kv_heads, "head_dim": w.head_dim,
-                       "page_size": w.page_size, "parallelism": "replicas only" if world > 1 else "single GPU",
-                       "l2": (f"inputs larger than L2: Q+O {qo_bytes / 1e9:.2f} GB + unique KV {kv_bytes / 1e9:.2f} GB "
+            "config": dict(describe_config(w, world),
+                           l2=(f"inputs larger than L2: Q+O {qo_bytes / 1e9:.2f} GB + unique KV {kv_bytes / 1e9:.2f} GB "
                               "touched per step vs 126 MB of L2; no explicit flush" if flush is None else
                               f"inputs ({touched / 1e6:.1f} MB touched per step) fit L2: a 256 MB buffer is overwritten "
                               "between steps; ms_per_step is the sum of append and attention event times"),
-                       "step": "wpp_plan_tiles + plan H2D + wpp_kv_append + wpp_prefill_attention_varlen",
-                       "tiles": int(info.num_tiles), "ctas": int(info.num_ctas), "key_steps": int(info.key_steps)},
+                           step="wpp_plan_tiles + plan H2D + wpp_kv_append + wpp_prefill_attention_varlen",
+                           tiles=int(info.num_tiles), ctas=int(info.num_ctas), key_steps=int(info.key_steps)),
             "tflops": flops / (ms_step * 1e-3) / 1e12 * world,
             "served_tokens_per_s": world * float((w.prefix_lens.astype(np.int64) + w.chunk_lens).sum()) / (ms_step * 1e-3),
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline, "cpu_baseline": cpu,
-            "phases": phases,
+            "phases": phases, "other_configs": others,
         }
         print(json.dumps(line))
     replicas.finalize()

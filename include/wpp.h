@@ -24,7 +24,7 @@
  *     every row start and stride must be a multiple of 16 bytes.
  *   - Problems the host can see are reported before anything is launched.  Problems
  *     only the device can see (a page id outside [0, num_pages), a bounded wait that
- *     ran out) set *status_dev (first error wins, never cleared by the library), the
+ *     ran out, lengths on the device that differ from the plan's) set *status_dev (first error wins, never cleared by the library), the
  *     affected work is skipped, and nothing traps; read it after your own sync.
  *   - A request appears at most once per wave; successive chunks of a request go in
  *     successive calls on the same stream (Section 4.6: order is preserved on each
@@ -49,7 +49,8 @@ typedef enum {
     WPP_ERR_BOUNDS = 3,             /* ceil((P_i + C_i) / B) > max_blocks_per_req, or page id out of range */
     WPP_ERR_POSITION_MISMATCH = 4,  /* span start != tokens actually cached (Section 4.6: execution fails) */
     WPP_ERR_WORKSPACE_TOO_SMALL = 5,
-    WPP_ERR_PLAN_MISMATCH = 6,      /* plan buffer corrupt, too small, or built for another batch description */
+    WPP_ERR_PLAN_MISMATCH = 6,      /* plan buffer corrupt, too small, or built for another batch description; device
+                                       side: a request's prefix_lens / chunk_lens are not those the plan was made for */
     WPP_ERR_CUDA = 7,               /* CUDA runtime/driver error; see wpp_last_cuda_error */
     WPP_ERR_TIMEOUT = 8,            /* device side: a bounded barrier wait expired; the tile was abandoned */
     WPP_ERR_ALIASED_APPEND = 9      /* wpp_validate_batch: two writers, or a writer and a reader, share a slot */
@@ -60,8 +61,13 @@ enum { WPP_BF16 = 1 };
 /* Opaque per-device context: SM count, shared-memory limit, driver entry points.  Owns host memory only. */
 typedef struct wpp_ctx wpp_ctx;
 
-/* Create a context for CUDA device `cuda_device` (makes no device allocation).  WPP_ERR_CUDA if the device or
- * driver is unusable (there is no CPU fallback).  *out is host memory owned by the library until wpp_destroy. */
+/* Create a context for CUDA device `cuda_device`.  It makes no cudaMalloc; it does look up the device address of
+ * the library's built-in scratch array (see wpp_prefill_attention_varlen_static), which is what makes the CUDA
+ * runtime place that array (wpp_static_scratch_bytes() bytes) on the device: create the context at start-up, before
+ * the KV pool is sized from the free memory.  WPP_ERR_CUDA if the device or driver is unusable (there is no CPU
+ * fallback).  *out is host memory owned by the library until wpp_destroy.  Every launching entry point must be
+ * called with the context's device current (WPP_ERR_INVALID_ARG otherwise).  The context caches the tensor maps
+ * it encodes, keyed by (pointer, extents, strides); it may be used from several host threads. */
 int wpp_create(wpp_ctx** out, int cuda_device);
 int wpp_destroy(wpp_ctx* ctx);
 const char* wpp_status_string(int status);
@@ -143,7 +149,8 @@ int wpp_plan_tiles(const wpp_ctx* ctx_or_null, const wpp_batch_desc* desc,
 int wpp_validate_batch(const wpp_batch_desc* desc, const int32_t* block_tables_host,
                        const int32_t* prefix_lens_host, const int32_t* chunk_lens_host);
 
-/* KV append ("prefill fills the cache", Sections 1 and 4.1 steps 3-5): for every new token t of request i,
+/* KV append (the chunk's K/V go into the blocks reserved for them, Section 4.1 steps 3-5): for every new token t of
+ * request i,
  * pos = P_i + t, page = block_tables[i][pos / B], slot = pos % B; copies k_new[q_off_i + t][h][0..d) and
  * v_new[...] bit for bit to k_cache / v_cache [page][h][slot][0..d).  No other pool byte is written.
  *   k_new, v_new : device, bf16 [T][Hkv][d] (read).     k_cache, v_cache : device pools (written).
@@ -152,7 +159,9 @@ int wpp_validate_batch(const wpp_batch_desc* desc, const int32_t* block_tables_h
  *   plan_host    : the host plan it was copied from (read during the call only, for launch sizing).
  *   status_dev   : device int32, sticky first-error word (may be NULL).
  * One kernel on cuda_stream, 16-byte vector copies.  A page id outside [0, num_pages) sets
- * *status_dev = WPP_ERR_BOUNDS and that token is skipped. */
+ * *status_dev = WPP_ERR_BOUNDS and that token is skipped.  A request whose prefix_lens[i] or chunk_lens[i] on the
+ * device differ from the lengths the plan was made for sets WPP_ERR_PLAN_MISMATCH and none of its tokens is written
+ * (Section 4.6: a position mismatch fails execution rather than writing against the wrong cache state). */
 int wpp_kv_append(const wpp_ctx* ctx, const wpp_batch_desc* desc, const void* k_new, const void* v_new,
                   void* k_cache, void* v_cache, const int32_t* block_tables, const int32_t* prefix_lens,
                   const int32_t* chunk_lens, const void* plan_host, const void* plan_dev, int32_t* status_dev,
@@ -172,6 +181,8 @@ int wpp_kv_append(const wpp_ctx* ctx, const wpp_batch_desc* desc, const void* k_
  *                   counter the persistent CTAs take their tiles from (zeroed by this call on the stream) and
  *                   the split-KV partial results; contents are undefined afterwards.  Two calls that may run
  *                   at the same time need a workspace each.
+ * A request whose prefix_lens[i] or chunk_lens[i] on the device differ from the plan's sets *status_dev =
+ * WPP_ERR_PLAN_MISMATCH; its tiles are skipped (its output rows are not computed; rows of split tiles read as zero).
  * Enqueues a 256-byte memset and one persistent kernel, plus one combine kernel iff the plan has split tiles.
  * Results are bit-reproducible for a given plan, whichever CTA takes which tile (no atomics on outputs; partials
  * are merged in a fixed order). */
@@ -192,8 +203,9 @@ int wpp_prefill_attention_varlen(const wpp_ctx* ctx, const wpp_batch_desc* desc,
  *   - Arguments as for wpp_prefill_attention_varlen, without workspace / workspace_bytes.
  *   - A plan that needs more scratch than the array holds is rejected with WPP_ERR_WORKSPACE_TOO_SMALL before
  *     anything is launched (plan with fewer key splits, or use the caller-workspace entry point).
- *   - The first call on a device looks up the array's device address, with the context's device current
- *     (WPP_ERR_INVALID_ARG otherwise); make that first call before any stream capture begins.
+ *   - The array's device address is looked up by wpp_create (once per device, with that device current), so that
+ *     the memory is placed at start-up and no call of this entry point has anything left to set up; create the
+ *     context before any stream capture begins.
  *   - All calls on a device share the one array and it keeps whatever the last call left in it.  The call zeroes
  *     the tile counter itself (a memset node on the stream) and every partial row is written before the combine
  *     pass reads it, but two calls whose kernels overlap on the GPU, e.g. on different streams, race on it:

@@ -7,6 +7,9 @@
 #include <stdlib.h>
 #include <string.h>
 
+#include <mutex>
+#include <new>
+
 #include "../../include/wpp.h"
 #include "wpp_device.h"
 #include "wpp_host.h"
@@ -16,6 +19,21 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
+// A tensor map depends only on (base pointer, extents, strides, box); serving loops call with the same pools and
+// the same query buffers wave after wave, so the context keeps the maps it has encoded.
+struct MapKey {
+    const void* base;
+    uint64_t dims[4], strides[3];
+    uint32_t box[4];
+    int rank;
+};
+struct MapEntry {
+    MapKey key;
+    CUtensorMap map;
+    uint64_t used;      // 0 = empty; else the tick of the last use (least recently used entry is replaced)
+};
+constexpr int kMapCacheEntries = 32;
+
 struct wpp_ctx {
     int device;
     int sm_count;
@@ -23,7 +41,46 @@ struct wpp_ctx {
     int last_cuda_error;
     int64_t launches;
     EncodeTiledFn encode_tiled;
+    void* static_scratch;           // device address of the built-in scratch array on this context's device
+    std::mutex* map_lock;
+    uint64_t map_tick;
+    MapEntry maps[kMapCacheEntries];
 };
+
+// ---------------------------------------------------------------------------------------------------------------
+// Built-in scratch for the entry point that allocates nothing (wpp_prefill_attention_varlen_static, below).
+// Some callers of this library cannot call cudaMalloc when a wave is due: the serving process has handed all free
+// device memory to the KV page pool, and an allocation on the execution path would fail or stall the stream.
+#define WPP_STATIC_SCRATCH_BYTES (16u << 20)
+static __device__ __align__(256) unsigned char wpp_static_scratch[WPP_STATIC_SCRATCH_BYTES];
+
+extern "C" size_t wpp_static_scratch_bytes(void) { return (size_t)WPP_STATIC_SCRATCH_BYTES; }
+
+// In host code the array's name is only a handle, not a device address.  The address is looked up once per
+// device, with that device current (the symbol resolves to the current device's copy).  The look-up is also
+// what makes the CUDA runtime load this module on the device, i.e. what reserves the 16 MiB there: it runs
+// inside wpp_create, at start-up, so that no later call has to find memory for it.
+static std::mutex g_scratch_lock;
+static void* g_scratch_ptr[64];
+
+static cudaError_t static_scratch_address(int device, void** out) {
+    std::lock_guard<std::mutex> guard(g_scratch_lock);
+    if (device < 0 || device >= 64) return cudaErrorInvalidDevice;
+    if (!g_scratch_ptr[device]) {
+        int cur = -1;
+        cudaError_t e = cudaGetDevice(&cur);
+        if (e != cudaSuccess) return e;
+        if (cur != device && (e = cudaSetDevice(device)) != cudaSuccess) return e;
+        void* ptr = nullptr;
+        e = cudaGetSymbolAddress(&ptr, wpp_static_scratch);
+        if (cur != device) cudaSetDevice(cur);
+        if (e != cudaSuccess) return e;
+        if (!ptr) return cudaErrorInvalidSymbol;
+        g_scratch_ptr[device] = ptr;
+    }
+    *out = g_scratch_ptr[device];
+    return cudaSuccess;
+}
 
 extern "C" int wpp_ctx_sm_count(const wpp_ctx* ctx) { return ctx ? ctx->sm_count : 148; }
 
@@ -54,13 +111,32 @@ extern "C" int wpp_create(wpp_ctx** out, int cuda_device) {
         return WPP_ERR_CUDA;
     }
     c->encode_tiled = reinterpret_cast<EncodeTiledFn>(fn);
+    if (static_scratch_address(cuda_device, &c->static_scratch) != cudaSuccess) {
+        free(c);
+        return WPP_ERR_CUDA;
+    }
+    c->map_lock = new (std::nothrow) std::mutex();
+    if (!c->map_lock) {
+        free(c);
+        return WPP_ERR_INVALID_ARG;
+    }
     *out = c;
     return WPP_OK;
 }
 
 extern "C" int wpp_destroy(wpp_ctx* ctx) {
+    if (ctx) delete ctx->map_lock;
     free(ctx);
     return WPP_OK;
+}
+
+// Every launching entry point runs with the context's device current: a call made with another device current
+// would launch there with this device's pointers and tensor maps.
+extern "C" int wpp_ctx_check_device(const wpp_ctx* ctx) {
+    int cur = -1;
+    cudaError_t e = cudaGetDevice(&cur);
+    if (e != cudaSuccess) return cuda_fail(ctx, (int)e);
+    return cur == ctx->device ? WPP_OK : WPP_ERR_INVALID_ARG;
 }
 
 extern "C" int wpp_last_cuda_error(const wpp_ctx* ctx) { return ctx ? ctx->last_cuda_error : 0; }
@@ -69,6 +145,7 @@ extern "C" int64_t wpp_launch_count(const wpp_ctx* ctx) { return ctx ? ctx->laun
 extern "C" int wpp_selftest_bounded_wait(const wpp_ctx* ctx, int64_t limit_cycles, int32_t* status_dev,
                                          int64_t* waited_cycles_dev, void* cuda_stream) {
     if (!ctx || !status_dev || limit_cycles < 1 || limit_cycles > (1ll << 30)) return WPP_ERR_INVALID_ARG;
+    if (int rc = wpp_ctx_check_device(ctx)) return rc;
     int e = wpp_launch_selftest_wait((long long)limit_cycles, status_dev,
                                      reinterpret_cast<long long*>(waited_cycles_dev), cuda_stream);
     if (e != 0) return cuda_fail(ctx, e);
@@ -78,9 +155,30 @@ extern "C" int wpp_selftest_bounded_wait(const wpp_ctx* ctx, int64_t limit_cycle
 
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
 
-// bf16 tensor map with 128-byte swizzle; dims/strides innermost first, strides in bytes for dims 1..rank-1
-static int make_map(const wpp_ctx* ctx, CUtensorMap* m, const void* base, int rank, const uint64_t* dims,
+// bf16 tensor map with 128-byte swizzle; dims/strides innermost first, strides in bytes for dims 1..rank-1.
+// Looked up in the context's cache first (six maps per attention call; encoding them costs more than a small
+// wave's kernel).
+static int make_map(const wpp_ctx* cctx, CUtensorMap* m, const void* base, int rank, const uint64_t* dims,
                     const uint64_t* strides_bytes, const uint32_t* box) {
+    wpp_ctx* ctx = const_cast<wpp_ctx*>(cctx);
+    MapKey key;
+    memset(&key, 0, sizeof(key));
+    key.base = base;
+    key.rank = rank;
+    for (int i = 0; i < rank; ++i) { key.dims[i] = dims[i]; key.box[i] = box[i]; }
+    for (int i = 0; i < rank - 1; ++i) key.strides[i] = strides_bytes[i];
+    std::lock_guard<std::mutex> guard(*ctx->map_lock);
+    const uint64_t tick = ++ctx->map_tick;
+    int victim = 0;
+    for (int i = 0; i < kMapCacheEntries; ++i) {
+        MapEntry& en = ctx->maps[i];
+        if (en.used && memcmp(&en.key, &key, sizeof(key)) == 0) {
+            en.used = tick;
+            *m = en.map;
+            return WPP_OK;
+        }
+        if (en.used < ctx->maps[victim].used) victim = i;
+    }
     cuuint64_t gd[4];
     cuuint64_t gs[3];
     cuuint32_t bx[4], es[4];
@@ -90,6 +188,10 @@ static int make_map(const wpp_ctx* ctx, CUtensorMap* m, const void* base, int ra
                                    gs, bx, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return cuda_fail(ctx, (int)r);
+    MapEntry& en = ctx->maps[victim];
+    memcpy(&en.key, &key, sizeof(key));
+    en.map = *m;
+    en.used = tick;
     return WPP_OK;
 }
 
@@ -104,6 +206,7 @@ extern "C" int wpp_kv_append(const wpp_ctx* ctx, const wpp_batch_desc* desc, con
     const WppPlanHeader* hd = nullptr;
     if ((rc = wpp_check_plan(plan_host, &d, &hd)) != WPP_OK) return rc;
     if (hd->total_new_tokens == 0) return WPP_OK;
+    if ((rc = wpp_ctx_check_device(ctx)) != WPP_OK) return rc;
     if (!k_new || !v_new || !k_cache || !v_cache || !block_tables || !prefix_lens || !chunk_lens || !plan_dev)
         return WPP_ERR_INVALID_ARG;
     if (!aligned16(k_new) || !aligned16(v_new) || !aligned16(k_cache) || !aligned16(v_cache) || !aligned16(plan_dev))
@@ -117,6 +220,7 @@ extern "C" int wpp_kv_append(const wpp_ctx* ctx, const wpp_batch_desc* desc, con
     p.v_cache = static_cast<uint4*>(v_cache);
     p.block_tables = block_tables;
     p.prefix_lens = prefix_lens;
+    p.chunk_lens = chunk_lens;
     p.status = status_dev;
     p.kvnew_token_stride = d.kvnew_token_stride / 8;
     p.kvnew_head_stride = d.kvnew_head_stride / 8;
@@ -150,6 +254,7 @@ extern "C" int wpp_prefill_attention_varlen(const wpp_ctx* ctx, const wpp_batch_
     if ((rc = wpp_check_plan(plan_host, &d, &hd)) != WPP_OK) return rc;
     if (hd->tile_m > WPP_MAX_TILE_M) return WPP_ERR_PLAN_MISMATCH;
     if (hd->total_new_tokens == 0 || hd->num_units == 0) return WPP_OK;
+    if ((rc = wpp_ctx_check_device(ctx)) != WPP_OK) return rc;
     if (!q || !out || !k_cache || !v_cache || !block_tables || !prefix_lens || !chunk_lens || !plan_dev)
         return WPP_ERR_INVALID_ARG;
     if (!aligned16(q) || !aligned16(out) || !aligned16(k_cache) || !aligned16(v_cache) || !aligned16(plan_dev))
@@ -197,12 +302,6 @@ extern "C" int wpp_prefill_attention_varlen(const wpp_ctx* ctx, const wpp_batch_
     p.num_pages = d.num_pages;
     const double scale = d.sm_scale > 0.f ? (double)d.sm_scale : 1.0 / sqrt((double)d.head_dim);
     p.scale_log2 = (float)(scale * 1.4426950408889634);
-#if defined(WPP_TRACE) || defined(WPP_STATS)
-    {   // tuning builds: the address of a device timeline buffer comes through the environment
-        const char* t = getenv("WPP_TRACE_PTR");
-        p.trace = t ? reinterpret_cast<uint32_t*>(strtoull(t, nullptr, 0)) : nullptr;
-    }
-#endif
 
     // the counter the CTAs take their tiles from starts at zero (a memset node on the caller's stream)
     int e = (int)cudaMemsetAsync(workspace, 0, WPP_WS_HEADER_BYTES, (cudaStream_t)cuda_stream);
@@ -231,45 +330,23 @@ extern "C" int wpp_prefill_attention_varlen(const wpp_ctx* ctx, const wpp_batch_
 }
 
 // ---------------------------------------------------------------------------------------------------------------
-// Entry point that allocates nothing: split-KV partials live in a scratch array inside the library image.
-// Some callers of this library cannot call cudaMalloc when a wave is due: the serving process has handed all free
-// device memory to the KV page pool, and an allocation on the execution path would fail or stall the stream.
-#define WPP_STATIC_SCRATCH_BYTES (16u << 20)
-static __device__ __align__(256) unsigned char wpp_static_scratch[WPP_STATIC_SCRATCH_BYTES];
-
-// In host code the array's name is only a handle; its device address is looked up once per device.
-static void* g_static_scratch_ptr[64];
-static bool g_static_scratch_ready[64];
-
-extern "C" size_t wpp_static_scratch_bytes(void) { return (size_t)WPP_STATIC_SCRATCH_BYTES; }
-
+// Entry point that allocates nothing: the tile counter and the split-KV partials live in the built-in scratch array
+// whose address wpp_create looked up.
 extern "C" int wpp_prefill_attention_varlen_static(const wpp_ctx* ctx, const wpp_batch_desc* desc, const void* q,
                                                    void* out, float* lse_or_null, const void* k_cache,
                                                    const void* v_cache, const int32_t* block_tables,
                                                    const int32_t* prefix_lens, const int32_t* chunk_lens,
                                                    const void* plan_host, const void* plan_dev, int32_t* status_dev,
                                                    void* cuda_stream) {
-    if (!ctx || ctx->device < 0 || ctx->device >= 64) return WPP_ERR_INVALID_ARG;
+    if (!ctx || !ctx->static_scratch) return WPP_ERR_INVALID_ARG;
     wpp_batch_desc d;
     int rc = wpp_resolve_desc(desc, &d);
     if (rc != WPP_OK) return rc;
     const WppPlanHeader* hd = nullptr;
     if ((rc = wpp_check_plan(plan_host, &d, &hd)) != WPP_OK) return rc;
     if (hd->workspace_bytes > (uint64_t)WPP_STATIC_SCRATCH_BYTES) return WPP_ERR_WORKSPACE_TOO_SMALL;
-    if (!g_static_scratch_ready[ctx->device]) {
-        // set-up, once per device, with that device current: the symbol resolves to the current device's copy
-        int cur = -1;
-        cudaError_t e = cudaGetDevice(&cur);
-        if (e != cudaSuccess) return cuda_fail(ctx, (int)e);
-        if (cur != ctx->device) return WPP_ERR_INVALID_ARG;
-        void* ptr = nullptr;
-        e = cudaGetSymbolAddress(&ptr, wpp_static_scratch);
-        if (e != cudaSuccess || !ptr) return cuda_fail(ctx, (int)e);
-        g_static_scratch_ptr[ctx->device] = ptr;
-        g_static_scratch_ready[ctx->device] = true;
-    }
     return wpp_prefill_attention_varlen(ctx, desc, q, out, lse_or_null, k_cache, v_cache, block_tables, prefix_lens,
-                                        chunk_lens, plan_host, plan_dev, g_static_scratch_ptr[ctx->device],
+                                        chunk_lens, plan_host, plan_dev, ctx->static_scratch,
                                         (size_t)WPP_STATIC_SCRATCH_BYTES, status_dev, cuda_stream);
 }
 
@@ -285,6 +362,7 @@ extern "C" int wpp_kda_chunk(const wpp_ctx* ctx, const wpp_kda_desc* desc, const
     if (desc->d_k != 128 || desc->d_v != 128) return WPP_ERR_UNSUPPORTED;
     if (desc->num_requests > 65535) return WPP_ERR_UNSUPPORTED;      // one grid row per request
     if (desc->num_requests == 0) return WPP_OK;
+    if (int rc = wpp_ctx_check_device(ctx)) return rc;
     if (!row_offsets || !state_in || !state_out) return WPP_ERR_INVALID_ARG;
     if (desc->num_slots > 0 && !state_pool) return WPP_ERR_INVALID_ARG;
     if (desc->total_tokens > 0 && (!q || !k || !v || !alpha || !beta || !out)) return WPP_ERR_INVALID_ARG;

@@ -11,10 +11,14 @@ namespace wpp {
 
 // One thread moves one 16-byte vector of K and the matching vector of V.  A vector index decomposes as
 // (token, kv head, vector within the head row); the request is found by bisection in the row offsets.
+// A request whose span on the device (prefix_lens, chunk_lens) is not the span the plan was made for is refused:
+// nothing of it is written and the status word becomes WPP_ERR_PLAN_MISMATCH (Section 4.6: a position mismatch
+// fails execution instead of writing against the wrong cache state).
 __global__ void __launch_bounds__(256) wpp_append_kernel(const AppendParams p) {
     const char* plan = static_cast<const char*>(p.plan);
     const WppPlanHeader* hd = reinterpret_cast<const WppPlanHeader*>(plan);
     const int32_t* q_offsets = reinterpret_cast<const int32_t*>(plan + hd->off_q_offsets);
+    const int32_t* plan_prefix = reinterpret_cast<const int32_t*>(plan + hd->off_prefix);
     const int64_t per_token = (int64_t)p.num_kv_heads * p.vec_per_row;
     const int64_t total = p.total_new_tokens * per_token;
     const int64_t stride = (int64_t)gridDim.x * blockDim.x;
@@ -27,7 +31,12 @@ __global__ void __launch_bounds__(256) wpp_append_kernel(const AppendParams p) {
             const int mid = (lo + hi) >> 1;
             if (q_offsets[mid] <= tok) lo = mid; else hi = mid;
         }
-        const int pos = p.prefix_lens[lo] + (int)(tok - q_offsets[lo]);
+        const int P = p.prefix_lens[lo];
+        if (P != plan_prefix[lo] || p.chunk_lens[lo] != q_offsets[lo + 1] - q_offsets[lo]) {
+            if (p.status) atomicCAS(p.status, 0, WPP_ERR_PLAN_MISMATCH);
+            continue;
+        }
+        const int pos = P + (int)(tok - q_offsets[lo]);
         const int blk = pos / p.page_size, slot = pos - blk * p.page_size;
         const int page = (blk < p.max_blocks) ? p.block_tables[(int64_t)lo * p.max_blocks + blk] : -1;
         if (page < 0 || page >= p.num_pages) {

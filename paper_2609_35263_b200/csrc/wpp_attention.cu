@@ -45,27 +45,12 @@ __host__ __device__ constexpr uint32_t col_p(int hf) { return 128u + 64u * hf; }
 __host__ __device__ constexpr uint32_t col_o(int hf) { return 256u + 128u * hf; }   // O of half hf
 // registers per thread after the warpgroups re-split the register file (8 x kRegsSoftmax + 4 x kRegsEpilogue +
 // 4 x kRegsUtil <= 2048 per thread slot of 32 lanes, i.e. 65536 in all)
-#ifndef WPP_REGS_SOFTMAX
-#define WPP_REGS_SOFTMAX 192
-#define WPP_REGS_EPILOGUE 64
-#define WPP_REGS_UTIL 64
-#endif
-constexpr int kRegsSoftmax = WPP_REGS_SOFTMAX, kRegsEpilogue = WPP_REGS_EPILOGUE, kRegsUtil = WPP_REGS_UTIL;
+constexpr int kRegsSoftmax = 192, kRegsEpilogue = 64, kRegsUtil = 64;
 static_assert(8 * kRegsSoftmax + 4 * kRegsEpilogue + 4 * kRegsUtil <= 2048, "register file exceeded");
-// arrivals on s_free and p_ready: every softmax thread (128), or one elected lane per warp after __syncwarp (4)
-#ifndef WPP_ELECT_ARRIVE
-#define WPP_ELECT_ARRIVE 0
-#endif
-constexpr uint32_t kSoftmaxArrivals = WPP_ELECT_ARRIVE ? 4 : 128;
-#ifndef WPP_RESCALE_COLS
-#define WPP_RESCALE_COLS 16
-#endif
-constexpr int kRescaleCols = WPP_RESCALE_COLS;   // columns of O in flight while a moved reference rescales it
+constexpr uint32_t kSoftmaxArrivals = 128;   // every softmax thread arrives on s_free and p_ready itself
+constexpr int kRescaleCols = 16;    // columns of O in flight while a moved reference rescales it
 constexpr float kRefSlack = 16.f;   // a row keeps its reference while its scores stay below reference + 16 (log2)
-#ifndef WPP_EXP_BLOCK
-#define WPP_EXP_BLOCK 8
-#endif
-constexpr int kExpBlock = WPP_EXP_BLOCK;   // score pairs whose exponentials are in flight together
+constexpr int kExpBlock = 8;        // score pairs whose exponentials are in flight together
 
 template <int D>
 struct Cfg {
@@ -84,34 +69,6 @@ struct Cfg {
     static_assert(kSmemBytes <= 232448, "more shared memory than a CTA can have");
 };
 
-// Optional wait accounting for tuning (compiled out unless WPP_STATS is defined): one thread of each role adds
-// the clocks it spent in each kind of wait to p.trace, read as unsigned long long [role][8].
-#ifdef WPP_STATS
-#define STAT_DECL()                                                                                        \
-    uint32_t stat0_ = 0, stat1_ = 0, stat2_ = 0, stat3_ = 0, stat4_ = 0, stat5_ = 0, stat6_ = 0;           \
-    const long long stat_begin_ = clock64()
-#define STAT_T0() const uint32_t st0_ = (uint32_t)clock64()
-#define STAT_ADD(k) stat##k##_ += (uint32_t)clock64() - st0_
-#define STAT_INC(k) stat##k##_ += 1u
-#define STAT_FLUSH(role, leader)                                                                          \
-    do {                                                                                                  \
-        if (p.trace && (leader)) {                                                                        \
-            unsigned long long* t_ = reinterpret_cast<unsigned long long*>(p.trace) + (role) * 8;         \
-            atomicAdd(t_ + 0, (unsigned long long)stat0_); atomicAdd(t_ + 1, (unsigned long long)stat1_); \
-            atomicAdd(t_ + 2, (unsigned long long)stat2_); atomicAdd(t_ + 3, (unsigned long long)stat3_); \
-            atomicAdd(t_ + 4, (unsigned long long)stat4_); atomicAdd(t_ + 5, (unsigned long long)stat5_); \
-            atomicAdd(t_ + 6, (unsigned long long)stat6_);                                                \
-            atomicAdd(t_ + 7, (unsigned long long)(clock64() - stat_begin_));                             \
-        }                                                                                                 \
-    } while (0)
-#else
-#define STAT_DECL() do { } while (0)
-#define STAT_T0() do { } while (0)
-#define STAT_ADD(k) do { } while (0)
-#define STAT_INC(k) do { } while (0)
-#define STAT_FLUSH(role, leader) do { } while (0)
-#endif
-
 struct Ring {
     uint32_t stage, phase;
     __device__ __forceinline__ void advance(uint32_t n) {
@@ -124,17 +81,23 @@ struct UnitView {
     int request, kv_begin, n_steps;      // n_steps = max over halves
     int n[2];                            // key steps of each half (0: nothing to compute)
     int P, kv_len, q_off;
+    bool mismatch;                       // the launch's lengths are not the plan's
 };
-__device__ __forceinline__ UnitView view_of(const WppUnit& un, const AttnParams& p, const int32_t* q_offsets) {
+// A request whose span on the device differs from the span the plan was made for gets no key steps (every role
+// skips the tile, `mismatch` tells the producer to report it): the tile geometry belongs to other lengths.
+__device__ __forceinline__ UnitView view_of(const WppUnit& un, const AttnParams& p, const int32_t* q_offsets,
+                                            const int32_t* plan_prefix) {
     UnitView v;
     v.request = un.request;
     v.kv_begin = un.kv_begin;
     v.P = p.prefix_lens[un.request];
-    v.kv_len = v.P + p.chunk_lens[un.request];
+    const int C = p.chunk_lens[un.request];
+    v.kv_len = v.P + C;
     v.q_off = q_offsets[un.request];
+    v.mismatch = (v.P != plan_prefix[un.request]) || (C != q_offsets[un.request + 1] - v.q_off);
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
-        const int end = un.rows[h] > 0 ? (v.P + un.row0[h] + un.rows[h] + 127) / 128 : 0;
+        const int end = (un.rows[h] > 0 && !v.mismatch) ? (v.P + un.row0[h] + un.rows[h] + 127) / 128 : 0;
         v.n[h] = max(0, min(un.kv_end, end) - un.kv_begin);
     }
     v.n_steps = max(v.n[0], v.n[1]);
@@ -212,6 +175,7 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     const char* plan = static_cast<const char*>(p.plan);
     const WppPlanHeader* hd = reinterpret_cast<const WppPlanHeader*>(plan);
     const int32_t* q_offsets = reinterpret_cast<const int32_t*>(plan + hd->off_q_offsets);
+    const int32_t* plan_prefix = reinterpret_cast<const int32_t*>(plan + hd->off_prefix);
     const WppUnit* units = reinterpret_cast<const WppUnit*>(plan + hd->off_units);
     const int num_units = hd->num_units;
     // next tile index for a consuming role: -1 = no more tiles, -2 = the wait was abandoned
@@ -237,7 +201,6 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             Ring ring_k = {0, 0}, ring_v = {0, 0};
             uint32_t q_phase = 0;
             bool dead = false;
-            STAT_DECL();
             while (!dead) {
                 // take the next tile of the planner's order and tell the other roles
                 int u = 0;
@@ -255,7 +218,8 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 }
                 if (u < 0) break;
                 const WppUnit un = units[u];
-                const UnitView v = view_of(un, p, q_offsets);
+                const UnitView v = view_of(un, p, q_offsets, plan_prefix);
+                if (v.mismatch && lane == 0 && p.status) atomicCAS(p.status, 0, WPP_ERR_PLAN_MISMATCH);
                 if (v.n_steps == 0) continue;
                 const int n_pages = (v.kv_len + B - 1) / B;
                 const int kvh = un.head[0] / p.group;
@@ -274,9 +238,7 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                         pid = 0;
                     }
                     const uint32_t slot = slot0 + ring.stage;
-                    STAT_T0();
                     const bool ok = mbar_wait(bSlotEmpty + 8 * slot, ring.phase ^ 1u, abort_flag);
-                    STAT_ADD(0);
                     if (!__all_sync(0xffffffffu, ok)) return false;
                     const uint32_t full = bSlotFull + 8 * slot;
                     if (lane == 0) mbar_arrive_expect_tx(full, (uint32_t)cnt * B * D * 2);
@@ -288,9 +250,7 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 };
                 // K(0) only needs a ring slot, which frees up before the previous tile's Q does
                 if (!load_tile(&tm_k, 0, ring_k, n_v, n_k)) { dead = true; break; }
-                STAT_T0();
                 const bool ok = mbar_wait(bQEmpty, q_phase ^ 1u, abort_flag);
-                STAT_ADD(1);
                 if (!__all_sync(0xffffffffu, ok)) { dead = true; break; }
                 q_phase ^= 1u;
                 {
@@ -316,7 +276,6 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     if (!dead && k + 1 < v.n_steps && !load_tile(&tm_k, k + 1, ring_k, n_v, n_k)) dead = true;
                 }
             }
-            STAT_FLUSH(4, lane == 0);
         } else if (warp == 12 && lane == 0) {
             // ================================================================ issuer of S = Q K^T (one thread)
             // S_A(0), S_B(0), S_A(1), S_B(1), ...: each S goes into the landing buffer as soon as the previous one
@@ -328,25 +287,20 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             const uint64_t k_desc0 = smem_desc_sw128(sKV + n_v * C::kTileBytes, 16, 1024);   // + stage * (kTileBytes >> 4)
             const uint32_t tS = tmem + kColS;
             bool dead = false;
-            STAT_DECL();
             while (!dead) {
                 const int u = next_tile();
                 if (u < 0) break;
                 const WppUnit un = units[u];
-                const UnitView v = view_of(un, p, q_offsets);
+                const UnitView v = view_of(un, p, q_offsets, plan_prefix);
                 if (v.n_steps == 0) continue;
                 {
-                    STAT_T0();
                     const bool ok = mbar_wait(bQFull, q_phase, abort_flag);
-                    STAT_ADD(4);
                     if (!ok) break;
                 }
                 q_phase ^= 1u;
                 for (int k = 0; k < v.n_steps; ++k) {
                     {
-                        STAT_T0();
                         const bool ok = mbar_wait(bSlotFull + 8 * (n_v + ring.stage), ring.phase, abort_flag);   // K(k)
-                        STAT_ADD(0);
                         if (!ok) { dead = true; break; }
                     }
                     const uint64_t kd = k_desc0 + (uint64_t)(ring.stage * (C::kTileBytes >> 4));
@@ -354,15 +308,12 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     for (int hf = 0; hf < 2; ++hf) {
                         if (k >= v.n[hf]) continue;
                         {
-                            STAT_T0();
                             const bool ok = mbar_wait(bSFree, sfree_phase ^ 1u, abort_flag);
-                            STAT_ADD(2);
                             if (!ok) { dead = true; break; }
                         }
                         sfree_phase ^= 1u;
                         tc_fence_after();
                         const uint64_t qd = q_desc0 + (uint64_t)(hf * (C::kTileBytes >> 4));
-                        STAT_T0();
 #pragma unroll
                         for (int kk = 0; kk < D / 16; ++kk) {
                             const uint64_t off = (uint64_t)(((kk >> 2) * C::kHalfBytes + (kk & 3) * 32) >> 4);
@@ -370,7 +321,6 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                             else mma_ss_accumulate(tS, qd + off, kd + off, idesc_qk);
                         }
                         mma_commit(bSFull(hf));
-                        STAT_ADD(6);
                     }
                     if (dead) break;
                     mma_commit(bSlotEmpty + 8 * (n_v + ring.stage));                  // K(k) has been read
@@ -378,7 +328,6 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 }
                 if (!dead) mma_commit(bQEmpty);           // every S of the tile has been issued: Q may be replaced
             }
-            STAT_FLUSH(0, true);
         } else if (warp == 14 && lane == 0) {
             // ================================================================ issuer of O += P V (one thread)
             // O_A += P_A V(0), O_B += P_B V(0), O_A += P_A V(1), ...: each product waits for its P.
@@ -387,18 +336,15 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             constexpr uint32_t idesc_pv = idesc_bf16(D, 0, 1);
             const uint64_t v_desc0 = smem_desc_sw128(sKV, C::kHalfBytes, 1024);       // + stage * (kTileBytes >> 4)
             bool dead = false;
-            STAT_DECL();
             while (!dead) {
                 const int u = next_tile();
                 if (u < 0) break;
                 const WppUnit un = units[u];
-                const UnitView v = view_of(un, p, q_offsets);
+                const UnitView v = view_of(un, p, q_offsets, plan_prefix);
                 if (v.n_steps == 0) continue;
                 for (int k = 0; k < v.n_steps; ++k) {
                     {
-                        STAT_T0();
                         const bool ok = mbar_wait(bSlotFull + 8 * ring.stage, ring.phase, abort_flag);           // V(k)
-                        STAT_ADD(0);
                         if (!ok) { dead = true; break; }
                     }
                     const int valid = v.kv_len - (v.kv_begin + k) * 128;      // keys of this step that exist
@@ -417,36 +363,29 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                         const int n = v.n[hf];
                         if (k >= n) continue;
                         {
-                            STAT_T0();
                             const bool ok = mbar_wait(bPReady(hf), p_phase[hf], abort_flag);     // P written, O fixed
-                            STAT_ADD(1);
                             if (!ok) { dead = true; break; }
                         }
                         p_phase[hf] ^= 1u;
                         if (k == 0) {
                             // the first product of a tile overwrites O: the previous tile's epilogue must have read it
-                            STAT_T0();
                             const bool ok = mbar_wait(bOFree(hf), of_phase[hf] ^ 1u, abort_flag);
-                            STAT_ADD(3);
                             if (!ok) { dead = true; break; }
                             of_phase[hf] ^= 1u;
                         }
                         tc_fence_after();
                         const uint32_t tP = tmem + col_p(hf), tO = tmem + col_o(hf);
-                        STAT_T0();
                         if (k > 0) mma_ts_accumulate(tO, tP, vd, idesc_pv); else mma_ts_overwrite(tO, tP, vd, idesc_pv);
 #pragma unroll
                         for (int kk = 1; kk < 8; ++kk) mma_ts_accumulate(tO, tP + kk * 8, vd + (uint64_t)(kk * 128), idesc_pv);
                         mma_commit(bPFree(hf));
                         if (k + 1 == n) mma_commit(bOFinal(hf));
-                        STAT_ADD(5);
                     }
                     if (dead) break;
                     mma_commit(bSlotEmpty + 8 * ring.stage);                          // V(k) has been read
                     ring.advance(n_v);
                 }
             }
-            STAT_FLUSH(1, true);
         }
     } else if (wg == 2) {
         // ================================================================ epilogue (one thread per output row)
@@ -459,7 +398,7 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             const int u = next_tile();
             if (!__all_sync(0xffffffffu, u != -2) || u < 0) break;
             const WppUnit un = units[u];
-            const UnitView v = view_of(un, p, q_offsets);
+            const UnitView v = view_of(un, p, q_offsets, plan_prefix);
             // ---- epilogue of both halves
 #pragma unroll
             for (int hf = 0; hf < 2; ++hf) {
@@ -535,12 +474,11 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         const float c = p.scale_log2;
         const uint64_t c2 = pack2(c, c);
         bool dead = false;
-        STAT_DECL();
         while (!dead) {
             const int u = next_tile();
             if (!__all_sync(0xffffffffu, u != -2) || u < 0) break;
             const WppUnit un = units[u];
-            const UnitView v = view_of(un, p, q_offsets);
+            const UnitView v = view_of(un, p, q_offsets, plan_prefix);
             const int n = v.n[hf];
             if (n == 0) continue;
             const int first_pos = v.P + un.row0[hf];          // last key visible to row 0 of this half
@@ -553,17 +491,11 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             float m_ref = -INFINITY, l_run = 0.f, nmc = 0.f;
             for (int j = 0; j < n; ++j) {
                 {
-                    STAT_T0();
                     const bool ok = mbar_wait(bSFull(hf), s_phase, abort_flag);
-                    STAT_ADD(0);
-                    STAT_INC(2);
                     if (!__all_sync(0xffffffffu, ok)) { dead = true; break; }
                 }
                 s_phase ^= 1u;
                 tc_fence_after();
-#ifdef WPP_STATS_FINE
-                const uint32_t sta_ = (uint32_t)clock64();
-#endif
                 // copy S out of the landing buffer and hand the buffer back at once
                 float s[128];
 #pragma unroll
@@ -571,27 +503,7 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     tmem_ld32(lane_addr + kColS + q4 * 32, reinterpret_cast<uint32_t*>(s) + q4 * 32);
                 tmem_wait_ld();
                 tc_fence_before();
-                if (WPP_ELECT_ARRIVE) {
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(bSFree);
-                } else {
-                    mbar_arrive(bSFree);
-                }
-#ifdef WPP_STATS_FINE
-                const uint32_t stb_ = (uint32_t)clock64();
-                stat4_ += stb_ - sta_;
-#endif
-#ifdef WPP_EXPERIMENT_NO_SOFTMAX
-                // tuning experiment: how fast is the tile loop when the softmax costs nothing (results are garbage)
-                {
-                    const bool okp = mbar_wait(bPFree(hf), pf_phase ^ 1u, abort_flag);
-                    if (!__all_sync(0xffffffffu, okp)) { dead = true; break; }
-                    pf_phase ^= 1u;
-                }
-                tc_fence_before();
-                mbar_arrive(bPReady(hf));
-                continue;
-#endif
+                mbar_arrive(bSFree);
                 const int key0 = (v.kv_begin + j) * 128;
                 if (key0 + 127 > first_pos) {                 // only steps that touch the diagonal are masked
                     const int limit = row_last - key0;
@@ -649,10 +561,6 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                         }
                     }
                 }
-#ifdef WPP_STATS_FINE
-                const uint32_t stm_ = (uint32_t)clock64();
-                stat3_ += stm_ - stb_;
-#endif
                 // p = 2^(s*c - m_ref*c) for the whole row: bf16 pairs for the tensor cores, fp32 row sum.  The packed
                 // pair i takes the place of score i, which pair i/2 has consumed: the row never needs more than its
                 // 128 registers.
@@ -673,14 +581,8 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                         for (int k = 0; k < kExpBlock; ++k) {
                             float x0, x1;
                             unpack2(x2[k], x0, x1);
-#ifdef WPP_EXPERIMENT_CHEAP_EXP
-                            // tuning experiment: the same loop without the special-function unit (results are garbage)
-                            e[2 * k] = __saturatef(x0 * 0.01f + 0.5f);
-                            e[2 * k + 1] = __saturatef(x1 * 0.01f + 0.5f);
-#else
                             e[2 * k] = fast_exp2(x0);
                             e[2 * k + 1] = fast_exp2(x1);
-#endif
                         }
 #pragma unroll
                         for (int k = 0; k < kExpBlock; ++k) {
@@ -693,15 +595,9 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     unpack2(fadd2(sum2a, sum2b), t0, t1);
                     l_run += t0 + t1;
                 }
-#ifdef WPP_STATS_FINE
-                const uint32_t stc_ = (uint32_t)clock64();
-                stat5_ += stc_ - stm_;
-#endif
                 if (!waited) {
                     // P(j-1) must have been consumed before P(j) replaces it
-                    STAT_T0();
                     const bool okp = mbar_wait(bPFree(hf), pf_phase ^ 1u, abort_flag);
-                    STAT_ADD(1);
                     if (!__all_sync(0xffffffffu, okp)) { dead = true; break; }
                     pf_phase ^= 1u;
                     tc_fence_after();
@@ -712,15 +608,7 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 for (int c8 = 0; c8 < 64; c8 += 8) tmem_st8(lane_addr + col_p(hf) + c8, pk + c8);
                 tmem_wait_st();
                 tc_fence_before();
-                if (WPP_ELECT_ARRIVE) {
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(bPReady(hf));
-                } else {
-                    mbar_arrive(bPReady(hf));
-                }
-#ifdef WPP_STATS_FINE
-                stat6_ += (uint32_t)clock64() - stc_;
-#endif
+                mbar_arrive(bPReady(hf));
             }
             if (dead) break;
             {
@@ -733,17 +621,18 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             s_final[hf * 128 + r] = make_float2(-nmc, l_run);
             mbar_arrive(bFinalReady(hf));
         }
-        STAT_FLUSH(2 + hf, r == 0);
     }
 
-    // ---- teardown: every loop above is bounded, so every thread gets here
+    // ---- teardown: every loop above is bounded, so every thread gets here.  The abort flag is read after the
+    //      barrier: a role that gave up late (after thread 0 had finished its own work) is still reported.
+    tc_fence_before();
+    __syncthreads();
     if (*abort_flag) {
         const long long t0 = clock64();
         while (clock64() - t0 < 400000) { }     // let copies and tensor-core work in flight land
         if (threadIdx.x == 0 && p.status) atomicCAS(p.status, 0, WPP_ERR_TIMEOUT);
+        __syncthreads();
     }
-    tc_fence_before();
-    __syncthreads();
     if (warp == 12) {
         tc_fence_after();
         tmem_dealloc(tmem, kTmemCols);

@@ -22,7 +22,6 @@ struct AttnParams {
     int64_t o_token_stride, o_head_stride;
     int32_t num_q_heads, group, page_size, max_blocks, num_pages;
     float scale_log2;                // sm_scale * log2(e)
-    uint32_t* trace;                 // tuning builds only (WPP_TRACE): timeline buffer, else null
 };
 
 struct AppendParams {
@@ -33,6 +32,7 @@ struct AppendParams {
     uint4* v_cache;
     const int32_t* block_tables;
     const int32_t* prefix_lens;
+    const int32_t* chunk_lens;
     int32_t* status;
     int64_t kvnew_token_stride, kvnew_head_stride;       // in 16-byte units
     int64_t kv_page_stride, kv_head_stride, kv_token_stride;

@@ -120,6 +120,7 @@ extern "C" int wpp_hash_blocks(const wpp_ctx* ctx, const int32_t* tokens, const 
     if (!ctx || num_requests < 0 || block_size < 1 || total_blocks < 0) return WPP_ERR_INVALID_ARG;
     if (num_requests == 0 || total_blocks == 0) return WPP_OK;
     if (!tokens || !token_offsets || !block_offsets || !hashes_out) return WPP_ERR_INVALID_ARG;
+    if (int rc = wpp_ctx_check_device(ctx)) return rc;
     cudaStream_t st = (cudaStream_t)cuda_stream;
     int64_t blocks = (total_blocks * 32 + 255) / 256;
     if (blocks > 148 * 16) blocks = 148 * 16;

@@ -15,6 +15,7 @@ int wpp_resolve_desc(const wpp_batch_desc* in, wpp_batch_desc* out);
 uint64_t wpp_desc_hash(const wpp_batch_desc* resolved);
 int wpp_check_plan(const void* plan_host, const wpp_batch_desc* resolved, const struct WppPlanHeader** out);
 int wpp_ctx_sm_count(const wpp_ctx* ctx);
+int wpp_ctx_check_device(const wpp_ctx* ctx);   /* WPP_OK iff the context's device is the current one */
 #ifdef __cplusplus
 }
 #endif

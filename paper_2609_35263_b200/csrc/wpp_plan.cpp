@@ -62,7 +62,9 @@ static uint64_t fnv1a(uint64_t h, const void* p, size_t n) {
     return h;
 }
 
-// Hash of everything a plan depends on except the lengths (those are covered by q_offsets checks).
+// Hash of everything a plan depends on except the lengths.  Those travel inside the plan (row offsets and a copy
+// of prefix_lens); the kernels compare them with the device arrays they are launched with and refuse a request
+// whose span differs (WPP_ERR_PLAN_MISMATCH in the status word).
 uint64_t wpp_desc_hash(const wpp_batch_desc* d) {
     uint64_t h = 0xcbf29ce484222325ull;
     const int32_t ints[] = {d->num_requests, d->num_q_heads, d->num_kv_heads, d->head_dim, d->page_size,
@@ -96,7 +98,7 @@ static size_t plan_bytes_bound(const wpp_batch_desc* d, const wpp_plan_opts* o, 
     const int64_t base = q_tiles * d->num_q_heads;
     const int64_t units = o->force_kv_splits >= 2 ? base * o->force_kv_splits : base + 2 * (int64_t)o->max_ctas;
     size_t n = sizeof(WppPlanHeader);
-    n += align_up(sizeof(int32_t) * (size_t)(d->num_requests + 1), 16);
+    n += 2 * align_up(sizeof(int32_t) * (size_t)(d->num_requests + 1), 16);   // row offsets, prefix copy
     n += align_up(sizeof(int32_t) * (size_t)(o->max_ctas + 1), 16);
     n += sizeof(WppUnit) * (size_t)units;
     n += sizeof(WppCombine) * (size_t)base * 2;
@@ -290,6 +292,8 @@ int wpp_plan_tiles(const wpp_ctx* ctx, const wpp_batch_desc* desc, const int32_t
     size_t off = sizeof(WppPlanHeader);
     hd.off_q_offsets = (uint32_t)off;
     off += align_up(sizeof(int32_t) * (size_t)(R + 1), 16);
+    hd.off_prefix = (uint32_t)off;
+    off += align_up(sizeof(int32_t) * (size_t)(R + 1), 16);
     hd.off_units = (uint32_t)off;
     off += sizeof(WppUnit) * (size_t)n_units;
     hd.off_combine = (uint32_t)off;
@@ -303,6 +307,8 @@ int wpp_plan_tiles(const wpp_ctx* ctx, const wpp_batch_desc* desc, const int32_t
     int32_t* qo = reinterpret_cast<int32_t*>(p + hd.off_q_offsets);
     qo[0] = 0;
     for (int i = 0; i < R; ++i) qo[i + 1] = qo[i] + chunk_lens[i];
+    int32_t* pp = reinterpret_cast<int32_t*>(p + hd.off_prefix);
+    for (int i = 0; i < R; ++i) pp[i] = prefix_lens[i];
     WppUnit* us = reinterpret_cast<WppUnit*>(p + hd.off_units);
     for (int64_t k = 0; k < n_units; ++k) us[k] = units[(size_t)order[(size_t)k]];
     if (!combines.empty())

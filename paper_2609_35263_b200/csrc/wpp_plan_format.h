@@ -4,21 +4,22 @@
 #include <stdint.h>
 
 #define WPP_PLAN_MAGIC 0x31505057u /* "WPP1" */
-#define WPP_PLAN_VERSION 5u
+#define WPP_PLAN_VERSION 6u
 #define WPP_TILE_N 128             /* keys per step */
 #define WPP_WS_HEADER_BYTES 256
 #define WPP_HALF_M 128             /* query rows per tensor-core tile (one TMEM lane per row) */
 
 struct WppPlanHeader {
     uint32_t magic, version;
-    uint64_t desc_hash;             // hash of the batch description + lengths the plan was made for
+    uint64_t desc_hash;             // hash of the batch description the plan was made for (the lengths are stored)
     int32_t num_requests, num_ctas, num_units, num_combine;
     int32_t num_split_slots;        // partial-result slots of 2 x 128 rows each in the workspace
     int32_t tile_m, tile_n, head_dim;
     int64_t total_new_tokens, key_steps, flops;
     uint64_t workspace_bytes, plan_bytes;
     uint32_t off_q_offsets;         // int32 [R+1]   exclusive scan of chunk_lens
-    uint32_t reserved0;
+    uint32_t off_prefix;            // int32 [R]     prefix_lens the plan was made for: the kernels compare them (and
+                                    //               the row offsets) with the lengths they are launched with
     uint32_t off_units;             // WppUnit [num_units] in the order the persistent CTAs take them
     uint32_t off_combine;           // WppCombine [num_combine]
     uint32_t pad[8];

@@ -7,9 +7,12 @@ KV-head sharding needs no exchange inside attention: heads are independent, so r
 heads [r Hkv/W, (r+1) Hkv/W) and their query heads through strided views of the same tensors.
 
 The hand-off is asynchronous point-to-point: a fixed-size header (wave id, span count, token count, the spans as
-(request id, starting token, length)) followed by the activations, received into a ring of buffers so that wave w+1
-arrives while wave w computes.  A follower checks every span against the tokens it has itself materialised for that
-request and fails the wave on a mismatch (Section 4.6)."""
+(request id, starting token, length)) and the activations.  Both messages have a fixed size (the activations always
+travel as the link's full wave buffer, `max_wave_tokens` rows, of which the header says how many count), so a stage
+can post both receives of wave w+1 before it knows anything about that wave, i.e. before it starts computing wave
+w: the transfer overlaps the compute.  Waves are planned to fill the budget, so little of the buffer is padding.  A
+follower checks every span against the tokens it has itself materialised for that request and fails the wave on a
+mismatch (Section 4.6)."""
 from __future__ import annotations
 
 from typing import Dict, List, Sequence, Tuple
@@ -54,7 +57,7 @@ def check_spans(spans: Sequence[Span], materialised: Dict[int, int]) -> None:
 
 
 class StageLink:
-    """Sends waves to the next stage and receives them from the previous one."""
+    """Sends waves to the next stage and receives them from the previous one (a middle stage does both)."""
 
     HEADER = 4           # wave id, number of spans, number of tokens, hidden size
 
@@ -64,51 +67,64 @@ class StageLink:
         self.prev = rank - 1 if rank > 0 else None
         self.next = rank + 1 if rank + 1 < world else None
         self.device = torch.device(device)
-        self._hdr = [torch.zeros(self.HEADER + 3 * max_lanes, dtype=torch.int64, device=self.device) for _ in range(depth)]
-        self._act = [torch.empty((max_wave_tokens, hidden), dtype=dtype, device=self.device) for _ in range(depth)]
+        hdr = lambda: torch.zeros(self.HEADER + 3 * max_lanes, dtype=torch.int64, device=self.device)
+        act = lambda: torch.zeros((max_wave_tokens, hidden), dtype=dtype, device=self.device)
+        self._hdr = [hdr() for _ in range(depth)] if self.prev is not None else []
+        self._act = [act() for _ in range(depth)] if self.prev is not None else []
         self._slot = 0
-        self._posted = None          # (slot, work) of the header receive in flight
-        self._sent: List = []        # (work handles, tensors kept alive)
+        self._posted = None          # (slot, header work, activation work) of the receives in flight
+        # send side: a ring of staging buffers; a buffer is reused once its two sends have completed
+        self._out_hdr = [hdr() for _ in range(depth)] if self.next is not None else []
+        self._out_act = [act() for _ in range(depth)] if self.next is not None else []
+        self._out_work: List = [None] * depth
+        self._out_slot = 0
 
     # ---- towards the next stage
     def send_wave(self, wave_id: int, spans: Sequence[Span], activations: torch.Tensor) -> None:
         if self.next is None:
             raise RuntimeError("the last stage has nowhere to send")
         n = len(spans)
-        if n > self.max_lanes or activations.shape[0] != sum(s[2] for s in spans) or activations.shape[1] != self.hidden:
+        tokens = int(activations.shape[0])
+        if (n > self.max_lanes or tokens != sum(s[2] for s in spans) or activations.shape[1] != self.hidden
+                or tokens > self._out_act[0].shape[0]):
             raise ValueError("wave does not fit the link or spans and activations disagree")
+        slot = self._out_slot
+        self._out_slot = (slot + 1) % len(self._out_hdr)
+        if self._out_work[slot] is not None:
+            for w in self._out_work[slot]:
+                w.wait()
         hdr = torch.zeros(self.HEADER + 3 * self.max_lanes, dtype=torch.int64)
-        hdr[:4] = torch.tensor([wave_id, n, activations.shape[0], self.hidden])
+        hdr[:4] = torch.tensor([wave_id, n, tokens, self.hidden])
         if n:
             hdr[4:4 + 3 * n] = torch.tensor(spans, dtype=torch.int64).reshape(-1)
-        hdr = hdr.to(self.device)
-        works = [dist.isend(hdr, self.next)]
-        if activations.shape[0]:
-            works.append(dist.isend(activations, self.next))
-        self._sent.append((works, (hdr, activations)))
-        self._sent = [s for s in self._sent if not all(w.is_completed() for w in s[0])]
+        self._out_hdr[slot].copy_(hdr)
+        self._out_act[slot][:tokens].copy_(activations)
+        self._out_work[slot] = [dist.isend(self._out_hdr[slot], self.next), dist.isend(self._out_act[slot], self.next)]
 
     def flush(self) -> None:
-        for works, _ in self._sent:
-            for w in works:
-                w.wait()
-        self._sent = []
+        for i, works in enumerate(self._out_work):
+            if works is not None:
+                for w in works:
+                    w.wait()
+                self._out_work[i] = None
 
     # ---- from the previous stage
     def post_recv(self) -> None:
-        """Start receiving the next wave's header; call it before computing the current wave."""
+        """Start receiving the next wave, header and activations; call it before computing the current wave so
+        that the transfer runs under the compute."""
         if self.prev is None:
             raise RuntimeError("the first stage has nothing to receive")
         if self._posted is None:
             slot = self._slot
-            self._posted = (slot, dist.irecv(self._hdr[slot], self.prev))
+            self._posted = (slot, dist.irecv(self._hdr[slot], self.prev), dist.irecv(self._act[slot], self.prev))
 
     def recv_wave(self):
         """(wave id, spans, activations) of the next wave; the activations are a view of a ring buffer that stays
-        valid until `depth - 1` further waves have been received."""
+        valid until `depth - 1` further receives have been posted."""
         self.post_recv()
-        slot, work = self._posted
-        work.wait()
+        slot, hdr_work, act_work = self._posted
+        hdr_work.wait()
+        act_work.wait()
         self._posted = None
         self._slot = (slot + 1) % len(self._hdr)
         hdr = self._hdr[slot].cpu()
@@ -116,7 +132,4 @@ class StageLink:
         if hidden != self.hidden or n > self.max_lanes or tokens > self._act[slot].shape[0]:
             raise ValueError("incoming wave does not fit the link")
         spans = [tuple(int(x) for x in hdr[4 + 3 * i:7 + 3 * i]) for i in range(n)]
-        act = self._act[slot][:tokens]
-        if tokens:
-            dist.recv(act, self.prev)
-        return wave_id, spans, act
+        return wave_id, spans, self._act[slot][:tokens]

@@ -28,15 +28,19 @@ def device_inputs(w, inp=None, device="cuda"):
 
 
 def run_wave(w, dev_inp, opts=None, sm_scale=0.0, want_lse=True, poison_out=True, do_append=True,
-             do_attention=True):
-    """plan -> H2D plan -> wpp_kv_append -> wpp_prefill_attention_varlen on the current stream."""
+             do_attention=True, launch_prefix_lens=None, launch_chunk_lens=None):
+    """plan -> H2D plan -> wpp_kv_append -> wpp_prefill_attention_varlen on the current stream.
+    launch_prefix_lens / launch_chunk_lens: device arrays the kernels get instead of the lengths the plan was made
+    for (a host-made mismatch)."""
     c = ctx()
     d = desc_of(w, sm_scale)
     plan = wpp.wpp_plan_tiles(c, d, w.prefix_lens, w.chunk_lens, opts=opts).to_device()
     dev = torch.device("cuda")
     bt = torch.from_numpy(w.block_tables).to(dev)
-    P = torch.from_numpy(w.prefix_lens).to(dev)
-    C = torch.from_numpy(w.chunk_lens).to(dev)
+    P = torch.from_numpy(np.asarray(w.prefix_lens if launch_prefix_lens is None else launch_prefix_lens,
+                                    dtype=np.int32)).to(dev)
+    C = torch.from_numpy(np.asarray(w.chunk_lens if launch_chunk_lens is None else launch_chunk_lens,
+                                    dtype=np.int32)).to(dev)
     status = torch.zeros(1, dtype=torch.int32, device=dev)
     T = w.total_new_tokens
     out = torch.empty(T, w.num_q_heads, w.head_dim, dtype=torch.bfloat16, device=dev)
@@ -85,3 +89,28 @@ def assert_close(gpu_out_f64, ref, what=""):
     assert e["mean_abs"] <= REL_MEAN_TOL * e["rms_ref"] + 1e-6, f"{what}: relative mean gate {e}"
     assert e["max_abs"] <= REL_MAX_TOL * e["max_ref"] + 2e-3, f"{what}: relative max gate {e}"
     return e
+
+
+# ---------------------------------------------------------------------------------------------------------------
+# Workloads whose pools are too large to copy to the host as a whole: the oracle gets one request at a time.
+def request_slice(w, dev_inp, i):
+    """Host copy of everything request `i` touches, as a one-request problem with a private pool.
+
+    The request's pages are gathered through its block-table row from the device pools (call this BEFORE the wave
+    runs: the append writes into those pages) and renumbered 0..n-1; q / k_new / v_new are the request's rows.
+    Returns a dict the oracle's entry points accept (bf16 CPU tensors, int32 arrays)."""
+    P, C = int(w.prefix_lens[i]), int(w.chunk_lens[i])
+    nb = (P + C + w.page_size - 1) // w.page_size
+    ids = torch.from_numpy(w.block_tables[i, :nb].astype(np.int64)).to(dev_inp["k_pool"].device)
+    off = w.q_offsets
+    r0, r1 = int(off[i]), int(off[i + 1])
+    return dict(q=dev_inp["q"][r0:r1].cpu(), k_new=dev_inp["k_new"][r0:r1].cpu(), v_new=dev_inp["v_new"][r0:r1].cpu(),
+                k_pool=dev_inp["k_pool"][ids].cpu(), v_pool=dev_inp["v_pool"][ids].cpu(),
+                block_tables=np.arange(nb, dtype=np.int32).reshape(1, nb),
+                prefix_lens=np.array([P], dtype=np.int32), chunk_lens=np.array([C], dtype=np.int32),
+                page_ids=ids, rows=(r0, r1))
+
+
+def appended_pages_of(dev_inp, sl):
+    """The request's pages as they are on the device now (after the wave), in the slice's numbering."""
+    return dev_inp["k_pool"][sl["page_ids"]], dev_inp["v_pool"][sl["page_ids"]]

@@ -227,6 +227,39 @@ def test_bad_page_id_sets_status_without_trapping():
     _full_parity(w2)
 
 
+@pytest.mark.parametrize("splits", [1, 2])
+def test_plan_launched_with_other_lengths_is_refused_per_request(splits):
+    """Section 4.6: a position mismatch fails execution instead of running against the wrong cache state.  The
+    plan is made for one set of spans; the device arrays are altered afterwards (on the host): the requests
+    whose span differs are refused - status WPP_ERR_PLAN_MISMATCH, none of their slots written, none of their
+    rows computed - the others run normally, nothing traps and the context stays usable."""
+    w = W.custom_workload([200, 128, 0, 300], [150, 260, 70, 129], 4, 2, 128, 64, seed=29, spare_pages=4)
+    inp = cpu_inputs(w)
+    P_dev = w.prefix_lens.copy()
+    C_dev = w.chunk_lens.copy()
+    P_dev[1] += 64          # this rank's cache of request 1 ends elsewhere
+    C_dev[3] -= 1           # request 3's span has another length
+    res = H.run_wave(w, H.device_inputs(w, inp), opts=wpp.PlanOpts(0, 0, splits, 0), launch_prefix_lens=P_dev,
+                     launch_chunk_lens=C_dev)
+    assert res["status"] == 6                                    # WPP_ERR_PLAN_MISMATCH
+    # the oracle's wave without the refused requests: their chunks are empty
+    C_ok = w.chunk_lens.copy()
+    C_ok[[1, 3]] = 0
+    off = w.q_offsets
+    keep = np.concatenate([np.arange(off[i], off[i + 1]) for i in (0, 2)])
+    kp, vp = oracle.oracle_append(inp["k_new"][keep], inp["v_new"][keep], inp["k_pool"], inp["v_pool"],
+                                  w.block_tables, w.prefix_lens, C_ok)
+    assert np.array_equal(bits(res["k_pool"]), kp), "a refused request's slots were written"
+    assert np.array_equal(bits(res["v_pool"]), vp)
+    ref, ref_lse = oracle.oracle_attention(inp["q"][keep], kp, vp, w.block_tables, w.prefix_lens, C_ok)
+    H.assert_close(f64(res["out"][keep]), ref, "requests whose spans agree")
+    for i in (1, 3):
+        rows = res["out"][off[i]:off[i + 1]].float()
+        # unsplit tiles leave the rows as the caller's poison; split tiles read as zero after the combine
+        assert bool((torch.isnan(rows) | (rows == 0)).all()), "a refused request's rows were computed"
+    _full_parity(W.custom_workload([64], [64], 2, 1, 128, 64, seed=17))      # the context still works
+
+
 def test_cfg2_sampled_rows():
     """Ragged batch of 16: the oracle checks a seeded sample of (request, row, head) plus boundary rows."""
     w = W.cfg2()
