@@ -496,8 +496,11 @@ def run_kda(args):
     ro, s_in, s_out = torch.from_numpy(w.row_offsets).to(dev), i32(w.state_in), i32(w.state_out)
     status = torch.zeros(1, dtype=torch.int32, device=dev)
     out = torch.empty((w.total_tokens, w.num_heads, w.d_v), dtype=torch.bfloat16, device=dev)
+    P_dev = i32(w.prefix_lens)
+    ws = torch.empty(wpp.wpp_kda_workspace_bytes(int(w.chunk_lens.size), w.num_heads, w.total_tokens), dtype=torch.uint8,
+                     device=dev) if args.kda_layout in (0, 3) else None
     step = lambda: wpp.wpp_kda_chunk(ctx, d["q"], d["k"], d["v"], d["alpha"], d["beta"], ro, d["state_pool"], s_in, s_out,
-                                     out=out, status=status, layout=args.kda_layout)
+                                     out=out, prefix_lens=P_dev, status=status, layout=args.kda_layout, workspace=ws)
     warm, steps = max(3, args.warmup), max(1, args.steps)
     for _ in range(warm):
         step()

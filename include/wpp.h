@@ -354,7 +354,12 @@ int wpp_hint_probe_recurrent(const wpp_hint_index* idx, int32_t window, const ui
  * with S (d_k x d_v, fp32) resumed from the state after exactly the reused prefix - a recurrent layer cannot
  * resume from anything else - and written back at the chunk end and, optionally, at sparse periodic boundaries.
  * Heads are independent.  No normalisation or scaling of q or k is applied here (the update has none).
- * Arithmetic: fp32 throughout (inputs widened, fp32 fused multiply-adds in token order), outputs rounded to bf16. */
+ * Two forms compute it.  The chunk-parallel form (layout 3) works on blocks of 64 sequence positions: per block the
+ * products Kt Kh^T, Qt Kh^T (Kt, Kh, Qt: keys and queries scaled by the decay products inside the block), Kt S_0,
+ * T (V - Kt S_0), Qt S_0, tril(Qt Kh^T) U and Kb^T U run on the tensor cores with the fp32 state in tensor memory;
+ * every operand is split into two bf16 terms (16 significant bits, three MMAs per product), accumulation is fp32.
+ * It needs a workspace (wpp_kda_workspace_bytes).  The token-by-token forms (layouts 1, 2) use fp32 fused
+ * multiply-adds on CUDA cores in token order and need no workspace.  Outputs are rounded to bf16, states stay fp32. */
 typedef struct {
     int32_t num_requests;   /* R >= 0 */
     int32_t num_heads;      /* H >= 1: state heads */
@@ -363,8 +368,10 @@ typedef struct {
     int32_t num_slots;      /* slots of state_pool, each H * d_k * d_v floats */
     int32_t snap_interval;  /* > 0: snapshot whenever the tokens folded into S reach a multiple of it; 0: none */
     int32_t max_snaps;      /* row length of snap_slots (0 when snap_interval is 0) */
-    int32_t layout;         /* 0: the library chooses; 1: one CTA per (request, head); 2: four CTAs per (request,
-                             * head), 32 columns each - a shorter token chain, chosen when 4 R H <= the SM count */
+    int32_t layout;         /* 0: the library chooses (the chunk-parallel form when a large enough workspace is given
+                             * and the wave has at least 64 tokens per request on average, else 1 or 2);
+                             * 1: token by token, one CTA per (request, head); 2: token by token, four CTAs per
+                             * (request, head) of 32 columns each; 3: chunk-parallel on the tensor cores */
     int64_t total_tokens;   /* T = row_offsets[R] */
 } wpp_kda_desc;
 
@@ -382,14 +389,23 @@ typedef struct {
  *   snap_slots  : device int32 [R, max_snaps] or NULL: slot for the n-th boundary inside the chunk, -1 = skip;
  *                 boundaries past max_snaps are skipped.
  *   out         : device bf16 [T, H, d_v].
+ *   workspace   : device scratch for the chunk-parallel form, 1024-byte aligned, wpp_kda_workspace_bytes(desc)
+ *                 bytes (about 160 KB per 64 tokens and head); may be NULL (0 bytes) for the other forms.  Contents
+ *                 are undefined afterwards; calls that may overlap on the GPU need a workspace each.
  *   status_dev  : device int32 or NULL; a slot id outside [-1, num_slots) sets it to WPP_ERR_BOUNDS (if it was 0)
  *                 and that request's state is neither read (zero state used) nor written there.
  * A request with an empty chunk copies state_in to state_out.  Returns WPP_ERR_INVALID_ARG for null or misaligned
- * pointers or negative sizes, WPP_ERR_UNSUPPORTED for d_k, d_v other than 128, WPP_ERR_CUDA for a launch failure. */
+ * pointers or negative sizes, WPP_ERR_UNSUPPORTED for d_k, d_v other than 128, WPP_ERR_WORKSPACE_TOO_SMALL when
+ * layout 3 is asked for without enough workspace, WPP_ERR_CUDA for a launch failure.  The chunk-parallel form
+ * enqueues three kernels (block offsets, per-block preparation, the chain over the blocks), the others one. */
 int wpp_kda_chunk(const wpp_ctx* ctx, const wpp_kda_desc* desc, const void* q, const void* k, const void* v,
                   const float* alpha, const float* beta, const int64_t* row_offsets, const int32_t* prefix_lens,
                   float* state_pool, const int32_t* state_in, const int32_t* state_out, const int32_t* snap_slots,
-                  void* out, int32_t* status_dev, void* cuda_stream);
+                  void* out, void* workspace, size_t workspace_bytes, int32_t* status_dev, void* cuda_stream);
+
+/* Bytes of workspace the chunk-parallel form of wpp_kda_chunk needs for a wave of this description (depends on
+ * num_requests, num_heads and total_tokens only); 0 for an invalid description. */
+size_t wpp_kda_workspace_bytes(const wpp_kda_desc* desc);
 
 #ifdef __cplusplus
 }

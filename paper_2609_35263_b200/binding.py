@@ -89,7 +89,7 @@ EXPORTS = ["wpp_create", "wpp_destroy", "wpp_status_string", "wpp_last_cuda_erro
            "wpp_selftest_bounded_wait", "wpp_wave_ladder", "wpp_plan_waves",
            "wpp_hash_blocks", "wpp_hash_blocks_host", "wpp_hint_index_create", "wpp_hint_index_destroy",
            "wpp_hint_index_add", "wpp_hint_index_remove", "wpp_hint_index_size", "wpp_hint_probe",
-           "wpp_hint_probe_recurrent", "wpp_kda_chunk"]
+           "wpp_hint_probe_recurrent", "wpp_kda_chunk", "wpp_kda_workspace_bytes"]
 
 _lib = None
 
@@ -140,7 +140,9 @@ def load_library() -> ctypes.CDLL:
         lib.wpp_wave_ladder.argtypes = [ctypes.POINTER(WaveConfig), vp, ctypes.c_int32, ctypes.POINTER(ctypes.c_int32)]
         lib.wpp_plan_waves.argtypes = [ctypes.POINTER(WaveConfig), ctypes.POINTER(WaveState), vp, ctypes.c_int32, vp,
                                        ctypes.c_int32, ctypes.c_int32, vp, ctypes.POINTER(WaveInfo)]
-        lib.wpp_kda_chunk.argtypes = [vp, ctypes.POINTER(KdaDesc)] + [vp] * 14
+        lib.wpp_kda_chunk.argtypes = [vp, ctypes.POINTER(KdaDesc)] + [vp] * 13 + [ctypes.c_size_t, vp, vp]
+        lib.wpp_kda_workspace_bytes.restype = ctypes.c_size_t
+        lib.wpp_kda_workspace_bytes.argtypes = [ctypes.POINTER(KdaDesc)]
         _lib = lib
     return _lib
 
@@ -432,15 +434,24 @@ class HintIndex:
         return int(m.value), int(p.value)
 
 
+def wpp_kda_workspace_bytes(num_requests: int, num_heads: int, total_tokens: int) -> int:
+    """Bytes of workspace the chunk-parallel (tensor-core) form of wpp_kda_chunk needs for such a wave."""
+    desc = KdaDesc(int(num_requests), int(num_heads), 128, 128, 0, 0, 0, 0, int(total_tokens))
+    return int(load_library().wpp_kda_workspace_bytes(ctypes.byref(desc)))
+
+
 def wpp_kda_chunk(ctx: Context, q, k, v, alpha, beta, row_offsets, state_pool, state_in, state_out, out=None,
-                  prefix_lens=None, snap_interval: int = 0, snap_slots=None, status=None, stream=None, layout: int = 0):
+                  prefix_lens=None, snap_interval: int = 0, snap_slots=None, status=None, stream=None, layout: int = 0,
+                  workspace=None):
     """Queue the recurrent-state (KDA) layer of one wave on `stream` (Section 3.1 update, Section 3.2 snapshots).
 
     q, k: cuda bf16 [T, H, 128]; v: cuda bf16 [T, H, 128]; alpha: cuda fp32 [T, H, 128]; beta: cuda fp32 [T, H];
     row_offsets: cuda int64 [R+1]; state_pool: cuda fp32 [slots, H, 128, 128] (updated in place); state_in,
     state_out: cuda int32 [R] (-1: zero state / do not store); snap_slots: cuda int32 [R, max_snaps] with
-    prefix_lens (cuda int32 [R]) and snap_interval > 0 for periodic snapshots; layout 0 lets the library choose
-    between one and four CTAs per (request, head).  Returns the cuda bf16 output."""
+    prefix_lens (cuda int32 [R]) and snap_interval > 0 for periodic snapshots.  layout 0 lets the library choose:
+    the chunk-parallel tensor-core form when `workspace` (cuda uint8, wpp_kda_workspace_bytes bytes, 1024-byte
+    aligned) is given and the chunks average 64 tokens or more, else a token-by-token form; 1, 2: token by token
+    with one / four CTAs per (request, head); 3: chunk-parallel.  Returns the cuda bf16 output."""
     T, H, dk = (int(x) for x in q.shape)
     dv = int(v.shape[2])
     R = int(row_offsets.numel()) - 1
@@ -448,8 +459,10 @@ def wpp_kda_chunk(ctx: Context, q, k, v, alpha, beta, row_offsets, state_pool, s
         out = torch.empty((T, H, dv), dtype=torch.bfloat16, device=q.device)
     max_snaps = 0 if snap_slots is None else int(snap_slots.shape[1])
     desc = KdaDesc(R, H, dk, dv, int(state_pool.shape[0]), int(snap_interval), max_snaps, int(layout), T)
+    ws_bytes = 0 if workspace is None else int(workspace.numel() * workspace.element_size())
     st = load_library().wpp_kda_chunk(ctx.handle, ctypes.byref(desc), _ptr(q), _ptr(k), _ptr(v), _ptr(alpha), _ptr(beta),
                                       _ptr(row_offsets), _ptr(prefix_lens), _ptr(state_pool), _ptr(state_in),
-                                      _ptr(state_out), _ptr(snap_slots), _ptr(out), _ptr(status), _stream(stream))
+                                      _ptr(state_out), _ptr(snap_slots), _ptr(out), _ptr(workspace), ws_bytes,
+                                      _ptr(status), _stream(stream))
     _check(st, "wpp_kda_chunk")
     return out

@@ -8,7 +8,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libwpp.so")
 SOURCES = ["wpp_plan.cpp", "wpp_waves.cpp", "wpp_hints.cu", "wpp_api.cu", "wpp_append_combine.cu", "wpp_attention.cu",
-           "wpp_kda.cu"]
+           "wpp_kda.cu", "wpp_kda_tc.cu"]
 HEADERS = ["wpp_host.h", "wpp_plan_format.h", "wpp_device.h", "wpp_ptx.cuh", os.path.join("..", "..", "include", "wpp.h")]
 
 
@@ -28,7 +28,7 @@ def is_stale() -> bool:
 
 
 def build(force: bool = False, verbose: bool = False, defines=(), out: str = None) -> str:
-    """Compile the library; `defines` (e.g. ["WPP_EMU_PAIRS_OF_4=2"]) and `out` build a tuning variant."""
+    """Compile the library; `defines` (a list of NAME=VALUE strings) and `out` build a variant beside it."""
     if out is None and not force and not is_stale():
         return LIB
     target = out or LIB

@@ -350,15 +350,43 @@ extern "C" int wpp_prefill_attention_varlen_static(const wpp_ctx* ctx, const wpp
                                         (size_t)WPP_STATIC_SCRATCH_BYTES, status_dev, cuda_stream);
 }
 
+// ---------------------------------------------------------------------------------------------------------------
+// Recurrent-state layer.  Workspace of the chunk-parallel form: block offsets, then per (block, head) the cut mask,
+// the decay products at sub-block ends and the ten operand arrays the preparation kernel leaves for the chain kernel.
+struct KdaWorkspace {
+    int64_t max_blocks, n_bh;
+    size_t off_blk, off_mask, off_e, off_op[6], off_sq[4], bytes;
+};
+static size_t up1k(size_t x) { return (x + 1023) / 1024 * 1024; }
+static KdaWorkspace kda_workspace(const wpp_kda_desc* d) {
+    KdaWorkspace w;
+    w.max_blocks = d->total_tokens / 64 + 2 * (int64_t)d->num_requests;      // a chunk of C tokens touches <= C/64 + 2 blocks
+    w.n_bh = w.max_blocks * d->num_heads;
+    size_t off = 0;
+    w.off_blk = off;  off += up1k(sizeof(int32_t) * ((size_t)d->num_requests + 1));
+    w.off_mask = off; off += up1k(sizeof(uint64_t) * (size_t)w.n_bh);
+    w.off_e = off;    off += up1k(sizeof(float) * (size_t)w.n_bh * 64 * 128);
+    for (int i = 0; i < 6; ++i) { w.off_op[i] = off; off += up1k(2 * (size_t)w.n_bh * 64 * 128); }
+    for (int i = 0; i < 4; ++i) { w.off_sq[i] = off; off += up1k(2 * (size_t)w.n_bh * 64 * 64); }
+    w.bytes = off;
+    return w;
+}
+static bool kda_desc_ok(const wpp_kda_desc* desc) {
+    return desc && desc->num_requests >= 0 && desc->num_heads >= 1 && desc->num_slots >= 0 && desc->snap_interval >= 0 &&
+           desc->max_snaps >= 0 && desc->total_tokens >= 0 && desc->layout >= 0 && desc->layout <= 3;
+}
+
+extern "C" size_t wpp_kda_workspace_bytes(const wpp_kda_desc* desc) {
+    if (!kda_desc_ok(desc)) return 0;
+    return kda_workspace(desc).bytes;
+}
+
 extern "C" int wpp_kda_chunk(const wpp_ctx* ctx, const wpp_kda_desc* desc, const void* q, const void* k, const void* v,
                              const float* alpha, const float* beta, const int64_t* row_offsets,
                              const int32_t* prefix_lens, float* state_pool, const int32_t* state_in,
-                             const int32_t* state_out, const int32_t* snap_slots, void* out, int32_t* status_dev,
-                             void* cuda_stream) {
-    if (!ctx || !desc) return WPP_ERR_INVALID_ARG;
-    if (desc->num_requests < 0 || desc->num_heads < 1 || desc->num_slots < 0 || desc->snap_interval < 0 ||
-        desc->max_snaps < 0 || desc->total_tokens < 0 || desc->layout < 0 || desc->layout > 2)
-        return WPP_ERR_INVALID_ARG;
+                             const int32_t* state_out, const int32_t* snap_slots, void* out, void* workspace,
+                             size_t workspace_bytes, int32_t* status_dev, void* cuda_stream) {
+    if (!ctx || !kda_desc_ok(desc)) return WPP_ERR_INVALID_ARG;
     if (desc->d_k != 128 || desc->d_v != 128) return WPP_ERR_UNSUPPORTED;
     if (desc->num_requests > 65535) return WPP_ERR_UNSUPPORTED;      // one grid row per request
     if (desc->num_requests == 0) return WPP_OK;
@@ -369,6 +397,69 @@ extern "C" int wpp_kda_chunk(const wpp_ctx* ctx, const wpp_kda_desc* desc, const
     if (desc->snap_interval > 0 && !prefix_lens) return WPP_ERR_INVALID_ARG;
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(alpha) || !aligned16(out) || !aligned16(state_pool))
         return WPP_ERR_INVALID_ARG;
+    // Which form: the chunk-parallel tensor-core form needs a workspace and pays off from about a block of tokens
+    // per request; the token-by-token forms need none.
+    const KdaWorkspace w = kda_workspace(desc);
+    bool tensor_form = desc->layout == 3;
+    if (desc->layout == 0)
+        tensor_form = workspace && workspace_bytes >= w.bytes && desc->total_tokens >= 64 * (int64_t)desc->num_requests;
+    if (tensor_form) {
+        if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 1023) != 0) return WPP_ERR_INVALID_ARG;
+        if (workspace_bytes < w.bytes) return WPP_ERR_WORKSPACE_TOO_SMALL;
+        if (w.n_bh * 64 > 0x7fffffffll || desc->total_tokens > 0x7fffffffll) return WPP_ERR_UNSUPPORTED;
+        char* ws = static_cast<char*>(workspace);
+        wpp::KdaTcParams p;
+        memset(&p, 0, sizeof(p));
+        p.q = static_cast<const __nv_bfloat16*>(q);
+        p.k = static_cast<const __nv_bfloat16*>(k);
+        p.v = static_cast<const __nv_bfloat16*>(v);
+        p.alpha = alpha;
+        p.beta = beta;
+        p.row_offsets = row_offsets;
+        p.prefix_lens = prefix_lens;
+        p.state_pool = state_pool;
+        p.state_in = state_in;
+        p.state_out = state_out;
+        p.snap_slots = desc->max_snaps > 0 ? snap_slots : nullptr;
+        p.out = static_cast<__nv_bfloat16*>(out);
+        p.status = status_dev;
+        p.num_requests = desc->num_requests;
+        p.num_heads = desc->num_heads;
+        p.num_slots = desc->num_slots;
+        p.snap_interval = desc->snap_interval;
+        p.max_snaps = desc->max_snaps;
+        p.blk_off = reinterpret_cast<int32_t*>(ws + w.off_blk);
+        p.ws_mask = reinterpret_cast<unsigned long long*>(ws + w.off_mask);
+        p.ws_e = reinterpret_cast<float*>(ws + w.off_e);
+        __nv_bfloat16** ops[6] = {&p.ws_kt_h, &p.ws_kt_l, &p.ws_qt_h, &p.ws_qt_l, &p.ws_kb_h, &p.ws_kb_l};
+        __nv_bfloat16** sqs[4] = {&p.ws_t_h, &p.ws_t_l, &p.ws_m_h, &p.ws_m_l};
+        CUtensorMap maps[11];
+        int rc;
+        for (int i = 0; i < 6; ++i) {
+            *ops[i] = reinterpret_cast<__nv_bfloat16*>(ws + w.off_op[i]);
+            const uint64_t dims[2] = {128, (uint64_t)w.n_bh * 64};
+            const uint64_t strides[1] = {256};
+            const uint32_t box[2] = {64, 64};
+            if ((rc = make_map(ctx, &maps[i], *ops[i], 2, dims, strides, box)) != WPP_OK) return rc;
+        }
+        for (int i = 0; i < 4; ++i) {
+            *sqs[i] = reinterpret_cast<__nv_bfloat16*>(ws + w.off_sq[i]);
+            const uint64_t dims[2] = {64, (uint64_t)w.n_bh * 64};
+            const uint64_t strides[1] = {128};
+            const uint32_t box[2] = {64, 64};
+            if ((rc = make_map(ctx, &maps[6 + i], *sqs[i], 2, dims, strides, box)) != WPP_OK) return rc;
+        }
+        {
+            const uint64_t dims[3] = {128, (uint64_t)desc->num_heads, (uint64_t)desc->total_tokens};
+            const uint64_t strides[2] = {256, (uint64_t)desc->num_heads * 256};
+            const uint32_t box[3] = {64, 1, 64};
+            if ((rc = make_map(ctx, &maps[10], v, 3, dims, strides, box)) != WPP_OK) return rc;
+        }
+        int e = wpp_launch_kda_tc(&p, maps, (int)w.max_blocks, cuda_stream);
+        if (e != 0) return cuda_fail(ctx, e);
+        const_cast<wpp_ctx*>(ctx)->launches += 3;
+        return WPP_OK;
+    }
     wpp::KdaParams p;
     memset(&p, 0, sizeof(p));
     p.q = static_cast<const __nv_bfloat16*>(q);

@@ -67,9 +67,34 @@ struct KdaParams {
     int32_t num_requests, num_heads, num_slots, snap_interval, max_snaps;
 };
 
+// Chunk-parallel (tensor-core) form of the recurrent layer: the inputs of KdaParams plus the workspace arrays the
+// preparation kernel fills for the chain kernel.  bh = (global block index) * num_heads + head.
+struct KdaTcParams {
+    const __nv_bfloat16* q;
+    const __nv_bfloat16* k;
+    const __nv_bfloat16* v;
+    const float* alpha;
+    const float* beta;
+    const int64_t* row_offsets;
+    const int32_t* prefix_lens;
+    float* state_pool;
+    const int32_t* state_in;
+    const int32_t* state_out;
+    const int32_t* snap_slots;
+    __nv_bfloat16* out;
+    int32_t* status;
+    int32_t num_requests, num_heads, num_slots, snap_interval, max_snaps;
+    int32_t* blk_off;               // [R+1] exclusive scan of the requests' block counts
+    unsigned long long* ws_mask;    // [bh] bit t: token t of the block starts a sub-block
+    float* ws_e;                    // [bh][64][128] decay product at a sub-block's last token (other rows unused)
+    __nv_bfloat16 *ws_kt_h, *ws_kt_l, *ws_qt_h, *ws_qt_l, *ws_kb_h, *ws_kb_l;   // [bh][64][128]
+    __nv_bfloat16 *ws_t_h, *ws_t_l, *ws_m_h, *ws_m_l;                           // [bh][64][64]
+};
+
 }  // namespace wpp
 
 extern "C" {
+int wpp_launch_kda_tc(const wpp::KdaTcParams* p, const CUtensorMap* maps, int max_blocks, void* stream);
 int wpp_launch_attention(int head_dim, const CUtensorMap* tq, const CUtensorMap* tk, const CUtensorMap* tv,
                          const wpp::AttnParams* p, int num_ctas, void* stream);
 int wpp_launch_append(const wpp::AppendParams* p, int num_sms, void* stream);

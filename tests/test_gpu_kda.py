@@ -1,8 +1,10 @@
 """wpp_kda_chunk (CUDA, through the C ABI) against the fp64 oracle of the recurrent-state layer (Section 3.1 update,
 Section 3.2 snapshots), element by element on seeded inputs, plus the properties that hold at any size.
 
-Tolerances: the kernel computes in fp32 (relative error of a step about 1e-7, a few 1e-6 after thousands of
-contracting steps) and rounds outputs to bf16 (relative 2^-9); states stay fp32.
+Tolerances: the token-by-token forms (layouts 1, 2) compute in fp32 (relative error of a step about 1e-7, a few
+1e-6 after thousands of contracting steps); the chunk-parallel tensor-core form (layout 3) multiplies operands of
+16 significant bits (two bf16 terms each, relative 2^-17 per factor) and accumulates in fp32, so a product of 64 or
+128 terms carries about 1e-5 of its typical term; all forms round outputs to bf16 (relative 2^-9), states stay fp32.
   outputs : |delta| <= 2^-8 |ref| + 1e-4 max|ref|          states : |delta| <= 1e-4 max|ref|"""
 import numpy as np
 import pytest
@@ -30,12 +32,14 @@ def _gpu(w, t, state_in=None, state_out=None, layout=0):
     d = {k: v.to(dev) for k, v in t.items()}
     i32 = lambda a: None if a is None else torch.from_numpy(np.ascontiguousarray(a, dtype=np.int32)).to(dev)
     status = torch.zeros(1, dtype=torch.int32, device=dev)
+    T, Hh = int(t["q"].shape[0]), int(t["q"].shape[1])
+    ws = torch.full((wpp.wpp_kda_workspace_bytes(len(w.chunk_lens), Hh, T),), 0xFF, dtype=torch.uint8, device=dev)
     out = wpp.wpp_kda_chunk(H.ctx(), d["q"], d["k"], d["v"], d["alpha"], d["beta"],
                             torch.from_numpy(w.row_offsets).to(dev), d["state_pool"],
                             i32(w.state_in if state_in is None else state_in),
                             i32(w.state_out if state_out is None else state_out),
                             prefix_lens=i32(w.prefix_lens), snap_interval=w.snap_interval,
-                            snap_slots=i32(w.snap_slots), status=status, layout=layout)
+                            snap_slots=i32(w.snap_slots), status=status, layout=layout, workspace=ws)
     torch.cuda.synchronize()
     return out.float().cpu().double().numpy(), d["state_pool"].cpu().double().numpy(), int(status.item())
 
@@ -57,7 +61,7 @@ def _close_state(got, ref, what):
     ([300], [0], 0, 3),                                                            # one request from the zero state
     ([15, 16, 17, 31, 32, 33], [1, 2, 3, 4, 5, 6], 7, 1),                          # around the staging size; odd interval
 ])
-@pytest.mark.parametrize("layout", [1, 2])          # one CTA per (request, head) / four column slices
+@pytest.mark.parametrize("layout", [1, 2, 3])       # one CTA per (request, head) / four column slices / chunk-parallel
 def test_ragged_batches_match_the_oracle(lens, prefix, interval, H_, layout):
     w = W.kda_workload("ragged", 11, lens, H_, prefix, snap_interval=interval)
     t = w.tensors()
@@ -75,7 +79,7 @@ def test_ragged_batches_match_the_oracle(lens, prefix, interval, H_, layout):
             assert np.array_equal(got_pool[s], t["state_pool"][s].double().numpy())
 
 
-@pytest.mark.parametrize("layout", [1, 2])
+@pytest.mark.parametrize("layout", [1, 2, 3])
 def test_a_long_chain_stays_within_tolerance(layout):
     w = W.kda_workload("long", 5, [2048], 1, [4096])
     t = w.tensors()
@@ -86,11 +90,12 @@ def test_a_long_chain_stays_within_tolerance(layout):
     _close_state(got_pool, ref_pool, "state pool")
 
 
-@pytest.mark.parametrize("layout", [1, 2])
-@pytest.mark.parametrize("cut", [(64, 32), (37, 20)])
+@pytest.mark.parametrize("layout,cut", [(1, (64, 32)), (1, (37, 20)), (2, (64, 32)), (2, (37, 20)), (3, (59, 64))])
 def test_splitting_a_chunk_and_resuming_is_bit_identical(layout, cut):
-    """Section 3.2: the state after exactly r tokens is all a recurrent layer needs; the kernel's arithmetic per
-    token does not depend on where a chunk starts, so one call and two resumed calls agree to the bit."""
+    """Section 3.2: the state after exactly r tokens is all a recurrent layer needs.  The token-by-token forms'
+    arithmetic per token does not depend on where a chunk starts, so one call and two resumed calls agree to the bit
+    for any cut; the chunk-parallel form works on blocks of 64 sequence positions, so it does for cuts at multiples
+    of 64 (request 0 has 5 cached tokens: its cut after 59 tokens is position 64)."""
     w = W.kda_workload("whole", 3, [100, 64], 2, [5, 0], resume=[True, False])
     t = w.tensors()
     whole_o, whole_pool, _ = _gpu(w, t, layout=layout)
@@ -101,7 +106,7 @@ def test_splitting_a_chunk_and_resuming_is_bit_identical(layout, cut):
         lens = [cut[i] if first else int(w.chunk_lens[i]) - cut[i] for i in range(2)]
         sel = np.concatenate([np.arange(rows[i] + (0 if first else cut[i]), rows[i] + (cut[i] if first else w.chunk_lens[i]))
                               for i in range(2)])
-        wp = W.kda_workload("part", 3, lens, 2, [5, 0])
+        wp = W.kda_workload("part", 3, lens, 2, [5, 0] if first else [5 + cut[0], cut[1]])
         wp.num_slots = w.num_slots
         tp = {k: (v[sel].contiguous() if k != "state_pool" else pool) for k, v in t.items()}
         s_in = w.state_in if first else w.state_out          # the second call resumes from what the first stored
@@ -113,7 +118,32 @@ def test_splitting_a_chunk_and_resuming_is_bit_identical(layout, cut):
     assert np.array_equal(pool.double().numpy(), whole_pool)
 
 
-@pytest.mark.parametrize("layout", [1, 2])
+def test_splitting_inside_a_block_stays_within_tolerance_in_the_chunk_parallel_form():
+    """A cut that is not a multiple of 64 moves a block boundary of the chunk-parallel form: the two resumed calls
+    then round differently from the single call, and both stay within the tolerances against the oracle."""
+    w = W.kda_workload("whole", 3, [100, 64], 2, [5, 0], resume=[True, False])
+    t = w.tensors()
+    ref_o, ref_pool = _oracle(w, t)
+    rows, cut = w.row_offsets, (37, 20)
+    parts_o = np.zeros_like(ref_o)
+    pool = t["state_pool"].clone()
+    for first in (True, False):
+        lens = [cut[i] if first else int(w.chunk_lens[i]) - cut[i] for i in range(2)]
+        sel = np.concatenate([np.arange(rows[i] + (0 if first else cut[i]), rows[i] + (cut[i] if first else w.chunk_lens[i]))
+                              for i in range(2)])
+        wp = W.kda_workload("part", 3, lens, 2, [5, 0] if first else [5 + cut[0], cut[1]])
+        wp.num_slots = w.num_slots
+        tp = {k: (v[sel].contiguous() if k != "state_pool" else pool) for k, v in t.items()}
+        o, new_pool, status = _gpu(wp, tp, state_in=w.state_in if first else w.state_out, state_out=w.state_out, layout=3)
+        assert status == 0
+        parts_o[sel] = o
+        pool = torch.from_numpy(new_pool).float()
+    _close_out(parts_o, ref_o, "outputs of the two resumed calls")
+    for i in range(2):
+        _close_state(pool[w.state_out[i]].double().numpy(), ref_pool[w.state_out[i]], "final state")
+
+
+@pytest.mark.parametrize("layout", [1, 2, 3])
 def test_tiny_and_zero_decays(layout):
     """Decays of exactly 0 (a channel forgets everything), of 1e-6 and 1e-20, and runs of small ones."""
     w = W.kda_workload("decays", 17, [90, 40], 2, [3, 0])
@@ -133,7 +163,7 @@ def test_tiny_and_zero_decays(layout):
     _close_state(got_pool, ref_pool, "state pool")
 
 
-@pytest.mark.parametrize("layout", [1, 2])
+@pytest.mark.parametrize("layout", [1, 2, 3])
 def test_in_place_slots_and_pure_decay(layout):
     # state_out == state_in updates a slot in place; with beta = 0 and alpha = 1 the state must not change at all
     w = W.kda_workload("inplace", 9, [50, 20], 2, [10, 10])
