@@ -355,7 +355,7 @@ extern "C" int wpp_prefill_attention_varlen_static(const wpp_ctx* ctx, const wpp
 // the decay products at sub-block ends and the ten operand arrays the preparation kernel leaves for the chain kernel.
 struct KdaWorkspace {
     int64_t max_blocks, n_bh;
-    size_t off_blk, off_mask, off_e, off_op[6], off_sq[4], bytes;
+    size_t off_blk, off_mask, off_e, off_u0, off_op[6], off_sq[2], bytes;
 };
 static size_t up1k(size_t x) { return (x + 1023) / 1024 * 1024; }
 static KdaWorkspace kda_workspace(const wpp_kda_desc* d) {
@@ -366,8 +366,9 @@ static KdaWorkspace kda_workspace(const wpp_kda_desc* d) {
     w.off_blk = off;  off += up1k(sizeof(int32_t) * ((size_t)d->num_requests + 1));
     w.off_mask = off; off += up1k(sizeof(uint64_t) * (size_t)w.n_bh);
     w.off_e = off;    off += up1k(sizeof(float) * (size_t)w.n_bh * 64 * 128);
+    w.off_u0 = off;   off += up1k(sizeof(float) * (size_t)w.n_bh * 64 * 128);
     for (int i = 0; i < 6; ++i) { w.off_op[i] = off; off += up1k(2 * (size_t)w.n_bh * 64 * 128); }
-    for (int i = 0; i < 4; ++i) { w.off_sq[i] = off; off += up1k(2 * (size_t)w.n_bh * 64 * 64); }
+    for (int i = 0; i < 2; ++i) { w.off_sq[i] = off; off += up1k(2 * (size_t)w.n_bh * 64 * 64); }
     w.bytes = off;
     return w;
 }
@@ -431,9 +432,10 @@ extern "C" int wpp_kda_chunk(const wpp_ctx* ctx, const wpp_kda_desc* desc, const
         p.blk_off = reinterpret_cast<int32_t*>(ws + w.off_blk);
         p.ws_mask = reinterpret_cast<unsigned long long*>(ws + w.off_mask);
         p.ws_e = reinterpret_cast<float*>(ws + w.off_e);
-        __nv_bfloat16** ops[6] = {&p.ws_kt_h, &p.ws_kt_l, &p.ws_qt_h, &p.ws_qt_l, &p.ws_kb_h, &p.ws_kb_l};
-        __nv_bfloat16** sqs[4] = {&p.ws_t_h, &p.ws_t_l, &p.ws_m_h, &p.ws_m_l};
-        CUtensorMap maps[11];
+        p.ws_u0 = reinterpret_cast<float*>(ws + w.off_u0);
+        __nv_bfloat16** ops[6] = {&p.ws_w0_h, &p.ws_w0_l, &p.ws_qt_h, &p.ws_qt_l, &p.ws_kb_h, &p.ws_kb_l};
+        __nv_bfloat16** sqs[2] = {&p.ws_m_h, &p.ws_m_l};
+        CUtensorMap maps[8];
         int rc;
         for (int i = 0; i < 6; ++i) {
             *ops[i] = reinterpret_cast<__nv_bfloat16*>(ws + w.off_op[i]);
@@ -442,18 +444,12 @@ extern "C" int wpp_kda_chunk(const wpp_ctx* ctx, const wpp_kda_desc* desc, const
             const uint32_t box[2] = {64, 64};
             if ((rc = make_map(ctx, &maps[i], *ops[i], 2, dims, strides, box)) != WPP_OK) return rc;
         }
-        for (int i = 0; i < 4; ++i) {
+        for (int i = 0; i < 2; ++i) {
             *sqs[i] = reinterpret_cast<__nv_bfloat16*>(ws + w.off_sq[i]);
             const uint64_t dims[2] = {64, (uint64_t)w.n_bh * 64};
             const uint64_t strides[1] = {128};
             const uint32_t box[2] = {64, 64};
             if ((rc = make_map(ctx, &maps[6 + i], *sqs[i], 2, dims, strides, box)) != WPP_OK) return rc;
-        }
-        {
-            const uint64_t dims[3] = {128, (uint64_t)desc->num_heads, (uint64_t)desc->total_tokens};
-            const uint64_t strides[2] = {256, (uint64_t)desc->num_heads * 256};
-            const uint32_t box[3] = {64, 1, 64};
-            if ((rc = make_map(ctx, &maps[10], v, 3, dims, strides, box)) != WPP_OK) return rc;
         }
         int e = wpp_launch_kda_tc(&p, maps, (int)w.max_blocks, cuda_stream);
         if (e != 0) return cuda_fail(ctx, e);

@@ -87,8 +87,9 @@ struct KdaTcParams {
     int32_t* blk_off;               // [R+1] exclusive scan of the requests' block counts
     unsigned long long* ws_mask;    // [bh] bit t: token t of the block starts a sub-block
     float* ws_e;                    // [bh][64][128] decay product at a sub-block's last token (other rows unused)
-    __nv_bfloat16 *ws_kt_h, *ws_kt_l, *ws_qt_h, *ws_qt_l, *ws_kb_h, *ws_kb_l;   // [bh][64][128]
-    __nv_bfloat16 *ws_t_h, *ws_t_l, *ws_m_h, *ws_m_l;                           // [bh][64][64]
+    __nv_bfloat16 *ws_w0_h, *ws_w0_l, *ws_qt_h, *ws_qt_l, *ws_kb_h, *ws_kb_l;   // [bh][64][128] hi / lo bf16 terms
+    __nv_bfloat16 *ws_m_h, *ws_m_l;                                             // [bh][64][64]
+    float* ws_u0;                                                               // [bh][64][128]
 };
 
 }  // namespace wpp

@@ -6,13 +6,15 @@
 //     u_t  = beta_t (v_t - (Diag(alpha_t) S_{t-1})^T k_t)                       so that S_t = Diag(alpha_t) S_{t-1} + k_t u_t^T
 //     S_t  = Diag(G_t) S_0' + sum_{s <= t} Diag(G_t / G_s) k_s u_s^T
 // and, with Kt = K o G (rows k_t o G_t), Kh = K / G, Qt = Q o G, Kb = Kh o G_{b-1}:
-//     A = tril(diag(beta) Kt Kh^T, -1),   (I + A) U = diag(beta) (V - Kt S_0'),   i.e.  U = T (V - Kt S_0'),  T = (I + A)^-1 diag(beta)
-//     O = Qt S_0' + tril(Qt Kh^T) U,       S_b = Diag(G_{b-1}) S_0' + Kb^T U.
-// Everything that does not involve the state is computed for all blocks in parallel by the PREPARATION kernel
-// (one CTA per 64-token block and head: decay products, Kt, Kh, Qt, Kb, the products Kt Kh^T and Qt Kh^T on the tensor
-// cores, the inverse of the unit lower triangular 64 x 64 matrix on CUDA cores) and left in a workspace; the CHAIN
-// kernel (one CTA per request and head) then walks the blocks in order with five tensor-core products per block
-// (Kt S_0', T (V - W), Qt S_0', M U, Kb^T U) and the 128 x 128 fp32 state resident in tensor memory.
+//     A = tril(diag(beta) Kt Kh^T, -1),   (I + A) U = diag(beta) (V - Kt S_0'),   T = (I + A)^-1 diag(beta),
+//     U = U0 - W0 S_0'   with   U0 = T V,  W0 = T Kt   (neither depends on the state),
+//     O = Qt S_0' + M U  with   M = tril(Qt Kh^T),       S_b = Diag(G_{b-1}) S_0' + Kb^T U.
+// Everything that does not involve the state is computed for all blocks in parallel by the PREPARATION kernel (one
+// CTA per 64-token block and head: decay products, Kt, Kh, Qt, Kb, the products Kt Kh^T, Qt Kh^T, T Kt and T V on the
+// tensor cores, the inverse of the unit lower triangular 64 x 64 matrix on CUDA cores) and left in a workspace; the
+// CHAIN kernel (one CTA per request and head) then walks the blocks in order with four tensor-core products per
+// block (W0 S_0', Qt S_0', M U, Kb^T U) and the 128 x 128 fp32 state resident in tensor memory.  Per block the
+// chain from state to state is: scale and split the state, one product, form and split U, one product.
 //
 // Precision.  The state must stay within 1e-4 of its largest element, which single bf16 operands (8 significant
 // bits) cannot give.  Every operand is therefore split into two bf16 terms, x = hi + lo with hi = bf16(x) and lo =
@@ -23,11 +25,13 @@
 // position reproduces the unsplit result bit for bit).  A block is cut into sub-blocks, processed as steps of
 // their own, wherever the state is needed (a periodic snapshot) and wherever a channel's decay product inside the
 // block would fall below 2^-40: the token that causes it starts a new sub-block, where its own alpha is applied to
-// the state directly instead of through a quotient G_t / G_s.  Decays of exactly 0 are therefore exact.
+// the state directly instead of through a quotient G_t / G_s.  Decays of exactly 0 are therefore exact.  (T and M
+// are block diagonal over the sub-blocks, so one set of operands serves all steps of a block; a step zeroes the
+// rows of U outside its own tokens.)
 //
 // Orientation on the tensor cores: everything is kept transposed, with the value dimension d_v = 128 on the 128
-// rows (tensor-memory lanes): S^T [d_v x d_k], W^T = S_0'^T Kt^T [d_v x 64], U^T = (V - W)^T T^T, O^T = S_0'^T Qt^T +
-// U^T M^T, S_b^T = Diag-scaled S_0'^T + U^T Kb.  Thread r of the chain warps owns row r: column r of the state.
+// rows (tensor-memory lanes): S^T [d_v x d_k], X^T = S_0'^T W0^T [d_v x 64], O^T = S_0'^T Qt^T + U^T M^T,
+// S_b^T = Diag-scaled S_0'^T + U^T Kb.  Thread r of a row warpgroup owns row r: column r of the state.
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
@@ -125,27 +129,35 @@ __global__ void __launch_bounds__(1024) kda_tc_setup_kernel(const KdaTcParams p)
 }
 
 // ---------------------------------------------------------------------------------------------------------------
-// Preparation: one CTA (128 threads) per (block, head).
+// Preparation: one CTA (128 threads) per (block, head).  Shared memory is three regions of 32 KB that change roles:
+//   R0: alpha, then the decay products G (fp32 [64][128]); then Qt as an MMA operand; then T (hi tile, lo tile) and,
+//       behind them, the inverse it is made from
+//   R1: Kt as an MMA operand (A of Kt Kh^T, later B of T Kt)
+//   R2: Kh as an MMA operand; then the triangular matrix (fp32 [64][64]) and the V tile
+// An operand tile has 64 rows (tokens); as the A operand of a 128-row MMA its rows 64.. are whatever follows it in
+// shared memory: those rows of the result are never read.
 struct PrepSmem {
-    static constexpr int kOffG = 0;                          // fp32 [64][128]: alpha, then decay products
-    static constexpr int kOffA = kOffG + kL * kD * 4;        // Kt (later Qt) as MMA operand: hi0 hi1 lo0 lo1 tiles
-    static constexpr int kOffB = kOffA + 4 * kTileBytes;     // Kh: hi0 hi1 lo0 lo1; later the triangular matrix (fp32)
-    static constexpr int kOffMisc = kOffB + 4 * kTileBytes;  // beta[64], barrier, tmem slot, reduction scratch
-    static constexpr int kBytes = kOffMisc + 1024 + 1024;    // + alignment slack
+    static constexpr int kOffR0 = 0;
+    static constexpr int kOffR1 = kOffR0 + 4 * kTileBytes;
+    static constexpr int kOffR2 = kOffR1 + 4 * kTileBytes;
+    static constexpr int kOffMisc = kOffR2 + 4 * kTileBytes;  // beta[64], reduction scratch, tmem slot, barrier
+    static constexpr int kBytes = kOffMisc + 1024 + 1024;     // + alignment slack
 };
 
 __global__ void __launch_bounds__(128) kda_tc_prep_kernel(const KdaTcParams p) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* sm = smem_raw + (base - smem_u32(smem_raw));
-    float* G = reinterpret_cast<float*>(sm + PrepSmem::kOffG);
-    uint8_t* tileA = sm + PrepSmem::kOffA;
-    uint8_t* tileB = sm + PrepSmem::kOffB;
+    float* G = reinterpret_cast<float*>(sm + PrepSmem::kOffR0);
+    uint8_t* r0 = sm + PrepSmem::kOffR0;
+    uint8_t* r1 = sm + PrepSmem::kOffR1;
+    uint8_t* r2 = sm + PrepSmem::kOffR2;
     float* s_beta = reinterpret_cast<float*>(sm + PrepSmem::kOffMisc);              // [64]
     int* s_red = reinterpret_cast<int*>(sm + PrepSmem::kOffMisc + 256);             // [4]
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(sm + PrepSmem::kOffMisc + 512);
     volatile uint32_t* abort_flag = tmem_slot + 1;
     const uint32_t bar = base + PrepSmem::kOffMisc + 528;
+    const uint32_t a0 = base + PrepSmem::kOffR0, a1 = base + PrepSmem::kOffR1, a2 = base + PrepSmem::kOffR2;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int head = blockIdx.y, H = p.num_heads, R = p.num_requests;
@@ -162,6 +174,7 @@ __global__ void __launch_bounds__(128) kda_tc_prep_kernel(const KdaTcParams p) {
     const int t_lo = max(0, g.P - blk * kL), t_hi = min(kL, g.P + g.C - blk * kL);     // active tokens [t_lo, t_hi)
     const int64_t row_t0 = g.row0 + ((int64_t)blk * kL - g.P);                         // row of token 0 (may be < 0)
     const size_t bh = (size_t)gb * H + head;
+    const size_t tile_elems = (size_t)kL * kD;
 
     if (tid == 0) {
         mbar_init(bar, 1);
@@ -169,7 +182,7 @@ __global__ void __launch_bounds__(128) kda_tc_prep_kernel(const KdaTcParams p) {
         fence_barrier_init();
     }
     if (warp == 0) {
-        tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), 128);
+        tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), 256);
         tmem_relinquish();
     }
     // ---- alpha and beta of the block (inactive tokens: alpha 1, beta 0)
@@ -224,188 +237,287 @@ __global__ void __launch_bounds__(128) kda_tc_prep_kernel(const KdaTcParams p) {
     if (tid == 0) p.ws_mask[bh] = mask;
     __syncthreads();
 
-    // ---- Kt = k G, Kh = k / G, Kb = Kh G_end as hi/lo bf16: Kt and Kh to shared memory (MMA operands), Kt and Kb
-    //      to the workspace.  A thread handles 8 consecutive channels of a token at a time.
-    const size_t tile_elems = (size_t)kL * kD;
+    // ---- Kt = k G, Kh = k / G, Kb = Kh G_end, Qt = q G as hi/lo bf16.  Kt and Kh go to shared memory (MMA operands), Kb
+    //      and Qt to the workspace; Qt also waits in registers for the region the decay products occupy.  A thread handles
+    //      8 consecutive channels of a token at a time.
+    uint4 qt_h[8], qt_l[8];
+#pragma unroll
     for (int it = 0; it < 8; ++it) {
         const int item = it * 128 + tid, t = item >> 4, ch = item & 15, c0 = ch * 8;
         const bool active = t >= t_lo && t < t_hi;
         uint4 kt_h = make_uint4(0, 0, 0, 0), kt_l = kt_h, kh_h = kt_h, kh_l = kt_h, kb_h = kt_h, kb_l = kt_h;
+        qt_h[it] = kt_h; qt_l[it] = kt_h;
         if (active) {
             const uint4 raw = *reinterpret_cast<const uint4*>(p.k + ((row_t0 + t) * H + head) * kD + c0);
+            const uint4 rawq = *reinterpret_cast<const uint4*>(p.q + ((row_t0 + t) * H + head) * kD + c0);
             const int e_t = sub_end(mask, t, t_hi) - 1;
-            const uint32_t rw[4] = {raw.x, raw.y, raw.z, raw.w};
-            uint32_t o[6][4];
+            const uint32_t rw[4] = {raw.x, raw.y, raw.z, raw.w}, rq[4] = {rawq.x, rawq.y, rawq.z, rawq.w};
+            uint32_t o[8][4];
 #pragma unroll
             for (int w = 0; w < 4; ++w) {
                 const float k0 = __uint_as_float(rw[w] << 16), k1 = __uint_as_float(rw[w] & 0xffff0000u);
+                const float q0 = __uint_as_float(rq[w] << 16), q1 = __uint_as_float(rq[w] & 0xffff0000u);
                 const float g0 = G[t * kD + c0 + 2 * w], g1 = G[t * kD + c0 + 2 * w + 1];
                 const float e0 = G[e_t * kD + c0 + 2 * w], e1 = G[e_t * kD + c0 + 2 * w + 1];
+                const float i0 = __frcp_rn(g0), i1 = __frcp_rn(g1);       // g >= 2^-40: finite
                 split2(k0 * g0, k1 * g1, o[0][w], o[1][w]);
-                split2(k0 / g0, k1 / g1, o[2][w], o[3][w]);
-                split2(k0 * (e0 / g0), k1 * (e1 / g1), o[4][w], o[5][w]);
+                split2(k0 * i0, k1 * i1, o[2][w], o[3][w]);
+                split2(k0 * (e0 * i0), k1 * (e1 * i1), o[4][w], o[5][w]);
+                split2(q0 * g0, q1 * g1, o[6][w], o[7][w]);
             }
             kt_h = make_uint4(o[0][0], o[0][1], o[0][2], o[0][3]); kt_l = make_uint4(o[1][0], o[1][1], o[1][2], o[1][3]);
             kh_h = make_uint4(o[2][0], o[2][1], o[2][2], o[2][3]); kh_l = make_uint4(o[3][0], o[3][1], o[3][2], o[3][3]);
             kb_h = make_uint4(o[4][0], o[4][1], o[4][2], o[4][3]); kb_l = make_uint4(o[5][0], o[5][1], o[5][2], o[5][3]);
+            qt_h[it] = make_uint4(o[6][0], o[6][1], o[6][2], o[6][3]); qt_l[it] = make_uint4(o[7][0], o[7][1], o[7][2], o[7][3]);
         }
         const uint32_t off = (uint32_t)((ch >> 3) * kTileBytes) + sw_off(t, ch & 7);
-        *reinterpret_cast<uint4*>(tileA + off) = kt_h;
-        *reinterpret_cast<uint4*>(tileA + 2 * kTileBytes + off) = kt_l;
-        *reinterpret_cast<uint4*>(tileB + off) = kh_h;
-        *reinterpret_cast<uint4*>(tileB + 2 * kTileBytes + off) = kh_l;
+        *reinterpret_cast<uint4*>(r1 + off) = kt_h;
+        *reinterpret_cast<uint4*>(r1 + 2 * kTileBytes + off) = kt_l;
+        *reinterpret_cast<uint4*>(r2 + off) = kh_h;
+        *reinterpret_cast<uint4*>(r2 + 2 * kTileBytes + off) = kh_l;
         const size_t go = bh * tile_elems + (size_t)t * kD + c0;
-        *reinterpret_cast<uint4*>(p.ws_kt_h + go) = kt_h;
-        *reinterpret_cast<uint4*>(p.ws_kt_l + go) = kt_l;
         *reinterpret_cast<uint4*>(p.ws_kb_h + go) = kb_h;
         *reinterpret_cast<uint4*>(p.ws_kb_l + go) = kb_l;
+        *reinterpret_cast<uint4*>(p.ws_qt_h + go) = qt_h[it];
+        *reinterpret_cast<uint4*>(p.ws_qt_l + go) = qt_l[it];
+    }
+    __syncthreads();                       // every read of the decay products is done: Qt takes their place
+#pragma unroll
+    for (int it = 0; it < 8; ++it) {
+        const int item = it * 128 + tid, t = item >> 4, ch = item & 15;
+        const uint32_t off = (uint32_t)((ch >> 3) * kTileBytes) + sw_off(t, ch & 7);
+        *reinterpret_cast<uint4*>(r0 + off) = qt_h[it];
+        *reinterpret_cast<uint4*>(r0 + 2 * kTileBytes + off) = qt_l[it];
     }
     fence_proxy_async_smem();
     __syncthreads();
 
-    // D[128 x 64] (rows 64.. are never read: the A tiles have 64 rows, the rows after them are whatever follows in
-    // shared memory) = A (hi + lo) x B (hi + lo)^T without the lo x lo term
-    constexpr uint32_t idesc = idesc_bf16(64, 0, 0);
-    auto issue_product = [&](uint32_t d_col) {
-        const uint32_t a_hi = base + PrepSmem::kOffA, a_lo = a_hi + 2 * kTileBytes;
-        const uint32_t b_hi = base + PrepSmem::kOffB, b_lo = b_hi + 2 * kTileBytes;
-        const uint32_t aa[3] = {a_hi, a_hi, a_lo}, bb[3] = {b_hi, b_lo, b_hi};
-        bool first = true;
+    // ---- Kt Kh^T -> columns [0, 64), Qt Kh^T -> columns [64, 128): (hi + lo)(hi + lo)^T without the lo x lo term
+    if (tid == 0) {
+        tc_fence_after();
+        constexpr uint32_t idesc = idesc_bf16(64, 0, 0);
+        const uint32_t aa_base[2] = {a1, a0};
 #pragma unroll
-        for (int term = 0; term < 3; ++term) {
-            const uint64_t ad = smem_desc_sw128(aa[term], 16, 1024), bd = smem_desc_sw128(bb[term], 16, 1024);
+        for (int prod = 0; prod < 2; ++prod) {
+            const uint32_t a_hi = aa_base[prod], a_lo = a_hi + 2 * kTileBytes, b_hi = a2, b_lo = a2 + 2 * kTileBytes;
+            const uint32_t aa[3] = {a_hi, a_hi, a_lo}, bb[3] = {b_hi, b_lo, b_hi};
 #pragma unroll
-            for (int kk = 0; kk < 8; ++kk) {
-                const uint64_t off = (uint64_t)(((kk >> 2) * kTileBytes + (kk & 3) * 32) >> 4);
-                mma_ss(tmem + d_col, ad + off, bd + off, idesc, first ? 0u : 1u);
-                first = false;
+            for (int term = 0; term < 3; ++term) {
+                const uint64_t ad = smem_desc_sw128(aa[term], 16, 1024), bd = smem_desc_sw128(bb[term], 16, 1024);
+#pragma unroll
+                for (int kk = 0; kk < 8; ++kk) {
+                    const uint64_t off = (uint64_t)(((kk >> 2) * kTileBytes + (kk & 3) * 32) >> 4);
+                    mma_ss(tmem + prod * 64, ad + off, bd + off, idesc, (term | kk) ? 1u : 0u);
+                }
             }
         }
         mma_commit(bar);
-    };
-    if (tid == 0) {
-        tc_fence_after();
-        issue_product(0);
     }
-    bool ok = mbar_wait(bar, 0, abort_flag);
-
-    // ---- Qt = q G over the Kt tiles (the first product has completed), also to the workspace
-    for (int it = 0; it < 8 && ok; ++it) {
-        const int item = it * 128 + tid, t = item >> 4, ch = item & 15, c0 = ch * 8;
-        uint4 q_h = make_uint4(0, 0, 0, 0), q_l = q_h;
-        if (t >= t_lo && t < t_hi) {
-            const uint4 raw = *reinterpret_cast<const uint4*>(p.q + ((row_t0 + t) * H + head) * kD + c0);
-            const uint32_t rw[4] = {raw.x, raw.y, raw.z, raw.w};
-            uint32_t o[2][4];
+    // the block's values, on their way while the products run
+    uint4 vraw[8];
 #pragma unroll
-            for (int w = 0; w < 4; ++w) {
-                const float q0 = __uint_as_float(rw[w] << 16), q1 = __uint_as_float(rw[w] & 0xffff0000u);
-                split2(q0 * G[t * kD + c0 + 2 * w], q1 * G[t * kD + c0 + 2 * w + 1], o[0][w], o[1][w]);
-            }
-            q_h = make_uint4(o[0][0], o[0][1], o[0][2], o[0][3]);
-            q_l = make_uint4(o[1][0], o[1][1], o[1][2], o[1][3]);
-        }
-        const uint32_t off = (uint32_t)((ch >> 3) * kTileBytes) + sw_off(t, ch & 7);
-        *reinterpret_cast<uint4*>(tileA + off) = q_h;
-        *reinterpret_cast<uint4*>(tileA + 2 * kTileBytes + off) = q_l;
-        const size_t go = bh * tile_elems + (size_t)t * kD + c0;
-        *reinterpret_cast<uint4*>(p.ws_qt_h + go) = q_h;
-        *reinterpret_cast<uint4*>(p.ws_qt_l + go) = q_l;
+    for (int it = 0; it < 8; ++it) {
+        const int item = it * 128 + tid, t = item >> 4, c0 = (item & 15) * 8;
+        vraw[it] = make_uint4(0, 0, 0, 0);
+        if (t >= t_lo && t < t_hi) vraw[it] = *reinterpret_cast<const uint4*>(p.v + ((row_t0 + t) * H + head) * kD + c0);
     }
-    fence_proxy_async_smem();
-    tc_fence_before();
-    __syncthreads();
-    if (tid == 0 && ok) {
-        tc_fence_after();
-        issue_product(64);
-    }
-    ok = ok && mbar_wait(bar, 1, abort_flag);
+    bool ok = __syncthreads_and(mbar_wait(bar, 0, abort_flag));
     tc_fence_after();
 
     // ---- rows of the two products (thread t < 64 owns token t = tensor-memory lane t).  The triangular matrix goes
-    //      to shared memory (over the Kh tiles: both products have completed), M = tril(Qt Kh^T) to the workspace.
-    float* Amat = reinterpret_cast<float*>(tileB);          // [64][64] fp32: beta_t (Kt Kh^T)[t][s] for s < t in the sub-block
+    //      to shared memory (over the Kh tiles: both products have completed), M = tril(Qt Kh^T) to the workspace;
+    //      the V tile goes behind the triangular matrix.
+    float* Amat = reinterpret_cast<float*>(r2);          // [64][64] fp32: beta_t (Kt Kh^T)[t][s] for s < t in the sub-block
+    uint8_t* vtile = r2 + 2 * kTileBytes;                // two 64-column tiles, tokens as rows
+#pragma unroll
+    for (int it = 0; it < 8; ++it) {
+        const int item = it * 128 + tid, t = item >> 4, ch = item & 15;
+        *reinterpret_cast<uint4*>(vtile + (ch >> 3) * kTileBytes + sw_off(t, ch & 7)) = vraw[it];
+    }
     if (warp < 2 && ok) {
         const int t = tid;
         const bool active = t >= t_lo && t < t_hi;
         const int s0 = active ? sub_start(mask, t) : kL;    // columns [s0, t) (and t itself for M) count
         const uint32_t lane_addr = tmem + ((uint32_t)(warp * 32) << 16);
         const float bt = s_beta[t];
-        float x[32];
+        float x[64];
+        tmem_ld32(lane_addr, reinterpret_cast<uint32_t*>(x));
+        tmem_ld32(lane_addr + 32, reinterpret_cast<uint32_t*>(x) + 32);
+        tmem_wait_ld();
 #pragma unroll
-        for (int half = 0; half < 2; ++half) {
-            tmem_ld32(lane_addr + half * 32, reinterpret_cast<uint32_t*>(x));
-            tmem_wait_ld();
-#pragma unroll
-            for (int i = 0; i < 32; ++i) {
-                const int s = half * 32 + i;
-                Amat[t * kL + s] = (active && s >= s0 && s < t) ? bt * x[i] : 0.f;
-            }
+        for (int s4 = 0; s4 < 16; ++s4) {
+            float4 a;
+            a.x = (active && 4 * s4 + 0 >= s0 && 4 * s4 + 0 < t) ? bt * x[4 * s4 + 0] : 0.f;
+            a.y = (active && 4 * s4 + 1 >= s0 && 4 * s4 + 1 < t) ? bt * x[4 * s4 + 1] : 0.f;
+            a.z = (active && 4 * s4 + 2 >= s0 && 4 * s4 + 2 < t) ? bt * x[4 * s4 + 2] : 0.f;
+            a.w = (active && 4 * s4 + 3 >= s0 && 4 * s4 + 3 < t) ? bt * x[4 * s4 + 3] : 0.f;
+            *reinterpret_cast<float4*>(Amat + t * kL + 4 * s4) = a;
         }
+        tmem_ld32(lane_addr + 64, reinterpret_cast<uint32_t*>(x));
+        tmem_ld32(lane_addr + 96, reinterpret_cast<uint32_t*>(x) + 32);
+        tmem_wait_ld();
         __nv_bfloat16* mh = p.ws_m_h + (bh * kL + t) * kL;
         __nv_bfloat16* ml = p.ws_m_l + (bh * kL + t) * kL;
 #pragma unroll
-        for (int half = 0; half < 2; ++half) {
-            tmem_ld32(lane_addr + 64 + half * 32, reinterpret_cast<uint32_t*>(x));
-            tmem_wait_ld();
-            uint32_t oh[16], ol[16];
-#pragma unroll
-            for (int i = 0; i < 16; ++i) {
-                const int s = half * 32 + 2 * i;
-                const float m0 = (active && s >= s0 && s <= t) ? x[2 * i] : 0.f;
-                const float m1 = (active && s + 1 >= s0 && s + 1 <= t) ? x[2 * i + 1] : 0.f;
-                split2(m0, m1, oh[i], ol[i]);
-            }
+        for (int i8 = 0; i8 < 8; ++i8) {
+            uint32_t oh[4], ol[4];
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
-                *reinterpret_cast<uint4*>(mh + half * 32 + i * 8) = make_uint4(oh[4 * i], oh[4 * i + 1], oh[4 * i + 2], oh[4 * i + 3]);
-                *reinterpret_cast<uint4*>(ml + half * 32 + i * 8) = make_uint4(ol[4 * i], ol[4 * i + 1], ol[4 * i + 2], ol[4 * i + 3]);
+                const int s = i8 * 8 + 2 * i;
+                const float m0 = (active && s >= s0 && s <= t) ? x[s] : 0.f;
+                const float m1 = (active && s + 1 >= s0 && s + 1 <= t) ? x[s + 1] : 0.f;
+                split2(m0, m1, oh[i], ol[i]);
             }
+            *reinterpret_cast<uint4*>(mh + i8 * 8) = make_uint4(oh[0], oh[1], oh[2], oh[3]);
+            *reinterpret_cast<uint4*>(ml + i8 * 8) = make_uint4(ol[0], ol[1], ol[2], ol[3]);
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    // ---- T = (I + A)^-1 diag(beta).  The unit lower triangular 64 x 64 matrix L = I + A is inverted in 16 x 16 blocks:
+    //      the four diagonal blocks by forward substitution (64 threads, one column each), then the blocks below the
+    //      diagonal, one block diagonal after the other, from X_ij = -X_ii sum_{j <= k < i} L_ik X_kj as small products
+    //      on all 128 threads (two elements of each 16 x 16 block per thread).  X lives behind the T tiles in R0; the
+    //      sums are staged where the T tiles will go.
+    float* Xm = reinterpret_cast<float*>(r0 + 2 * kTileBytes);        // [64][64] fp32
+    float* Tmp = reinterpret_cast<float*>(r0);                        // up to three 16 x 16 blocks
+    if (ok) {
+        for (int i = tid; i < kL * kL; i += 128) Xm[i] = 0.f;
+        __syncthreads();
+        if (tid < kL) {
+            const int bi = tid >> 4, c = tid & 15;
+            float x[16];
+#pragma unroll
+            for (int r = 0; r < 16; ++r) {
+                float acc = (r == c) ? 1.f : 0.f;
+#pragma unroll
+                for (int q = 0; q < r; ++q) acc = fmaf(-Amat[(bi * 16 + r) * kL + bi * 16 + q], x[q], acc);
+                x[r] = acc;
+                Xm[(bi * 16 + r) * kL + bi * 16 + c] = acc;
+            }
+        }
+        __syncthreads();
+        const int er = tid >> 3, ec = (tid & 7) * 2;                  // this thread's two elements of a block
+#pragma unroll 1
+        for (int d = 1; d < 4; ++d) {
+            // sums S_ij = sum_k L_ik X_kj for the blocks (i, j = i - d)
+#pragma unroll 1
+            for (int i = d; i < 4; ++i) {
+                const int j = i - d;
+                float s0 = 0.f, s1 = 0.f;
+#pragma unroll 1
+                for (int k = j; k < i; ++k) {
+#pragma unroll
+                    for (int q = 0; q < 16; ++q) {
+                        const float l = Amat[(i * 16 + er) * kL + k * 16 + q];
+                        const float2 xv = *reinterpret_cast<const float2*>(Xm + (k * 16 + q) * kL + j * 16 + ec);
+                        s0 = fmaf(l, xv.x, s0);
+                        s1 = fmaf(l, xv.y, s1);
+                    }
+                }
+                *reinterpret_cast<float2*>(Tmp + (i - d) * 256 + er * 16 + ec) = make_float2(s0, s1);
+            }
+            __syncthreads();
+#pragma unroll 1
+            for (int i = d; i < 4; ++i) {
+                const int j = i - d;
+                float s0 = 0.f, s1 = 0.f;
+#pragma unroll
+                for (int q = 0; q < 16; ++q) {
+                    const float x = Xm[(i * 16 + er) * kL + i * 16 + q];
+                    const float2 tv = *reinterpret_cast<const float2*>(Tmp + (i - d) * 256 + q * 16 + ec);
+                    s0 = fmaf(x, tv.x, s0);
+                    s1 = fmaf(x, tv.y, s1);
+                }
+                *reinterpret_cast<float2*>(Xm + (i * 16 + er) * kL + j * 16 + ec) = make_float2(-s0, -s1);
+            }
+            __syncthreads();
+        }
+        // T[t][c] = X[t][c] beta_c as hi/lo operand tiles (hi at R0, lo behind it): thread -> (row, 32 columns)
+        {
+            const int t = tid >> 1, cb = (tid & 1) * 32;
+            uint4 th[4], tl[4];
+#pragma unroll
+            for (int j8 = 0; j8 < 4; ++j8) {
+                uint32_t oh[4], ol[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int c = cb + j8 * 8 + 2 * i;
+                    split2(Xm[t * kL + c] * s_beta[c], Xm[t * kL + c + 1] * s_beta[c + 1], oh[i], ol[i]);
+                }
+                th[j8] = make_uint4(oh[0], oh[1], oh[2], oh[3]);
+                tl[j8] = make_uint4(ol[0], ol[1], ol[2], ol[3]);
+            }
+            __syncthreads();               // the staging area is free: the tiles take its place
+#pragma unroll
+            for (int j8 = 0; j8 < 4; ++j8) {
+                const uint32_t off = sw_off(t, (cb >> 3) + j8);
+                *reinterpret_cast<uint4*>(r0 + off) = th[j8];
+                *reinterpret_cast<uint4*>(r0 + kTileBytes + off) = tl[j8];
+            }
+        }
+    }
+    fence_proxy_async_smem();
+    tc_fence_before();
+    __syncthreads();
+    // ---- W0 = T Kt -> columns [0, 128), U0 = T V -> columns [128, 256)   (V is bf16: it has no lo term)
+    if (tid == 0 && ok) {
+        tc_fence_after();
+        constexpr uint32_t idesc = idesc_bf16(128, 0, 1);
+        const uint32_t t_hi_a = a0, t_lo_a = a0 + kTileBytes;
+        const uint32_t kt_hi = a1, kt_lo = a1 + 2 * kTileBytes, v_a = a2 + 2 * kTileBytes;
+        const uint32_t aa[5] = {t_hi_a, t_hi_a, t_lo_a, t_hi_a, t_lo_a}, bb[5] = {kt_hi, kt_lo, kt_hi, v_a, v_a};
+#pragma unroll
+        for (int term = 0; term < 5; ++term) {
+            const uint64_t ad = smem_desc_sw128(aa[term], 16, 1024), bd = smem_desc_sw128(bb[term], kTileBytes, 1024);
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk)
+                mma_ss(tmem + (term >= 3 ? 128 : 0), ad + (uint64_t)(kk * 2), bd + (uint64_t)(kk * 128), idesc,
+                       ((term == 0 || term == 3) && kk == 0) ? 0u : 1u);
+        }
+        mma_commit(bar);
+    }
+    ok = __syncthreads_and(ok && mbar_wait(bar, 1, abort_flag));
+    tc_fence_after();
+    if (warp < 2 && ok) {
+        const int t = tid;
+        const uint32_t lane_addr = tmem + ((uint32_t)(warp * 32) << 16);
+        __nv_bfloat16* wh = p.ws_w0_h + bh * tile_elems + (size_t)t * kD;
+        __nv_bfloat16* wl = p.ws_w0_l + bh * tile_elems + (size_t)t * kD;
+        float* u0 = p.ws_u0 + bh * tile_elems + (size_t)t * kD;
+#pragma unroll 1
+        for (int c0 = 0; c0 < kD; c0 += 32) {
+            float x[32];
+            tmem_ld32(lane_addr + c0, reinterpret_cast<uint32_t*>(x));
+            tmem_wait_ld();
+#pragma unroll
+            for (int i8 = 0; i8 < 4; ++i8) {
+                uint32_t oh[4], ol[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) split2(x[i8 * 8 + 2 * i], x[i8 * 8 + 2 * i + 1], oh[i], ol[i]);
+                *reinterpret_cast<uint4*>(wh + c0 + i8 * 8) = make_uint4(oh[0], oh[1], oh[2], oh[3]);
+                *reinterpret_cast<uint4*>(wl + c0 + i8 * 8) = make_uint4(ol[0], ol[1], ol[2], ol[3]);
+            }
+            tmem_ld32(lane_addr + 128 + c0, reinterpret_cast<uint32_t*>(x));
+            tmem_wait_ld();
+#pragma unroll
+            for (int i4 = 0; i4 < 8; ++i4)
+                *reinterpret_cast<float4*>(u0 + c0 + i4 * 4) = make_float4(x[4 * i4], x[4 * i4 + 1], x[4 * i4 + 2], x[4 * i4 + 3]);
         }
     }
     tc_fence_before();
     __syncthreads();
     if (warp == 0) {
         tc_fence_after();
-        tmem_dealloc(tmem, 128);
+        tmem_dealloc(tmem, 256);
     }
-    if (!ok) {
-        if (tid == 0 && p.status) atomicCAS(p.status, 0, WPP_ERR_TIMEOUT);
-        return;
-    }
-    // ---- T = (I + A)^-1 diag(beta) by forward substitution: thread c owns column c (T[t][c] = 0 for t < c)
-    if (tid < kL) {
-        const int c = tid;
-        float Tc[kL];
-#pragma unroll
-        for (int t = 0; t < kL; ++t) {
-            float acc = (t == c) ? s_beta[t] : 0.f;
-            const float4* arow = reinterpret_cast<const float4*>(Amat + t * kL);
-#pragma unroll
-            for (int s4 = 0; s4 < (t + 3) / 4; ++s4) {
-                const float4 a = arow[s4];
-                if (4 * s4 + 0 < t) acc = fmaf(-a.x, Tc[4 * s4 + 0], acc);
-                if (4 * s4 + 1 < t) acc = fmaf(-a.y, Tc[4 * s4 + 1], acc);
-                if (4 * s4 + 2 < t) acc = fmaf(-a.z, Tc[4 * s4 + 2], acc);
-                if (4 * s4 + 3 < t) acc = fmaf(-a.w, Tc[4 * s4 + 3], acc);
-            }
-            Tc[t] = acc;
-        }
-        __nv_bfloat16* th = p.ws_t_h + bh * kL * kL + c;
-        __nv_bfloat16* tl = p.ws_t_l + bh * kL * kL + c;
-#pragma unroll
-        for (int t = 0; t < kL; ++t) {
-            const __nv_bfloat16 h = __float2bfloat16_rn(Tc[t]);
-            th[t * kL] = h;
-            tl[t * kL] = __float2bfloat16_rn(Tc[t] - __bfloat162float(h));
-        }
-    }
+    if (!ok && tid == 0 && p.status) atomicCAS(p.status, 0, WPP_ERR_TIMEOUT);
 }
 
 // ---------------------------------------------------------------------------------------------------------------
-// Chain: one CTA per (request, head).  Warps 0-3: the state's rows (thread r = tensor-memory lane r = column r of S);
-// warps 4-7: output epilogue; warp 8: producer (TMA loads of the block's operands, step records); warp 9: one thread
-// issues the MMAs.
+// Chain: one CTA per (request, head).  Warps 0-3 and 4-7: two row warpgroups (thread r of either = tensor-memory lane r
+// = column r of S); they share the per-step conversions half and half, and the second one also writes the outputs.
+// Warp 8: operand loader (TMA); warp 9: one thread issues the MMAs; warp 10: publishes the step records.
 constexpr int kStepRing = 4;
 struct Ring {
     uint32_t stage, phase;
@@ -416,35 +528,33 @@ struct Ring {
 struct StepRec {
     int a, b;            // tokens [a, b) of the block; a < 0: no more steps
     int first, last;     // first / last step of its block (operand buffers are acquired / released there)
-    int store_slot;      // state slot to write after the step (periodic snapshot or the chunk's end), or -1
+    int store_slot;      // state slot to write after the step (periodic snapshot), or -1
     int pad[3];
     int64_t row_t0;      // row of the block's token 0 in the packed arrays
 };
 struct ChainSmem {
-    // operand tiles of one block, each a pair (hi, lo); 128-channel operands have two 64-column tiles per part
-    static constexpr int kOffKt = 0;                          // hi0 hi1 lo0 lo1
-    static constexpr int kOffQt = kOffKt + 4 * kTileBytes;
+    // operand tiles of one block, each a pair (hi, lo) of two 64-column tiles
+    static constexpr int kOffW0 = 0;                          // hi0 hi1 lo0 lo1
+    static constexpr int kOffQt = kOffW0 + 4 * kTileBytes;
     static constexpr int kOffKb = kOffQt + 4 * kTileBytes;
-    static constexpr int kOffT = kOffKb + 4 * kTileBytes;     // hi lo
-    static constexpr int kOffM = kOffT + 2 * kTileBytes;
-    static constexpr int kOffV = kOffM + 2 * kTileBytes;      // two 64-column tiles
-    static constexpr int kOffVec = kOffV + 2 * kTileBytes;    // per ring slot: alpha of the step's first token, decay product at its end
+    static constexpr int kOffM = kOffKb + 4 * kTileBytes;     // hi lo
+    static constexpr int kOffU0 = kOffM + 2 * kTileBytes;     // fp32 [64][128], plain rows
+    static constexpr int kOffVec = kOffU0 + kL * kD * 4;      // per ring slot: alpha of the step's first token, decay product at its end
     static constexpr int kOffRec = kOffVec + kStepRing * 2 * kD * 4;
     static constexpr int kOffBars = kOffRec + kStepRing * (int)sizeof(StepRec);
-    static constexpr int kNumBars = 2 * kStepRing + 12 + 8;
+    static constexpr int kNumBars = 2 * kStepRing + 10 + 6;
     static constexpr int kOffMisc = kOffBars + 8 * kNumBars;
     static constexpr int kBytes = kOffMisc + 64 + 1024;
 };
-// tensor-memory columns
-constexpr uint32_t kColS = 0, kColShl = 128, kColWU = 256, kColRU = 320, kColO = 384;
+// tensor-memory columns: state, its hi/lo operand form, X = W0 S_0' (fp32), U as hi/lo operand, output accumulator
+constexpr uint32_t kColS = 0, kColShl = 128, kColX = 256, kColU = 320, kColO = 384;
 
-__global__ void __launch_bounds__(320, 1)
-kda_tc_chain_kernel(const __grid_constant__ CUtensorMap tm_kt_h, const __grid_constant__ CUtensorMap tm_kt_l,
+__global__ void __launch_bounds__(352, 1)
+kda_tc_chain_kernel(const __grid_constant__ CUtensorMap tm_w0_h, const __grid_constant__ CUtensorMap tm_w0_l,
                     const __grid_constant__ CUtensorMap tm_qt_h, const __grid_constant__ CUtensorMap tm_qt_l,
                     const __grid_constant__ CUtensorMap tm_kb_h, const __grid_constant__ CUtensorMap tm_kb_l,
-                    const __grid_constant__ CUtensorMap tm_t_h, const __grid_constant__ CUtensorMap tm_t_l,
                     const __grid_constant__ CUtensorMap tm_m_h, const __grid_constant__ CUtensorMap tm_m_l,
-                    const __grid_constant__ CUtensorMap tm_v, const KdaTcParams p) {
+                    const KdaTcParams p) {
     using CS = ChainSmem;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -453,16 +563,16 @@ kda_tc_chain_kernel(const __grid_constant__ CUtensorMap tm_kt_h, const __grid_co
     auto bStepFull = [&](int s) { return bars + 8 * s; };
     auto bStepEmpty = [&](int s) { return bars + 8 * (kStepRing + s); };
     const uint32_t b0 = bars + 16 * kStepRing;
-    // operand buffers (one block in flight each): full / empty
-    const uint32_t bKtFull = b0, bKtEmpty = b0 + 8, bQtFull = b0 + 16, bQtEmpty = b0 + 24, bKbFull = b0 + 32,
-                   bKbEmpty = b0 + 40, bTFull = b0 + 48, bTEmpty = b0 + 56, bMFull = b0 + 64, bMEmpty = b0 + 72,
-                   bVFull = b0 + 80, bVEmpty = b0 + 88;
-    const uint32_t b1 = b0 + 96;
-    const uint32_t bShlReady = b1, bWReady = b1 + 8, bRhsReady = b1 + 16, bUReady = b1 + 24, bUhlReady = b1 + 32,
-                   bSReady = b1 + 40, bOReady = b1 + 48, bOFree = b1 + 56;
+    // operand buffers (one block in flight each): full at b0 + 16 i, empty at b0 + 16 i + 8 (W0 Qt Kb M U0)
+    const uint32_t bW0Full = b0, bW0Empty = b0 + 8, bQtFull = b0 + 16, bQtEmpty = b0 + 24, bKbFull = b0 + 32,
+                   bKbEmpty = b0 + 40, bMFull = b0 + 48, bMEmpty = b0 + 56, bU0Full = b0 + 64, bU0Empty = b0 + 72;
+    const uint32_t b1 = b0 + 80;
+    const uint32_t bShlReady = b1, bXReady = b1 + 8, bUhlReady = b1 + 16, bSReady = b1 + 24, bOReady = b1 + 32,
+                   bOFree = b1 + 40;
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(sm + CS::kOffMisc);
     volatile uint32_t* abort_flag = tmem_slot + 1;
-    float* s_vec = reinterpret_cast<float*>(sm + CS::kOffVec);
+    const float* s_vec = reinterpret_cast<const float*>(sm + CS::kOffVec);
+    const float* s_u0 = reinterpret_cast<const float*>(sm + CS::kOffU0);
     volatile StepRec* s_rec = reinterpret_cast<volatile StepRec*>(sm + CS::kOffRec);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -489,12 +599,12 @@ kda_tc_chain_kernel(const __grid_constant__ CUtensorMap tm_kt_h, const __grid_co
     }
 
     if (tid == 0) {
-        for (int s = 0; s < kStepRing; ++s) { mbar_init(bStepFull(s), 1); mbar_init(bStepEmpty(s), 128 + 128 + 1); }
-        for (int i = 0; i < 5; ++i) { mbar_init(b0 + 16 * i, 1); mbar_init(b0 + 16 * i + 8, 1); }
-        mbar_init(bVFull, 1);
-        mbar_init(bVEmpty, 128);          // the value tile is released by the 128 row threads
-        mbar_init(bShlReady, 128); mbar_init(bWReady, 1); mbar_init(bRhsReady, 128); mbar_init(bUReady, 1);
-        mbar_init(bUhlReady, 128); mbar_init(bSReady, 1); mbar_init(bOReady, 1); mbar_init(bOFree, 128);
+        for (int s = 0; s < kStepRing; ++s) { mbar_init(bStepFull(s), 1); mbar_init(bStepEmpty(s), 256 + 1); }
+        for (int i = 0; i < 4; ++i) { mbar_init(b0 + 16 * i, 1); mbar_init(b0 + 16 * i + 8, 1); }
+        mbar_init(bU0Full, 1);
+        mbar_init(bU0Empty, 256);          // the U0 tile is released by the 256 row threads
+        mbar_init(bShlReady, 256); mbar_init(bXReady, 1); mbar_init(bUhlReady, 256); mbar_init(bSReady, 1);
+        mbar_init(bOReady, 1); mbar_init(bOFree, 128);
         *abort_flag = 0u;
         fence_barrier_init();
     }
@@ -509,11 +619,49 @@ kda_tc_chain_kernel(const __grid_constant__ CUtensorMap tm_kt_h, const __grid_co
     const int gb0 = p.blk_off[req];
 
     if (warp == 8) {
-        // ================================================================ producer
-        uint32_t ph_e[6] = {0, 0, 0, 0, 0, 0};      // parity of the operand buffers' empty barriers (Kt Qt Kb T M V)
+        // ================================================================ operand loader
+        // One buffer per operand; a block's operands are released, in this order, as its last step proceeds (W0 after
+        // X, Qt after the first output product, U0 by the row threads, Kb after the state product, M after the second
+        // output product), and each is requested again for the next block the moment it is free.
+        uint32_t ph_e = 0;
+        for (int b = 0; b < g.n_blocks; ++b) {
+            const size_t bh = (size_t)(gb0 + b) * H + head;
+            const int row = (int)(bh * kL);
+            const CUtensorMap* mh[4] = {&tm_w0_h, &tm_qt_h, nullptr, &tm_kb_h};
+            const CUtensorMap* ml[4] = {&tm_w0_l, &tm_qt_l, nullptr, &tm_kb_l};
+            const uint32_t dst4[4] = {base + CS::kOffW0, base + CS::kOffQt, 0u, base + CS::kOffKb};
+            bool okw = true;
+#pragma unroll
+            for (int buf = 0; buf < 5 && okw; ++buf) {
+                // buffers in release order: 0 W0, 1 Qt, 2 U0 (barrier index 4), 3 Kb (index 2), 4 M (index 3)
+                const int bi = buf == 2 ? 4 : buf == 3 ? 2 : buf == 4 ? 3 : buf;
+                const uint32_t full = b0 + 16 * bi, empty = full + 8;
+                okw = mbar_wait(empty, ph_e ^ 1u, abort_flag);
+                okw = __all_sync(0xffffffffu, okw);
+                if (!okw) break;
+                if (buf == 2) {
+                    if (lane == 0) {
+                        mbar_arrive_expect_tx(full, kL * kD * 4);
+                        bulk_load(base + CS::kOffU0, p.ws_u0 + bh * (size_t)kL * kD, kL * kD * 4, full);
+                    }
+                } else if (buf == 4) {
+                    if (lane == 0) mbar_arrive_expect_tx(full, 2 * kTileBytes);
+                    __syncwarp();
+                    if (lane < 2) tma_load_2d(base + CS::kOffM + lane * kTileBytes, lane ? &tm_m_l : &tm_m_h, full, 0, row);
+                } else {
+                    if (lane == 0) mbar_arrive_expect_tx(full, 4 * kTileBytes);
+                    __syncwarp();
+                    if (lane < 4)
+                        tma_load_2d(dst4[buf] + lane * kTileBytes, (lane & 2) ? ml[buf] : mh[buf], full, (lane & 1) * 64, row);
+                }
+            }
+            if (!okw) break;
+            ph_e ^= 1u;
+        }
+    } else if (warp == 10) {
+        // ================================================================ step records
         Ring step = {0, 0};
         bool dead = false;
-        // periodic snapshots: next sequence position at which one is due
         const int interval = p.snap_interval;
         int64_t next_snap = interval > 0 ? ((int64_t)g.P / interval + 1) * interval : -1;
         int n_snap = 0;
@@ -531,47 +679,6 @@ kda_tc_chain_kernel(const __grid_constant__ CUtensorMap tm_kt_h, const __grid_co
             const size_t bh = (size_t)(gb0 + b) * H + head;
             const int t_lo = max(0, g.P - blk * kL), t_hi = min(kL, g.P + g.C - blk * kL);
             const int64_t row_t0 = g.row0 + ((int64_t)blk * kL - g.P);
-            // ---- operand loads of the block: each waits for its buffer (lanes 0..5 own one buffer each)
-            {
-                bool okw = true;
-                if (lane < 6) okw = mbar_wait(b0 + 16 * lane + 8, ph_e[lane] ^ 1u, abort_flag);
-                if (!__all_sync(0xffffffffu, okw)) { dead = true; break; }
-#pragma unroll
-                for (int i = 0; i < 6; ++i) ph_e[i] ^= 1u;
-                const int row = (int)(bh * kL);
-                if (lane == 0) {
-                    mbar_arrive_expect_tx(bKtFull, 4 * kTileBytes);
-                    tma_load_2d(base + CS::kOffKt, &tm_kt_h, bKtFull, 0, row);
-                    tma_load_2d(base + CS::kOffKt + kTileBytes, &tm_kt_h, bKtFull, 64, row);
-                    tma_load_2d(base + CS::kOffKt + 2 * kTileBytes, &tm_kt_l, bKtFull, 0, row);
-                    tma_load_2d(base + CS::kOffKt + 3 * kTileBytes, &tm_kt_l, bKtFull, 64, row);
-                } else if (lane == 1) {
-                    mbar_arrive_expect_tx(bQtFull, 4 * kTileBytes);
-                    tma_load_2d(base + CS::kOffQt, &tm_qt_h, bQtFull, 0, row);
-                    tma_load_2d(base + CS::kOffQt + kTileBytes, &tm_qt_h, bQtFull, 64, row);
-                    tma_load_2d(base + CS::kOffQt + 2 * kTileBytes, &tm_qt_l, bQtFull, 0, row);
-                    tma_load_2d(base + CS::kOffQt + 3 * kTileBytes, &tm_qt_l, bQtFull, 64, row);
-                } else if (lane == 2) {
-                    mbar_arrive_expect_tx(bKbFull, 4 * kTileBytes);
-                    tma_load_2d(base + CS::kOffKb, &tm_kb_h, bKbFull, 0, row);
-                    tma_load_2d(base + CS::kOffKb + kTileBytes, &tm_kb_h, bKbFull, 64, row);
-                    tma_load_2d(base + CS::kOffKb + 2 * kTileBytes, &tm_kb_l, bKbFull, 0, row);
-                    tma_load_2d(base + CS::kOffKb + 3 * kTileBytes, &tm_kb_l, bKbFull, 64, row);
-                } else if (lane == 3) {
-                    mbar_arrive_expect_tx(bTFull, 2 * kTileBytes);
-                    tma_load_2d(base + CS::kOffT, &tm_t_h, bTFull, 0, row);
-                    tma_load_2d(base + CS::kOffT + kTileBytes, &tm_t_l, bTFull, 0, row);
-                } else if (lane == 4) {
-                    mbar_arrive_expect_tx(bMFull, 2 * kTileBytes);
-                    tma_load_2d(base + CS::kOffM, &tm_m_h, bMFull, 0, row);
-                    tma_load_2d(base + CS::kOffM + kTileBytes, &tm_m_l, bMFull, 0, row);
-                } else if (lane == 5) {
-                    mbar_arrive_expect_tx(bVFull, 2 * kTileBytes);
-                    tma_load_3d(base + CS::kOffV, &tm_v, bVFull, 0, head, (int)row_t0);
-                    tma_load_3d(base + CS::kOffV + kTileBytes, &tm_v, bVFull, 64, head, (int)row_t0);
-                }
-            }
-            // ---- the block's steps
             uint64_t mask = 0;
             if (lane == 0) mask = p.ws_mask[bh];
             mask = __shfl_sync(0xffffffffu, mask, 0);
@@ -608,16 +715,18 @@ kda_tc_chain_kernel(const __grid_constant__ CUtensorMap tm_kt_h, const __grid_co
     } else if (warp == 9 && lane == 0) {
         // ================================================================ MMA issuer
         Ring step = {0, 0};
-        uint32_t ph_kt = 0, ph_qt = 0, ph_kb = 0, ph_t = 0, ph_m = 0;
-        uint32_t ph_shl = 0, ph_rhs = 0, ph_uhl = 0, ph_ofree = 0;
+        uint32_t ph_w0 = 0, ph_qt = 0, ph_kb = 0, ph_m = 0;
+        uint32_t ph_shl = 0, ph_uhl = 0, ph_ofree = 0;
         constexpr uint32_t idesc64 = idesc_bf16(64, 0, 0), idesc128mn = idesc_bf16(128, 0, 1);
-        const uint32_t tS = tmem + kColS, tShl = tmem + kColShl, tWU = tmem + kColWU, tRU = tmem + kColRU, tO = tmem + kColO;
+        const uint32_t tS = tmem + kColS, tShl = tmem + kColShl, tX = tmem + kColX, tU = tmem + kColU, tO = tmem + kColO;
         // A (hi + lo, in tensor memory, `acols` columns per part) x B^T (hi + lo tiles in shared memory, K-major)
         auto product_k = [&](uint32_t d, uint32_t a_tm, uint32_t acols, uint32_t b_hi, uint32_t b_lo, int ksteps, bool overwrite) {
             const uint32_t aa[3] = {a_tm, a_tm, a_tm + acols}, bb[3] = {b_hi, b_lo, b_hi};
             bool first = overwrite;
+#pragma unroll
             for (int term = 0; term < 3; ++term) {
                 const uint64_t bd = smem_desc_sw128(bb[term], 16, 1024);
+#pragma unroll 4
                 for (int kk = 0; kk < ksteps; ++kk) {
                     const uint64_t off = (uint64_t)(((kk >> 2) * kTileBytes + (kk & 3) * 32) >> 4);
                     mma_ts(d, aa[term] + kk * 8, bd + off, idesc64, first ? 0u : 1u);
@@ -625,37 +734,29 @@ kda_tc_chain_kernel(const __grid_constant__ CUtensorMap tm_kt_h, const __grid_co
                 }
             }
         };
-        bool dead = false;
         bool first_step = true;
-        while (!dead) {
+        while (true) {
             if (!mbar_wait(bStepFull(step.stage), step.phase, abort_flag)) break;
             const int a = s_rec[step.stage].a;
             const bool first = s_rec[step.stage].first, last = s_rec[step.stage].last;
             mbar_arrive(bStepEmpty(step.stage));
             step.advance(kStepRing);
             if (a < 0) break;
-            // ---- W^T = S_0'^T Kt^T
+            // ---- X^T = S_0'^T W0^T
             if (!mbar_wait(bShlReady, ph_shl, abort_flag)) break;
             ph_shl ^= 1u;
-            if (first) { if (!mbar_wait(bKtFull, ph_kt, abort_flag)) break; ph_kt ^= 1u; }
+            if (first) { if (!mbar_wait(bW0Full, ph_w0, abort_flag)) break; ph_w0 ^= 1u; }
             tc_fence_after();
-            product_k(tWU, tShl, 64, base + CS::kOffKt, base + CS::kOffKt + 2 * kTileBytes, 8, true);
-            mma_commit(bWReady);
-            if (last) mma_commit(bKtEmpty);
-            // ---- U^T = (V - W)^T T^T
-            if (!mbar_wait(bRhsReady, ph_rhs, abort_flag)) break;
-            ph_rhs ^= 1u;
-            if (first) { if (!mbar_wait(bTFull, ph_t, abort_flag)) break; ph_t ^= 1u; }
-            tc_fence_after();
-            product_k(tWU, tRU, 32, base + CS::kOffT, base + CS::kOffT + kTileBytes, 4, true);
-            mma_commit(bUReady);
-            if (last) mma_commit(bTEmpty);
+            product_k(tX, tShl, 64, base + CS::kOffW0, base + CS::kOffW0 + 2 * kTileBytes, 8, true);
+            mma_commit(bXReady);
+            if (last) mma_commit(bW0Empty);
             // ---- O^T = S_0'^T Qt^T (the previous step's output must have been read out)
             if (!first_step) { if (!mbar_wait(bOFree, ph_ofree, abort_flag)) break; ph_ofree ^= 1u; }
             first_step = false;
             if (first) { if (!mbar_wait(bQtFull, ph_qt, abort_flag)) break; ph_qt ^= 1u; }
             tc_fence_after();
             product_k(tO, tShl, 64, base + CS::kOffQt, base + CS::kOffQt + 2 * kTileBytes, 8, true);
+            if (last) mma_commit(bQtEmpty);
             // ---- S_b^T += U^T Kb   (the accumulator was preset to the decayed S_0'),   O^T += U^T M^T
             if (!mbar_wait(bUhlReady, ph_uhl, abort_flag)) break;
             ph_uhl ^= 1u;
@@ -663,35 +764,55 @@ kda_tc_chain_kernel(const __grid_constant__ CUtensorMap tm_kt_h, const __grid_co
             tc_fence_after();
             {
                 const uint32_t kb_hi = base + CS::kOffKb, kb_lo = kb_hi + 2 * kTileBytes;
-                const uint32_t aa[3] = {tRU, tRU, tRU + 32}, bb[3] = {kb_hi, kb_lo, kb_hi};
+                const uint32_t aa[3] = {tU, tU, tU + 32}, bb[3] = {kb_hi, kb_lo, kb_hi};
+#pragma unroll
                 for (int term = 0; term < 3; ++term) {
                     const uint64_t bd = smem_desc_sw128(bb[term], kTileBytes, 1024);      // MN-major: 64-column halves kTileBytes apart
+#pragma unroll
                     for (int kk = 0; kk < 4; ++kk) mma_ts(tS, aa[term] + kk * 8, bd + (uint64_t)(kk * 128), idesc128mn, 1u);
                 }
             }
             mma_commit(bSReady);
             if (last) mma_commit(bKbEmpty);
             if (first) { if (!mbar_wait(bMFull, ph_m, abort_flag)) break; ph_m ^= 1u; }
-            product_k(tO, tRU, 32, base + CS::kOffM, base + CS::kOffM + kTileBytes, 4, false);
+            product_k(tO, tU, 32, base + CS::kOffM, base + CS::kOffM + kTileBytes, 4, false);
             mma_commit(bOReady);
-            if (last) { mma_commit(bQtEmpty); mma_commit(bMEmpty); }
+            if (last) mma_commit(bMEmpty);
         }
-    } else if (warp >= 4 && warp < 8) {
-        // ================================================================ output epilogue (thread = value column r)
-        const int r = tid - 128;
+    } else if (warp < 8) {
+        // ================================================================ the state's rows (thread r = column r of S)
+        const int wg = warp >> 2;                      // 0: channels [0, 64), tokens [0, 32);  1: the other halves + outputs
+        const int r = tid & 127;
         const uint32_t lane_addr = tmem + ((uint32_t)((warp & 3) * 32) << 16);
-        Ring step = {0, 0};
+        const int cbase = wg * 64;                     // this warpgroup's channels (columns of S^T)
+        // initial state: S[c][r] for this warpgroup's c
+        {
+            const float* src = slot_in >= 0 ? p.state_pool + ((size_t)slot_in * H + head) * head_floats + r : nullptr;
+#pragma unroll 1
+            for (int c0 = cbase; c0 < cbase + 64; c0 += 32) {
+                float x[32];
+#pragma unroll
+                for (int i = 0; i < 32; ++i) x[i] = src ? src[(size_t)(c0 + i) * kD] : 0.f;
+                tmem_st32(lane_addr + kColS + c0, reinterpret_cast<const uint32_t*>(x));
+            }
+            tmem_wait_st();
+        }
+        auto store_state = [&](int slot) {
+            float* dst = p.state_pool + ((size_t)slot * H + head) * head_floats + r;
+#pragma unroll 1
+            for (int c0 = cbase; c0 < cbase + 64; c0 += 32) {
+                float x[32];
+                tmem_ld32(lane_addr + kColS + c0, reinterpret_cast<uint32_t*>(x));
+                tmem_wait_ld();
+#pragma unroll
+                for (int i = 0; i < 32; ++i) dst[(size_t)(c0 + i) * kD] = x[i];
+            }
+        };
+        // outputs of a finished step (second warpgroup): rows [a, b) of the block
         uint32_t ph_o = 0;
-        while (true) {
-            const bool okw = mbar_wait(bStepFull(step.stage), step.phase, abort_flag);
-            if (!__all_sync(0xffffffffu, okw)) break;
-            const int a = s_rec[step.stage].a, b = s_rec[step.stage].b;
-            const int64_t row_t0 = s_rec[step.stage].row_t0;
-            mbar_arrive(bStepEmpty(step.stage));
-            step.advance(kStepRing);
-            if (a < 0) break;
+        auto write_outputs = [&](int a, int b, int64_t row_t0) -> bool {
             const bool oko = mbar_wait(bOReady, ph_o, abort_flag);
-            if (!__all_sync(0xffffffffu, oko)) break;
+            if (!__all_sync(0xffffffffu, oko)) return false;
             ph_o ^= 1u;
             tc_fence_after();
             float o[64];
@@ -703,40 +824,14 @@ kda_tc_chain_kernel(const __grid_constant__ CUtensorMap tm_kt_h, const __grid_co
 #pragma unroll
             for (int t = 0; t < kL; ++t)
                 if (t >= a && t < b) p.out[((row_t0 + t) * H + head) * kD + r] = __float2bfloat16_rn(o[t]);
-        }
-    } else if (warp < 4) {
-        // ================================================================ the state's rows (thread r = column r of S)
-        const int r = tid;
-        const uint32_t lane_addr = tmem + ((uint32_t)(warp * 32) << 16);
-        // initial state: S[c][r] for all c
-        {
-            const float* src = slot_in >= 0 ? p.state_pool + ((size_t)slot_in * H + head) * head_floats + r : nullptr;
-#pragma unroll 1
-            for (int c0 = 0; c0 < kD; c0 += 32) {
-                float x[32];
-#pragma unroll
-                for (int i = 0; i < 32; ++i) x[i] = src ? src[(size_t)(c0 + i) * kD] : 0.f;
-                tmem_st32(lane_addr + kColS + c0, reinterpret_cast<const uint32_t*>(x));
-            }
-            tmem_wait_st();
-        }
-        auto store_state = [&](int slot) {
-            float* dst = p.state_pool + ((size_t)slot * H + head) * head_floats + r;
-#pragma unroll 1
-            for (int c0 = 0; c0 < kD; c0 += 32) {
-                float x[32];
-                tmem_ld32(lane_addr + kColS + c0, reinterpret_cast<uint32_t*>(x));
-                tmem_wait_ld();
-#pragma unroll
-                for (int i = 0; i < 32; ++i) dst[(size_t)(c0 + i) * kD] = x[i];
-            }
+            return true;
         };
         Ring step = {0, 0};
-        uint32_t ph_w = 0, ph_u = 0, ph_s = 0, ph_v = 0;
+        uint32_t ph_x = 0, ph_s = 0, ph_u0 = 0;
         bool s_pending = false;          // an S_b product is in flight: wait for it before touching S
         bool dead = false;
-        const uint8_t* vt = sm + CS::kOffV + (r >> 6) * kTileBytes;
-        const int vj = (r & 63) >> 3, vb = (r & 7) * 2;
+        int prev_a = -1, prev_b = -1;    // the step whose outputs are still to be written
+        int64_t prev_row = 0;
         while (!dead) {
             const bool okw = mbar_wait(bStepFull(step.stage), step.phase, abort_flag);
             if (!__all_sync(0xffffffffu, okw)) { dead = true; break; }
@@ -744,6 +839,7 @@ kda_tc_chain_kernel(const __grid_constant__ CUtensorMap tm_kt_h, const __grid_co
             const int a = s_rec[slot_ring].a, b = s_rec[slot_ring].b;
             const bool first = s_rec[slot_ring].first, last = s_rec[slot_ring].last;
             const int store_slot = s_rec[slot_ring].store_slot;
+            const int64_t row_t0 = s_rec[slot_ring].row_t0;
             if (a < 0) { mbar_arrive(bStepEmpty(slot_ring)); break; }
             const float* v_alpha = s_vec + slot_ring * 2 * kD;
             const float* v_end = v_alpha + kD;
@@ -755,91 +851,70 @@ kda_tc_chain_kernel(const __grid_constant__ CUtensorMap tm_kt_h, const __grid_co
                 s_pending = false;
             }
             tc_fence_after();
-#pragma unroll 1
-            for (int c0 = 0; c0 < kD; c0 += 32) {
-                float x[32];
-                uint32_t hi[16], lo[16];
-                tmem_ld32(lane_addr + kColS + c0, reinterpret_cast<uint32_t*>(x));
+            {
+                float x[64];
+                tmem_ld32(lane_addr + kColS + cbase, reinterpret_cast<uint32_t*>(x));
+                tmem_ld32(lane_addr + kColS + cbase + 32, reinterpret_cast<uint32_t*>(x) + 32);
                 tmem_wait_ld();
+                uint32_t hi[32], lo[32];
 #pragma unroll
-                for (int i = 0; i < 16; ++i) {
-                    const float y0 = x[2 * i] * v_alpha[c0 + 2 * i], y1 = x[2 * i + 1] * v_alpha[c0 + 2 * i + 1];
+                for (int i = 0; i < 32; ++i) {
+                    const float2 al = *reinterpret_cast<const float2*>(v_alpha + cbase + 2 * i);
+                    const float2 en = *reinterpret_cast<const float2*>(v_end + cbase + 2 * i);
+                    const float y0 = x[2 * i] * al.x, y1 = x[2 * i + 1] * al.y;
                     split2(y0, y1, hi[i], lo[i]);
-                    x[2 * i] = y0 * v_end[c0 + 2 * i];
-                    x[2 * i + 1] = y1 * v_end[c0 + 2 * i + 1];
+                    x[2 * i] = y0 * en.x;
+                    x[2 * i + 1] = y1 * en.y;
                 }
-                tmem_st32(lane_addr + kColS + c0, reinterpret_cast<const uint32_t*>(x));
-                tmem_st8(lane_addr + kColShl + c0 / 2, hi);
-                tmem_st8(lane_addr + kColShl + c0 / 2 + 8, hi + 8);
-                tmem_st8(lane_addr + kColShl + 64 + c0 / 2, lo);
-                tmem_st8(lane_addr + kColShl + 64 + c0 / 2 + 8, lo + 8);
+                tmem_st32(lane_addr + kColS + cbase, reinterpret_cast<const uint32_t*>(x));
+                tmem_st32(lane_addr + kColS + cbase + 32, reinterpret_cast<const uint32_t*>(x) + 32);
+                tmem_st32(lane_addr + kColShl + cbase / 2, hi);
+                tmem_st32(lane_addr + kColShl + 64 + cbase / 2, lo);
             }
             tmem_wait_st();
             tc_fence_before();
             mbar_arrive(bShlReady);
             mbar_arrive(bStepEmpty(slot_ring));      // the record and its vectors have been consumed
-            // ---- (V - W)^T for the step's tokens, zero elsewhere
+            // ---- the second warpgroup writes the previous step's outputs while X is being computed
+            if (wg == 1 && prev_a >= 0) {
+                if (!write_outputs(prev_a, prev_b, prev_row)) { dead = true; break; }
+            }
+            // ---- U^T = (U0 - X)^T for the step's tokens, zero elsewhere, as the hi/lo operand
             if (first) {
-                const bool okv = mbar_wait(bVFull, ph_v, abort_flag);
-                if (!__all_sync(0xffffffffu, okv)) { dead = true; break; }
-                ph_v ^= 1u;
+                const bool oku = mbar_wait(bU0Full, ph_u0, abort_flag);
+                if (!__all_sync(0xffffffffu, oku)) { dead = true; break; }
+                ph_u0 ^= 1u;
             }
             {
-                const bool okw2 = mbar_wait(bWReady, ph_w, abort_flag);
-                if (!__all_sync(0xffffffffu, okw2)) { dead = true; break; }
-                ph_w ^= 1u;
+                const bool okx = mbar_wait(bXReady, ph_x, abort_flag);
+                if (!__all_sync(0xffffffffu, okx)) { dead = true; break; }
+                ph_x ^= 1u;
             }
             tc_fence_after();
-#pragma unroll
-            for (int half = 0; half < 2; ++half) {
+            {
+                const int tb = wg * 32;
                 float x[32];
                 uint32_t hi[16], lo[16];
-                tmem_ld32(lane_addr + kColWU + half * 32, reinterpret_cast<uint32_t*>(x));
+                tmem_ld32(lane_addr + kColX + tb, reinterpret_cast<uint32_t*>(x));
                 tmem_wait_ld();
 #pragma unroll
                 for (int i = 0; i < 16; ++i) {
-                    float rr[2];
-#pragma unroll
-                    for (int e = 0; e < 2; ++e) {
-                        const int t = half * 32 + 2 * i + e;
-                        const float vv = __bfloat162float(*reinterpret_cast<const __nv_bfloat16*>(vt + sw_off(t, vj) + vb));
-                        rr[e] = (t >= a && t < b) ? vv - x[2 * i + e] : 0.f;
-                    }
-                    split2(rr[0], rr[1], hi[i], lo[i]);
+                    const int t0 = tb + 2 * i;
+                    const float u0 = (t0 >= a && t0 < b) ? s_u0[t0 * kD + r] - x[2 * i] : 0.f;
+                    const float u1 = (t0 + 1 >= a && t0 + 1 < b) ? s_u0[(t0 + 1) * kD + r] - x[2 * i + 1] : 0.f;
+                    split2(u0, u1, hi[i], lo[i]);
                 }
-                tmem_st8(lane_addr + kColRU + half * 16, hi);
-                tmem_st8(lane_addr + kColRU + half * 16 + 8, hi + 8);
-                tmem_st8(lane_addr + kColRU + 32 + half * 16, lo);
-                tmem_st8(lane_addr + kColRU + 32 + half * 16 + 8, lo + 8);
-            }
-            tmem_wait_st();
-            tc_fence_before();
-            mbar_arrive(bRhsReady);
-            if (last) mbar_arrive(bVEmpty);
-            // ---- U^T as the hi/lo operand
-            {
-                const bool oku = mbar_wait(bUReady, ph_u, abort_flag);
-                if (!__all_sync(0xffffffffu, oku)) { dead = true; break; }
-                ph_u ^= 1u;
-            }
-            tc_fence_after();
-#pragma unroll
-            for (int half = 0; half < 2; ++half) {
-                float x[32];
-                uint32_t hi[16], lo[16];
-                tmem_ld32(lane_addr + kColWU + half * 32, reinterpret_cast<uint32_t*>(x));
-                tmem_wait_ld();
-#pragma unroll
-                for (int i = 0; i < 16; ++i) split2(x[2 * i], x[2 * i + 1], hi[i], lo[i]);
-                tmem_st8(lane_addr + kColRU + half * 16, hi);
-                tmem_st8(lane_addr + kColRU + half * 16 + 8, hi + 8);
-                tmem_st8(lane_addr + kColRU + 32 + half * 16, lo);
-                tmem_st8(lane_addr + kColRU + 32 + half * 16 + 8, lo + 8);
+                tmem_st8(lane_addr + kColU + tb / 2, hi);
+                tmem_st8(lane_addr + kColU + tb / 2 + 8, hi + 8);
+                tmem_st8(lane_addr + kColU + 32 + tb / 2, lo);
+                tmem_st8(lane_addr + kColU + 32 + tb / 2 + 8, lo + 8);
             }
             tmem_wait_st();
             tc_fence_before();
             mbar_arrive(bUhlReady);
+            if (last) mbar_arrive(bU0Empty);
             s_pending = true;
+            prev_a = a; prev_b = b; prev_row = row_t0;
             step.advance(kStepRing);
             if (store_slot >= 0) {
                 const bool oks = mbar_wait(bSReady, ph_s, abort_flag);
@@ -850,6 +925,7 @@ kda_tc_chain_kernel(const __grid_constant__ CUtensorMap tm_kt_h, const __grid_co
                 store_state(store_slot);
             }
         }
+        if (!dead && wg == 1 && prev_a >= 0) dead = !write_outputs(prev_a, prev_b, prev_row);
         if (!dead && slot_out >= 0) {
             bool oks = true;
             if (s_pending) oks = mbar_wait(bSReady, ph_s, abort_flag);
@@ -860,7 +936,7 @@ kda_tc_chain_kernel(const __grid_constant__ CUtensorMap tm_kt_h, const __grid_co
         }
     }
 
-    // ---- teardown
+    // ---- teardown (the second warpgroup has seen the last output product land: nothing is in flight)
     tc_fence_before();
     __syncthreads();
     if (*abort_flag) {
@@ -897,7 +973,7 @@ extern "C" int wpp_launch_kda_tc(const wpp::KdaTcParams* p, const CUtensorMap* m
         kda_tc_prep_kernel<<<grid_a, 128, PrepSmem::kBytes, st>>>(*p);
     }
     dim3 grid_b((unsigned)p->num_heads, (unsigned)p->num_requests);
-    kda_tc_chain_kernel<<<grid_b, 320, ChainSmem::kBytes, st>>>(maps[0], maps[1], maps[2], maps[3], maps[4], maps[5], maps[6],
-                                                               maps[7], maps[8], maps[9], maps[10], *p);
+    kda_tc_chain_kernel<<<grid_b, 352, ChainSmem::kBytes, st>>>(maps[0], maps[1], maps[2], maps[3], maps[4], maps[5], maps[6],
+                                                               maps[7], *p);
     return (int)cudaGetLastError();
 }
