@@ -533,21 +533,27 @@ struct StepRec {
     int64_t row_t0;      // row of the block's token 0 in the packed arrays
 };
 struct ChainSmem {
-    // operand tiles of one block, each a pair (hi, lo) of two 64-column tiles
-    static constexpr int kOffW0 = 0;                          // hi0 hi1 lo0 lo1
-    static constexpr int kOffQt = kOffW0 + 4 * kTileBytes;
-    static constexpr int kOffKb = kOffQt + 4 * kTileBytes;
+    // operand tiles of one block.  WQ: W0 and Qt stacked as one 128-row operand per 64-column tile (rows 0..63 W0,
+    // rows 64..127 Qt), so that X = W0 S_0' and the first part of the outputs, Qt S_0', are ONE product of N = 128:
+    // [W0 hi0 | Qt hi0][W0 hi1 | Qt hi1][W0 lo0 | Qt lo0][W0 lo1 | Qt lo1]
+    static constexpr int kOffWQ = 0;
+    static constexpr int kOffKb = kOffWQ + 8 * kTileBytes;    // hi0 hi1 lo0 lo1
     static constexpr int kOffM = kOffKb + 4 * kTileBytes;     // hi lo
     static constexpr int kOffU0 = kOffM + 2 * kTileBytes;     // fp32 [64][128], plain rows
-    static constexpr int kOffVec = kOffU0 + kL * kD * 4;      // per ring slot: alpha of the step's first token, decay product at its end
+    static constexpr int kOffOut = kOffU0 + kL * kD * 4;      // bf16 [64][128]: a step's outputs on their way to global memory
+    static constexpr int kOffVec = kOffOut + kL * kD * 2;     // per ring slot: alpha of the step's first token, decay product at its end
     static constexpr int kOffRec = kOffVec + kStepRing * 2 * kD * 4;
     static constexpr int kOffBars = kOffRec + kStepRing * (int)sizeof(StepRec);
-    static constexpr int kNumBars = 2 * kStepRing + 10 + 6;
+    static constexpr int kNumBars = 2 * kStepRing + 8 + 7;
     static constexpr int kOffMisc = kOffBars + 8 * kNumBars;
     static constexpr int kBytes = kOffMisc + 64 + 1024;
 };
-// tensor-memory columns: state, its hi/lo operand form, X = W0 S_0' (fp32), U as hi/lo operand, output accumulator
-constexpr uint32_t kColS = 0, kColShl = 128, kColX = 256, kColU = 320, kColO = 384;
+// tensor-memory columns: the state, its hi/lo operand form, and two result regions used by alternate steps.  A result
+// region holds X = W0 S_0' in its first 64 columns - replaced in place by U as a hi/lo operand: tokens 0..31 hi in
+// columns [0, 16), lo in [16, 32), tokens 32..63 hi in [32, 48), lo in [48, 64) - and the output accumulator in its
+// last 64 columns.
+constexpr uint32_t kColS = 0, kColShl = 128, kColD = 256;
+__device__ __forceinline__ uint32_t col_d(int step) { return kColD + 128u * (uint32_t)(step & 1); }
 
 __global__ void __launch_bounds__(352, 1)
 kda_tc_chain_kernel(const __grid_constant__ CUtensorMap tm_w0_h, const __grid_constant__ CUtensorMap tm_w0_l,
@@ -563,12 +569,14 @@ kda_tc_chain_kernel(const __grid_constant__ CUtensorMap tm_w0_h, const __grid_co
     auto bStepFull = [&](int s) { return bars + 8 * s; };
     auto bStepEmpty = [&](int s) { return bars + 8 * (kStepRing + s); };
     const uint32_t b0 = bars + 16 * kStepRing;
-    // operand buffers (one block in flight each): full at b0 + 16 i, empty at b0 + 16 i + 8 (W0 Qt Kb M U0)
-    const uint32_t bW0Full = b0, bW0Empty = b0 + 8, bQtFull = b0 + 16, bQtEmpty = b0 + 24, bKbFull = b0 + 32,
-                   bKbEmpty = b0 + 40, bMFull = b0 + 48, bMEmpty = b0 + 56, bU0Full = b0 + 64, bU0Empty = b0 + 72;
-    const uint32_t b1 = b0 + 80;
-    const uint32_t bShlReady = b1, bXReady = b1 + 8, bUhlReady = b1 + 16, bSReady = b1 + 24, bOReady = b1 + 32,
-                   bOFree = b1 + 40;
+    // operand buffers (one block in flight each), in the order a block's last step releases them: WQ, U0, Kb, M
+    const uint32_t bWQFull = b0, bWQEmpty = b0 + 8, bU0Full = b0 + 16, bU0Empty = b0 + 24, bKbFull = b0 + 32,
+                   bKbEmpty = b0 + 40, bMFull = b0 + 48, bMEmpty = b0 + 56;
+    const uint32_t b1 = b0 + 64;
+    const uint32_t bShlReady = b1, bXReady = b1 + 8, bUhlReady = b1 + 16, bSReady = b1 + 24, bOReady = b1 + 32;
+    // o_free, one per result region: a waiter may lag a barrier by at most one phase, and the issuing thread asks for
+    // the read-out of two steps back while the row threads may already have signalled the one after it
+    auto bOFree = [&](int n) { return b1 + 40 + 8 * (uint32_t)(n & 1); };
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(sm + CS::kOffMisc);
     volatile uint32_t* abort_flag = tmem_slot + 1;
     const float* s_vec = reinterpret_cast<const float*>(sm + CS::kOffVec);
@@ -600,11 +608,12 @@ kda_tc_chain_kernel(const __grid_constant__ CUtensorMap tm_w0_h, const __grid_co
 
     if (tid == 0) {
         for (int s = 0; s < kStepRing; ++s) { mbar_init(bStepFull(s), 1); mbar_init(bStepEmpty(s), 256 + 1); }
-        for (int i = 0; i < 4; ++i) { mbar_init(b0 + 16 * i, 1); mbar_init(b0 + 16 * i + 8, 1); }
+        mbar_init(bWQFull, 1); mbar_init(bWQEmpty, 1); mbar_init(bKbFull, 1); mbar_init(bKbEmpty, 1);
+        mbar_init(bMFull, 1); mbar_init(bMEmpty, 1);
         mbar_init(bU0Full, 1);
         mbar_init(bU0Empty, 256);          // the U0 tile is released by the 256 row threads
         mbar_init(bShlReady, 256); mbar_init(bXReady, 1); mbar_init(bUhlReady, 256); mbar_init(bSReady, 1);
-        mbar_init(bOReady, 1); mbar_init(bOFree, 128);
+        mbar_init(bOReady, 1); mbar_init(bOFree(0), 128); mbar_init(bOFree(1), 128);
         *abort_flag = 0u;
         fence_barrier_init();
     }
@@ -620,42 +629,41 @@ kda_tc_chain_kernel(const __grid_constant__ CUtensorMap tm_w0_h, const __grid_co
 
     if (warp == 8) {
         // ================================================================ operand loader
-        // One buffer per operand; a block's operands are released, in this order, as its last step proceeds (W0 after
-        // X, Qt after the first output product, U0 by the row threads, Kb after the state product, M after the second
-        // output product), and each is requested again for the next block the moment it is free.
+        // One buffer per operand; a block's operands are released, in this order, as its last step proceeds (WQ after
+        // the first product, U0 by the row threads, Kb after the state product, M after the second output product),
+        // and each is requested again for the next block the moment it is free.
         uint32_t ph_e = 0;
         for (int b = 0; b < g.n_blocks; ++b) {
             const size_t bh = (size_t)(gb0 + b) * H + head;
             const int row = (int)(bh * kL);
-            const CUtensorMap* mh[4] = {&tm_w0_h, &tm_qt_h, nullptr, &tm_kb_h};
-            const CUtensorMap* ml[4] = {&tm_w0_l, &tm_qt_l, nullptr, &tm_kb_l};
-            const uint32_t dst4[4] = {base + CS::kOffW0, base + CS::kOffQt, 0u, base + CS::kOffKb};
-            bool okw = true;
-#pragma unroll
-            for (int buf = 0; buf < 5 && okw; ++buf) {
-                // buffers in release order: 0 W0, 1 Qt, 2 U0 (barrier index 4), 3 Kb (index 2), 4 M (index 3)
-                const int bi = buf == 2 ? 4 : buf == 3 ? 2 : buf == 4 ? 3 : buf;
-                const uint32_t full = b0 + 16 * bi, empty = full + 8;
-                okw = mbar_wait(empty, ph_e ^ 1u, abort_flag);
-                okw = __all_sync(0xffffffffu, okw);
-                if (!okw) break;
-                if (buf == 2) {
-                    if (lane == 0) {
-                        mbar_arrive_expect_tx(full, kL * kD * 4);
-                        bulk_load(base + CS::kOffU0, p.ws_u0 + bh * (size_t)kL * kD, kL * kD * 4, full);
-                    }
-                } else if (buf == 4) {
-                    if (lane == 0) mbar_arrive_expect_tx(full, 2 * kTileBytes);
-                    __syncwarp();
-                    if (lane < 2) tma_load_2d(base + CS::kOffM + lane * kTileBytes, lane ? &tm_m_l : &tm_m_h, full, 0, row);
-                } else {
-                    if (lane == 0) mbar_arrive_expect_tx(full, 4 * kTileBytes);
-                    __syncwarp();
-                    if (lane < 4)
-                        tma_load_2d(dst4[buf] + lane * kTileBytes, (lane & 2) ? ml[buf] : mh[buf], full, (lane & 1) * 64, row);
-                }
-            }
+            bool okw = __all_sync(0xffffffffu, mbar_wait(bWQEmpty, ph_e ^ 1u, abort_flag));
             if (!okw) break;
+            if (lane == 0) mbar_arrive_expect_tx(bWQFull, 8 * kTileBytes);
+            __syncwarp();
+            if (lane < 8) {
+                // lane = 4 * (lo part) + 2 * (column half) + (0: W0, 1: Qt)
+                const bool lo_part = lane & 4, qt = lane & 1;
+                const int half = (lane >> 1) & 1;
+                const CUtensorMap* tm = qt ? (lo_part ? &tm_qt_l : &tm_qt_h) : (lo_part ? &tm_w0_l : &tm_w0_h);
+                tma_load_2d(base + CS::kOffWQ + ((lane >> 1) * 2 + (lane & 1)) * kTileBytes, tm, bWQFull, half * 64, row);
+            }
+            okw = __all_sync(0xffffffffu, mbar_wait(bU0Empty, ph_e ^ 1u, abort_flag));
+            if (!okw) break;
+            if (lane == 0) {
+                mbar_arrive_expect_tx(bU0Full, kL * kD * 4);
+                bulk_load(base + CS::kOffU0, p.ws_u0 + bh * (size_t)kL * kD, kL * kD * 4, bU0Full);
+            }
+            okw = __all_sync(0xffffffffu, mbar_wait(bKbEmpty, ph_e ^ 1u, abort_flag));
+            if (!okw) break;
+            if (lane == 0) mbar_arrive_expect_tx(bKbFull, 4 * kTileBytes);
+            __syncwarp();
+            if (lane < 4)
+                tma_load_2d(base + CS::kOffKb + lane * kTileBytes, (lane & 2) ? &tm_kb_l : &tm_kb_h, bKbFull, (lane & 1) * 64, row);
+            okw = __all_sync(0xffffffffu, mbar_wait(bMEmpty, ph_e ^ 1u, abort_flag));
+            if (!okw) break;
+            if (lane == 0) mbar_arrive_expect_tx(bMFull, 2 * kTileBytes);
+            __syncwarp();
+            if (lane < 2) tma_load_2d(base + CS::kOffM + lane * kTileBytes, lane ? &tm_m_l : &tm_m_h, bMFull, 0, row);
             ph_e ^= 1u;
         }
     } else if (warp == 10) {
@@ -715,26 +723,14 @@ kda_tc_chain_kernel(const __grid_constant__ CUtensorMap tm_w0_h, const __grid_co
     } else if (warp == 9 && lane == 0) {
         // ================================================================ MMA issuer
         Ring step = {0, 0};
-        uint32_t ph_w0 = 0, ph_qt = 0, ph_kb = 0, ph_m = 0;
-        uint32_t ph_shl = 0, ph_uhl = 0, ph_ofree = 0;
-        constexpr uint32_t idesc64 = idesc_bf16(64, 0, 0), idesc128mn = idesc_bf16(128, 0, 1);
-        const uint32_t tS = tmem + kColS, tShl = tmem + kColShl, tX = tmem + kColX, tU = tmem + kColU, tO = tmem + kColO;
-        // A (hi + lo, in tensor memory, `acols` columns per part) x B^T (hi + lo tiles in shared memory, K-major)
-        auto product_k = [&](uint32_t d, uint32_t a_tm, uint32_t acols, uint32_t b_hi, uint32_t b_lo, int ksteps, bool overwrite) {
-            const uint32_t aa[3] = {a_tm, a_tm, a_tm + acols}, bb[3] = {b_hi, b_lo, b_hi};
-            bool first = overwrite;
-#pragma unroll
-            for (int term = 0; term < 3; ++term) {
-                const uint64_t bd = smem_desc_sw128(bb[term], 16, 1024);
-#pragma unroll 4
-                for (int kk = 0; kk < ksteps; ++kk) {
-                    const uint64_t off = (uint64_t)(((kk >> 2) * kTileBytes + (kk & 3) * 32) >> 4);
-                    mma_ts(d, aa[term] + kk * 8, bd + off, idesc64, first ? 0u : 1u);
-                    first = false;
-                }
-            }
-        };
-        bool first_step = true;
+        uint32_t ph_wq = 0, ph_kb = 0, ph_m = 0, ph_shl = 0, ph_uhl = 0, ph_ofree[2] = {0, 0};
+        constexpr uint32_t idesc64 = idesc_bf16(64, 0, 0), idesc128 = idesc_bf16(128, 0, 0), idesc128mn = idesc_bf16(128, 0, 1);
+        const uint32_t tS = tmem + kColS, tShl = tmem + kColShl;
+        // descriptors of the operand buffers (they never move)
+        const uint64_t wq_hi = smem_desc_sw128(base + CS::kOffWQ, 16, 1024), wq_lo = smem_desc_sw128(base + CS::kOffWQ + 4 * kTileBytes, 16, 1024);
+        const uint64_t kb_hi = smem_desc_sw128(base + CS::kOffKb, kTileBytes, 1024), kb_lo = smem_desc_sw128(base + CS::kOffKb + 2 * kTileBytes, kTileBytes, 1024);
+        const uint64_t m_hi = smem_desc_sw128(base + CS::kOffM, 16, 1024), m_lo = smem_desc_sw128(base + CS::kOffM + kTileBytes, 16, 1024);
+        int n = 0;                     // step counter: selects the result region
         while (true) {
             if (!mbar_wait(bStepFull(step.stage), step.phase, abort_flag)) break;
             const int a = s_rec[step.stage].a;
@@ -742,42 +738,51 @@ kda_tc_chain_kernel(const __grid_constant__ CUtensorMap tm_w0_h, const __grid_co
             mbar_arrive(bStepEmpty(step.stage));
             step.advance(kStepRing);
             if (a < 0) break;
-            // ---- X^T = S_0'^T W0^T
+            const uint32_t tD = tmem + col_d(n);
+            // ---- [X^T | O^T] = S_0'^T [W0; Qt]^T   (the region's previous outputs, two steps back, must have been read)
+            if (n >= 2) { if (!mbar_wait(bOFree(n), ph_ofree[n & 1], abort_flag)) break; ph_ofree[n & 1] ^= 1u; }
             if (!mbar_wait(bShlReady, ph_shl, abort_flag)) break;
             ph_shl ^= 1u;
-            if (first) { if (!mbar_wait(bW0Full, ph_w0, abort_flag)) break; ph_w0 ^= 1u; }
+            if (first) { if (!mbar_wait(bWQFull, ph_wq, abort_flag)) break; ph_wq ^= 1u; }
             tc_fence_after();
-            product_k(tX, tShl, 64, base + CS::kOffW0, base + CS::kOffW0 + 2 * kTileBytes, 8, true);
+#pragma unroll
+            for (int term = 0; term < 3; ++term) {
+                const uint32_t a_tm = tShl + (term == 2 ? 64u : 0u);
+                const uint64_t bd = (term == 1) ? wq_lo : wq_hi;
+#pragma unroll
+                for (int kk = 0; kk < 8; ++kk) {
+                    const uint64_t off = (uint64_t)(((kk >> 2) * 2 * kTileBytes + (kk & 3) * 32) >> 4);
+                    if (term == 0 && kk == 0) mma_ts_overwrite(tD, a_tm, bd + off, idesc128);
+                    else mma_ts_accumulate(tD, a_tm + kk * 8, bd + off, idesc128);
+                }
+            }
             mma_commit(bXReady);
-            if (last) mma_commit(bW0Empty);
-            // ---- O^T = S_0'^T Qt^T (the previous step's output must have been read out)
-            if (!first_step) { if (!mbar_wait(bOFree, ph_ofree, abort_flag)) break; ph_ofree ^= 1u; }
-            first_step = false;
-            if (first) { if (!mbar_wait(bQtFull, ph_qt, abort_flag)) break; ph_qt ^= 1u; }
-            tc_fence_after();
-            product_k(tO, tShl, 64, base + CS::kOffQt, base + CS::kOffQt + 2 * kTileBytes, 8, true);
-            if (last) mma_commit(bQtEmpty);
+            if (last) mma_commit(bWQEmpty);
             // ---- S_b^T += U^T Kb   (the accumulator was preset to the decayed S_0'),   O^T += U^T M^T
             if (!mbar_wait(bUhlReady, ph_uhl, abort_flag)) break;
             ph_uhl ^= 1u;
             if (first) { if (!mbar_wait(bKbFull, ph_kb, abort_flag)) break; ph_kb ^= 1u; }
             tc_fence_after();
-            {
-                const uint32_t kb_hi = base + CS::kOffKb, kb_lo = kb_hi + 2 * kTileBytes;
-                const uint32_t aa[3] = {tU, tU, tU + 32}, bb[3] = {kb_hi, kb_lo, kb_hi};
 #pragma unroll
-                for (int term = 0; term < 3; ++term) {
-                    const uint64_t bd = smem_desc_sw128(bb[term], kTileBytes, 1024);      // MN-major: 64-column halves kTileBytes apart
+            for (int term = 0; term < 3; ++term) {
+                const uint64_t bd = (term == 1) ? kb_lo : kb_hi;          // MN-major: 64-column halves kTileBytes apart
 #pragma unroll
-                    for (int kk = 0; kk < 4; ++kk) mma_ts(tS, aa[term] + kk * 8, bd + (uint64_t)(kk * 128), idesc128mn, 1u);
-                }
+                for (int kk = 0; kk < 4; ++kk)
+                    mma_ts_accumulate(tS, tD + (kk >> 1) * 32 + (kk & 1) * 8 + (term == 2 ? 16u : 0u), bd + (uint64_t)(kk * 128), idesc128mn);
             }
             mma_commit(bSReady);
             if (last) mma_commit(bKbEmpty);
             if (first) { if (!mbar_wait(bMFull, ph_m, abort_flag)) break; ph_m ^= 1u; }
-            product_k(tO, tU, 32, base + CS::kOffM, base + CS::kOffM + kTileBytes, 4, false);
+#pragma unroll
+            for (int term = 0; term < 3; ++term) {
+                const uint64_t bd = (term == 1) ? m_lo : m_hi;
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk)
+                    mma_ts_accumulate(tD + 64, tD + (kk >> 1) * 32 + (kk & 1) * 8 + (term == 2 ? 16u : 0u), bd + (uint64_t)(kk * 2), idesc64);
+            }
             mma_commit(bOReady);
             if (last) mma_commit(bMEmpty);
+            ++n;
         }
     } else if (warp < 8) {
         // ================================================================ the state's rows (thread r = column r of S)
@@ -808,22 +813,33 @@ kda_tc_chain_kernel(const __grid_constant__ CUtensorMap tm_w0_h, const __grid_co
                 for (int i = 0; i < 32; ++i) dst[(size_t)(c0 + i) * kD] = x[i];
             }
         };
-        // outputs of a finished step (second warpgroup): rows [a, b) of the block
+        // outputs of a finished step (second warpgroup): rows [a, b) of the block, from result region `n`.  A thread
+        // holds one value column of all 64 tokens; the tile is turned round in shared memory so that global memory
+        // sees 16-byte stores of whole rows.
         uint32_t ph_o = 0;
-        auto write_outputs = [&](int a, int b, int64_t row_t0) -> bool {
+        __nv_bfloat16* s_out = reinterpret_cast<__nv_bfloat16*>(sm + CS::kOffOut);
+        auto write_outputs = [&](int a, int b, int64_t row_t0, int n) -> bool {
             const bool oko = mbar_wait(bOReady, ph_o, abort_flag);
             if (!__all_sync(0xffffffffu, oko)) return false;
             ph_o ^= 1u;
             tc_fence_after();
             float o[64];
-            tmem_ld32(lane_addr + kColO, reinterpret_cast<uint32_t*>(o));
-            tmem_ld32(lane_addr + kColO + 32, reinterpret_cast<uint32_t*>(o) + 32);
+            tmem_ld32(lane_addr + col_d(n) + 64, reinterpret_cast<uint32_t*>(o));
+            tmem_ld32(lane_addr + col_d(n) + 96, reinterpret_cast<uint32_t*>(o) + 32);
             tmem_wait_ld();
             tc_fence_before();
-            mbar_arrive(bOFree);
+            mbar_arrive(bOFree(n));
 #pragma unroll
-            for (int t = 0; t < kL; ++t)
-                if (t >= a && t < b) p.out[((row_t0 + t) * H + head) * kD + r] = __float2bfloat16_rn(o[t]);
+            for (int t = 0; t < kL; ++t) s_out[t * kD + r] = __float2bfloat16_rn(o[t]);
+            named_bar(1, 128);
+#pragma unroll
+            for (int it = 0; it < 8; ++it) {
+                const int item = it * 128 + r, t = item >> 4, c0 = (item & 15) * 8;
+                if (t >= a && t < b)
+                    *reinterpret_cast<uint4*>(p.out + ((row_t0 + t) * H + head) * kD + c0) =
+                        *reinterpret_cast<const uint4*>(s_out + t * kD + c0);
+            }
+            named_bar(1, 128);                   // the tile may be overwritten by the next step's outputs
             return true;
         };
         Ring step = {0, 0};
@@ -832,6 +848,7 @@ kda_tc_chain_kernel(const __grid_constant__ CUtensorMap tm_w0_h, const __grid_co
         bool dead = false;
         int prev_a = -1, prev_b = -1;    // the step whose outputs are still to be written
         int64_t prev_row = 0;
+        int n = 0;
         while (!dead) {
             const bool okw = mbar_wait(bStepFull(step.stage), step.phase, abort_flag);
             if (!__all_sync(0xffffffffu, okw)) { dead = true; break; }
@@ -866,20 +883,16 @@ kda_tc_chain_kernel(const __grid_constant__ CUtensorMap tm_w0_h, const __grid_co
                     x[2 * i] = y0 * en.x;
                     x[2 * i + 1] = y1 * en.y;
                 }
-                tmem_st32(lane_addr + kColS + cbase, reinterpret_cast<const uint32_t*>(x));
-                tmem_st32(lane_addr + kColS + cbase + 32, reinterpret_cast<const uint32_t*>(x) + 32);
                 tmem_st32(lane_addr + kColShl + cbase / 2, hi);
                 tmem_st32(lane_addr + kColShl + 64 + cbase / 2, lo);
+                tmem_st32(lane_addr + kColS + cbase, reinterpret_cast<const uint32_t*>(x));
+                tmem_st32(lane_addr + kColS + cbase + 32, reinterpret_cast<const uint32_t*>(x) + 32);
             }
             tmem_wait_st();
             tc_fence_before();
             mbar_arrive(bShlReady);
             mbar_arrive(bStepEmpty(slot_ring));      // the record and its vectors have been consumed
-            // ---- the second warpgroup writes the previous step's outputs while X is being computed
-            if (wg == 1 && prev_a >= 0) {
-                if (!write_outputs(prev_a, prev_b, prev_row)) { dead = true; break; }
-            }
-            // ---- U^T = (U0 - X)^T for the step's tokens, zero elsewhere, as the hi/lo operand
+            // ---- U^T = (U0 - X)^T for the step's tokens, zero elsewhere, as the hi/lo operand, in place of X
             if (first) {
                 const bool oku = mbar_wait(bU0Full, ph_u0, abort_flag);
                 if (!__all_sync(0xffffffffu, oku)) { dead = true; break; }
@@ -895,7 +908,7 @@ kda_tc_chain_kernel(const __grid_constant__ CUtensorMap tm_w0_h, const __grid_co
                 const int tb = wg * 32;
                 float x[32];
                 uint32_t hi[16], lo[16];
-                tmem_ld32(lane_addr + kColX + tb, reinterpret_cast<uint32_t*>(x));
+                tmem_ld32(lane_addr + col_d(n) + tb, reinterpret_cast<uint32_t*>(x));
                 tmem_wait_ld();
 #pragma unroll
                 for (int i = 0; i < 16; ++i) {
@@ -904,18 +917,23 @@ kda_tc_chain_kernel(const __grid_constant__ CUtensorMap tm_w0_h, const __grid_co
                     const float u1 = (t0 + 1 >= a && t0 + 1 < b) ? s_u0[(t0 + 1) * kD + r] - x[2 * i + 1] : 0.f;
                     split2(u0, u1, hi[i], lo[i]);
                 }
-                tmem_st8(lane_addr + kColU + tb / 2, hi);
-                tmem_st8(lane_addr + kColU + tb / 2 + 8, hi + 8);
-                tmem_st8(lane_addr + kColU + 32 + tb / 2, lo);
-                tmem_st8(lane_addr + kColU + 32 + tb / 2 + 8, lo + 8);
+                tmem_st8(lane_addr + col_d(n) + tb, hi);
+                tmem_st8(lane_addr + col_d(n) + tb + 8, hi + 8);
+                tmem_st8(lane_addr + col_d(n) + tb + 16, lo);
+                tmem_st8(lane_addr + col_d(n) + tb + 24, lo + 8);
             }
             tmem_wait_st();
             tc_fence_before();
             mbar_arrive(bUhlReady);
             if (last) mbar_arrive(bU0Empty);
             s_pending = true;
+            // ---- the second warpgroup writes the previous step's outputs while the state product runs
+            if (wg == 1 && prev_a >= 0) {
+                if (!write_outputs(prev_a, prev_b, prev_row, n - 1)) { dead = true; break; }
+            }
             prev_a = a; prev_b = b; prev_row = row_t0;
             step.advance(kStepRing);
+            ++n;
             if (store_slot >= 0) {
                 const bool oks = mbar_wait(bSReady, ph_s, abort_flag);
                 if (!__all_sync(0xffffffffu, oks)) { dead = true; break; }
@@ -925,7 +943,7 @@ kda_tc_chain_kernel(const __grid_constant__ CUtensorMap tm_w0_h, const __grid_co
                 store_state(store_slot);
             }
         }
-        if (!dead && wg == 1 && prev_a >= 0) dead = !write_outputs(prev_a, prev_b, prev_row);
+        if (!dead && wg == 1 && prev_a >= 0) dead = !write_outputs(prev_a, prev_b, prev_row, n - 1);
         if (!dead && slot_out >= 0) {
             bool oks = true;
             if (s_pending) oks = mbar_wait(bSReady, ph_s, abort_flag);
