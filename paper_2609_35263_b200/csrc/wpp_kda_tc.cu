@@ -53,8 +53,8 @@ constexpr int kTileBytes = kL * 128;   // one 64-row x 128-byte swizzled tile (8
 // hi/lo split of two fp32 values into two packed bf16 pairs (element 0 in the low half)
 __device__ __forceinline__ void split2(float x0, float x1, uint32_t& hi, uint32_t& lo) {
     hi = pack_bf16x2(x0, x1);
-    const float h0 = __uint_as_float(hi << 16), h1 = __uint_as_float(hi & 0xffff0000u);
-    lo = pack_bf16x2(x0 - h0, x1 - h1);
+    const float2 d = __fadd2_rn(make_float2(x0, x1), make_float2(-__uint_as_float(hi << 16), -__uint_as_float(hi & 0xffff0000u)));
+    lo = pack_bf16x2(d.x, d.y);
 }
 
 // byte offset of 16-byte chunk j of row t inside a 128-byte-swizzled tile of 128-byte rows
@@ -129,7 +129,7 @@ __global__ void __launch_bounds__(1024) kda_tc_setup_kernel(const KdaTcParams p)
 }
 
 // ---------------------------------------------------------------------------------------------------------------
-// Preparation: one CTA (128 threads) per (block, head).  Shared memory is three regions of 32 KB that change roles:
+// Preparation: one CTA (256 threads) per (block, head).  Shared memory is three regions of 32 KB that change roles:
 //   R0: alpha, then the decay products G (fp32 [64][128]); then Qt as an MMA operand; then T (hi tile, lo tile) and,
 //       behind them, the inverse it is made from
 //   R1: Kt as an MMA operand (A of Kt Kh^T, later B of T Kt)
@@ -144,7 +144,9 @@ struct PrepSmem {
     static constexpr int kBytes = kOffMisc + 1024 + 1024;     // + alignment slack
 };
 
-__global__ void __launch_bounds__(128) kda_tc_prep_kernel(const KdaTcParams p) {
+constexpr int kPrepThreads = 256;
+
+__global__ void __launch_bounds__(kPrepThreads, 2) kda_tc_prep_kernel(const KdaTcParams p) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* sm = smem_raw + (base - smem_u32(smem_raw));
@@ -153,7 +155,8 @@ __global__ void __launch_bounds__(128) kda_tc_prep_kernel(const KdaTcParams p) {
     uint8_t* r1 = sm + PrepSmem::kOffR1;
     uint8_t* r2 = sm + PrepSmem::kOffR2;
     float* s_beta = reinterpret_cast<float*>(sm + PrepSmem::kOffMisc);              // [64]
-    int* s_red = reinterpret_cast<int*>(sm + PrepSmem::kOffMisc + 256);             // [4]
+    float* s_red = reinterpret_cast<float*>(sm + PrepSmem::kOffMisc + 256);         // [8]
+    int* s_redi = reinterpret_cast<int*>(sm + PrepSmem::kOffMisc + 320);            // [4]
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(sm + PrepSmem::kOffMisc + 512);
     volatile uint32_t* abort_flag = tmem_slot + 1;
     const uint32_t bar = base + PrepSmem::kOffMisc + 528;
@@ -186,64 +189,118 @@ __global__ void __launch_bounds__(128) kda_tc_prep_kernel(const KdaTcParams p) {
         tmem_relinquish();
     }
     // ---- alpha and beta of the block (inactive tokens: alpha 1, beta 0)
-    for (int it = 0; it < 16; ++it) {
-        const int item = it * 128 + tid, t = item >> 5, c4 = (item & 31) * 4;
-        float4 a = make_float4(1.f, 1.f, 1.f, 1.f);
-        if (t >= t_lo && t < t_hi) a = *reinterpret_cast<const float4*>(p.alpha + ((row_t0 + t) * H + head) * kD + c4);
-        *reinterpret_cast<float4*>(G + t * kD + c4) = a;
-    }
+    auto load_alpha = [&]() {
+#pragma unroll
+        for (int it = 0; it < 8; ++it) {
+            const int item = it * kPrepThreads + tid, t = item >> 5, c4 = (item & 31) * 4;
+            float4 a = make_float4(1.f, 1.f, 1.f, 1.f);
+            if (t >= t_lo && t < t_hi) a = *reinterpret_cast<const float4*>(p.alpha + ((row_t0 + t) * H + head) * kD + c4);
+            *reinterpret_cast<float4*>(G + t * kD + c4) = a;
+        }
+    };
+    load_alpha();
     if (tid < kL) s_beta[tid] = (tid >= t_lo && tid < t_hi) ? p.beta[(row_t0 + tid) * H + head] : 0.f;
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
 
-    // ---- cuts.  A sub-block starts at the first active token, after every token that completes a periodic
-    //      snapshot position, and at every token whose alpha would push a channel's decay product below 2^-40.
+    // ---- cuts and decay products.  A sub-block starts at the first active token and after every token that completes
+    //      a periodic snapshot position; with those cuts alone the decay products (from each sub-block's start, the
+    //      start's own alpha excluded) are formed by two threads per channel, one per half of the block, the second
+    //      half picking up the first half's last value.  Only if some product fell below 2^-40 are the extra cuts
+    //      found, one at a time, by the slow path below.
     uint64_t mask = 1ull << t_lo;
     if (p.snap_interval > 0) {
         for (int t = t_lo; t + 1 < t_hi; ++t)
             if (((int64_t)blk * kL + t + 1) % p.snap_interval == 0) mask |= 1ull << (t + 1);
     }
-    for (int round = 0; round < kL; ++round) {
-        // thread c follows channel c: the first token whose decay product (from its sub-block's start) is too small
-        int first_bad = kL;
-        float gacc = 1.f;
-        for (int t = t_lo + 1; t < t_hi; ++t) {
-            if ((mask >> t) & 1ull) { gacc = 1.f; continue; }
-            gacc *= G[t * kD + tid];
-            if (gacc < kMinGamma) { first_bad = t; break; }
-        }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) first_bad = min(first_bad, __shfl_xor_sync(0xffffffffu, first_bad, o));
-        if (lane == 0) s_red[warp] = first_bad;
-        __syncthreads();
-        first_bad = min(min(s_red[0], s_red[1]), min(s_red[2], s_red[3]));
-        __syncthreads();
-        if (first_bad >= kL) break;
-        mask |= 1ull << first_bad;
-    }
-    // decay products in place of alpha; the last row of every sub-block goes to the workspace (the chain scales
-    // the state by it)
+    const int ch = tid & 127, half = tid >> 7;
+    float gmin = 1.f;
     {
         float gacc = 1.f;
-        for (int t = 0; t < kL; ++t) {
-            if (t < t_lo || t >= t_hi) { G[t * kD + tid] = 1.f; continue; }
-            gacc = ((mask >> t) & 1ull) ? 1.f : gacc * G[t * kD + tid];
-            G[t * kD + tid] = gacc;
-            if (t + 1 == t_hi || ((mask >> (t + 1)) & 1ull)) p.ws_e[(bh * kL + t) * kD + tid] = gacc;
+        const int tb = half * 32;
+#pragma unroll 8
+        for (int t = tb; t < tb + 32; ++t) {
+            const bool active = t >= t_lo && t < t_hi;
+            gacc = (!active || ((mask >> t) & 1ull)) ? 1.f : gacc * G[t * kD + ch];
+            G[t * kD + ch] = gacc;
+        }
+    }
+    __syncthreads();
+    if (half == 1) {
+        // tokens 32.. up to the first cut in this half continue the first half's product
+        const uint64_t cuts = mask >> 32;
+        const int n_carry = cuts ? (__ffsll((long long)cuts) - 1) : 32;
+        const float carry = (31 >= t_lo && 31 < t_hi) ? G[31 * kD + ch] : 1.f;
+        for (int t = 32; t < 32 + n_carry; ++t)
+            if (t >= t_lo && t < t_hi) G[t * kD + ch] *= carry;
+    }
+    __syncthreads();
+    {
+        const int tb = half * 32;
+#pragma unroll 8
+        for (int t = tb; t < tb + 32; ++t) gmin = fminf(gmin, G[t * kD + ch]);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) gmin = fminf(gmin, __shfl_xor_sync(0xffffffffu, gmin, o));
+        if (lane == 0) s_red[warp] = gmin;
+        __syncthreads();
+        gmin = fminf(fminf(fminf(s_red[0], s_red[1]), fminf(s_red[2], s_red[3])),
+                     fminf(fminf(s_red[4], s_red[5]), fminf(s_red[6], s_red[7])));
+    }
+    if (!(gmin >= kMinGamma)) {
+        // ---- slow path (rare): some channel decays below 2^-40 inside a sub-block.  The token that causes it starts a
+        //      new sub-block; thread c < 128 follows channel c, the cuts are found one at a time.
+        __syncthreads();
+        load_alpha();
+        __syncthreads();
+        for (int round = 0; round < kL; ++round) {
+            int first_bad = kL;
+            if (tid < 128) {
+                float gacc = 1.f;
+                for (int t = t_lo + 1; t < t_hi; ++t) {
+                    if ((mask >> t) & 1ull) { gacc = 1.f; continue; }
+                    gacc *= G[t * kD + tid];
+                    if (!(gacc >= kMinGamma)) { first_bad = t; break; }
+                }
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) first_bad = min(first_bad, __shfl_xor_sync(0xffffffffu, first_bad, o));
+                if (lane == 0) s_redi[warp] = first_bad;
+            }
+            __syncthreads();
+            first_bad = min(min(s_redi[0], s_redi[1]), min(s_redi[2], s_redi[3]));
+            __syncthreads();
+            if (first_bad >= kL) break;
+            mask |= 1ull << first_bad;
+        }
+        if (tid < 128) {
+            float gacc = 1.f;
+            for (int t = 0; t < kL; ++t) {
+                if (t < t_lo || t >= t_hi) { G[t * kD + tid] = 1.f; continue; }
+                gacc = ((mask >> t) & 1ull) ? 1.f : gacc * G[t * kD + tid];
+                G[t * kD + tid] = gacc;
+            }
+        }
+        __syncthreads();
+    }
+    // the last row of every sub-block goes to the workspace (the chain scales the state by it)
+    if (tid < 128) {
+        int a = t_lo;
+        while (a < t_hi) {
+            const int e = sub_end(mask, a, t_hi);
+            p.ws_e[(bh * kL + e - 1) * kD + tid] = G[(e - 1) * kD + tid];
+            a = e;
         }
     }
     if (tid == 0) p.ws_mask[bh] = mask;
-    __syncthreads();
 
     // ---- Kt = k G, Kh = k / G, Kb = Kh G_end, Qt = q G as hi/lo bf16.  Kt and Kh go to shared memory (MMA operands), Kb
     //      and Qt to the workspace; Qt also waits in registers for the region the decay products occupy.  A thread handles
     //      8 consecutive channels of a token at a time.
-    uint4 qt_h[8], qt_l[8];
+    uint4 qt_h[4], qt_l[4];
 #pragma unroll
-    for (int it = 0; it < 8; ++it) {
-        const int item = it * 128 + tid, t = item >> 4, ch = item & 15, c0 = ch * 8;
+    for (int it = 0; it < 4; ++it) {
+        const int item = it * kPrepThreads + tid, t = item >> 4, c8 = item & 15, c0 = c8 * 8;
         const bool active = t >= t_lo && t < t_hi;
         uint4 kt_h = make_uint4(0, 0, 0, 0), kt_l = kt_h, kh_h = kt_h, kh_l = kt_h, kb_h = kt_h, kb_l = kt_h;
         qt_h[it] = kt_h; qt_l[it] = kt_h;
@@ -257,20 +314,20 @@ __global__ void __launch_bounds__(128) kda_tc_prep_kernel(const KdaTcParams p) {
             for (int w = 0; w < 4; ++w) {
                 const float k0 = __uint_as_float(rw[w] << 16), k1 = __uint_as_float(rw[w] & 0xffff0000u);
                 const float q0 = __uint_as_float(rq[w] << 16), q1 = __uint_as_float(rq[w] & 0xffff0000u);
-                const float g0 = G[t * kD + c0 + 2 * w], g1 = G[t * kD + c0 + 2 * w + 1];
-                const float e0 = G[e_t * kD + c0 + 2 * w], e1 = G[e_t * kD + c0 + 2 * w + 1];
-                const float i0 = __frcp_rn(g0), i1 = __frcp_rn(g1);       // g >= 2^-40: finite
-                split2(k0 * g0, k1 * g1, o[0][w], o[1][w]);
+                const float2 gg = *reinterpret_cast<const float2*>(G + t * kD + c0 + 2 * w);
+                const float2 ee = *reinterpret_cast<const float2*>(G + e_t * kD + c0 + 2 * w);
+                const float i0 = __frcp_rn(gg.x), i1 = __frcp_rn(gg.y);       // g >= 2^-40: finite
+                split2(k0 * gg.x, k1 * gg.y, o[0][w], o[1][w]);
                 split2(k0 * i0, k1 * i1, o[2][w], o[3][w]);
-                split2(k0 * (e0 * i0), k1 * (e1 * i1), o[4][w], o[5][w]);
-                split2(q0 * g0, q1 * g1, o[6][w], o[7][w]);
+                split2(k0 * (ee.x * i0), k1 * (ee.y * i1), o[4][w], o[5][w]);
+                split2(q0 * gg.x, q1 * gg.y, o[6][w], o[7][w]);
             }
             kt_h = make_uint4(o[0][0], o[0][1], o[0][2], o[0][3]); kt_l = make_uint4(o[1][0], o[1][1], o[1][2], o[1][3]);
             kh_h = make_uint4(o[2][0], o[2][1], o[2][2], o[2][3]); kh_l = make_uint4(o[3][0], o[3][1], o[3][2], o[3][3]);
             kb_h = make_uint4(o[4][0], o[4][1], o[4][2], o[4][3]); kb_l = make_uint4(o[5][0], o[5][1], o[5][2], o[5][3]);
             qt_h[it] = make_uint4(o[6][0], o[6][1], o[6][2], o[6][3]); qt_l[it] = make_uint4(o[7][0], o[7][1], o[7][2], o[7][3]);
         }
-        const uint32_t off = (uint32_t)((ch >> 3) * kTileBytes) + sw_off(t, ch & 7);
+        const uint32_t off = (uint32_t)((c8 >> 3) * kTileBytes) + sw_off(t, c8 & 7);
         *reinterpret_cast<uint4*>(r1 + off) = kt_h;
         *reinterpret_cast<uint4*>(r1 + 2 * kTileBytes + off) = kt_l;
         *reinterpret_cast<uint4*>(r2 + off) = kh_h;
@@ -283,9 +340,9 @@ __global__ void __launch_bounds__(128) kda_tc_prep_kernel(const KdaTcParams p) {
     }
     __syncthreads();                       // every read of the decay products is done: Qt takes their place
 #pragma unroll
-    for (int it = 0; it < 8; ++it) {
-        const int item = it * 128 + tid, t = item >> 4, ch = item & 15;
-        const uint32_t off = (uint32_t)((ch >> 3) * kTileBytes) + sw_off(t, ch & 7);
+    for (int it = 0; it < 4; ++it) {
+        const int item = it * kPrepThreads + tid, t = item >> 4, c8 = item & 15;
+        const uint32_t off = (uint32_t)((c8 >> 3) * kTileBytes) + sw_off(t, c8 & 7);
         *reinterpret_cast<uint4*>(r0 + off) = qt_h[it];
         *reinterpret_cast<uint4*>(r0 + 2 * kTileBytes + off) = qt_l[it];
     }
@@ -314,62 +371,66 @@ __global__ void __launch_bounds__(128) kda_tc_prep_kernel(const KdaTcParams p) {
         mma_commit(bar);
     }
     // the block's values, on their way while the products run
-    uint4 vraw[8];
+    uint4 vraw[4];
 #pragma unroll
-    for (int it = 0; it < 8; ++it) {
-        const int item = it * 128 + tid, t = item >> 4, c0 = (item & 15) * 8;
+    for (int it = 0; it < 4; ++it) {
+        const int item = it * kPrepThreads + tid, t = item >> 4, c0 = (item & 15) * 8;
         vraw[it] = make_uint4(0, 0, 0, 0);
         if (t >= t_lo && t < t_hi) vraw[it] = *reinterpret_cast<const uint4*>(p.v + ((row_t0 + t) * H + head) * kD + c0);
     }
     bool ok = __syncthreads_and(mbar_wait(bar, 0, abort_flag));
     tc_fence_after();
 
-    // ---- rows of the two products (thread t < 64 owns token t = tensor-memory lane t).  The triangular matrix goes
-    //      to shared memory (over the Kh tiles: both products have completed), M = tril(Qt Kh^T) to the workspace;
-    //      the V tile goes behind the triangular matrix.
-    float* Amat = reinterpret_cast<float*>(r2);          // [64][64] fp32: beta_t (Kt Kh^T)[t][s] for s < t in the sub-block
+    // ---- rows of the two products (token t = tensor-memory lane t): warps 0, 1 take Kt Kh^T, whose strictly lower part
+    //      within a sub-block, scaled by beta_t, is the triangular matrix (to shared memory, over the Kh tiles: both
+    //      products have completed); warps 4, 5 take M = tril(Qt Kh^T), which goes to the workspace.  The V tile goes behind
+    //      the triangular matrix.
+    float* Amat = reinterpret_cast<float*>(r2);          // [64][64] fp32
     uint8_t* vtile = r2 + 2 * kTileBytes;                // two 64-column tiles, tokens as rows
 #pragma unroll
-    for (int it = 0; it < 8; ++it) {
-        const int item = it * 128 + tid, t = item >> 4, ch = item & 15;
-        *reinterpret_cast<uint4*>(vtile + (ch >> 3) * kTileBytes + sw_off(t, ch & 7)) = vraw[it];
+    for (int it = 0; it < 4; ++it) {
+        const int item = it * kPrepThreads + tid, t = item >> 4, c8 = item & 15;
+        *reinterpret_cast<uint4*>(vtile + (c8 >> 3) * kTileBytes + sw_off(t, c8 & 7)) = vraw[it];
     }
-    if (warp < 2 && ok) {
-        const int t = tid;
+    if ((warp & 3) < 2 && ok) {
+        const int t = (warp & 3) * 32 + lane;
         const bool active = t >= t_lo && t < t_hi;
         const int s0 = active ? sub_start(mask, t) : kL;    // columns [s0, t) (and t itself for M) count
-        const uint32_t lane_addr = tmem + ((uint32_t)(warp * 32) << 16);
-        const float bt = s_beta[t];
+        const uint32_t lane_addr = tmem + ((uint32_t)((warp & 3) * 32) << 16);
         float x[64];
-        tmem_ld32(lane_addr, reinterpret_cast<uint32_t*>(x));
-        tmem_ld32(lane_addr + 32, reinterpret_cast<uint32_t*>(x) + 32);
-        tmem_wait_ld();
+        if (warp < 4) {
+            const float bt = s_beta[t];
+            tmem_ld32(lane_addr, reinterpret_cast<uint32_t*>(x));
+            tmem_ld32(lane_addr + 32, reinterpret_cast<uint32_t*>(x) + 32);
+            tmem_wait_ld();
 #pragma unroll
-        for (int s4 = 0; s4 < 16; ++s4) {
-            float4 a;
-            a.x = (active && 4 * s4 + 0 >= s0 && 4 * s4 + 0 < t) ? bt * x[4 * s4 + 0] : 0.f;
-            a.y = (active && 4 * s4 + 1 >= s0 && 4 * s4 + 1 < t) ? bt * x[4 * s4 + 1] : 0.f;
-            a.z = (active && 4 * s4 + 2 >= s0 && 4 * s4 + 2 < t) ? bt * x[4 * s4 + 2] : 0.f;
-            a.w = (active && 4 * s4 + 3 >= s0 && 4 * s4 + 3 < t) ? bt * x[4 * s4 + 3] : 0.f;
-            *reinterpret_cast<float4*>(Amat + t * kL + 4 * s4) = a;
-        }
-        tmem_ld32(lane_addr + 64, reinterpret_cast<uint32_t*>(x));
-        tmem_ld32(lane_addr + 96, reinterpret_cast<uint32_t*>(x) + 32);
-        tmem_wait_ld();
-        __nv_bfloat16* mh = p.ws_m_h + (bh * kL + t) * kL;
-        __nv_bfloat16* ml = p.ws_m_l + (bh * kL + t) * kL;
-#pragma unroll
-        for (int i8 = 0; i8 < 8; ++i8) {
-            uint32_t oh[4], ol[4];
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const int s = i8 * 8 + 2 * i;
-                const float m0 = (active && s >= s0 && s <= t) ? x[s] : 0.f;
-                const float m1 = (active && s + 1 >= s0 && s + 1 <= t) ? x[s + 1] : 0.f;
-                split2(m0, m1, oh[i], ol[i]);
+            for (int s4 = 0; s4 < 16; ++s4) {
+                float4 a;
+                a.x = (active && 4 * s4 + 0 >= s0 && 4 * s4 + 0 < t) ? bt * x[4 * s4 + 0] : 0.f;
+                a.y = (active && 4 * s4 + 1 >= s0 && 4 * s4 + 1 < t) ? bt * x[4 * s4 + 1] : 0.f;
+                a.z = (active && 4 * s4 + 2 >= s0 && 4 * s4 + 2 < t) ? bt * x[4 * s4 + 2] : 0.f;
+                a.w = (active && 4 * s4 + 3 >= s0 && 4 * s4 + 3 < t) ? bt * x[4 * s4 + 3] : 0.f;
+                *reinterpret_cast<float4*>(Amat + t * kL + 4 * s4) = a;
             }
-            *reinterpret_cast<uint4*>(mh + i8 * 8) = make_uint4(oh[0], oh[1], oh[2], oh[3]);
-            *reinterpret_cast<uint4*>(ml + i8 * 8) = make_uint4(ol[0], ol[1], ol[2], ol[3]);
+        } else {
+            tmem_ld32(lane_addr + 64, reinterpret_cast<uint32_t*>(x));
+            tmem_ld32(lane_addr + 96, reinterpret_cast<uint32_t*>(x) + 32);
+            tmem_wait_ld();
+            __nv_bfloat16* mh = p.ws_m_h + (bh * kL + t) * kL;
+            __nv_bfloat16* ml = p.ws_m_l + (bh * kL + t) * kL;
+#pragma unroll
+            for (int i8 = 0; i8 < 8; ++i8) {
+                uint32_t oh[4], ol[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int s = i8 * 8 + 2 * i;
+                    const float m0 = (active && s >= s0 && s <= t) ? x[s] : 0.f;
+                    const float m1 = (active && s + 1 >= s0 && s + 1 <= t) ? x[s + 1] : 0.f;
+                    split2(m0, m1, oh[i], ol[i]);
+                }
+                *reinterpret_cast<uint4*>(mh + i8 * 8) = make_uint4(oh[0], oh[1], oh[2], oh[3]);
+                *reinterpret_cast<uint4*>(ml + i8 * 8) = make_uint4(ol[0], ol[1], ol[2], ol[3]);
+            }
         }
     }
     tc_fence_before();
@@ -377,12 +438,12 @@ __global__ void __launch_bounds__(128) kda_tc_prep_kernel(const KdaTcParams p) {
     // ---- T = (I + A)^-1 diag(beta).  The unit lower triangular 64 x 64 matrix L = I + A is inverted in 16 x 16 blocks:
     //      the four diagonal blocks by forward substitution (64 threads, one column each), then the blocks below the
     //      diagonal, one block diagonal after the other, from X_ij = -X_ii sum_{j <= k < i} L_ik X_kj as small products
-    //      on all 128 threads (two elements of each 16 x 16 block per thread).  X lives behind the T tiles in R0; the
-    //      sums are staged where the T tiles will go.
+    //      (one element of each 16 x 16 block per thread).  X lives behind the T tiles in R0; the sums are staged where
+    //      the T tiles will go.
     float* Xm = reinterpret_cast<float*>(r0 + 2 * kTileBytes);        // [64][64] fp32
     float* Tmp = reinterpret_cast<float*>(r0);                        // up to three 16 x 16 blocks
     if (ok) {
-        for (int i = tid; i < kL * kL; i += 128) Xm[i] = 0.f;
+        for (int i = tid; i < kL * kL; i += kPrepThreads) Xm[i] = 0.f;
         __syncthreads();
         if (tid < kL) {
             const int bi = tid >> 4, c = tid & 15;
@@ -397,48 +458,54 @@ __global__ void __launch_bounds__(128) kda_tc_prep_kernel(const KdaTcParams p) {
             }
         }
         __syncthreads();
-        const int er = tid >> 3, ec = (tid & 7) * 2;                  // this thread's two elements of a block
+        // a thread owns a 1 x 4 patch of one block of the current diagonal: thread -> (block slot, row, 4 columns)
+        const int bs = tid >> 6, er = (tid >> 2) & 15, ec = (tid & 3) * 4;
 #pragma unroll 1
         for (int d = 1; d < 4; ++d) {
-            // sums S_ij = sum_k L_ik X_kj for the blocks (i, j = i - d)
-#pragma unroll 1
-            for (int i = d; i < 4; ++i) {
-                const int j = i - d;
-                float s0 = 0.f, s1 = 0.f;
+            const int i = d + bs, j = bs;                             // block (i, j = i - d), for bs < 4 - d
+            // sums S_ij = sum_k L_ik X_kj
+            if (i < 4) {
+                float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll 1
                 for (int k = j; k < i; ++k) {
 #pragma unroll
-                    for (int q = 0; q < 16; ++q) {
-                        const float l = Amat[(i * 16 + er) * kL + k * 16 + q];
-                        const float2 xv = *reinterpret_cast<const float2*>(Xm + (k * 16 + q) * kL + j * 16 + ec);
-                        s0 = fmaf(l, xv.x, s0);
-                        s1 = fmaf(l, xv.y, s1);
+                    for (int q4 = 0; q4 < 16; q4 += 4) {
+                        const float4 l = *reinterpret_cast<const float4*>(Amat + (i * 16 + er) * kL + k * 16 + q4);
+                        const float lq[4] = {l.x, l.y, l.z, l.w};
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) {
+                            const float4 xv = *reinterpret_cast<const float4*>(Xm + (k * 16 + q4 + q) * kL + j * 16 + ec);
+                            acc.x = fmaf(lq[q], xv.x, acc.x); acc.y = fmaf(lq[q], xv.y, acc.y);
+                            acc.z = fmaf(lq[q], xv.z, acc.z); acc.w = fmaf(lq[q], xv.w, acc.w);
+                        }
                     }
                 }
-                *reinterpret_cast<float2*>(Tmp + (i - d) * 256 + er * 16 + ec) = make_float2(s0, s1);
+                *reinterpret_cast<float4*>(Tmp + bs * 256 + er * 16 + ec) = acc;
             }
             __syncthreads();
-#pragma unroll 1
-            for (int i = d; i < 4; ++i) {
-                const int j = i - d;
-                float s0 = 0.f, s1 = 0.f;
+            if (i < 4) {
+                float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-                for (int q = 0; q < 16; ++q) {
-                    const float x = Xm[(i * 16 + er) * kL + i * 16 + q];
-                    const float2 tv = *reinterpret_cast<const float2*>(Tmp + (i - d) * 256 + q * 16 + ec);
-                    s0 = fmaf(x, tv.x, s0);
-                    s1 = fmaf(x, tv.y, s1);
+                for (int q4 = 0; q4 < 16; q4 += 4) {
+                    const float4 x = *reinterpret_cast<const float4*>(Xm + (i * 16 + er) * kL + i * 16 + q4);
+                    const float xq[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        const float4 tv = *reinterpret_cast<const float4*>(Tmp + bs * 256 + (q4 + q) * 16 + ec);
+                        acc.x = fmaf(xq[q], tv.x, acc.x); acc.y = fmaf(xq[q], tv.y, acc.y);
+                        acc.z = fmaf(xq[q], tv.z, acc.z); acc.w = fmaf(xq[q], tv.w, acc.w);
+                    }
                 }
-                *reinterpret_cast<float2*>(Xm + (i * 16 + er) * kL + j * 16 + ec) = make_float2(-s0, -s1);
+                *reinterpret_cast<float4*>(Xm + (i * 16 + er) * kL + j * 16 + ec) = make_float4(-acc.x, -acc.y, -acc.z, -acc.w);
             }
             __syncthreads();
         }
-        // T[t][c] = X[t][c] beta_c as hi/lo operand tiles (hi at R0, lo behind it): thread -> (row, 32 columns)
+        // T[t][c] = X[t][c] beta_c as hi/lo operand tiles (hi at R0, lo behind it): thread -> (row, 16 columns)
         {
-            const int t = tid >> 1, cb = (tid & 1) * 32;
-            uint4 th[4], tl[4];
+            const int t = tid >> 2, cb = (tid & 3) * 16;
+            uint4 th[2], tl[2];
 #pragma unroll
-            for (int j8 = 0; j8 < 4; ++j8) {
+            for (int j8 = 0; j8 < 2; ++j8) {
                 uint32_t oh[4], ol[4];
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
@@ -450,7 +517,7 @@ __global__ void __launch_bounds__(128) kda_tc_prep_kernel(const KdaTcParams p) {
             }
             __syncthreads();               // the staging area is free: the tiles take its place
 #pragma unroll
-            for (int j8 = 0; j8 < 4; ++j8) {
+            for (int j8 = 0; j8 < 2; ++j8) {
                 const uint32_t off = sw_off(t, (cb >> 3) + j8);
                 *reinterpret_cast<uint4*>(r0 + off) = th[j8];
                 *reinterpret_cast<uint4*>(r0 + kTileBytes + off) = tl[j8];
@@ -479,30 +546,38 @@ __global__ void __launch_bounds__(128) kda_tc_prep_kernel(const KdaTcParams p) {
     }
     ok = __syncthreads_and(ok && mbar_wait(bar, 1, abort_flag));
     tc_fence_after();
-    if (warp < 2 && ok) {
-        const int t = tid;
-        const uint32_t lane_addr = tmem + ((uint32_t)(warp * 32) << 16);
-        __nv_bfloat16* wh = p.ws_w0_h + bh * tile_elems + (size_t)t * kD;
-        __nv_bfloat16* wl = p.ws_w0_l + bh * tile_elems + (size_t)t * kD;
-        float* u0 = p.ws_u0 + bh * tile_elems + (size_t)t * kD;
+    // ---- rows of W0 (warps 0, 1: hi/lo bf16) and of U0 (warps 4, 5: fp32) to the workspace
+    if ((warp & 3) < 2 && ok) {
+        const int t = (warp & 3) * 32 + lane;
+        const uint32_t lane_addr = tmem + ((uint32_t)((warp & 3) * 32) << 16);
+        if (warp < 4) {
+            __nv_bfloat16* wh = p.ws_w0_h + bh * tile_elems + (size_t)t * kD;
+            __nv_bfloat16* wl = p.ws_w0_l + bh * tile_elems + (size_t)t * kD;
 #pragma unroll 1
-        for (int c0 = 0; c0 < kD; c0 += 32) {
-            float x[32];
-            tmem_ld32(lane_addr + c0, reinterpret_cast<uint32_t*>(x));
-            tmem_wait_ld();
+            for (int c0 = 0; c0 < kD; c0 += 32) {
+                float x[32];
+                tmem_ld32(lane_addr + c0, reinterpret_cast<uint32_t*>(x));
+                tmem_wait_ld();
 #pragma unroll
-            for (int i8 = 0; i8 < 4; ++i8) {
-                uint32_t oh[4], ol[4];
+                for (int i8 = 0; i8 < 4; ++i8) {
+                    uint32_t oh[4], ol[4];
 #pragma unroll
-                for (int i = 0; i < 4; ++i) split2(x[i8 * 8 + 2 * i], x[i8 * 8 + 2 * i + 1], oh[i], ol[i]);
-                *reinterpret_cast<uint4*>(wh + c0 + i8 * 8) = make_uint4(oh[0], oh[1], oh[2], oh[3]);
-                *reinterpret_cast<uint4*>(wl + c0 + i8 * 8) = make_uint4(ol[0], ol[1], ol[2], ol[3]);
+                    for (int i = 0; i < 4; ++i) split2(x[i8 * 8 + 2 * i], x[i8 * 8 + 2 * i + 1], oh[i], ol[i]);
+                    *reinterpret_cast<uint4*>(wh + c0 + i8 * 8) = make_uint4(oh[0], oh[1], oh[2], oh[3]);
+                    *reinterpret_cast<uint4*>(wl + c0 + i8 * 8) = make_uint4(ol[0], ol[1], ol[2], ol[3]);
+                }
             }
-            tmem_ld32(lane_addr + 128 + c0, reinterpret_cast<uint32_t*>(x));
-            tmem_wait_ld();
+        } else {
+            float* u0 = p.ws_u0 + bh * tile_elems + (size_t)t * kD;
+#pragma unroll 1
+            for (int c0 = 0; c0 < kD; c0 += 32) {
+                float x[32];
+                tmem_ld32(lane_addr + 128 + c0, reinterpret_cast<uint32_t*>(x));
+                tmem_wait_ld();
 #pragma unroll
-            for (int i4 = 0; i4 < 8; ++i4)
-                *reinterpret_cast<float4*>(u0 + c0 + i4 * 4) = make_float4(x[4 * i4], x[4 * i4 + 1], x[4 * i4 + 2], x[4 * i4 + 3]);
+                for (int i4 = 0; i4 < 8; ++i4)
+                    *reinterpret_cast<float4*>(u0 + c0 + i4 * 4) = make_float4(x[4 * i4], x[4 * i4 + 1], x[4 * i4 + 2], x[4 * i4 + 3]);
+            }
         }
     }
     tc_fence_before();
@@ -875,13 +950,15 @@ kda_tc_chain_kernel(const __grid_constant__ CUtensorMap tm_w0_h, const __grid_co
                 tmem_wait_ld();
                 uint32_t hi[32], lo[32];
 #pragma unroll
-                for (int i = 0; i < 32; ++i) {
-                    const float2 al = *reinterpret_cast<const float2*>(v_alpha + cbase + 2 * i);
-                    const float2 en = *reinterpret_cast<const float2*>(v_end + cbase + 2 * i);
-                    const float y0 = x[2 * i] * al.x, y1 = x[2 * i + 1] * al.y;
-                    split2(y0, y1, hi[i], lo[i]);
-                    x[2 * i] = y0 * en.x;
-                    x[2 * i + 1] = y1 * en.y;
+                for (int i4 = 0; i4 < 16; ++i4) {
+                    const float4 al = *reinterpret_cast<const float4*>(v_alpha + cbase + 4 * i4);
+                    const float4 en = *reinterpret_cast<const float4*>(v_end + cbase + 4 * i4);
+                    const float2 ya = __fmul2_rn(make_float2(x[4 * i4], x[4 * i4 + 1]), make_float2(al.x, al.y));
+                    const float2 yb = __fmul2_rn(make_float2(x[4 * i4 + 2], x[4 * i4 + 3]), make_float2(al.z, al.w));
+                    split2(ya.x, ya.y, hi[2 * i4], lo[2 * i4]);
+                    split2(yb.x, yb.y, hi[2 * i4 + 1], lo[2 * i4 + 1]);
+                    const float2 za = __fmul2_rn(ya, make_float2(en.x, en.y)), zb = __fmul2_rn(yb, make_float2(en.z, en.w));
+                    x[4 * i4] = za.x; x[4 * i4 + 1] = za.y; x[4 * i4 + 2] = zb.x; x[4 * i4 + 3] = zb.y;
                 }
                 tmem_st32(lane_addr + kColShl + cbase / 2, hi);
                 tmem_st32(lane_addr + kColShl + 64 + cbase / 2, lo);
@@ -988,7 +1065,7 @@ extern "C" int wpp_launch_kda_tc(const wpp::KdaTcParams* p, const CUtensorMap* m
     kda_tc_setup_kernel<<<1, 1024, 0, st>>>(*p);
     if (max_blocks > 0) {
         dim3 grid_a((unsigned)max_blocks, (unsigned)p->num_heads);
-        kda_tc_prep_kernel<<<grid_a, 128, PrepSmem::kBytes, st>>>(*p);
+        kda_tc_prep_kernel<<<grid_a, kPrepThreads, PrepSmem::kBytes, st>>>(*p);
     }
     dim3 grid_b((unsigned)p->num_heads, (unsigned)p->num_requests);
     kda_tc_chain_kernel<<<grid_b, 352, ChainSmem::kBytes, st>>>(maps[0], maps[1], maps[2], maps[3], maps[4], maps[5], maps[6],
