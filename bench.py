@@ -40,6 +40,9 @@ DRAM_SOURCE = ("estimate: 628.9 DRAM bytes per 128x128 key step (dram__bytes_rea
 # Recurrent layer: dram read + write bytes of one wpp_kda_chunk launch on the default wave (8 x 2,048 tokens, 32 heads)
 # / its 524,288 (token, head) pairs; other wave shapes scale with the pairs (the state traffic per request is small).
 KDA_DRAM_BYTES_PER_TOKEN_HEAD = 1571.3
+# Chunk-parallel form: (686.6 MB + 1160.2 MB) of the preparation kernel + (1233.3 MB + 137.7 MB) of the chain kernel on
+# the same wave / 524,288 pairs.
+KDA_TC_DRAM_BYTES_PER_TOKEN_HEAD = 6137.6
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -479,8 +482,9 @@ def run_kda(args):
     """The recurrent-state (KDA) layer of one wave (Section 3.1 update, Section 3.2 snapshots): `--kda-lanes`
     requests of `--kda-chunk` tokens, 32 state heads of 128 x 128, every request resuming from a snapshot and
     storing one at the chunk end.  Timed with CUDA events over back-to-back launches on inputs larger than L2;
-    the roofline is plain fp32 arithmetic: 7 flop per state element and token (one multiply and three fused
-    multiply-adds) against 148 SMs x 128 lanes x 2 flop x the maximum SM clock."""
+    the library's choice (--kda-layout 0) is the chunk-parallel tensor-core form, bounded by the algorithmic bytes at
+    HBM bandwidth; the token-by-token forms (--kda-layout 1, 2) are plain fp32 arithmetic: 7 flop per state element
+    and token against 148 SMs x 128 lanes x 2 flop x the maximum SM clock."""
     if int(os.environ.get("RANK", "0")) != 0:
         return
     import torch
@@ -531,21 +535,42 @@ def run_kda(args):
     if not np.all(np.abs(got - ref) <= 2.0 ** -8 * np.abs(ref) + 1e-4 * np.abs(ref).max()):
         raise SystemExit(f"wpp_kda_chunk disagrees with the oracle (max |delta| {err:.3e})")
     T, Hh = w.total_tokens, w.num_heads
-    flops = 7.0 * w.d_k * w.d_v * T * Hh
-    peak = 148 * 128 * 2 * 1965e6 / 1e12
+    flops = 7.0 * w.d_k * w.d_v * T * Hh             # the method's work: 7 flop per state element, token and head
     nbytes = T * Hh * (2 * w.d_k * 2 + 2 * w.d_v * 2 + 4 * w.d_k + 4) + 2 * w.chunk_lens.size * Hh * w.d_k * w.d_v * 4
+    peaks, peak_kind = load_peaks()
+    hbm = float(peaks.get("hbm_gbs", FALLBACK_PEAKS["hbm_gbs"]))
+    tensor_form = args.kda_layout == 3 or (args.kda_layout == 0 and T >= 64 * int(w.chunk_lens.size))
+    if tensor_form:
+        # Chunk-parallel form: the algorithmic bytes (q, k, v, alpha, beta in, outputs and states out) at the copy
+        # bandwidth bound it from below (7 d_k d_v flop per token and head are 0.04 ms of tensor time for the default
+        # wave, the bytes 0.13 ms); what it actually moves is three times that, because the preparation kernel hands
+        # its per-block operands to the chain kernel through the workspace.
+        roofline = {"bound": "hbm", "kernel": "kda_tc_prep_kernel + kda_tc_chain_kernel",
+                    "achieved": nbytes / (ms * 1e-3) / 1e9, "peak": hbm, "unit": "GB/s",
+                    "frac": nbytes / (ms * 1e-3) / 1e9 / hbm, "peak_source": f"of {peak_kind} (copy bandwidth)",
+                    "algorithmic_bytes": nbytes, "flop_per_token_head": 7 * w.d_k * w.d_v,
+                    "tflops_algorithmic": flops / (ms * 1e-3) / 1e12,
+                    "traffic": KDA_TC_DRAM_BYTES_PER_TOKEN_HEAD * T * Hh,
+                    "traffic_source": "estimate: dram read + write bytes of one preparation and one chain launch on the "
+                                      "8 x 2,048-token wave (ncu), per (token, head), x this wave's pairs; not measured "
+                                      "in this run"}
+    else:
+        peak = 148 * 128 * 2 * 1965e6 / 1e12
+        roofline = {"bound": "alu", "kernel": "wpp_kda_chunk_kernel", "achieved": flops / (ms * 1e-3) / 1e12,
+                    "peak": peak, "unit": "TFLOP/s", "frac": flops / (ms * 1e-3) / 1e12 / peak,
+                    "peak_source": "derived: 148 SMs x 128 fp32 lanes x 2 flop x 1965 MHz",
+                    "flop_per_token_head": 7 * w.d_k * w.d_v, "traffic": KDA_DRAM_BYTES_PER_TOKEN_HEAD * T * Hh,
+                    "traffic_source": "estimate from an ncu capture of the default wave, scaled by (token, head) pairs",
+                    "hbm_gbs_algorithmic": nbytes / (ms * 1e-3) / 1e9}
     line = {"metric": "recurrent-state (KDA) layer, new tokens/s through one layer", "value": T / (ms * 1e-3),
             "unit": "tokens/s", "n_gpus": 1, "steps": steps, "warmup": warm, "ms_per_step": ms, "higher_is_better": True,
-            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic", "gpu_launches": steps,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16 x 2 terms, fp32 accumulate" if tensor_form else "f32",
+            "data": "synthetic", "gpu_launches": steps * (3 if tensor_form else 1),
             "config": {"workload": w.name, "requests": int(w.chunk_lens.size), "chunk": int(w.chunk_lens[0]),
                        "state_heads": Hh, "d_k": w.d_k, "d_v": w.d_v, "layout": args.kda_layout,
+                       "form": "chunk-parallel on tensor cores" if tensor_form else "token by token on CUDA cores",
                        "l2": "inputs larger than L2"},
-            "clocks": clocks,
-            "roofline": {"bound": "alu", "kernel": "wpp_kda_chunk_kernel", "achieved": flops / (ms * 1e-3) / 1e12,
-                         "peak": peak, "unit": "TFLOP/s", "frac": flops / (ms * 1e-3) / 1e12 / peak,
-                         "peak_source": "derived: 148 SMs x 128 fp32 lanes x 2 flop x 1965 MHz",
-                         "flop_per_token_head": 7 * w.d_k * w.d_v, "traffic": KDA_DRAM_BYTES_PER_TOKEN_HEAD * T * Hh,
-                         "hbm_gbs_algorithmic": nbytes / (ms * 1e-3) / 1e9},
+            "clocks": clocks, "roofline": roofline,
             "cpu_baseline": {"value": (sl.stop - sl.start) / t_cpu / Hh, "unit": "tokens/s", "cores": 1, "kind": "oracle",
                              "sample": f"one (request, head) chain of {sl.stop - sl.start} tokens, scaled to {Hh} heads"},
             "parity": {"checked": f"request {req}, head {head}: all outputs against the fp64 oracle", "max_abs_err": err}}
@@ -573,7 +598,7 @@ def main():
     ap.add_argument("--kda", action="store_true", help="the recurrent-state (KDA) layer of one wave")
     ap.add_argument("--kda-lanes", type=int, default=8)
     ap.add_argument("--kda-chunk", type=int, default=2048)
-    ap.add_argument("--kda-layout", type=int, default=0, help="0: library chooses, 1: one CTA per (request, head), 2: four")
+    ap.add_argument("--kda-layout", type=int, default=0, help="0: library chooses, 1: one CTA per (request, head), 2: four, 3: chunk-parallel on tensor cores")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "native" else args.warmup
 

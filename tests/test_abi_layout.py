@@ -50,7 +50,7 @@ def test_entry_points_reject_a_null_context_without_touching_a_gpu():
     """Every device entry point validates its arguments on the host first: with no context nothing is launched."""
     lib = B.load_library()
     desc = B.KdaDesc(1, 1, 128, 128, 1, 0, 0, 0, 4)
-    assert lib.wpp_kda_chunk(None, ctypes.byref(desc), *([None] * 14)) == 1          # WPP_ERR_INVALID_ARG
+    assert lib.wpp_kda_chunk(None, ctypes.byref(desc), *([None] * 13), 0, None, None) == 1          # WPP_ERR_INVALID_ARG
     assert lib.wpp_hash_blocks(None, None, None, None, 1, 16, 0, None, None, 1, None) == 1
     bd = B.make_desc(1, 2, 1, 128, 16, 4, 8)
     assert lib.wpp_kv_append(None, ctypes.byref(bd), *([None] * 11)) == 1
