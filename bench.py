@@ -592,6 +592,8 @@ def main():
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
     ap.add_argument("--plan-order", type=int, default=0, help="0: stream order (default), 1: longest tile first")
     ap.add_argument("--max-ctas", type=int, default=0, help="persistent CTAs to launch (0: one per SM)")
+    ap.add_argument("--shape", type=int, default=0, help="attention kernel: 0 planner's choice, 1 SM-wide two-half CTAs, "
+                                                         "2 small single-half CTAs (two per SM)")
     ap.add_argument("--waves", action="store_true", help="time the wave-budget planner (host only) instead")
     ap.add_argument("--waves-sim", action="store_true", help="wave planner + kernels: simulated pipeline fill")
     ap.add_argument("--hints", action="store_true", help="chained block hashing on the GPU and the hint probe")
@@ -634,7 +636,7 @@ def main():
     ctx = wpp.Context(local_rank)
     desc = wpp.make_desc(w.num_requests, w.num_q_heads, w.num_kv_heads, w.head_dim, w.page_size,
                          w.max_blocks_per_req, w.num_pages)
-    opts = wpp.PlanOpts(0, 0, args.force_kv_splits, args.max_ctas, args.plan_order)
+    opts = wpp.PlanOpts(0, 0, args.force_kv_splits, args.max_ctas, args.plan_order, args.shape)
     T = w.total_new_tokens
 
     # ---- resident state and inputs on the device
@@ -858,7 +860,8 @@ def main():
                               f"inputs ({touched / 1e6:.1f} MB touched per step) fit L2: a 256 MB buffer is overwritten "
                               "between steps; ms_per_step is the sum of append and attention event times"),
                            step="wpp_plan_tiles + plan H2D + wpp_kv_append + wpp_prefill_attention_varlen",
-                           tiles=int(info.num_tiles), ctas=int(info.num_ctas), key_steps=int(info.key_steps)),
+                           tiles=int(info.num_tiles), ctas=int(info.num_ctas), key_steps=int(info.key_steps),
+                           kernel_shape=int(info.shape)),
             "tflops": flops / (ms_step * 1e-3) / 1e12 * world,
             "served_tokens_per_s": world * float((w.prefix_lens.astype(np.int64) + w.chunk_lens).sum()) / (ms_step * 1e-3),
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline, "cpu_baseline": cpu,

@@ -107,6 +107,11 @@ typedef struct {
                                  tiles that read the same (request, KV head) pages are neighbours and so run at the
                                  same time: the pages are fetched from DRAM once and shared through L2; 1: longest
                                  tile first */
+    int32_t shape;            /* which attention kernel runs the plan.  1: one CTA per SM working on both 128-row halves
+                                 of a tile against 128-key steps (long tiles: the two halves and the tensor pipe overlap
+                                 inside the CTA); 2: two small CTAs per SM, each working on one half against 64-key
+                                 steps (short tiles: one CTA's tile start and end hide under the other's steps);
+                                 0: the library decides from the mean number of key steps per half */
 } wpp_plan_opts;
 
 typedef struct {
@@ -117,6 +122,7 @@ typedef struct {
     int64_t total_new_tokens;   /* T */
     int64_t key_steps;          /* sum over tiles of 128-row x 128-key steps (work incl. tile quantisation) */
     int64_t flops;              /* algorithmic: 4 * d * Hq * sum_i (C_i P_i + C_i (C_i + 1) / 2) */
+    int64_t shape;              /* attention kernel the plan is for: 1 or 2, see wpp_plan_opts.shape */
     size_t workspace_bytes;     /* device scratch wpp_prefill_attention_varlen needs for this plan (never 0) */
     size_t plan_bytes;          /* bytes of plan_host actually used; copy that many to the device */
 } wpp_plan_info;
@@ -183,7 +189,8 @@ int wpp_kv_append(const wpp_ctx* ctx, const wpp_batch_desc* desc, const void* k_
  *                   at the same time need a workspace each.
  * A request whose prefix_lens[i] or chunk_lens[i] on the device differ from the plan's sets *status_dev =
  * WPP_ERR_PLAN_MISMATCH; its tiles are skipped (its output rows are not computed; rows of split tiles read as zero).
- * Enqueues a 256-byte memset and one persistent kernel, plus one combine kernel iff the plan has split tiles.
+ * Enqueues a 256-byte memset and one persistent kernel (the shape the plan names), plus one combine kernel iff the
+ * plan has split tiles.
  * Results are bit-reproducible for a given plan, whichever CTA takes which tile (no atomics on outputs; partials
  * are merged in a fixed order). */
 int wpp_prefill_attention_varlen(const wpp_ctx* ctx, const wpp_batch_desc* desc, const void* q, void* out,

@@ -46,14 +46,14 @@ class BatchDesc(ctypes.Structure):
 
 class PlanOpts(ctypes.Structure):
     _fields_ = [("tile_m", ctypes.c_int32), ("tile_n", ctypes.c_int32), ("force_kv_splits", ctypes.c_int32),
-                ("max_ctas", ctypes.c_int32), ("order", ctypes.c_int32)]
+                ("max_ctas", ctypes.c_int32), ("order", ctypes.c_int32), ("shape", ctypes.c_int32)]
 
 
 class PlanInfo(ctypes.Structure):
     _fields_ = [("num_tiles", ctypes.c_int64), ("num_split_tiles", ctypes.c_int64),
                 ("num_combine_tiles", ctypes.c_int64), ("num_ctas", ctypes.c_int64),
                 ("total_new_tokens", ctypes.c_int64), ("key_steps", ctypes.c_int64), ("flops", ctypes.c_int64),
-                ("workspace_bytes", ctypes.c_size_t), ("plan_bytes", ctypes.c_size_t)]
+                ("shape", ctypes.c_int64), ("workspace_bytes", ctypes.c_size_t), ("plan_bytes", ctypes.c_size_t)]
 
 
 class WaveConfig(ctypes.Structure):

@@ -7,7 +7,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libwpp.so")
-SOURCES = ["wpp_plan.cpp", "wpp_waves.cpp", "wpp_hints.cu", "wpp_api.cu", "wpp_append_combine.cu", "wpp_attention.cu",
+SOURCES = ["wpp_plan.cpp", "wpp_waves.cpp", "wpp_hints.cu", "wpp_api.cu", "wpp_append_combine.cu", "wpp_attention.cu", "wpp_attention_small.cu",
            "wpp_kda.cu", "wpp_kda_tc.cu"]
 HEADERS = ["wpp_host.h", "wpp_plan_format.h", "wpp_device.h", "wpp_ptx.cuh", os.path.join("..", "..", "include", "wpp.h")]
 

@@ -252,7 +252,7 @@ extern "C" int wpp_prefill_attention_varlen(const wpp_ctx* ctx, const wpp_batch_
     if (rc != WPP_OK) return rc;
     const WppPlanHeader* hd = nullptr;
     if ((rc = wpp_check_plan(plan_host, &d, &hd)) != WPP_OK) return rc;
-    if (hd->tile_m > WPP_MAX_TILE_M) return WPP_ERR_PLAN_MISMATCH;
+    if (hd->tile_m > WPP_MAX_TILE_M || hd->shape < 1 || hd->shape > 2) return WPP_ERR_PLAN_MISMATCH;
     if (hd->total_new_tokens == 0 || hd->num_units == 0) return WPP_OK;
     if ((rc = wpp_ctx_check_device(ctx)) != WPP_OK) return rc;
     if (!q || !out || !k_cache || !v_cache || !block_tables || !prefix_lens || !chunk_lens || !plan_dev)
@@ -276,7 +276,9 @@ extern "C" int wpp_prefill_attention_varlen(const wpp_ctx* ctx, const wpp_batch_
                                   (uint64_t)d.num_pages};
         const uint64_t strides[3] = {(uint64_t)d.kv_token_stride * 2, (uint64_t)d.kv_head_stride * 2,
                                      (uint64_t)d.kv_page_stride * 2};
-        const uint32_t box[4] = {64, (uint32_t)d.page_size, 1, 1};
+        // the small shape works on 64-key steps: its boxes have at most 64 rows (half a 128-token page)
+        const uint32_t box_rows = (hd->shape == 2 && d.page_size > 64) ? 64u : (uint32_t)d.page_size;
+        const uint32_t box[4] = {64, box_rows, 1, 1};
         if ((rc = make_map(ctx, &tk, k_cache, 4, dims, strides, box)) != WPP_OK) return rc;
         if ((rc = make_map(ctx, &tv, v_cache, 4, dims, strides, box)) != WPP_OK) return rc;
     }
@@ -306,7 +308,8 @@ extern "C" int wpp_prefill_attention_varlen(const wpp_ctx* ctx, const wpp_batch_
     // the counter the CTAs take their tiles from starts at zero (a memset node on the caller's stream)
     int e = (int)cudaMemsetAsync(workspace, 0, WPP_WS_HEADER_BYTES, (cudaStream_t)cuda_stream);
     if (e != 0) return cuda_fail(ctx, e);
-    e = wpp_launch_attention(d.head_dim, tq, &tk, &tv, &p, hd->num_ctas, cuda_stream);
+    e = hd->shape == 2 ? wpp_launch_attention_small(d.head_dim, tq, &tk, &tv, &p, hd->num_ctas, cuda_stream)
+                       : wpp_launch_attention(d.head_dim, tq, &tk, &tv, &p, hd->num_ctas, cuda_stream);
     if (e != 0) return cuda_fail(ctx, e);
     const_cast<wpp_ctx*>(ctx)->launches += 1;
     if (hd->num_combine > 0) {

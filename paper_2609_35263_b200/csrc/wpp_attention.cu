@@ -45,7 +45,7 @@ __host__ __device__ constexpr uint32_t col_p(int hf) { return 128u + 64u * hf; }
 __host__ __device__ constexpr uint32_t col_o(int hf) { return 256u + 128u * hf; }   // O of half hf
 // registers per thread after the warpgroups re-split the register file (8 x kRegsSoftmax + 4 x kRegsEpilogue +
 // 4 x kRegsUtil <= 2048 per thread slot of 32 lanes, i.e. 65536 in all)
-constexpr int kRegsSoftmax = 192, kRegsEpilogue = 64, kRegsUtil = 64;
+constexpr int kRegsSoftmax = 192, kRegsEpilogue = 72, kRegsUtil = 56;
 static_assert(8 * kRegsSoftmax + 4 * kRegsEpilogue + 4 * kRegsUtil <= 2048, "register file exceeded");
 constexpr uint32_t kSoftmaxArrivals = 128;   // every softmax thread arrives on s_free and p_ready itself
 constexpr int kRescaleCols = 16;    // columns of O in flight while a moved reference rescales it
@@ -63,9 +63,10 @@ struct Cfg {
     static constexpr int kTileQ = 2;                       // tile ids the producer may publish ahead
     static constexpr int kNumBars = 2 + 2 * kSlots + 1 + 6 * 2 + 2 * kTileQ;
     static constexpr int kOffFinal = kOffBars + 8 * kNumBars;          // float2 (m, l)[2][128]
-    static constexpr int kOffMisc = kOffFinal + 2 * 128 * 8;           // tmem ptr, abort flag, tile ids
+    static constexpr int kOffStage = (kOffFinal + 2 * 128 * 8 + 15) / 16 * 16;   // 4 x 2 KB: the epilogue warps' store staging (16-byte chunks)
+    static constexpr int kOffMisc = kOffStage + 4 * 2048;              // tmem ptr, abort flag, tile ids
     static constexpr int kUsedBytes = kOffMisc + 16 + 4 * kTileQ + 8;
-    static constexpr int kSmemBytes = kUsedBytes + 1024;               // + alignment slack (193 KB at D = 128)
+    static constexpr int kSmemBytes = kUsedBytes + 1024;               // + alignment slack (201 KB at D = 128)
     static_assert(kSmemBytes <= 232448, "more shared memory than a CTA can have");
 };
 
@@ -423,39 +424,43 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 const float2 ml = s_final[hf * 128 + r];
                 const float inv_l = (ml.y > 0.f) ? 1.f / ml.y : 0.f;
                 const float lse2 = (ml.y > 0.f) ? (ml.x + log2f(ml.y)) : -INFINITY;
+                uint8_t* stage = smem_gen + C::kOffStage + (warp & 3) * 2048;
                 if (un.split_slot < 0) {
-                    __nv_bfloat16* dst = p.out + tok * p.o_token_stride + (int64_t)head * p.o_head_stride;
+                    const __nv_bfloat16* dst = p.out + tok * p.o_token_stride + (int64_t)head * p.o_head_stride;
 #pragma unroll
                     for (int q4 = 0; q4 < D / 32; ++q4) {
                         float o[32];
                         tmem_ld32(lane_addr + col_o(hf) + q4 * 32, reinterpret_cast<uint32_t*>(o));
                         tmem_wait_ld();
-                        if (row_ok) {
+                        uint4 w[4];
 #pragma unroll
-                            for (int w4 = 0; w4 < 4; ++w4) {
-                                uint4 w;
-                                w.x = pack_bf16x2(o[8 * w4 + 0] * inv_l, o[8 * w4 + 1] * inv_l);
-                                w.y = pack_bf16x2(o[8 * w4 + 2] * inv_l, o[8 * w4 + 3] * inv_l);
-                                w.z = pack_bf16x2(o[8 * w4 + 4] * inv_l, o[8 * w4 + 5] * inv_l);
-                                w.w = pack_bf16x2(o[8 * w4 + 6] * inv_l, o[8 * w4 + 7] * inv_l);
-                                *reinterpret_cast<uint4*>(dst + q4 * 32 + w4 * 8) = w;
-                            }
+                        for (int w4 = 0; w4 < 4; ++w4) {
+                            w[w4].x = pack_bf16x2(o[8 * w4 + 0] * inv_l, o[8 * w4 + 1] * inv_l);
+                            w[w4].y = pack_bf16x2(o[8 * w4 + 2] * inv_l, o[8 * w4 + 3] * inv_l);
+                            w[w4].z = pack_bf16x2(o[8 * w4 + 4] * inv_l, o[8 * w4 + 5] * inv_l);
+                            w[w4].w = pack_bf16x2(o[8 * w4 + 6] * inv_l, o[8 * w4 + 7] * inv_l);
                         }
+                        warp_store_rows64(stage, lane, w, dst, row_ok, q4 * 64);
                     }
                     if (p.lse && row_ok) p.lse[tok * p.num_q_heads + head] = lse2 * 0.6931471805599453f;
                 } else {
-                    float* dst = p.ws_o + prow * D;
+                    const float* dst = p.ws_o + prow * D;
 #pragma unroll
                     for (int q4 = 0; q4 < D / 32; ++q4) {
                         float o[32];
                         tmem_ld32(lane_addr + col_o(hf) + q4 * 32, reinterpret_cast<uint32_t*>(o));
                         tmem_wait_ld();
-                        if (row_ok) {
 #pragma unroll
-                            for (int w4 = 0; w4 < 8; ++w4)
-                                *reinterpret_cast<float4*>(dst + q4 * 32 + w4 * 4) =
-                                    make_float4(o[4 * w4] * inv_l, o[4 * w4 + 1] * inv_l, o[4 * w4 + 2] * inv_l,
-                                                o[4 * w4 + 3] * inv_l);
+                        for (int h2 = 0; h2 < 2; ++h2) {
+                            uint4 w[4];
+#pragma unroll
+                            for (int w4 = 0; w4 < 4; ++w4) {
+                                w[w4].x = __float_as_uint(o[16 * h2 + 4 * w4 + 0] * inv_l);
+                                w[w4].y = __float_as_uint(o[16 * h2 + 4 * w4 + 1] * inv_l);
+                                w[w4].z = __float_as_uint(o[16 * h2 + 4 * w4 + 2] * inv_l);
+                                w[w4].w = __float_as_uint(o[16 * h2 + 4 * w4 + 3] * inv_l);
+                            }
+                            warp_store_rows64(stage, lane, w, dst, row_ok, q4 * 128 + h2 * 64);
                         }
                     }
                     if (row_ok) p.ws_lse[prow] = lse2;

@@ -98,6 +98,8 @@ extern "C" {
 int wpp_launch_kda_tc(const wpp::KdaTcParams* p, const CUtensorMap* maps, int max_blocks, void* stream);
 int wpp_launch_attention(int head_dim, const CUtensorMap* tq, const CUtensorMap* tk, const CUtensorMap* tv,
                          const wpp::AttnParams* p, int num_ctas, void* stream);
+int wpp_launch_attention_small(int head_dim, const CUtensorMap* tq, const CUtensorMap* tk, const CUtensorMap* tv,
+                               const wpp::AttnParams* p, int num_ctas, void* stream);
 int wpp_launch_append(const wpp::AppendParams* p, int num_sms, void* stream);
 int wpp_launch_combine(const wpp::CombineParams* p, int num_combine, void* stream);
 int wpp_launch_kda(const wpp::KdaParams* p, int num_sms, int layout, void* stream);

@@ -7,6 +7,8 @@
 
 #define WPP_DEFAULT_TILE_M 256
 #define WPP_MAX_TILE_M 256
+/* a plan whose halves average at most this many 128-key steps runs on the small kernel shape */
+#define WPP_SMALL_SHAPE_MAX_STEPS 1
 
 #ifdef __cplusplus
 extern "C" {

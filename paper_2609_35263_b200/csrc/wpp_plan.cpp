@@ -79,7 +79,7 @@ uint64_t wpp_desc_hash(const wpp_batch_desc* d) {
 static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 static int resolve_opts(const wpp_ctx* ctx, const wpp_plan_opts* in, wpp_plan_opts* o) {
-    wpp_plan_opts z = {0, 0, 0, 0, 0};
+    wpp_plan_opts z = {0, 0, 0, 0, 0, 0};
     *o = in ? *in : z;
     if (!o->tile_m) o->tile_m = WPP_DEFAULT_TILE_M;
     if (!o->tile_n) o->tile_n = WPP_TILE_N;
@@ -88,7 +88,7 @@ static int resolve_opts(const wpp_ctx* ctx, const wpp_plan_opts* in, wpp_plan_op
     if (o->tile_m > WPP_MAX_TILE_M) return WPP_ERR_UNSUPPORTED;
     if (o->tile_n != WPP_TILE_N) return WPP_ERR_UNSUPPORTED;
     if (o->force_kv_splits < 0 || o->force_kv_splits > 64 || o->max_ctas < 1 || o->max_ctas > 4096 ||
-        o->order < 0 || o->order > 1)
+        o->order < 0 || o->order > 1 || o->shape < 0 || o->shape > 2)
         return WPP_ERR_INVALID_ARG;
     return WPP_OK;
 }
@@ -237,7 +237,14 @@ int wpp_plan_tiles(const wpp_ctx* ctx, const wpp_batch_desc* desc, const int32_t
         }
     }
     const int64_t n_units = (int64_t)units.size();
-    if (n_units > 0x7fffffff) return WPP_ERR_INVALID_ARG;
+    if (n_units > 0x3fffffff) return WPP_ERR_INVALID_ARG;
+    // ---- kernel shape: short tiles (few key steps per half) go to the small CTAs, two per SM, where the start and end of
+    //      one tile hide under the other CTA's steps; long tiles to the SM-wide CTA whose two halves overlap each other
+    int64_t nonempty_halves = 0;
+    for (const WppUnit& u : units)
+        for (int h = 0; h < 2; ++h) nonempty_halves += u.rows[h] > 0;
+    int shape = o.shape;
+    if (shape == 0) shape = (key_steps <= WPP_SMALL_SHAPE_MAX_STEPS * nonempty_halves) ? 2 : 1;
 
     // ---- order of execution.  The persistent CTAs take tiles in this order at run time (a counter in the
     //      workspace), so tiles adjacent in the order run at the same time on different SMs.
@@ -246,7 +253,8 @@ int wpp_plan_tiles(const wpp_ctx* ctx, const wpp_batch_desc* desc, const int32_t
     //      so a page comes from DRAM once and is then hit in L2 by the other tiles; a prefix shared by many
     //      requests stays L2-resident while its KV head is being worked on.
     //      order 1: longest tile first (best balance, no regard for which tiles run together).
-    const int num_ctas = (int)std::max<int64_t>(1, std::min<int64_t>(o.max_ctas, n_units));
+    const int num_ctas = shape == 2 ? (int)std::max<int64_t>(1, std::min<int64_t>(2 * (int64_t)o.max_ctas, 2 * n_units))
+                                    : (int)std::max<int64_t>(1, std::min<int64_t>(o.max_ctas, n_units));
     std::vector<int32_t> order((size_t)n_units);
     for (int64_t u = 0; u < n_units; ++u) order[(size_t)u] = (int32_t)u;
     if (o.order == 1) {
@@ -285,6 +293,8 @@ int wpp_plan_tiles(const wpp_ctx* ctx, const wpp_batch_desc* desc, const int32_t
     hd.tile_m = TM;
     hd.tile_n = WPP_TILE_N;
     hd.head_dim = d.head_dim;
+    hd.shape = shape;
+    hd.nonempty_halves = (int32_t)std::min<int64_t>(nonempty_halves, 0x7fffffff);
     hd.total_new_tokens = T;
     hd.key_steps = key_steps;
     hd.flops = 4 * (int64_t)d.head_dim * Hq * pairs;
@@ -321,6 +331,7 @@ int wpp_plan_tiles(const wpp_ctx* ctx, const wpp_batch_desc* desc, const int32_t
     info->total_new_tokens = T;
     info->key_steps = key_steps;
     info->flops = hd.flops;
+    info->shape = shape;
     info->workspace_bytes = hd.workspace_bytes;
     info->plan_bytes = hd.plan_bytes;
     return WPP_OK;

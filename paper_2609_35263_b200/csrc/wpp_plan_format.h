@@ -4,7 +4,7 @@
 #include <stdint.h>
 
 #define WPP_PLAN_MAGIC 0x31505057u /* "WPP1" */
-#define WPP_PLAN_VERSION 6u
+#define WPP_PLAN_VERSION 7u
 #define WPP_TILE_N 128             /* keys per step */
 #define WPP_WS_HEADER_BYTES 256
 #define WPP_HALF_M 128             /* query rows per tensor-core tile (one TMEM lane per row) */
@@ -22,7 +22,9 @@ struct WppPlanHeader {
                                     //               the row offsets) with the lengths they are launched with
     uint32_t off_units;             // WppUnit [num_units] in the order the persistent CTAs take them
     uint32_t off_combine;           // WppCombine [num_combine]
-    uint32_t pad[8];
+    int32_t shape;                  // 1: two-half CTAs, one per SM; 2: single-half CTAs, two per SM (work item = half a unit)
+    int32_t nonempty_halves;
+    uint32_t pad[6];
 };
 
 // One work tile = two 128-row "halves" that share one K/V stream (same request, same KV head).  Each half

@@ -250,4 +250,30 @@ __device__ __forceinline__ float fmax3(float a, float b, float c) {
     return r;
 }
 
+// ------------------------------------------------------------------ row-per-thread results -> coalesced global stores
+// An epilogue thread holds one output ROW (a tensor-memory lane).  Storing it directly makes every warp store hit 32
+// rows at once: 32 partly written 32-byte sectors per instruction, which is what bounds short tiles.  Instead a warp
+// turns a 32-row x 64-byte block round in a 2 KB staging area of its own: lane r leaves its row's 64 bytes there
+// (16-byte chunks XOR-swizzled by row so that neither side has bank conflicts), then every lane stores one 16-byte
+// chunk of a row, four rows' worth of lanes side by side, so that a warp store writes eight complete 64-byte pieces.
+//   mine     : this lane's 64 bytes (columns [col_bytes, col_bytes + 64) of its row)
+//   row_ptr  : this lane's row in global memory (16-byte aligned), used only if row_ok
+__device__ __forceinline__ void warp_store_rows64(uint8_t* stage, int lane, const uint4 (&mine)[4], const void* row_ptr,
+                                                  bool row_ok, int col_bytes) {
+    const unsigned ok_mask = __ballot_sync(0xffffffffu, row_ok);
+    const int sw = (lane >> 1) & 3;
+#pragma unroll
+    for (int c = 0; c < 4; ++c) *reinterpret_cast<uint4*>(stage + lane * 64 + ((c ^ sw) << 4)) = mine[c];
+    __syncwarp();
+    const unsigned long long mine_ptr = reinterpret_cast<unsigned long long>(row_ptr);
+#pragma unroll
+    for (int it = 0; it < 4; ++it) {
+        const int row = it * 8 + (lane >> 2), c = lane & 3;
+        const unsigned long long dst = __shfl_sync(0xffffffffu, mine_ptr, row);
+        const uint4 v = *reinterpret_cast<const uint4*>(stage + row * 64 + ((c ^ ((row >> 1) & 3)) << 4));
+        if ((ok_mask >> row) & 1u) *reinterpret_cast<uint4*>(dst + col_bytes + (c << 4)) = v;
+    }
+    __syncwarp();
+}
+
 }  // namespace wpp

@@ -28,10 +28,13 @@ def device_inputs(w, inp=None, device="cuda"):
 
 
 def run_wave(w, dev_inp, opts=None, sm_scale=0.0, want_lse=True, poison_out=True, do_append=True,
-             do_attention=True, launch_prefix_lens=None, launch_chunk_lens=None):
+             do_attention=True, launch_prefix_lens=None, launch_chunk_lens=None, shape=None):
     """plan -> H2D plan -> wpp_kv_append -> wpp_prefill_attention_varlen on the current stream.
     launch_prefix_lens / launch_chunk_lens: device arrays the kernels get instead of the lengths the plan was made
-    for (a host-made mismatch)."""
+    for (a host-made mismatch).  shape: 1 or 2 overrides the planner's choice of attention kernel."""
+    if shape is not None:
+        o = opts or wpp.PlanOpts()
+        opts = wpp.PlanOpts(o.tile_m, o.tile_n, o.force_kv_splits, o.max_ctas, o.order, shape)
     c = ctx()
     d = desc_of(w, sm_scale)
     plan = wpp.wpp_plan_tiles(c, d, w.prefix_lens, w.chunk_lens, opts=opts).to_device()

@@ -25,4 +25,4 @@ def test_random_ragged_wave(seed):
     w = W.custom_workload(P, C, Hkv * G, Hkv, d, B, seed=seed, spare_pages=int(rng.integers(1, 6)))
     opts = wpp.PlanOpts(int(rng.choice([0, 128, 256])), 0, int(rng.choice([0, 0, 1, 2, 3])),
                         int(rng.choice([0, 1, 2, 5, 37, 148])), int(rng.integers(0, 2)))
-    _full_parity(w, opts=opts)
+    _full_parity(w, opts=opts)            # both kernel shapes

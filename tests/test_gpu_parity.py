@@ -12,17 +12,21 @@ from tests import gpu_harness as H
 pytestmark = pytest.mark.gpu
 
 
-def _full_parity(w, opts=None, inp=None, sm_scale=0.0):
+def _full_parity(w, opts=None, inp=None, sm_scale=0.0, shapes=(1, 2)):
+    """Both attention kernel shapes (unless the options name one) against the oracle; returns the last run."""
     inp = inp or cpu_inputs(w)
     kp, vp, ref, ref_lse = run_oracle(w, inp, sm_scale=sm_scale or None)
-    res = H.run_wave(w, H.device_inputs(w, inp), opts=opts, sm_scale=sm_scale)
-    assert res["status"] == 0
-    # append and page indexing: bit exact over the whole pools
-    assert np.array_equal(bits(res["k_pool"]), kp), "K pool differs"
-    assert np.array_equal(bits(res["v_pool"]), vp), "V pool differs"
-    e = H.assert_close(f64(res["out"]), ref, w.name)
-    lse = res["lse"].double().cpu().numpy()
-    assert np.isfinite(lse).all() and np.abs(lse - ref_lse).max() < 2e-2, np.abs(lse - ref_lse).max()
+    if opts is not None and opts.shape:
+        shapes = (opts.shape,)
+    for shape in shapes:
+        res = H.run_wave(w, H.device_inputs(w, inp), opts=opts, sm_scale=sm_scale, shape=shape)
+        assert res["status"] == 0 and res["plan"].info.shape == shape
+        # append and page indexing: bit exact over the whole pools
+        assert np.array_equal(bits(res["k_pool"]), kp), "K pool differs"
+        assert np.array_equal(bits(res["v_pool"]), vp), "V pool differs"
+        e = H.assert_close(f64(res["out"]), ref, f"{w.name} shape {shape}")
+        lse = res["lse"].double().cpu().numpy()
+        assert np.isfinite(lse).all() and np.abs(lse - ref_lse).max() < 2e-2, np.abs(lse - ref_lse).max()
     return res, e
 
 
@@ -87,15 +91,16 @@ def test_single_step_tiles_back_to_back(ctas):
     _, _, ref, _ = run_oracle(w, inp)
     first = None
     for rep in range(6):
-        res = H.run_wave(w, H.device_inputs(w, inp), opts=wpp.PlanOpts(256 if rep % 2 else 128, 0, 1, ctas))
+        res = H.run_wave(w, H.device_inputs(w, inp), opts=wpp.PlanOpts(256 if rep % 2 else 128, 0, 1, ctas), shape=1 + rep % 2 if rep < 4 else None)
         assert res["status"] == 0
         H.assert_close(f64(res["out"]), ref, f"single-step tiles, {ctas} CTAs, repeat {rep}")
 
 
-def test_single_key_is_bit_exact():
+@pytest.mark.parametrize("shape", [1, 2])
+def test_single_key_is_bit_exact(shape):
     w = W.custom_workload([0], [1], 4, 2, 128, 64, seed=8)
     inp = cpu_inputs(w)
-    res = H.run_wave(w, H.device_inputs(w, inp))
+    res = H.run_wave(w, H.device_inputs(w, inp), shape=shape)
     v0 = inp["v_new"][0]                                     # [Hkv, d]
     out = res["out"].cpu()
     for h in range(4):
@@ -122,16 +127,18 @@ def test_empty_wave_is_a_no_op():
     assert res["status"] == 0 and res["out"].numel() == 0
 
 
-def test_results_are_bit_reproducible():
+@pytest.mark.parametrize("shape", [1, 2])
+def test_results_are_bit_reproducible(shape):
     w = W.custom_workload([500, 77], [260, 300], 8, 2, 128, 64, seed=12)
     inp = cpu_inputs(w)
-    a = H.run_wave(w, H.device_inputs(w, inp), opts=wpp.PlanOpts(256, 0, 3, 0))
-    b = H.run_wave(w, H.device_inputs(w, inp), opts=wpp.PlanOpts(256, 0, 3, 0))
+    a = H.run_wave(w, H.device_inputs(w, inp), opts=wpp.PlanOpts(256, 0, 3, 0), shape=shape)
+    b = H.run_wave(w, H.device_inputs(w, inp), opts=wpp.PlanOpts(256, 0, 3, 0), shape=shape)
     assert torch.equal(a["out"].view(torch.int16), b["out"].view(torch.int16))
     assert torch.equal(a["lse"], b["lse"])
 
 
-def test_results_do_not_depend_on_which_cta_takes_which_tile():
+@pytest.mark.parametrize("shape", [1, 2])
+def test_results_do_not_depend_on_which_cta_takes_which_tile(shape):
     """Tiles are handed out at run time, so the assignment differs from run to run and with the order option; the
     tiles themselves (and the fixed combine order) are the same, so every bit of the result must be too."""
     w = W.custom_workload([1500, 40, 900, 0, 2048, 300], [700, 512, 130, 260, 64, 333], 8, 2, 128, 64, seed=21)
@@ -139,7 +146,7 @@ def test_results_do_not_depend_on_which_cta_takes_which_tile():
     ref = None
     for order in (0, 1, 0, 1):
         for splits in (1, 3):
-            r = H.run_wave(w, H.device_inputs(w, inp), opts=wpp.PlanOpts(256, 0, splits, 0, order))
+            r = H.run_wave(w, H.device_inputs(w, inp), opts=wpp.PlanOpts(256, 0, splits, 0, order), shape=shape)
             assert r["status"] == 0
             key = (splits,)
             ref = ref or {}
@@ -167,16 +174,17 @@ def test_stale_slots_unused_pages_and_scratch_poison_do_not_matter():
     _full_parity(w, inp=inp, opts=wpp.PlanOpts(0, 0, 2, 0))
 
 
-def test_page_permutation_gives_identical_bits():
+@pytest.mark.parametrize("shape", [1, 2])
+def test_page_permutation_gives_identical_bits(shape):
     w = W.custom_workload([200, 0], [130, 260], 4, 2, 128, 64, seed=14, spare_pages=4)
     inp = cpu_inputs(w)
-    a = H.run_wave(w, H.device_inputs(w, inp))
+    a = H.run_wave(w, H.device_inputs(w, inp), shape=shape)
     perm = np.random.default_rng(15).permutation(w.num_pages)
     kp = torch.empty_like(inp["k_pool"]); vp = torch.empty_like(inp["v_pool"])
     kp[perm] = inp["k_pool"]; vp[perm] = inp["v_pool"]
     w2 = W.custom_workload([200, 0], [130, 260], 4, 2, 128, 64, seed=14, spare_pages=4)
     w2.block_tables = np.where(w.block_tables >= 0, perm[np.maximum(w.block_tables, 0)], -1).astype(np.int32)
-    b = H.run_wave(w2, H.device_inputs(w2, dict(inp, k_pool=kp, v_pool=vp)))
+    b = H.run_wave(w2, H.device_inputs(w2, dict(inp, k_pool=kp, v_pool=vp)), shape=shape)
     assert torch.equal(a["out"].view(torch.int16), b["out"].view(torch.int16))
 
 
@@ -216,19 +224,21 @@ def test_a_wait_that_runs_out_reports_timeout_and_leaves_the_context_usable():
     _full_parity(W.custom_workload([64], [64], 2, 1, 128, 64, seed=17))      # the context still works
 
 
-def test_bad_page_id_sets_status_without_trapping():
+@pytest.mark.parametrize("shape", [1, 2])
+def test_bad_page_id_sets_status_without_trapping(shape):
     w = W.custom_workload([64], [64], 2, 1, 128, 64, seed=17)
     w.block_tables = w.block_tables.copy()
     w.block_tables[0, 1] = w.num_pages + 5
-    res = H.run_wave(w, H.device_inputs(w))
+    res = H.run_wave(w, H.device_inputs(w), shape=shape)
     assert res["status"] == 3          # WPP_ERR_BOUNDS
     # the context is still usable
     w2 = W.custom_workload([64], [64], 2, 1, 128, 64, seed=17)
     _full_parity(w2)
 
 
+@pytest.mark.parametrize("shape", [1, 2])
 @pytest.mark.parametrize("splits", [1, 2])
-def test_plan_launched_with_other_lengths_is_refused_per_request(splits):
+def test_plan_launched_with_other_lengths_is_refused_per_request(splits, shape):
     """Section 4.6: a position mismatch fails execution instead of running against the wrong cache state.  The
     plan is made for one set of spans; the device arrays are altered afterwards (on the host): the requests
     whose span differs are refused - status WPP_ERR_PLAN_MISMATCH, none of their slots written, none of their
@@ -240,7 +250,7 @@ def test_plan_launched_with_other_lengths_is_refused_per_request(splits):
     P_dev[1] += 64          # this rank's cache of request 1 ends elsewhere
     C_dev[3] -= 1           # request 3's span has another length
     res = H.run_wave(w, H.device_inputs(w, inp), opts=wpp.PlanOpts(0, 0, splits, 0), launch_prefix_lens=P_dev,
-                     launch_chunk_lens=C_dev)
+                     launch_chunk_lens=C_dev, shape=shape)
     assert res["status"] == 6                                    # WPP_ERR_PLAN_MISMATCH
     # the oracle's wave without the refused requests: their chunks are empty
     C_ok = w.chunk_lens.copy()

@@ -16,22 +16,23 @@ import paper_2609_35263_b200 as wpp
 from paper_2609_35263_b200 import binding
 
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
-HDR_FMT = "<IIQ" + "i" * 8 + "qqq" + "QQ" + "IIII"      # WppPlanHeader up to the section offsets
+HDR_FMT = "<IIQ" + "i" * 8 + "qqq" + "QQ" + "IIII" + "ii"      # WppPlanHeader up to the kernel shape
 
 
 def parse_plan(plan):
     raw = plan.host_bytes()
     f = struct.unpack_from(HDR_FMT, raw, 0)
     (magic, version, desc_hash, R, num_ctas, num_units, num_combine, num_slots, tile_m, tile_n, head_dim,
-     T, key_steps, flops, ws_bytes, plan_bytes, off_q, _reserved, off_units, off_comb) = f
+     T, key_steps, flops, ws_bytes, plan_bytes, off_q, off_prefix, off_units, off_comb, shape, nonempty_halves) = f
     assert magic == 0x31505057
     q_off = np.frombuffer(raw, dtype=np.int32, count=R + 1, offset=off_q)
     units = np.frombuffer(raw, dtype=np.int32, count=num_units * 12, offset=off_units).reshape(num_units, 12)
     comb = np.frombuffer(raw, dtype=np.int32, count=num_combine * 8, offset=off_comb).reshape(num_combine, 8)
     keys = ["request", "kv_begin", "kv_end", "split_slot", "row0_a", "row0_b", "rows_a", "rows_b", "head_a",
             "head_b", "cost", "pack"]
+    prefix = np.frombuffer(raw, dtype=np.int32, count=R, offset=off_prefix)
     return dict(R=R, num_ctas=num_ctas, tile_m=tile_m, T=T, key_steps=key_steps, flops=flops, slots=num_slots,
-                ws_bytes=ws_bytes, q_off=q_off, comb=comb,
+                ws_bytes=ws_bytes, q_off=q_off, comb=comb, shape=shape, nonempty_halves=nonempty_halves, prefix=prefix,
                 units=[dict(zip(keys, u.tolist())) for u in units])
 
 
@@ -74,7 +75,9 @@ def test_plan_covers_every_visible_pair_exactly_once(P, C, Hq, Hkv, tile_m, spli
     plan = wpp.wpp_plan_tiles(None, d, P, C, opts=wpp.PlanOpts(tile_m, 0, splits, 40), pin=False)
     pl = parse_plan(plan)
     assert pl["T"] == sum(C) and pl["q_off"].tolist() == np.concatenate([[0], np.cumsum(C)]).tolist()
-    assert 1 <= pl["num_ctas"] <= 40
+    assert pl["shape"] in (1, 2) and 1 <= pl["num_ctas"] <= 40 * pl["shape"]     # the small shape runs two CTAs per SM
+    assert pl["prefix"].tolist() == list(P)                                      # the spans the kernels check against
+    assert pl["nonempty_halves"] == sum((u["rows_a"] > 0) + (u["rows_b"] > 0) for u in pl["units"])
     G = Hq // Hkv
     cover = {}
     steps_total = 0
@@ -138,7 +141,7 @@ def test_plan_is_deterministic_and_its_order_balances():
     C = rng.integers(1, 2000, 24).tolist()
     d = desc(24, 16, 4, 128, 64, 200)
     for order in (0, 1):
-        opts = wpp.PlanOpts(0, 0, 0, 0, order)
+        opts = wpp.PlanOpts(0, 0, 0, 0, order, 1)
         a = wpp.wpp_plan_tiles(None, d, P, C, opts=opts, pin=False)
         b = wpp.wpp_plan_tiles(None, d, P, C, opts=opts, pin=False)
         assert a.host_bytes() == b.host_bytes()
@@ -159,7 +162,7 @@ def test_plan_is_deterministic_and_its_order_balances():
 
 def test_stream_order_runs_the_tiles_of_one_kv_stream_together():
     d = desc(3, 16, 4, 128, 64, 200)
-    pl = parse_plan(wpp.wpp_plan_tiles(None, d, [4096, 0, 8192], [1024, 512, 256], opts=wpp.PlanOpts(256, 0, 1, 8),
+    pl = parse_plan(wpp.wpp_plan_tiles(None, d, [4096, 0, 8192], [1024, 512, 256], opts=wpp.PlanOpts(256, 0, 1, 8, 0, 1),
                                        pin=False))
     # the first tiles (one per CTA) belong to KV head 0 of the costliest request (request 0: 4 row blocks x 4 heads)
     firsts = pl["units"][:pl["num_ctas"]]
@@ -237,3 +240,20 @@ def test_there_is_no_cpu_fallback():
         pytest.skip("a device is present")
     with pytest.raises(wpp.WppError):
         wpp.Context(0)
+
+
+def test_kernel_shape_follows_the_mean_key_steps_per_half():
+    """Short tiles go to the small kernel shape (two CTAs per SM), long ones to the SM-wide one; an explicit choice
+    is kept; the shape is part of the plan."""
+    d = desc(4, 8, 2, 128, 64, 300)
+    short = wpp.wpp_plan_tiles(None, d, [0, 0, 0, 0], [64, 100, 64, 128], pin=False)
+    long_ = wpp.wpp_plan_tiles(None, d, [16000, 9000, 12000, 8000], [256, 300, 64, 500], pin=False)
+    assert short.info.shape == 2 and parse_plan(short)["shape"] == 2
+    assert long_.info.shape == 1 and parse_plan(long_)["shape"] == 1
+    assert short.info.num_ctas == min(2 * 148, 2 * short.info.num_tiles)
+    for shape in (1, 2):
+        forced = wpp.wpp_plan_tiles(None, d, [0, 64, 0, 128], [256, 300, 64, 500], opts=wpp.PlanOpts(0, 0, 0, 0, 0, shape),
+                                    pin=False)
+        assert forced.info.shape == shape
+    with pytest.raises(wpp.WppError):
+        wpp.wpp_plan_tiles(None, d, [0] * 4, [64] * 4, opts=wpp.PlanOpts(0, 0, 0, 0, 0, 3), pin=False)
