@@ -33,8 +33,8 @@ METRIC = "prefill-attention tokens/s at concurrency 128, high prefix reuse"
 # ncu capture by the work of the launch timed here, and `roofline.traffic_source` says so in the JSON line.
 # Attention: dram__bytes_read.sum + dram__bytes_write.sum of one launch / its 128-row x 128-key steps, captured on the
 # 16-request cut of the concurrency-128 workload (--config cfg3_r16, 1.4 GB resident).
-DRAM_BYTES_PER_KEY_STEP = 628.9
-DRAM_SOURCE = ("estimate: 628.9 DRAM bytes per 128x128 key step (dram__bytes_read.sum + dram__bytes_write.sum of one "
+DRAM_BYTES_PER_KEY_STEP = 607.6
+DRAM_SOURCE = ("estimate: 607.6 DRAM bytes per 128x128 key step (dram__bytes_read.sum + dram__bytes_write.sum of one "
                "wpp_attn_kernel launch, ncu capture on the 16-request cut of this workload) x this launch's key steps; "
                "not measured in this run")
 # Recurrent layer: dram read + write bytes of one wpp_kda_chunk launch on the default wave (8 x 2,048 tokens, 32 heads)

@@ -213,6 +213,8 @@ int wpp_prefill_attention_varlen(const wpp_ctx* ctx, const wpp_batch_desc* desc,
  *   - The array's device address is looked up by wpp_create (once per device, with that device current), so that
  *     the memory is placed at start-up and no call of this entry point has anything left to set up; create the
  *     context before any stream capture begins.
+ *     (Like any CUDA kernel, the attention kernels are loaded onto the device by their first launch; this entry
+ *     point adds nothing to that.)
  *   - All calls on a device share the one array and it keeps whatever the last call left in it.  The call zeroes
  *     the tile counter itself (a memset node on the stream) and every partial row is written before the combine
  *     pass reads it, but two calls whose kernels overlap on the GPU, e.g. on different streams, race on it:
