@@ -34,6 +34,20 @@ constexpr uint32_t kColS = 0, kColP = 64, kColO = 128;
 constexpr float kRefSlack = 16.f;         // a row keeps its reference while its scores stay below reference + 16 (log2)
 constexpr int kRescaleCols = 16;
 
+// What every role derives from an item, identically.  A request whose span on the device differs from the plan's
+// gets no key steps (see the main kernel).
+struct ItemView {
+    int P, kv_len, q_off;
+    int step0, n;          // first 64-key step (absolute) and number of steps
+    bool mismatch;
+};
+// What the producer hands to the other roles with an item: the unit and everything derived from it, so that no
+// consumer repeats the dependent global reads (unit, then the request's lengths) at the start of every item.
+struct ItemRec {
+    WppUnit un;
+    int32_t it;            // item index (2 * unit + half), < 0: no more items
+    int32_t P, kv_len, q_off, step0, n, mismatch, pad;
+};
 template <int D>
 struct Cfg {
     static constexpr int kHalves = D / 64;                 // 64-element (128-byte) swizzled column blocks
@@ -49,7 +63,7 @@ struct Cfg {
     static constexpr int kNumBars = 2 + 4 * kSlots + 5 + 2 * kTileQ;
     static constexpr int kOffStage = (kOffBars + 8 * kNumBars + 15) / 16 * 16;   // 4 x 2 KB: the warps' store staging
     static constexpr int kOffMisc = kOffStage + 4 * 2048;
-    static constexpr int kUsedBytes = kOffMisc + 16 + 4 * kTileQ + 8;
+    static constexpr int kUsedBytes = kOffMisc + 16 + (int)sizeof(ItemRec) * kTileQ + 8;
     static constexpr int kSmemBytes = kUsedBytes + 1024;   // 105.4 KB at D = 128
 };
 
@@ -60,13 +74,6 @@ struct Ring {
     }
 };
 
-// What every role derives from an item, identically.  A request whose span on the device differs from the plan's
-// gets no key steps (see the main kernel).
-struct ItemView {
-    int P, kv_len, q_off;
-    int step0, n;          // first 64-key step (absolute) and number of steps
-    bool mismatch;
-};
 __device__ __forceinline__ ItemView view_of(const WppUnit& un, int hf, const AttnParams& p, const int32_t* q_offsets,
                                             const int32_t* plan_prefix) {
     ItemView v;
@@ -103,7 +110,7 @@ wpp_attn_small_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
     const uint32_t bTileFull = bSFull + 40, bTileEmpty = bTileFull + 8 * C::kTileQ;
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_gen + C::kOffMisc);
     volatile uint32_t* abort_flag = tmem_slot + 1;
-    volatile int32_t* tile_ids = reinterpret_cast<volatile int32_t*>(tmem_slot + 4);      // [kTileQ]
+    volatile ItemRec* item_q = reinterpret_cast<volatile ItemRec*>(tmem_slot + 4);        // [kTileQ]
     constexpr uint32_t kTileConsumers = 1 + 128;   // the issuing thread and the softmax threads
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -139,12 +146,21 @@ wpp_attn_small_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
     const WppUnit* units = reinterpret_cast<const WppUnit*>(plan + hd->off_units);
     const int num_items = 2 * hd->num_units;
     Ring tile_ring = {0, 0};
-    auto next_item = [&]() -> int {       // -1: no more items, -2: the wait was abandoned
-        if (!mbar_wait(bTileFull + 8 * tile_ring.stage, tile_ring.phase, abort_flag)) return -2;
-        const int id = tile_ids[tile_ring.stage];
+    // the next item for a consuming role; returns false when the wait was abandoned (rec.it < 0: no more items)
+    auto next_item = [&](WppUnit& un, int& hf, ItemView& v, int& it) -> bool {
+        if (!mbar_wait(bTileFull + 8 * tile_ring.stage, tile_ring.phase, abort_flag)) return false;
+        volatile ItemRec& r = item_q[tile_ring.stage];
+        it = r.it;
+        if (it >= 0) {
+            un.request = r.un.request; un.kv_begin = r.un.kv_begin; un.kv_end = r.un.kv_end; un.split_slot = r.un.split_slot;
+            un.row0[0] = r.un.row0[0]; un.row0[1] = r.un.row0[1]; un.rows[0] = r.un.rows[0]; un.rows[1] = r.un.rows[1];
+            un.head[0] = r.un.head[0]; un.head[1] = r.un.head[1]; un.cost = r.un.cost; un.pack = r.un.pack;
+            hf = it & 1;
+            v.P = r.P; v.kv_len = r.kv_len; v.q_off = r.q_off; v.step0 = r.step0; v.n = r.n; v.mismatch = r.mismatch != 0;
+        }
         mbar_arrive(bTileEmpty + 8 * tile_ring.stage);
         tile_ring.advance(C::kTileQ);
-        return id;
+        return true;
     };
     const int B = p.page_size;
     const int rows_box = B < kKeys ? B : kKeys;       // rows of one K/V box (the maps are built with this box)
@@ -154,24 +170,38 @@ wpp_attn_small_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
         Ring ring_k = {0, 0}, ring_v = {0, 0};
         uint32_t q_phase = 0;
         bool dead = false;
+        // item ids are taken one ahead: the atomic's round trip overlaps the previous item's load issue
+        int it_next = 0;
+        if (lane == 0) it_next = (int)atomicAdd(p.tile_counter, 1u);
         while (!dead) {
-            int it = 0;
-            if (lane == 0) it = (int)atomicAdd(p.tile_counter, 1u);
-            it = __shfl_sync(0xffffffffu, it, 0);
+            int it = __shfl_sync(0xffffffffu, it_next, 0);
             if (it >= num_items) it = -1;
+            if (it >= 0 && lane == 0) it_next = (int)atomicAdd(p.tile_counter, 1u);
+            WppUnit un;
+            ItemView v;
+            int hf = 0;
+            if (it >= 0) {
+                un = units[it >> 1];
+                hf = it & 1;
+                v = view_of(un, hf, p, q_offsets, plan_prefix);
+            }
             {
                 const bool ok = mbar_wait(bTileEmpty + 8 * tile_ring.stage, tile_ring.phase ^ 1u, abort_flag);
                 if (!__all_sync(0xffffffffu, ok)) break;
                 if (lane == 0) {
-                    tile_ids[tile_ring.stage] = it;
+                    volatile ItemRec& r = item_q[tile_ring.stage];
+                    r.it = it;
+                    if (it >= 0) {
+                        r.un.request = un.request; r.un.kv_begin = un.kv_begin; r.un.kv_end = un.kv_end; r.un.split_slot = un.split_slot;
+                        r.un.row0[0] = un.row0[0]; r.un.row0[1] = un.row0[1]; r.un.rows[0] = un.rows[0]; r.un.rows[1] = un.rows[1];
+                        r.un.head[0] = un.head[0]; r.un.head[1] = un.head[1]; r.un.cost = un.cost; r.un.pack = un.pack;
+                        r.P = v.P; r.kv_len = v.kv_len; r.q_off = v.q_off; r.step0 = v.step0; r.n = v.n; r.mismatch = v.mismatch;
+                    }
                     mbar_arrive(bTileFull + 8 * tile_ring.stage);
                 }
                 tile_ring.advance(C::kTileQ);
             }
             if (it < 0) break;
-            const WppUnit un = units[it >> 1];
-            const int hf = it & 1;
-            const ItemView v = view_of(un, hf, p, q_offsets, plan_prefix);
             if (v.mismatch && lane == 0 && p.status) atomicCAS(p.status, 0, WPP_ERR_PLAN_MISMATCH);
             if (v.n == 0) continue;
             const int kvh = un.head[hf] / p.group;
@@ -201,10 +231,9 @@ wpp_attn_small_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
                 ring.advance(C::kSlots);
                 return true;
             };
-            if (!load_tile(&tm_k, 0, ring_k, sK, bKFull, bKEmpty)) { dead = true; break; }
-            {
+            auto load_q = [&]() -> bool {
                 const bool ok = mbar_wait(bQEmpty, q_phase ^ 1u, abort_flag);
-                if (!__all_sync(0xffffffffu, ok)) { dead = true; break; }
+                if (!__all_sync(0xffffffffu, ok)) return false;
                 q_phase ^= 1u;
                 if (lane == 0) mbar_arrive_expect_tx(bQFull, C::kQBytes);
                 __syncwarp();
@@ -217,7 +246,14 @@ wpp_attn_small_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
                     tma_load_3d(sQ + h * C::kQHalfBytes + k * rph * 128, qm, bQFull, h * 64, un.head[hf] + k,
                                 v.q_off + un.row0[hf]);
                 }
-            }
+                return true;
+            };
+            // the queries need no page ids: they go first when their buffer is free already (the usual case after a
+            // short item), else the first K tile goes while the previous item still holds the Q buffer
+            const bool q_first = __all_sync(0xffffffffu, mbar_test(bQEmpty, q_phase ^ 1u) != 0u);
+            if (q_first && !load_q()) { dead = true; break; }
+            if (!load_tile(&tm_k, 0, ring_k, sK, bKFull, bKEmpty)) { dead = true; break; }
+            if (!q_first && !load_q()) { dead = true; break; }
             __syncwarp();
             for (int j = 0; j < v.n && !dead; ++j) {
                 if (!load_tile(&tm_v, j, ring_v, sV, bVFull, bVEmpty)) dead = true;
@@ -253,11 +289,10 @@ wpp_attn_small_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
             return true;
         };
         while (!dead) {
-            const int it = next_item();
-            if (it < 0) break;
-            const WppUnit un = units[it >> 1];
-            const int hf = it & 1;
-            const ItemView v = view_of(un, hf, p, q_offsets, plan_prefix);
+            WppUnit un;
+            ItemView v;
+            int hf = 0, it = -1;
+            if (!next_item(un, hf, v, it) || it < 0) break;
             if (v.n == 0) continue;
             if (!mbar_wait(bQFull, q_phase, abort_flag)) break;
             q_phase ^= 1u;
@@ -298,11 +333,11 @@ wpp_attn_small_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
         const uint64_t c2 = pack2(c, c);
         bool dead = false;
         while (!dead) {
-            const int it = next_item();
-            if (!__all_sync(0xffffffffu, it != -2) || it < 0) break;
-            const WppUnit un = units[it >> 1];
-            const int hf = it & 1;
-            const ItemView v = view_of(un, hf, p, q_offsets, plan_prefix);
+            WppUnit un;
+            ItemView v;
+            int hf = 0, it = -1;
+            const bool got = next_item(un, hf, v, it);
+            if (!__all_sync(0xffffffffu, got) || it < 0) break;
             if (un.rows[hf] == 0) continue;
             const int rph = 128 / un.pack, rr = r & (rph - 1);           // row inside its head's block
             const int head = un.head[hf] + r / rph;
@@ -437,7 +472,7 @@ wpp_attn_small_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
             uint8_t* stage = smem_gen + C::kOffStage + warp * 2048;
             if (un.split_slot < 0) {
                 const __nv_bfloat16* dst = p.out + tok * p.o_token_stride + (int64_t)head * p.o_head_stride;
-#pragma unroll
+#pragma unroll 1
                 for (int q4 = 0; q4 < D / 32; ++q4) {
                     float o[32];
                     tmem_ld32(lane_addr + kColO + q4 * 32, reinterpret_cast<uint32_t*>(o));
@@ -455,7 +490,7 @@ wpp_attn_small_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
                 if (p.lse && row_ok) p.lse[tok * p.num_q_heads + head] = lse2 * 0.6931471805599453f;
             } else {
                 const float* dst = p.ws_o + prow * D;
-#pragma unroll
+#pragma unroll 1
                 for (int q4 = 0; q4 < D / 32; ++q4) {
                     float o[32];
                     tmem_ld32(lane_addr + kColO + q4 * 32, reinterpret_cast<uint32_t*>(o));

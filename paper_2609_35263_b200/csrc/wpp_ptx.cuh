@@ -38,6 +38,19 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
     return ok;
 }
 
+// Non-blocking test of a phase (never suspends the thread).
+__device__ __forceinline__ uint32_t mbar_test(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok;
+}
+
 // Every wait in the kernels is bounded: after WPP_WAIT_LIMIT cycles the waiter raises the CTA's abort flag
 // and gives up; every other waiter of the CTA sees the flag within a few polls and gives up too.
 #ifndef WPP_WAIT_LIMIT
