@@ -398,7 +398,7 @@ typedef struct {
  *   snap_slots  : device int32 [R, max_snaps] or NULL: slot for the n-th boundary inside the chunk, -1 = skip;
  *                 boundaries past max_snaps are skipped.
  *   out         : device bf16 [T, H, d_v].
- *   workspace   : device scratch for the chunk-parallel form, 1024-byte aligned, wpp_kda_workspace_bytes(desc)
+ *   workspace   : device scratch for the chunk-parallel form, 256-byte aligned, wpp_kda_workspace_bytes(desc)
  *                 bytes (about 160 KB per 64 tokens and head); may be NULL (0 bytes) for the other forms.  Contents
  *                 are undefined afterwards; calls that may overlap on the GPU need a workspace each.
  *   status_dev  : device int32 or NULL; a slot id outside [-1, num_slots) sets it to WPP_ERR_BOUNDS (if it was 0)

@@ -449,7 +449,7 @@ def wpp_kda_chunk(ctx: Context, q, k, v, alpha, beta, row_offsets, state_pool, s
     row_offsets: cuda int64 [R+1]; state_pool: cuda fp32 [slots, H, 128, 128] (updated in place); state_in,
     state_out: cuda int32 [R] (-1: zero state / do not store); snap_slots: cuda int32 [R, max_snaps] with
     prefix_lens (cuda int32 [R]) and snap_interval > 0 for periodic snapshots.  layout 0 lets the library choose:
-    the chunk-parallel tensor-core form when `workspace` (cuda uint8, wpp_kda_workspace_bytes bytes, 1024-byte
+    the chunk-parallel tensor-core form when `workspace` (cuda uint8, wpp_kda_workspace_bytes bytes, 256-byte
     aligned) is given and the chunks average 64 tokens or more, else a token-by-token form; 1, 2: token by token
     with one / four CTAs per (request, head); 3: chunk-parallel.  Returns the cuda bf16 output."""
     T, H, dk = (int(x) for x in q.shape)

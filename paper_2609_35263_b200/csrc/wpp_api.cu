@@ -408,8 +408,8 @@ extern "C" int wpp_kda_chunk(const wpp_ctx* ctx, const wpp_kda_desc* desc, const
     if (desc->layout == 0)
         tensor_form = workspace && workspace_bytes >= w.bytes && desc->total_tokens >= 64 * (int64_t)desc->num_requests;
     if (tensor_form) {
-        if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 1023) != 0) return WPP_ERR_INVALID_ARG;
-        if (workspace_bytes < w.bytes) return WPP_ERR_WORKSPACE_TOO_SMALL;
+        if (!workspace || workspace_bytes < w.bytes) return WPP_ERR_WORKSPACE_TOO_SMALL;
+        if ((reinterpret_cast<uintptr_t>(workspace) & 255) != 0) return WPP_ERR_INVALID_ARG;
         if (w.n_bh * 64 > 0x7fffffffll || desc->total_tokens > 0x7fffffffll) return WPP_ERR_UNSUPPORTED;
         char* ws = static_cast<char*>(workspace);
         wpp::KdaTcParams p;

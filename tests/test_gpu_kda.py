@@ -205,6 +205,16 @@ def test_argument_errors():
         wpp.wpp_kda_chunk(H.ctx(), z(4, 1, 128), z(4, 1, 128), z(4, 1, 128), z(4, 1, 128, dt=torch.float32),
                           z(4, 1, dt=torch.float32), ro, pool, slot, slot, layout=3)
     assert e.value.status == 1
+    with pytest.raises(wpp.WppError) as e:                            # the chunk-parallel form needs its workspace
+        wpp.wpp_kda_chunk(H.ctx(), z(4, 1, 128), z(4, 1, 128), z(4, 1, 128), z(4, 1, 128, dt=torch.float32),
+                          z(4, 1, dt=torch.float32), ro, pool, slot, slot, layout=3)
+    assert e.value.status == 5
+    small = torch.empty(1024, dtype=torch.uint8, device=dev)
+    with pytest.raises(wpp.WppError) as e:
+        wpp.wpp_kda_chunk(H.ctx(), z(4, 1, 128), z(4, 1, 128), z(4, 1, 128), z(4, 1, 128, dt=torch.float32),
+                          z(4, 1, dt=torch.float32), ro, pool, slot, slot, layout=3, workspace=small)
+    assert e.value.status == 5
+    assert wpp.wpp_kda_workspace_bytes(1, 1, 4) > 1024
     with pytest.raises(wpp.WppError) as e:                            # periodic snapshots need prefix_lens
         wpp.wpp_kda_chunk(H.ctx(), z(4, 1, 128), z(4, 1, 128), z(4, 1, 128), z(4, 1, 128, dt=torch.float32),
                           z(4, 1, dt=torch.float32), ro, pool, slot, slot, snap_interval=2,
