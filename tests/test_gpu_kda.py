@@ -203,7 +203,7 @@ def test_argument_errors():
     pool = z(1, 1, 128, 128, dt=torch.float32)
     with pytest.raises(wpp.WppError) as e:                            # no such layout
         wpp.wpp_kda_chunk(H.ctx(), z(4, 1, 128), z(4, 1, 128), z(4, 1, 128), z(4, 1, 128, dt=torch.float32),
-                          z(4, 1, dt=torch.float32), ro, pool, slot, slot, layout=3)
+                          z(4, 1, dt=torch.float32), ro, pool, slot, slot, layout=4)
     assert e.value.status == 1
     with pytest.raises(wpp.WppError) as e:                            # the chunk-parallel form needs its workspace
         wpp.wpp_kda_chunk(H.ctx(), z(4, 1, 128), z(4, 1, 128), z(4, 1, 128), z(4, 1, 128, dt=torch.float32),
@@ -240,3 +240,31 @@ def test_full_size_wave_on_sampled_heads(lanes, chunk):
         ref_o, ref_pool = _oracle(sub, ts, heads=slice(head, head + 1))
         _close_out(got_o[sl, head:head + 1], ref_o, f"outputs of request {req} head {head}")
         _close_state(got_pool[w.state_out[req], head], ref_pool[w.state_out[req], 0], "final state")
+
+
+@pytest.mark.parametrize("seed", range(24))
+def test_random_waves_in_the_chunk_parallel_form(seed):
+    """Seeded random waves for the chunk-parallel form: chunk lengths around the block size, prefixes at every
+    alignment, snapshot intervals from 1 (every token is a sub-block of its own) to beyond a block, some channels with
+    zero and tiny decays (extra cuts), odd head counts, resumed and zero states - all against the oracle."""
+    rng = np.random.default_rng(4000 + seed)
+    R = int(rng.integers(1, 6))
+    H_ = int(rng.choice([1, 2, 3]))
+    lens = [int(x) for x in rng.choice([0, 1, 2, 31, 63, 64, 65, 100, 127, 128, 129, 200, 333], R)]
+    if sum(lens) == 0:
+        lens[0] = 70
+    prefix = [int(x) for x in rng.choice([0, 1, 5, 63, 64, 65, 100, 128, 1000, 4097], R)]
+    interval = int(rng.choice([0, 0, 1, 2, 3, 16, 50, 64, 65, 200]))
+    w = W.kda_workload("fuzz", 100 + seed, lens, H_, prefix, resume=rng.random(R) < 0.7, snap_interval=interval)
+    t = w.tensors()
+    if seed % 3 == 0 and w.total_tokens > 0:
+        a = t["alpha"].numpy()
+        T = a.shape[0]
+        for val, count in ((0.0, 6), (1e-9, 6), (1e-30, 4), (0.2, 200)):
+            idx = (rng.integers(0, T, count), rng.integers(0, H_, count), rng.integers(0, 128, count))
+            a[idx] = val
+    ref_o, ref_pool = _oracle(w, t)
+    got_o, got_pool, status = _gpu(w, t, layout=3)
+    assert status == 0 and np.isfinite(got_o).all() and np.isfinite(got_pool).all()
+    _close_out(got_o, ref_o, "outputs")
+    _close_state(got_pool, ref_pool, "state pool")
