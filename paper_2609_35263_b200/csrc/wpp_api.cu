@@ -438,7 +438,7 @@ extern "C" int wpp_kda_chunk(const wpp_ctx* ctx, const wpp_kda_desc* desc, const
         p.ws_u0 = reinterpret_cast<float*>(ws + w.off_u0);
         __nv_bfloat16** ops[6] = {&p.ws_w0_h, &p.ws_w0_l, &p.ws_qt_h, &p.ws_qt_l, &p.ws_kb_h, &p.ws_kb_l};
         __nv_bfloat16** sqs[2] = {&p.ws_m_h, &p.ws_m_l};
-        CUtensorMap maps[8];
+        CUtensorMap maps[13];
         int rc;
         for (int i = 0; i < 6; ++i) {
             *ops[i] = reinterpret_cast<__nv_bfloat16*>(ws + w.off_op[i]);
@@ -454,7 +454,27 @@ extern "C" int wpp_kda_chunk(const wpp_ctx* ctx, const wpp_kda_desc* desc, const
             const uint32_t box[2] = {64, 64};
             if ((rc = make_map(ctx, &maps[6 + i], *sqs[i], 2, dims, strides, box)) != WPP_OK) return rc;
         }
-        int e = wpp_launch_kda_tc(&p, maps, (int)w.max_blocks, cuda_stream);
+        // fp32 arrays (U0, alpha) as bf16 maps with twice the elements per row: the copies move bytes
+        {
+            const uint64_t dims[2] = {256, (uint64_t)w.n_bh * 64};
+            const uint64_t strides[1] = {512};
+            const uint32_t box[2] = {64, 64};
+            if ((rc = make_map(ctx, &maps[8], p.ws_u0, 2, dims, strides, box)) != WPP_OK) return rc;
+        }
+        if (desc->total_tokens > 0) {
+            const uint64_t H = (uint64_t)desc->num_heads, T = (uint64_t)desc->total_tokens;
+            const void* in[3] = {q, k, v};
+            const uint32_t box[3] = {64, 1, 64};
+            for (int i = 0; i < 3; ++i) {
+                const uint64_t dims[3] = {128, H, T};
+                const uint64_t strides[2] = {256, 256 * H};
+                if ((rc = make_map(ctx, &maps[9 + i], in[i], 3, dims, strides, box)) != WPP_OK) return rc;
+            }
+            const uint64_t dims[3] = {256, H, T};
+            const uint64_t strides[2] = {512, 512 * H};
+            if ((rc = make_map(ctx, &maps[12], alpha, 3, dims, strides, box)) != WPP_OK) return rc;
+        }
+        int e = wpp_launch_kda_tc(&p, maps, desc->total_tokens > 0 ? (int)w.max_blocks : 0, ctx->sm_count, cuda_stream);
         if (e != 0) return cuda_fail(ctx, e);
         const_cast<wpp_ctx*>(ctx)->launches += 3;
         return WPP_OK;

@@ -95,7 +95,8 @@ struct KdaTcParams {
 }  // namespace wpp
 
 extern "C" {
-int wpp_launch_kda_tc(const wpp::KdaTcParams* p, const CUtensorMap* maps, int max_blocks, void* stream);
+// maps: 0..5 the operand arrays W0, Qt, Kb (hi, lo each), 6..7 M (hi, lo), 8 U0, 9..12 q, k, v, alpha
+int wpp_launch_kda_tc(const wpp::KdaTcParams* p, const CUtensorMap* maps, int max_blocks, int num_sms, void* stream);
 int wpp_launch_attention(int head_dim, const CUtensorMap* tq, const CUtensorMap* tk, const CUtensorMap* tv,
                          const wpp::AttnParams* p, int num_ctas, void* stream);
 int wpp_launch_attention_small(int head_dim, const CUtensorMap* tq, const CUtensorMap* tk, const CUtensorMap* tv,

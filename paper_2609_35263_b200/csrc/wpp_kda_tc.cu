@@ -129,456 +129,598 @@ __global__ void __launch_bounds__(1024) kda_tc_setup_kernel(const KdaTcParams p)
 }
 
 // ---------------------------------------------------------------------------------------------------------------
-// Preparation: one CTA (256 threads) per (block, head).  Shared memory is three regions of 32 KB that change roles:
-//   R0: alpha, then the decay products G (fp32 [64][128]); then Qt as an MMA operand; then T (hi tile, lo tile) and,
-//       behind them, the inverse it is made from
-//   R1: Kt as an MMA operand (A of Kt Kh^T, later B of T Kt)
-//   R2: Kh as an MMA operand; then the triangular matrix (fp32 [64][64]) and the V tile
-// An operand tile has 64 rows (tokens); as the A operand of a 128-row MMA its rows 64.. are whatever follows it in
-// shared memory: those rows of the result are never read.
+// Preparation: persistent CTAs (256 threads, two per SM), each taking (block, head) items in turn.  Inputs arrive by
+// TMA a phase ahead of their use and results leave by TMA stores from swizzled staging tiles, so that no warp waits
+// on a global load and no store instruction touches 32 rows at once.  Shared memory:
+//   RA (64 KB): four slabs of 16 KB, slab s = 2 * term + khalf (term 0 = hi, 1 = lo; khalf = channels [64 khalf, +64)).
+//       Each slab is a Kt tile (64 tokens x 128 bytes, swizzled) followed by an 8 KB slot, so that the A operand of a
+//       128-row MMA that starts at the Kt tile has the slot as its rows 64..127.
+//       Kt tiles, in turn: the raw keys (in the hi tiles) and queries (in the lo tiles) as they arrive; Kt (a thread
+//       replaces the 16 bytes it read); staging of U0 on the way out.
+//       Slots, in turn: alpha and then the decay products G (fp32, 32 channels per slot, 16-byte chunks swizzled like a
+//       tile's); the Qt tiles (rows 64..127 of the first product's A operand: one MMA forms Kt Kh^T on lanes 0..63 and
+//       Qt Kh^T on lanes 64..127; the same tiles are the source of the Qt stores); then the triangular matrix (fp32,
+//       32 rows per slot, slots 0 and 1) and the V tiles (slots 2 and 3).
+//   R2 (32 KB): the Kh tiles (same order as the slabs, 8 KB each); then staging of M (16 KB) and the inverse (16 KB);
+//       then T as an A operand whose rows 64..127 repeat rows 0..63 (hi tile twice, lo tile twice), so that all 128
+//       lanes of the second products carry results and all eight warps read them out; then staging of W0.
+// fp32 arrays (alpha, U0) go through bf16 tensor maps with twice the elements per row: the copies move bytes.
 struct PrepSmem {
-    static constexpr int kOffR0 = 0;
-    static constexpr int kOffR1 = kOffR0 + 4 * kTileBytes;
-    static constexpr int kOffR2 = kOffR1 + 4 * kTileBytes;
-    static constexpr int kOffMisc = kOffR2 + 4 * kTileBytes;  // beta[64], reduction scratch, tmem slot, barrier
+    static constexpr int kSlab = 2 * kTileBytes;
+    static constexpr int kOffRA = 0;
+    static constexpr int kOffR2 = kOffRA + 4 * kSlab;
+    static constexpr int kOffTmp = kOffR2 + 4 * kTileBytes;   // three 16 x 16 fp32 blocks
+    static constexpr int kOffMisc = kOffTmp + 3 * 1024;       // beta[64], reduction scratch, tmem slot, barriers
     static constexpr int kBytes = kOffMisc + 1024 + 1024;     // + alignment slack
 };
 
 constexpr int kPrepThreads = 256;
 
-__global__ void __launch_bounds__(kPrepThreads, 2) kda_tc_prep_kernel(const KdaTcParams p) {
+__device__ __forceinline__ float rcp_approx(float x) {
+    float y;
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* m, uint32_t src, int c0, int c1) {
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+                 ::"l"(reinterpret_cast<uint64_t>(m)), "r"(src), "r"(c0), "r"(c1)
+                 : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read_all() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+
+struct PrepMaps {
+    CUtensorMap w0_h, w0_l, qt_h, qt_l, m_h, m_l, u0;     // workspace arrays (stores)
+    CUtensorMap q, k, v, alpha;                            // inputs (loads): (channel, head, row)
+};
+
+// The (block, head) item `item` of the wave: its request's geometry and the block's place in it.
+struct PrepItem {
+    int gb, head, blk, t_lo, t_hi;
+    int64_t row_t0;
+};
+__device__ __forceinline__ PrepItem prep_item(const KdaTcParams& p, int item) {
+    PrepItem it;
+    const int H = p.num_heads, R = p.num_requests;
+    it.gb = item / H;
+    it.head = item - it.gb * H;
+    int lo_r = 0, hi_r = R;                 // request: largest i with blk_off[i] <= gb (empty requests share offsets)
+    while (hi_r - lo_r > 1) {
+        const int mid = (lo_r + hi_r) >> 1;
+        if (p.blk_off[mid] <= it.gb) lo_r = mid; else hi_r = mid;
+    }
+    const ReqBlocks g = req_blocks(p, lo_r);
+    it.blk = g.first_block + (it.gb - p.blk_off[lo_r]);
+    it.t_lo = max(0, g.P - it.blk * kL);                                    // active tokens [t_lo, t_hi)
+    it.t_hi = min(kL, g.P + g.C - it.blk * kL);
+    it.row_t0 = g.row0 + ((int64_t)it.blk * kL - g.P);                      // row of token 0 (may be < 0)
+    return it;
+}
+
+__global__ void __launch_bounds__(kPrepThreads, 2)
+kda_tc_prep_kernel(const __grid_constant__ PrepMaps maps, const KdaTcParams p) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* sm = smem_raw + (base - smem_u32(smem_raw));
-    float* G = reinterpret_cast<float*>(sm + PrepSmem::kOffR0);
-    uint8_t* r0 = sm + PrepSmem::kOffR0;
-    uint8_t* r1 = sm + PrepSmem::kOffR1;
     uint8_t* r2 = sm + PrepSmem::kOffR2;
+    float* Tmp = reinterpret_cast<float*>(sm + PrepSmem::kOffTmp);
     float* s_beta = reinterpret_cast<float*>(sm + PrepSmem::kOffMisc);              // [64]
     float* s_red = reinterpret_cast<float*>(sm + PrepSmem::kOffMisc + 256);         // [8]
     int* s_redi = reinterpret_cast<int*>(sm + PrepSmem::kOffMisc + 320);            // [4]
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(sm + PrepSmem::kOffMisc + 512);
     volatile uint32_t* abort_flag = tmem_slot + 1;
-    const uint32_t bar = base + PrepSmem::kOffMisc + 528;
-    const uint32_t a0 = base + PrepSmem::kOffR0, a1 = base + PrepSmem::kOffR1, a2 = base + PrepSmem::kOffR2;
+    const uint32_t bar = base + PrepSmem::kOffMisc + 528;           // MMA completions (two per item)
+    const uint32_t bAlpha = bar + 8, bKQ = bar + 16, bV = bar + 24; // input arrivals (one each per item)
+    const uint32_t a0 = base + PrepSmem::kOffRA, a2 = base + PrepSmem::kOffR2;
+    constexpr int kSlab = PrepSmem::kSlab;
+    // element (t, c) of the decay products; row t of the triangular matrix
+    auto Gp = [&](int t, int c) -> float* {
+        return reinterpret_cast<float*>(sm + (c >> 5) * kSlab + kTileBytes + t * 128 + ((((c & 31) >> 2) ^ (t & 7)) << 4) +
+                                        (c & 3) * 4);
+    };
+    auto Arow = [&](int t) -> float* {
+        return reinterpret_cast<float*>(sm + (t >> 5) * kSlab + kTileBytes + (t & 31) * 256);
+    };
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int head = blockIdx.y, H = p.num_heads, R = p.num_requests;
-    const int gb = blockIdx.x;
-    if (gb >= p.blk_off[R]) return;
-    int lo_r = 0, hi_r = R;                 // request: largest i with blk_off[i] <= gb (empty requests share offsets)
-    while (hi_r - lo_r > 1) {
-        const int mid = (lo_r + hi_r) >> 1;
-        if (p.blk_off[mid] <= gb) lo_r = mid; else hi_r = mid;
-    }
-    const int req = lo_r;
-    const ReqBlocks g = req_blocks(p, req);
-    const int blk = g.first_block + (gb - p.blk_off[req]);
-    const int t_lo = max(0, g.P - blk * kL), t_hi = min(kL, g.P + g.C - blk * kL);     // active tokens [t_lo, t_hi)
-    const int64_t row_t0 = g.row0 + ((int64_t)blk * kL - g.P);                         // row of token 0 (may be < 0)
-    const size_t bh = (size_t)gb * H + head;
+    const int H = p.num_heads;
+    const int n_items = p.blk_off[p.num_requests] * H;
+    if ((int)blockIdx.x >= n_items) return;
     const size_t tile_elems = (size_t)kL * kD;
+
+    // alpha into the slots and the raw keys and queries into the Kt tiles of the item `it`
+    auto request_alpha = [&](const PrepItem& it) {
+        mbar_arrive_expect_tx(bAlpha, 4 * kTileBytes);
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+            tma_load_3d(a0 + j * kSlab + kTileBytes, &maps.alpha, bAlpha, 64 * j, it.head, (int)it.row_t0);
+    };
+    auto request_kq = [&](const PrepItem& it) {
+        mbar_arrive_expect_tx(bKQ, 4 * kTileBytes);
+#pragma unroll
+        for (int kh = 0; kh < 2; ++kh) {
+            tma_load_3d(a0 + kh * kSlab, &maps.k, bKQ, 64 * kh, it.head, (int)it.row_t0);
+            tma_load_3d(a0 + (2 + kh) * kSlab, &maps.q, bKQ, 64 * kh, it.head, (int)it.row_t0);
+        }
+    };
 
     if (tid == 0) {
         mbar_init(bar, 1);
+        mbar_init(bAlpha, 1);
+        mbar_init(bKQ, 1);
+        mbar_init(bV, 1);
         *abort_flag = 0u;
         fence_barrier_init();
+        const PrepItem first = prep_item(p, (int)blockIdx.x);
+        request_alpha(first);
+        request_kq(first);
     }
     if (warp == 0) {
         tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), 256);
         tmem_relinquish();
     }
-    // ---- alpha and beta of the block (inactive tokens: alpha 1, beta 0)
-    auto load_alpha = [&]() {
-#pragma unroll
-        for (int it = 0; it < 8; ++it) {
-            const int item = it * kPrepThreads + tid, t = item >> 5, c4 = (item & 31) * 4;
-            float4 a = make_float4(1.f, 1.f, 1.f, 1.f);
-            if (t >= t_lo && t < t_hi) a = *reinterpret_cast<const float4*>(p.alpha + ((row_t0 + t) * H + head) * kD + c4);
-            *reinterpret_cast<float4*>(G + t * kD + c4) = a;
-        }
-    };
-    load_alpha();
-    if (tid < kL) s_beta[tid] = (tid >= t_lo && tid < t_hi) ? p.beta[(row_t0 + tid) * H + head] : 0.f;
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
+    bool ok = true;
+    uint32_t in_phase = 0;
 
-    // ---- cuts and decay products.  A sub-block starts at the first active token and after every token that completes
-    //      a periodic snapshot position; with those cuts alone the decay products (from each sub-block's start, the
-    //      start's own alpha excluded) are formed by two threads per channel, one per half of the block, the second
-    //      half picking up the first half's last value.  Only if some product fell below 2^-40 are the extra cuts
-    //      found, one at a time, by the slow path below.
-    uint64_t mask = 1ull << t_lo;
-    if (p.snap_interval > 0) {
-        for (int t = t_lo; t + 1 < t_hi; ++t)
-            if (((int64_t)blk * kL + t + 1) % p.snap_interval == 0) mask |= 1ull << (t + 1);
-    }
-    const int ch = tid & 127, half = tid >> 7;
-    float gmin = 1.f;
-    {
-        float gacc = 1.f;
-        const int tb = half * 32;
-#pragma unroll 8
-        for (int t = tb; t < tb + 32; ++t) {
-            const bool active = t >= t_lo && t < t_hi;
-            gacc = (!active || ((mask >> t) & 1ull)) ? 1.f : gacc * G[t * kD + ch];
-            G[t * kD + ch] = gacc;
+    PrepItem cur = prep_item(p, (int)blockIdx.x);
+    // beta of the block (inactive tokens: 0); the later items' are fetched an item ahead
+    if (tid < kL) s_beta[tid] = (tid >= cur.t_lo && tid < cur.t_hi) ? p.beta[(cur.row_t0 + tid) * H + cur.head] : 0.f;
+    for (int item = (int)blockIdx.x;;) {
+        const int head = cur.head, blk = cur.blk, t_lo = cur.t_lo, t_hi = cur.t_hi;
+        const int64_t row_t0 = cur.row_t0;
+        const size_t bh = (size_t)cur.gb * H + head;
+        const int row_ws = (int)(bh * kL);                         // the item's first row in the workspace arrays
+
+        // ---- cuts and decay products.  A sub-block starts at the first active token and after every token that
+        //      completes a periodic snapshot position; with those cuts alone the decay products (from each sub-block's
+        //      start, the start's own alpha excluded) are formed by two threads per channel, one per half of the block,
+        //      the second half picking up the first half's last value.  Only if some product fell below 2^-40 are the
+        //      extra cuts found, one at a time, by the slow path below.
+        uint64_t mask = 1ull << t_lo;
+        if (p.snap_interval > 0) {
+            for (int t = t_lo; t + 1 < t_hi; ++t)
+                if (((int64_t)blk * kL + t + 1) % p.snap_interval == 0) mask |= 1ull << (t + 1);
         }
-    }
-    __syncthreads();
-    if (half == 1) {
-        // tokens 32.. up to the first cut in this half continue the first half's product
-        const uint64_t cuts = mask >> 32;
-        const int n_carry = cuts ? (__ffsll((long long)cuts) - 1) : 32;
-        const float carry = (31 >= t_lo && 31 < t_hi) ? G[31 * kD + ch] : 1.f;
-        for (int t = 32; t < 32 + n_carry; ++t)
-            if (t >= t_lo && t < t_hi) G[t * kD + ch] *= carry;
-    }
-    __syncthreads();
-    {
-        const int tb = half * 32;
+        ok = __syncthreads_and(mbar_wait(bAlpha, in_phase, abort_flag));
+        if (!ok) break;
+        const int ch = tid & 127, half = tid >> 7;
+        float gmin = 1.f;
+        {
+            float gacc = 1.f;
+            const int tb = half * 32;
 #pragma unroll 8
-        for (int t = tb; t < tb + 32; ++t) gmin = fminf(gmin, G[t * kD + ch]);
+            for (int t = tb; t < tb + 32; ++t) {
+                const bool active = t >= t_lo && t < t_hi;
+                float* gp = Gp(t, ch);
+                gacc = (!active || ((mask >> t) & 1ull)) ? 1.f : gacc * *gp;
+                *gp = gacc;
+            }
+        }
+        __syncthreads();
+        if (half == 1) {
+            // tokens 32.. up to the first cut in this half continue the first half's product
+            const uint64_t cuts = mask >> 32;
+            const int n_carry = cuts ? (__ffsll((long long)cuts) - 1) : 32;
+            const float carry = (31 >= t_lo && 31 < t_hi) ? *Gp(31, ch) : 1.f;
+            for (int t = 32; t < 32 + n_carry; ++t)
+                if (t >= t_lo && t < t_hi) *Gp(t, ch) *= carry;
+        }
+        __syncthreads();
+        {
+            const int tb = half * 32;
+#pragma unroll 8
+            for (int t = tb; t < tb + 32; ++t) gmin = fminf(gmin, *Gp(t, ch));
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) gmin = fminf(gmin, __shfl_xor_sync(0xffffffffu, gmin, o));
-        if (lane == 0) s_red[warp] = gmin;
-        __syncthreads();
-        gmin = fminf(fminf(fminf(s_red[0], s_red[1]), fminf(s_red[2], s_red[3])),
-                     fminf(fminf(s_red[4], s_red[5]), fminf(s_red[6], s_red[7])));
-    }
-    if (!(gmin >= kMinGamma)) {
-        // ---- slow path (rare): some channel decays below 2^-40 inside a sub-block.  The token that causes it starts a
-        //      new sub-block; thread c < 128 follows channel c, the cuts are found one at a time.
-        __syncthreads();
-        load_alpha();
-        __syncthreads();
-        for (int round = 0; round < kL; ++round) {
-            int first_bad = kL;
+            for (int o = 16; o > 0; o >>= 1) gmin = fminf(gmin, __shfl_xor_sync(0xffffffffu, gmin, o));
+            if (lane == 0) s_red[warp] = gmin;
+            __syncthreads();
+            gmin = fminf(fminf(fminf(s_red[0], s_red[1]), fminf(s_red[2], s_red[3])),
+                         fminf(fminf(s_red[4], s_red[5]), fminf(s_red[6], s_red[7])));
+        }
+        if (!(gmin >= kMinGamma)) {
+            // ---- slow path (rare): some channel decays below 2^-40 inside a sub-block.  The token that causes it starts
+            //      a new sub-block; thread c < 128 follows channel c, the cuts are found one at a time.
+            __syncthreads();
+            for (int i = tid; i < kL * (kD / 4); i += kPrepThreads) {
+                const int t = i >> 5, c4 = (i & 31) * 4;
+                float4 a = make_float4(1.f, 1.f, 1.f, 1.f);
+                if (t >= t_lo && t < t_hi) a = *reinterpret_cast<const float4*>(p.alpha + ((row_t0 + t) * H + head) * kD + c4);
+                *reinterpret_cast<float4*>(Gp(t, c4)) = a;
+            }
+            __syncthreads();
+            for (int round = 0; round < kL; ++round) {
+                int first_bad = kL;
+                if (tid < 128) {
+                    float gacc = 1.f;
+                    for (int t = t_lo + 1; t < t_hi; ++t) {
+                        if ((mask >> t) & 1ull) { gacc = 1.f; continue; }
+                        gacc *= *Gp(t, tid);
+                        if (!(gacc >= kMinGamma)) { first_bad = t; break; }
+                    }
+#pragma unroll
+                    for (int o = 16; o > 0; o >>= 1) first_bad = min(first_bad, __shfl_xor_sync(0xffffffffu, first_bad, o));
+                    if (lane == 0) s_redi[warp] = first_bad;
+                }
+                __syncthreads();
+                first_bad = min(min(s_redi[0], s_redi[1]), min(s_redi[2], s_redi[3]));
+                __syncthreads();
+                if (first_bad >= kL) break;
+                mask |= 1ull << first_bad;
+            }
             if (tid < 128) {
                 float gacc = 1.f;
-                for (int t = t_lo + 1; t < t_hi; ++t) {
-                    if ((mask >> t) & 1ull) { gacc = 1.f; continue; }
-                    gacc *= G[t * kD + tid];
-                    if (!(gacc >= kMinGamma)) { first_bad = t; break; }
+                for (int t = 0; t < kL; ++t) {
+                    if (t < t_lo || t >= t_hi) { *Gp(t, tid) = 1.f; continue; }
+                    gacc = ((mask >> t) & 1ull) ? 1.f : gacc * *Gp(t, tid);
+                    *Gp(t, tid) = gacc;
                 }
-#pragma unroll
-                for (int o = 16; o > 0; o >>= 1) first_bad = min(first_bad, __shfl_xor_sync(0xffffffffu, first_bad, o));
-                if (lane == 0) s_redi[warp] = first_bad;
             }
             __syncthreads();
-            first_bad = min(min(s_redi[0], s_redi[1]), min(s_redi[2], s_redi[3]));
-            __syncthreads();
-            if (first_bad >= kL) break;
-            mask |= 1ull << first_bad;
         }
+        // the last row of every sub-block goes to the workspace (the chain scales the state by it)
         if (tid < 128) {
-            float gacc = 1.f;
-            for (int t = 0; t < kL; ++t) {
-                if (t < t_lo || t >= t_hi) { G[t * kD + tid] = 1.f; continue; }
-                gacc = ((mask >> t) & 1ull) ? 1.f : gacc * G[t * kD + tid];
-                G[t * kD + tid] = gacc;
+            int a = t_lo;
+            while (a < t_hi) {
+                const int e = sub_end(mask, a, t_hi);
+                p.ws_e[(bh * kL + e - 1) * kD + tid] = *Gp(e - 1, tid);
+                a = e;
             }
         }
+        if (tid == 0) p.ws_mask[bh] = mask;
+
+        // ---- Kt = k G, Kh = k / G, Kb = Kh G_end, Qt = q G as hi/lo bf16.  Kt and Kh go to shared memory (MMA operands),
+        //      Kb to the workspace; Qt waits in registers for the slots the decay products occupy.  A thread handles 8
+        //      consecutive channels of a token at a time; the raw keys and queries sit where its Kt terms go.
+        ok = __syncthreads_and(mbar_wait(bKQ, in_phase, abort_flag));
+        if (!ok) break;
+        uint4 qt_h[4], qt_l[4];
+#pragma unroll
+        for (int it = 0; it < 4; ++it) {
+            const int idx = it * kPrepThreads + tid, t = idx >> 4, c8 = idx & 15, c0 = c8 * 8;
+            const bool active = t >= t_lo && t < t_hi;
+            const uint32_t sw = sw_off(t, c8 & 7);
+            const int kh = c8 >> 3;
+            uint4 kt_h = make_uint4(0, 0, 0, 0), kt_l = kt_h, kh_h = kt_h, kh_l = kt_h, kb_h = kt_h, kb_l = kt_h;
+            qt_h[it] = kt_h; qt_l[it] = kt_h;
+            if (active) {
+                const int e_t = sub_end(mask, t, t_hi) - 1;
+                const uint4 kraw = *reinterpret_cast<const uint4*>(sm + kh * kSlab + sw);
+                const uint4 qraw = *reinterpret_cast<const uint4*>(sm + (2 + kh) * kSlab + sw);
+                const uint32_t rw[4] = {kraw.x, kraw.y, kraw.z, kraw.w}, rq[4] = {qraw.x, qraw.y, qraw.z, qraw.w};
+                const float4 g0 = *reinterpret_cast<const float4*>(Gp(t, c0)), g1 = *reinterpret_cast<const float4*>(Gp(t, c0 + 4));
+                const float4 e0 = *reinterpret_cast<const float4*>(Gp(e_t, c0)), e1 = *reinterpret_cast<const float4*>(Gp(e_t, c0 + 4));
+                const float gg[8] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w};
+                const float ee[8] = {e0.x, e0.y, e0.z, e0.w, e1.x, e1.y, e1.z, e1.w};
+                uint32_t o[8][4];
+#pragma unroll
+                for (int w = 0; w < 4; ++w) {
+                    const float k0 = __uint_as_float(rw[w] << 16), k1 = __uint_as_float(rw[w] & 0xffff0000u);
+                    const float q0 = __uint_as_float(rq[w] << 16), q1 = __uint_as_float(rq[w] & 0xffff0000u);
+                    const float i0 = rcp_approx(gg[2 * w]), i1 = rcp_approx(gg[2 * w + 1]);      // g >= 2^-40: finite
+                    const float h0 = k0 * i0, h1 = k1 * i1;
+                    split2(k0 * gg[2 * w], k1 * gg[2 * w + 1], o[0][w], o[1][w]);
+                    split2(h0, h1, o[2][w], o[3][w]);
+                    split2(h0 * ee[2 * w], h1 * ee[2 * w + 1], o[4][w], o[5][w]);
+                    split2(q0 * gg[2 * w], q1 * gg[2 * w + 1], o[6][w], o[7][w]);
+                }
+                kt_h = make_uint4(o[0][0], o[0][1], o[0][2], o[0][3]); kt_l = make_uint4(o[1][0], o[1][1], o[1][2], o[1][3]);
+                kh_h = make_uint4(o[2][0], o[2][1], o[2][2], o[2][3]); kh_l = make_uint4(o[3][0], o[3][1], o[3][2], o[3][3]);
+                kb_h = make_uint4(o[4][0], o[4][1], o[4][2], o[4][3]); kb_l = make_uint4(o[5][0], o[5][1], o[5][2], o[5][3]);
+                qt_h[it] = make_uint4(o[6][0], o[6][1], o[6][2], o[6][3]); qt_l[it] = make_uint4(o[7][0], o[7][1], o[7][2], o[7][3]);
+            }
+            *reinterpret_cast<uint4*>(sm + kh * kSlab + sw) = kt_h;
+            *reinterpret_cast<uint4*>(sm + (2 + kh) * kSlab + sw) = kt_l;
+            *reinterpret_cast<uint4*>(r2 + kh * kTileBytes + sw) = kh_h;
+            *reinterpret_cast<uint4*>(r2 + (2 + kh) * kTileBytes + sw) = kh_l;
+            const size_t go = bh * tile_elems + (size_t)t * kD + c0;
+            *reinterpret_cast<uint4*>(p.ws_kb_h + go) = kb_h;
+            *reinterpret_cast<uint4*>(p.ws_kb_l + go) = kb_l;
+        }
+        __syncthreads();                   // every read of the decay products is done: Qt takes their place
+#pragma unroll
+        for (int it = 0; it < 4; ++it) {
+            const int idx = it * kPrepThreads + tid, t = idx >> 4, c8 = idx & 15;
+            const uint32_t off = (uint32_t)((c8 >> 3) * kSlab + kTileBytes) + sw_off(t, c8 & 7);
+            *reinterpret_cast<uint4*>(sm + off) = qt_h[it];
+            *reinterpret_cast<uint4*>(sm + 2 * kSlab + off) = qt_l[it];
+        }
+        fence_proxy_async_smem();
         __syncthreads();
-    }
-    // the last row of every sub-block goes to the workspace (the chain scales the state by it)
-    if (tid < 128) {
-        int a = t_lo;
-        while (a < t_hi) {
-            const int e = sub_end(mask, a, t_hi);
-            p.ws_e[(bh * kL + e - 1) * kD + tid] = G[(e - 1) * kD + tid];
-            a = e;
-        }
-    }
-    if (tid == 0) p.ws_mask[bh] = mask;
 
-    // ---- Kt = k G, Kh = k / G, Kb = Kh G_end, Qt = q G as hi/lo bf16.  Kt and Kh go to shared memory (MMA operands), Kb
-    //      and Qt to the workspace; Qt also waits in registers for the region the decay products occupy.  A thread handles
-    //      8 consecutive channels of a token at a time.
-    uint4 qt_h[4], qt_l[4];
-#pragma unroll
-    for (int it = 0; it < 4; ++it) {
-        const int item = it * kPrepThreads + tid, t = item >> 4, c8 = item & 15, c0 = c8 * 8;
-        const bool active = t >= t_lo && t < t_hi;
-        uint4 kt_h = make_uint4(0, 0, 0, 0), kt_l = kt_h, kh_h = kt_h, kh_l = kt_h, kb_h = kt_h, kb_l = kt_h;
-        qt_h[it] = kt_h; qt_l[it] = kt_h;
-        if (active) {
-            const uint4 raw = *reinterpret_cast<const uint4*>(p.k + ((row_t0 + t) * H + head) * kD + c0);
-            const uint4 rawq = *reinterpret_cast<const uint4*>(p.q + ((row_t0 + t) * H + head) * kD + c0);
-            const int e_t = sub_end(mask, t, t_hi) - 1;
-            const uint32_t rw[4] = {raw.x, raw.y, raw.z, raw.w}, rq[4] = {rawq.x, rawq.y, rawq.z, rawq.w};
-            uint32_t o[8][4];
-#pragma unroll
-            for (int w = 0; w < 4; ++w) {
-                const float k0 = __uint_as_float(rw[w] << 16), k1 = __uint_as_float(rw[w] & 0xffff0000u);
-                const float q0 = __uint_as_float(rq[w] << 16), q1 = __uint_as_float(rq[w] & 0xffff0000u);
-                const float2 gg = *reinterpret_cast<const float2*>(G + t * kD + c0 + 2 * w);
-                const float2 ee = *reinterpret_cast<const float2*>(G + e_t * kD + c0 + 2 * w);
-                const float i0 = __frcp_rn(gg.x), i1 = __frcp_rn(gg.y);       // g >= 2^-40: finite
-                split2(k0 * gg.x, k1 * gg.y, o[0][w], o[1][w]);
-                split2(k0 * i0, k1 * i1, o[2][w], o[3][w]);
-                split2(k0 * (ee.x * i0), k1 * (ee.y * i1), o[4][w], o[5][w]);
-                split2(q0 * gg.x, q1 * gg.y, o[6][w], o[7][w]);
-            }
-            kt_h = make_uint4(o[0][0], o[0][1], o[0][2], o[0][3]); kt_l = make_uint4(o[1][0], o[1][1], o[1][2], o[1][3]);
-            kh_h = make_uint4(o[2][0], o[2][1], o[2][2], o[2][3]); kh_l = make_uint4(o[3][0], o[3][1], o[3][2], o[3][3]);
-            kb_h = make_uint4(o[4][0], o[4][1], o[4][2], o[4][3]); kb_l = make_uint4(o[5][0], o[5][1], o[5][2], o[5][3]);
-            qt_h[it] = make_uint4(o[6][0], o[6][1], o[6][2], o[6][3]); qt_l[it] = make_uint4(o[7][0], o[7][1], o[7][2], o[7][3]);
-        }
-        const uint32_t off = (uint32_t)((c8 >> 3) * kTileBytes) + sw_off(t, c8 & 7);
-        *reinterpret_cast<uint4*>(r1 + off) = kt_h;
-        *reinterpret_cast<uint4*>(r1 + 2 * kTileBytes + off) = kt_l;
-        *reinterpret_cast<uint4*>(r2 + off) = kh_h;
-        *reinterpret_cast<uint4*>(r2 + 2 * kTileBytes + off) = kh_l;
-        const size_t go = bh * tile_elems + (size_t)t * kD + c0;
-        *reinterpret_cast<uint4*>(p.ws_kb_h + go) = kb_h;
-        *reinterpret_cast<uint4*>(p.ws_kb_l + go) = kb_l;
-        *reinterpret_cast<uint4*>(p.ws_qt_h + go) = qt_h[it];
-        *reinterpret_cast<uint4*>(p.ws_qt_l + go) = qt_l[it];
-    }
-    __syncthreads();                       // every read of the decay products is done: Qt takes their place
-#pragma unroll
-    for (int it = 0; it < 4; ++it) {
-        const int item = it * kPrepThreads + tid, t = item >> 4, c8 = item & 15;
-        const uint32_t off = (uint32_t)((c8 >> 3) * kTileBytes) + sw_off(t, c8 & 7);
-        *reinterpret_cast<uint4*>(r0 + off) = qt_h[it];
-        *reinterpret_cast<uint4*>(r0 + 2 * kTileBytes + off) = qt_l[it];
-    }
-    fence_proxy_async_smem();
-    __syncthreads();
-
-    // ---- Kt Kh^T -> columns [0, 64), Qt Kh^T -> columns [64, 128): (hi + lo)(hi + lo)^T without the lo x lo term
-    if (tid == 0) {
-        tc_fence_after();
-        constexpr uint32_t idesc = idesc_bf16(64, 0, 0);
-        const uint32_t aa_base[2] = {a1, a0};
-#pragma unroll
-        for (int prod = 0; prod < 2; ++prod) {
-            const uint32_t a_hi = aa_base[prod], a_lo = a_hi + 2 * kTileBytes, b_hi = a2, b_lo = a2 + 2 * kTileBytes;
+        // ---- [Kt; Qt] Kh^T -> columns [0, 64): lanes 0..63 carry Kt Kh^T, lanes 64..127 Qt Kh^T;
+        //      (hi + lo)(hi + lo)^T without the lo x lo term.  The Qt tiles leave for the workspace from where they are.
+        if (tid == 0) {
+            tc_fence_after();
+            constexpr uint32_t idesc = idesc_bf16(64, 0, 0);
+            const uint32_t a_hi = a0, a_lo = a0 + 2 * kSlab, b_hi = a2, b_lo = a2 + 2 * kTileBytes;
             const uint32_t aa[3] = {a_hi, a_hi, a_lo}, bb[3] = {b_hi, b_lo, b_hi};
 #pragma unroll
             for (int term = 0; term < 3; ++term) {
                 const uint64_t ad = smem_desc_sw128(aa[term], 16, 1024), bd = smem_desc_sw128(bb[term], 16, 1024);
 #pragma unroll
                 for (int kk = 0; kk < 8; ++kk) {
-                    const uint64_t off = (uint64_t)(((kk >> 2) * kTileBytes + (kk & 3) * 32) >> 4);
-                    mma_ss(tmem + prod * 64, ad + off, bd + off, idesc, (term | kk) ? 1u : 0u);
+                    const uint64_t offa = (uint64_t)(((kk >> 2) * kSlab + (kk & 3) * 32) >> 4);
+                    const uint64_t offb = (uint64_t)(((kk >> 2) * kTileBytes + (kk & 3) * 32) >> 4);
+                    mma_ss(tmem, ad + offa, bd + offb, idesc, (term | kk) ? 1u : 0u);
                 }
             }
+            mma_commit(bar);
+#pragma unroll
+            for (int kh = 0; kh < 2; ++kh) {
+                tma_store_2d(&maps.qt_h, a0 + kh * kSlab + kTileBytes, 64 * kh, row_ws);
+                tma_store_2d(&maps.qt_l, a0 + (2 + kh) * kSlab + kTileBytes, 64 * kh, row_ws);
+            }
+            bulk_commit();
+            bulk_wait_read_all();          // before the slots are written again
         }
-        mma_commit(bar);
-    }
-    // the block's values, on their way while the products run
-    uint4 vraw[4];
-#pragma unroll
-    for (int it = 0; it < 4; ++it) {
-        const int item = it * kPrepThreads + tid, t = item >> 4, c0 = (item & 15) * 8;
-        vraw[it] = make_uint4(0, 0, 0, 0);
-        if (t >= t_lo && t < t_hi) vraw[it] = *reinterpret_cast<const uint4*>(p.v + ((row_t0 + t) * H + head) * kD + c0);
-    }
-    bool ok = __syncthreads_and(mbar_wait(bar, 0, abort_flag));
-    tc_fence_after();
-
-    // ---- rows of the two products (token t = tensor-memory lane t): warps 0, 1 take Kt Kh^T, whose strictly lower part
-    //      within a sub-block, scaled by beta_t, is the triangular matrix (to shared memory, over the Kh tiles: both
-    //      products have completed); warps 4, 5 take M = tril(Qt Kh^T), which goes to the workspace.  The V tile goes behind
-    //      the triangular matrix.
-    float* Amat = reinterpret_cast<float*>(r2);          // [64][64] fp32
-    uint8_t* vtile = r2 + 2 * kTileBytes;                // two 64-column tiles, tokens as rows
-#pragma unroll
-    for (int it = 0; it < 4; ++it) {
-        const int item = it * kPrepThreads + tid, t = item >> 4, c8 = item & 15;
-        *reinterpret_cast<uint4*>(vtile + (c8 >> 3) * kTileBytes + sw_off(t, c8 & 7)) = vraw[it];
-    }
-    if ((warp & 3) < 2 && ok) {
-        const int t = (warp & 3) * 32 + lane;
-        const bool active = t >= t_lo && t < t_hi;
-        const int s0 = active ? sub_start(mask, t) : kL;    // columns [s0, t) (and t itself for M) count
-        const uint32_t lane_addr = tmem + ((uint32_t)((warp & 3) * 32) << 16);
-        float x[64];
-        if (warp < 4) {
-            const float bt = s_beta[t];
-            tmem_ld32(lane_addr, reinterpret_cast<uint32_t*>(x));
-            tmem_ld32(lane_addr + 32, reinterpret_cast<uint32_t*>(x) + 32);
-            tmem_wait_ld();
-#pragma unroll
-            for (int s4 = 0; s4 < 16; ++s4) {
-                float4 a;
-                a.x = (active && 4 * s4 + 0 >= s0 && 4 * s4 + 0 < t) ? bt * x[4 * s4 + 0] : 0.f;
-                a.y = (active && 4 * s4 + 1 >= s0 && 4 * s4 + 1 < t) ? bt * x[4 * s4 + 1] : 0.f;
-                a.z = (active && 4 * s4 + 2 >= s0 && 4 * s4 + 2 < t) ? bt * x[4 * s4 + 2] : 0.f;
-                a.w = (active && 4 * s4 + 3 >= s0 && 4 * s4 + 3 < t) ? bt * x[4 * s4 + 3] : 0.f;
-                *reinterpret_cast<float4*>(Amat + t * kL + 4 * s4) = a;
-            }
-        } else {
-            tmem_ld32(lane_addr + 64, reinterpret_cast<uint32_t*>(x));
-            tmem_ld32(lane_addr + 96, reinterpret_cast<uint32_t*>(x) + 32);
-            tmem_wait_ld();
-            __nv_bfloat16* mh = p.ws_m_h + (bh * kL + t) * kL;
-            __nv_bfloat16* ml = p.ws_m_l + (bh * kL + t) * kL;
-#pragma unroll
-            for (int i8 = 0; i8 < 8; ++i8) {
-                uint32_t oh[4], ol[4];
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const int s = i8 * 8 + 2 * i;
-                    const float m0 = (active && s >= s0 && s <= t) ? x[s] : 0.f;
-                    const float m1 = (active && s + 1 >= s0 && s + 1 <= t) ? x[s + 1] : 0.f;
-                    split2(m0, m1, oh[i], ol[i]);
-                }
-                *reinterpret_cast<uint4*>(mh + i8 * 8) = make_uint4(oh[0], oh[1], oh[2], oh[3]);
-                *reinterpret_cast<uint4*>(ml + i8 * 8) = make_uint4(ol[0], ol[1], ol[2], ol[3]);
-            }
-        }
-    }
-    tc_fence_before();
-    __syncthreads();
-    // ---- T = (I + A)^-1 diag(beta).  The unit lower triangular 64 x 64 matrix L = I + A is inverted in 16 x 16 blocks:
-    //      the four diagonal blocks by forward substitution (64 threads, one column each), then the blocks below the
-    //      diagonal, one block diagonal after the other, from X_ij = -X_ii sum_{j <= k < i} L_ik X_kj as small products
-    //      (one element of each 16 x 16 block per thread).  X lives behind the T tiles in R0; the sums are staged where
-    //      the T tiles will go.
-    float* Xm = reinterpret_cast<float*>(r0 + 2 * kTileBytes);        // [64][64] fp32
-    float* Tmp = reinterpret_cast<float*>(r0);                        // up to three 16 x 16 blocks
-    if (ok) {
-        for (int i = tid; i < kL * kL; i += kPrepThreads) Xm[i] = 0.f;
-        __syncthreads();
-        if (tid < kL) {
-            const int bi = tid >> 4, c = tid & 15;
-            float x[16];
-#pragma unroll
-            for (int r = 0; r < 16; ++r) {
-                float acc = (r == c) ? 1.f : 0.f;
-#pragma unroll
-                for (int q = 0; q < r; ++q) acc = fmaf(-Amat[(bi * 16 + r) * kL + bi * 16 + q], x[q], acc);
-                x[r] = acc;
-                Xm[(bi * 16 + r) * kL + bi * 16 + c] = acc;
-            }
-        }
-        __syncthreads();
-        // a thread owns a 1 x 4 patch of one block of the current diagonal: thread -> (block slot, row, 4 columns)
-        const int bs = tid >> 6, er = (tid >> 2) & 15, ec = (tid & 3) * 4;
-#pragma unroll 1
-        for (int d = 1; d < 4; ++d) {
-            const int i = d + bs, j = bs;                             // block (i, j = i - d), for bs < 4 - d
-            // sums S_ij = sum_k L_ik X_kj
-            if (i < 4) {
-                float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll 1
-                for (int k = j; k < i; ++k) {
-#pragma unroll
-                    for (int q4 = 0; q4 < 16; q4 += 4) {
-                        const float4 l = *reinterpret_cast<const float4*>(Amat + (i * 16 + er) * kL + k * 16 + q4);
-                        const float lq[4] = {l.x, l.y, l.z, l.w};
-#pragma unroll
-                        for (int q = 0; q < 4; ++q) {
-                            const float4 xv = *reinterpret_cast<const float4*>(Xm + (k * 16 + q4 + q) * kL + j * 16 + ec);
-                            acc.x = fmaf(lq[q], xv.x, acc.x); acc.y = fmaf(lq[q], xv.y, acc.y);
-                            acc.z = fmaf(lq[q], xv.z, acc.z); acc.w = fmaf(lq[q], xv.w, acc.w);
-                        }
-                    }
-                }
-                *reinterpret_cast<float4*>(Tmp + bs * 256 + er * 16 + ec) = acc;
-            }
-            __syncthreads();
-            if (i < 4) {
-                float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-                for (int q4 = 0; q4 < 16; q4 += 4) {
-                    const float4 x = *reinterpret_cast<const float4*>(Xm + (i * 16 + er) * kL + i * 16 + q4);
-                    const float xq[4] = {x.x, x.y, x.z, x.w};
-#pragma unroll
-                    for (int q = 0; q < 4; ++q) {
-                        const float4 tv = *reinterpret_cast<const float4*>(Tmp + bs * 256 + (q4 + q) * 16 + ec);
-                        acc.x = fmaf(xq[q], tv.x, acc.x); acc.y = fmaf(xq[q], tv.y, acc.y);
-                        acc.z = fmaf(xq[q], tv.z, acc.z); acc.w = fmaf(xq[q], tv.w, acc.w);
-                    }
-                }
-                *reinterpret_cast<float4*>(Xm + (i * 16 + er) * kL + j * 16 + ec) = make_float4(-acc.x, -acc.y, -acc.z, -acc.w);
-            }
-            __syncthreads();
-        }
-        // T[t][c] = X[t][c] beta_c as hi/lo operand tiles (hi at R0, lo behind it): thread -> (row, 16 columns)
-        {
-            const int t = tid >> 2, cb = (tid & 3) * 16;
-            uint4 th[2], tl[2];
-#pragma unroll
-            for (int j8 = 0; j8 < 2; ++j8) {
-                uint32_t oh[4], ol[4];
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const int c = cb + j8 * 8 + 2 * i;
-                    split2(Xm[t * kL + c] * s_beta[c], Xm[t * kL + c + 1] * s_beta[c + 1], oh[i], ol[i]);
-                }
-                th[j8] = make_uint4(oh[0], oh[1], oh[2], oh[3]);
-                tl[j8] = make_uint4(ol[0], ol[1], ol[2], ol[3]);
-            }
-            __syncthreads();               // the staging area is free: the tiles take its place
-#pragma unroll
-            for (int j8 = 0; j8 < 2; ++j8) {
-                const uint32_t off = sw_off(t, (cb >> 3) + j8);
-                *reinterpret_cast<uint4*>(r0 + off) = th[j8];
-                *reinterpret_cast<uint4*>(r0 + kTileBytes + off) = tl[j8];
-            }
-        }
-    }
-    fence_proxy_async_smem();
-    tc_fence_before();
-    __syncthreads();
-    // ---- W0 = T Kt -> columns [0, 128), U0 = T V -> columns [128, 256)   (V is bf16: it has no lo term)
-    if (tid == 0 && ok) {
+        ok = __syncthreads_and(mbar_wait(bar, 0, abort_flag));
+        if (!ok) break;
         tc_fence_after();
-        constexpr uint32_t idesc = idesc_bf16(128, 0, 1);
-        const uint32_t t_hi_a = a0, t_lo_a = a0 + kTileBytes;
-        const uint32_t kt_hi = a1, kt_lo = a1 + 2 * kTileBytes, v_a = a2 + 2 * kTileBytes;
-        const uint32_t aa[5] = {t_hi_a, t_hi_a, t_lo_a, t_hi_a, t_lo_a}, bb[5] = {kt_hi, kt_lo, kt_hi, v_a, v_a};
-#pragma unroll
-        for (int term = 0; term < 5; ++term) {
-            const uint64_t ad = smem_desc_sw128(aa[term], 16, 1024), bd = smem_desc_sw128(bb[term], kTileBytes, 1024);
-#pragma unroll
-            for (int kk = 0; kk < 4; ++kk)
-                mma_ss(tmem + (term >= 3 ? 128 : 0), ad + (uint64_t)(kk * 2), bd + (uint64_t)(kk * 128), idesc,
-                       ((term == 0 || term == 3) && kk == 0) ? 0u : 1u);
+        // the block's values into slots 2 and 3, on their way while the inverse is formed
+        if (tid == 0) {
+            mbar_arrive_expect_tx(bV, 2 * kTileBytes);
+            tma_load_3d(a0 + 2 * kSlab + kTileBytes, &maps.v, bV, 0, head, (int)row_t0);
+            tma_load_3d(a0 + 3 * kSlab + kTileBytes, &maps.v, bV, 64, head, (int)row_t0);
         }
-        mma_commit(bar);
-    }
-    ok = __syncthreads_and(ok && mbar_wait(bar, 1, abort_flag));
-    tc_fence_after();
-    // ---- rows of W0 (warps 0, 1: hi/lo bf16) and of U0 (warps 4, 5: fp32) to the workspace
-    if ((warp & 3) < 2 && ok) {
-        const int t = (warp & 3) * 32 + lane;
-        const uint32_t lane_addr = tmem + ((uint32_t)((warp & 3) * 32) << 16);
-        if (warp < 4) {
-            __nv_bfloat16* wh = p.ws_w0_h + bh * tile_elems + (size_t)t * kD;
-            __nv_bfloat16* wl = p.ws_w0_l + bh * tile_elems + (size_t)t * kD;
-#pragma unroll 1
-            for (int c0 = 0; c0 < kD; c0 += 32) {
-                float x[32];
-                tmem_ld32(lane_addr + c0, reinterpret_cast<uint32_t*>(x));
-                tmem_wait_ld();
+
+        // ---- rows of the two products.  Warps w with (w & 3) < 2 own lanes of Kt Kh^T, whose strictly lower part within
+        //      a sub-block, scaled by beta_t, is the triangular matrix (to slots 0 and 1); the others own lanes of
+        //      M = tril(Qt Kh^T), which goes to the workspace through staging tiles in R2 (the Kh tiles are spent).
+        //      Warps 0..3 take columns [0, 32), warps 4..7 columns [32, 64).
+        {
+            const int qd = warp & 3, cb = (warp >> 2) * 32;
+            const int t = (qd & 1) * 32 + lane;
+            const bool active = t >= t_lo && t < t_hi;
+            const int s0 = active ? sub_start(mask, t) : kL;    // columns [s0, t) (and t itself for M) count
+            float x[32];
+            tmem_ld32(tmem + ((uint32_t)(qd * 32) << 16) + cb, reinterpret_cast<uint32_t*>(x));
+            tmem_wait_ld();
+            if (qd < 2) {
+                const float bt = s_beta[t];
+                float* arow = Arow(t) + cb;
+#pragma unroll
+                for (int s4 = 0; s4 < 8; ++s4) {
+                    float4 a;
+                    a.x = (active && cb + 4 * s4 + 0 >= s0 && cb + 4 * s4 + 0 < t) ? bt * x[4 * s4 + 0] : 0.f;
+                    a.y = (active && cb + 4 * s4 + 1 >= s0 && cb + 4 * s4 + 1 < t) ? bt * x[4 * s4 + 1] : 0.f;
+                    a.z = (active && cb + 4 * s4 + 2 >= s0 && cb + 4 * s4 + 2 < t) ? bt * x[4 * s4 + 2] : 0.f;
+                    a.w = (active && cb + 4 * s4 + 3 >= s0 && cb + 4 * s4 + 3 < t) ? bt * x[4 * s4 + 3] : 0.f;
+                    *reinterpret_cast<float4*>(arow + 4 * s4) = a;
+                }
+            } else {
 #pragma unroll
                 for (int i8 = 0; i8 < 4; ++i8) {
                     uint32_t oh[4], ol[4];
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) split2(x[i8 * 8 + 2 * i], x[i8 * 8 + 2 * i + 1], oh[i], ol[i]);
-                    *reinterpret_cast<uint4*>(wh + c0 + i8 * 8) = make_uint4(oh[0], oh[1], oh[2], oh[3]);
-                    *reinterpret_cast<uint4*>(wl + c0 + i8 * 8) = make_uint4(ol[0], ol[1], ol[2], ol[3]);
+                    for (int i = 0; i < 4; ++i) {
+                        const int s = i8 * 8 + 2 * i;
+                        const float m0 = (active && cb + s >= s0 && cb + s <= t) ? x[s] : 0.f;
+                        const float m1 = (active && cb + s + 1 >= s0 && cb + s + 1 <= t) ? x[s + 1] : 0.f;
+                        split2(m0, m1, oh[i], ol[i]);
+                    }
+                    const uint32_t off = sw_off(t, (cb >> 3) + i8);
+                    *reinterpret_cast<uint4*>(r2 + off) = make_uint4(oh[0], oh[1], oh[2], oh[3]);
+                    *reinterpret_cast<uint4*>(r2 + kTileBytes + off) = make_uint4(ol[0], ol[1], ol[2], ol[3]);
                 }
             }
-        } else {
-            float* u0 = p.ws_u0 + bh * tile_elems + (size_t)t * kD;
-#pragma unroll 1
-            for (int c0 = 0; c0 < kD; c0 += 32) {
-                float x[32];
-                tmem_ld32(lane_addr + 128 + c0, reinterpret_cast<uint32_t*>(x));
-                tmem_wait_ld();
+        }
+        fence_proxy_async_smem();
+        tc_fence_before();
+        __syncthreads();
+        if (tid == 0) {
+            tma_store_2d(&maps.m_h, a2, 0, row_ws);
+            tma_store_2d(&maps.m_l, a2 + kTileBytes, 0, row_ws);
+            bulk_commit();
+        }
+        // ---- T = (I + A)^-1 diag(beta).  The unit lower triangular 64 x 64 matrix L = I + A is inverted in 16 x 16
+        //      blocks: the four diagonal blocks by forward substitution (64 threads, one column each), then the blocks
+        //      below the diagonal, one block diagonal after the other, from X_ij = -X_ii sum_{j <= k < i} L_ik X_kj as
+        //      small products (one 1 x 4 patch of a 16 x 16 block per thread).  X lives in the upper half of R2, where
+        //      (and over the staging tiles of M) the T tiles go afterwards.
+        float* Xm = reinterpret_cast<float*>(r2 + 2 * kTileBytes);        // [64][64] fp32
+        {
+            for (int i = tid; i < kL * kL; i += kPrepThreads) Xm[i] = 0.f;
+            __syncthreads();
+            if (tid < kL) {
+                const int bi = tid >> 4, c = tid & 15;
+                float x[16];
 #pragma unroll
-                for (int i4 = 0; i4 < 8; ++i4)
-                    *reinterpret_cast<float4*>(u0 + c0 + i4 * 4) = make_float4(x[4 * i4], x[4 * i4 + 1], x[4 * i4 + 2], x[4 * i4 + 3]);
+                for (int r = 0; r < 16; ++r) {
+                    float acc = (r == c) ? 1.f : 0.f;
+                    const float* arow = Arow(bi * 16 + r) + bi * 16;
+#pragma unroll
+                    for (int q = 0; q < r; ++q) acc = fmaf(-arow[q], x[q], acc);
+                    x[r] = acc;
+                    Xm[(bi * 16 + r) * kL + bi * 16 + c] = acc;
+                }
+            }
+            __syncthreads();
+            // a thread owns a 1 x 4 patch of one block of the current diagonal: thread -> (block slot, row, 4 columns)
+            const int bs = tid >> 6, er = (tid >> 2) & 15, ec = (tid & 3) * 4;
+#pragma unroll 1
+            for (int d = 1; d < 4; ++d) {
+                const int i = d + bs, j = bs;                             // block (i, j = i - d), for bs < 4 - d
+                // sums S_ij = sum_k L_ik X_kj
+                if (i < 4) {
+                    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+                    const float* arow = Arow(i * 16 + er);
+#pragma unroll 1
+                    for (int k = j; k < i; ++k) {
+#pragma unroll
+                        for (int q4 = 0; q4 < 16; q4 += 4) {
+                            const float4 l = *reinterpret_cast<const float4*>(arow + k * 16 + q4);
+                            const float lq[4] = {l.x, l.y, l.z, l.w};
+#pragma unroll
+                            for (int q = 0; q < 4; ++q) {
+                                const float4 xv = *reinterpret_cast<const float4*>(Xm + (k * 16 + q4 + q) * kL + j * 16 + ec);
+                                acc.x = fmaf(lq[q], xv.x, acc.x); acc.y = fmaf(lq[q], xv.y, acc.y);
+                                acc.z = fmaf(lq[q], xv.z, acc.z); acc.w = fmaf(lq[q], xv.w, acc.w);
+                            }
+                        }
+                    }
+                    *reinterpret_cast<float4*>(Tmp + bs * 256 + er * 16 + ec) = acc;
+                }
+                __syncthreads();
+                if (i < 4) {
+                    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                    for (int q4 = 0; q4 < 16; q4 += 4) {
+                        const float4 x = *reinterpret_cast<const float4*>(Xm + (i * 16 + er) * kL + i * 16 + q4);
+                        const float xq[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) {
+                            const float4 tv = *reinterpret_cast<const float4*>(Tmp + bs * 256 + (q4 + q) * 16 + ec);
+                            acc.x = fmaf(xq[q], tv.x, acc.x); acc.y = fmaf(xq[q], tv.y, acc.y);
+                            acc.z = fmaf(xq[q], tv.z, acc.z); acc.w = fmaf(xq[q], tv.w, acc.w);
+                        }
+                    }
+                    *reinterpret_cast<float4*>(Xm + (i * 16 + er) * kL + j * 16 + ec) = make_float4(-acc.x, -acc.y, -acc.z, -acc.w);
+                }
+                __syncthreads();
+            }
+            // T[t][c] = X[t][c] beta_c as hi/lo operand tiles, each stored twice: thread -> (row, 16 columns)
+            {
+                const int t = tid >> 2, cb = (tid & 3) * 16;
+                uint4 th[2], tl[2];
+#pragma unroll
+                for (int j8 = 0; j8 < 2; ++j8) {
+                    uint32_t oh[4], ol[4];
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const int c = cb + j8 * 8 + 2 * i;
+                        split2(Xm[t * kL + c] * s_beta[c], Xm[t * kL + c + 1] * s_beta[c + 1], oh[i], ol[i]);
+                    }
+                    th[j8] = make_uint4(oh[0], oh[1], oh[2], oh[3]);
+                    tl[j8] = make_uint4(ol[0], ol[1], ol[2], ol[3]);
+                }
+                if (tid == 0) bulk_wait_read_all();     // the staging tiles of M have been read
+                __syncthreads();                        // and so has the inverse: the tiles take their place
+#pragma unroll
+                for (int j8 = 0; j8 < 2; ++j8) {
+                    const uint32_t off = sw_off(t, (cb >> 3) + j8);
+                    *reinterpret_cast<uint4*>(r2 + off) = th[j8];
+                    *reinterpret_cast<uint4*>(r2 + kTileBytes + off) = th[j8];
+                    *reinterpret_cast<uint4*>(r2 + 2 * kTileBytes + off) = tl[j8];
+                    *reinterpret_cast<uint4*>(r2 + 3 * kTileBytes + off) = tl[j8];
+                }
             }
         }
+        // rows of V that belong to no token of this request (a block at either end of a chunk) are whatever lies
+        // next to the chunk in the array: they meet zero columns of T, but must be finite for that to give zero
+        if (t_lo > 0 || t_hi < kL) {
+            ok = __syncthreads_and(mbar_wait(bV, in_phase, abort_flag));
+            if (!ok) break;
+            for (int i = tid; i < kL * 16; i += kPrepThreads) {
+                const int t = i >> 4, c8 = i & 15;
+                if (t < t_lo || t >= t_hi)
+                    *reinterpret_cast<uint4*>(sm + (2 + (c8 >> 3)) * kSlab + kTileBytes + sw_off(t, c8 & 7)) = make_uint4(0, 0, 0, 0);
+            }
+        }
+        fence_proxy_async_smem();
+        tc_fence_before();
+        __syncthreads();
+        // ---- W0 = T Kt -> columns [0, 128), U0 = T V -> columns [128, 256)   (V is bf16: it has no lo term); lanes
+        //      64..127 repeat lanes 0..63
+        if (tid == 0) {
+            const bool okv = mbar_wait(bV, in_phase, abort_flag);
+            tc_fence_after();
+            constexpr uint32_t idesc = idesc_bf16(128, 0, 1);
+            const uint32_t t_hi_a = a2, t_lo_a = a2 + 2 * kTileBytes;
+            const uint32_t kt_hi = a0, kt_lo = a0 + 2 * kSlab, v_a = a0 + 2 * kSlab + kTileBytes;
+            const uint32_t aa[5] = {t_hi_a, t_hi_a, t_lo_a, t_hi_a, t_lo_a}, bb[5] = {kt_hi, kt_lo, kt_hi, v_a, v_a};
+            if (okv) {
+#pragma unroll
+                for (int term = 0; term < 5; ++term) {
+                    const uint64_t ad = smem_desc_sw128(aa[term], 16, 1024), bd = smem_desc_sw128(bb[term], kSlab, 1024);
+#pragma unroll
+                    for (int kk = 0; kk < 4; ++kk)
+                        mma_ss(tmem + (term >= 3 ? 128 : 0), ad + (uint64_t)(kk * 2), bd + (uint64_t)(kk * 128), idesc,
+                               ((term == 0 || term == 3) && kk == 0) ? 0u : 1u);
+                }
+            }
+            mma_commit(bar);
+        }
+        ok = __syncthreads_and(mbar_wait(bar, 1, abort_flag));
+        if (!ok) break;
+        tc_fence_after();
+        // the next item's alpha is requested as soon as the slots are free, and its beta fetched
+        const int next = item + (int)gridDim.x;
+        const bool more = next < n_items;
+        PrepItem nxt = cur;
+        float beta_next = 0.f;
+        if (more) {
+            nxt = prep_item(p, next);
+            if (tid == 0) request_alpha(nxt);
+            if (tid < kL && tid >= nxt.t_lo && tid < nxt.t_hi) beta_next = p.beta[(nxt.row_t0 + tid) * H + nxt.head];
+        }
+        // ---- rows of W0 (warps 0..3: hi/lo bf16, staged in R2) and of U0 (warps 4..7: fp32, staged in the Kt tiles); a
+        //      warp's lanes are tokens 32 (w & 1) + lane, and it takes columns [64 ((w & 3) >> 1), +64)
+        {
+            const int qd = warp & 3, t = (qd & 1) * 32 + lane, cbase = (qd >> 1) * 64;
+            const uint32_t lane_addr = tmem + ((uint32_t)(qd * 32) << 16) + (warp >= 4 ? 128 : 0) + cbase;
+            if (warp < 4) {
+                uint8_t* hi_tile = r2 + (cbase >> 6) * kTileBytes;            // khalf = cbase / 64
+                uint8_t* lo_tile = r2 + (2 + (cbase >> 6)) * kTileBytes;
+#pragma unroll 1
+                for (int c0 = 0; c0 < 64; c0 += 32) {
+                    float x[32];
+                    tmem_ld32(lane_addr + c0, reinterpret_cast<uint32_t*>(x));
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int i8 = 0; i8 < 4; ++i8) {
+                        uint32_t oh[4], ol[4];
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) split2(x[i8 * 8 + 2 * i], x[i8 * 8 + 2 * i + 1], oh[i], ol[i]);
+                        const uint32_t off = sw_off(t, (c0 >> 3) + i8);
+                        *reinterpret_cast<uint4*>(hi_tile + off) = make_uint4(oh[0], oh[1], oh[2], oh[3]);
+                        *reinterpret_cast<uint4*>(lo_tile + off) = make_uint4(ol[0], ol[1], ol[2], ol[3]);
+                    }
+                }
+            } else {
+#pragma unroll 1
+                for (int c0 = 0; c0 < 64; c0 += 32) {
+                    float x[32];
+                    tmem_ld32(lane_addr + c0, reinterpret_cast<uint32_t*>(x));
+                    tmem_wait_ld();
+                    uint8_t* tile = sm + ((cbase + c0) >> 5) * kSlab;         // 32 fp32 columns per tile
+#pragma unroll
+                    for (int i4 = 0; i4 < 8; ++i4)
+                        *reinterpret_cast<float4*>(tile + sw_off(t, i4)) = make_float4(x[4 * i4], x[4 * i4 + 1], x[4 * i4 + 2], x[4 * i4 + 3]);
+                }
+            }
+        }
+        if (tid < kL) s_beta[tid] = beta_next;
+        fence_proxy_async_smem();
+        tc_fence_before();
+        __syncthreads();
+        tc_fence_after();
+        if (tid == 0) {
+#pragma unroll
+            for (int kh = 0; kh < 2; ++kh) {
+                tma_store_2d(&maps.w0_h, a2 + kh * kTileBytes, 64 * kh, row_ws);
+                tma_store_2d(&maps.w0_l, a2 + (2 + kh) * kTileBytes, 64 * kh, row_ws);
+            }
+#pragma unroll
+            for (int j = 0; j < 4; ++j) tma_store_2d(&maps.u0, a0 + j * kSlab, 64 * j, row_ws);
+            bulk_commit();
+            bulk_wait_read_all();          // the Kt tiles and R2 are free again
+            if (more) request_kq(nxt);
+        }
+        if (!more) break;
+        cur = nxt;
+        item = next;
+        in_phase ^= 1u;
+    }
+    if (tid == 0) {
+        // a wait that gave up leaves copies in flight: give them time to land before the CTA's shared memory is released
+        if (!ok)
+            for (int i = 0; i < 200; ++i) __nanosleep(1000);
+        bulk_wait_all();
     }
     tc_fence_before();
     __syncthreads();
@@ -1049,7 +1191,8 @@ kda_tc_chain_kernel(const __grid_constant__ CUtensorMap tm_w0_h, const __grid_co
 }  // namespace kdatc
 }  // namespace wpp
 
-extern "C" int wpp_launch_kda_tc(const wpp::KdaTcParams* p, const CUtensorMap* maps, int max_blocks, void* stream) {
+extern "C" int wpp_launch_kda_tc(const wpp::KdaTcParams* p, const CUtensorMap* maps, int max_blocks, int num_sms,
+                                 void* stream) {
     using namespace wpp::kdatc;
     static bool attr_set[64] = {};
     int dev = 0;
@@ -1064,8 +1207,12 @@ extern "C" int wpp_launch_kda_tc(const wpp::KdaTcParams* p, const CUtensorMap* m
     cudaStream_t st = (cudaStream_t)stream;
     kda_tc_setup_kernel<<<1, 1024, 0, st>>>(*p);
     if (max_blocks > 0) {
-        dim3 grid_a((unsigned)max_blocks, (unsigned)p->num_heads);
-        kda_tc_prep_kernel<<<grid_a, kPrepThreads, PrepSmem::kBytes, st>>>(*p);
+        PrepMaps pm;
+        pm.w0_h = maps[0]; pm.w0_l = maps[1]; pm.qt_h = maps[2]; pm.qt_l = maps[3]; pm.m_h = maps[6]; pm.m_l = maps[7];
+        pm.u0 = maps[8]; pm.q = maps[9]; pm.k = maps[10]; pm.v = maps[11]; pm.alpha = maps[12];
+        const long long items = (long long)max_blocks * p->num_heads;
+        const unsigned grid_a = (unsigned)(items < 2ll * num_sms ? items : 2ll * num_sms);
+        kda_tc_prep_kernel<<<grid_a, kPrepThreads, PrepSmem::kBytes, st>>>(pm, *p);
     }
     dim3 grid_b((unsigned)p->num_heads, (unsigned)p->num_requests);
     kda_tc_chain_kernel<<<grid_b, 352, ChainSmem::kBytes, st>>>(maps[0], maps[1], maps[2], maps[3], maps[4], maps[5], maps[6],
