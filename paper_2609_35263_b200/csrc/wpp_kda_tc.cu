@@ -149,8 +149,8 @@ struct PrepSmem {
     static constexpr int kSlab = 2 * kTileBytes;
     static constexpr int kOffRA = 0;
     static constexpr int kOffR2 = kOffRA + 4 * kSlab;
-    static constexpr int kOffTmp = kOffR2 + 4 * kTileBytes;   // three 16 x 16 fp32 blocks
-    static constexpr int kOffMisc = kOffTmp + 3 * 1024;       // beta[64], reduction scratch, tmem slot, barriers
+    static constexpr int kOffTmp = kOffR2 + 4 * kTileBytes;   // a 32 x 32 fp32 block (products of the inverse)
+    static constexpr int kOffMisc = kOffTmp + 4 * 1024;       // beta[64], reduction scratch, tmem slot, barriers
     static constexpr int kBytes = kOffMisc + 1024 + 1024;     // + alignment slack
 };
 
@@ -219,8 +219,10 @@ kda_tc_prep_kernel(const __grid_constant__ PrepMaps maps, const KdaTcParams p) {
         return reinterpret_cast<float*>(sm + (c >> 5) * kSlab + kTileBytes + t * 128 + ((((c & 31) >> 2) ^ (t & 7)) << 4) +
                                         (c & 3) * 4);
     };
-    auto Arow = [&](int t) -> float* {
-        return reinterpret_cast<float*>(sm + (t >> 5) * kSlab + kTileBytes + (t & 31) * 256);
+    // (rows of 64 floats; the 16-byte chunks of a row are XOR-swizzled by the row so that a column walk across rows
+    // and row-per-lane stores spread over the banks); the inverse X is laid out the same way
+    auto Ap = [&](int t, int c) -> float* {
+        return reinterpret_cast<float*>(sm + (t >> 5) * kSlab + kTileBytes + (t & 31) * 256) + ((((c >> 2) ^ (t & 7)) << 2) | (c & 3));
     };
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -290,38 +292,68 @@ kda_tc_prep_kernel(const __grid_constant__ PrepMaps maps, const KdaTcParams p) {
         if (!ok) break;
         const int ch = tid & 127, half = tid >> 7;
         float gmin = 1.f;
-        {
-            float gacc = 1.f;
-            const int tb = half * 32;
+        if (mask == 1ull && t_hi == kL) {
+            // the usual block: all 64 tokens, no cut inside.  The second half forms its own products in registers while
+            // the first half runs, then scales them by the first half's last value.
+            if (half == 0) {
+                float gacc = 1.f;
+                *Gp(0, ch) = 1.f;
+#pragma unroll
+                for (int t = 1; t < 32; ++t) {
+                    float* gp = Gp(t, ch);
+                    gacc *= *gp;
+                    *gp = gacc;
+                    gmin = fminf(gmin, gacc);
+                }
+                named_bar(1, kPrepThreads);
+            } else {
+                float x[32];
+                x[0] = *Gp(32, ch);
+#pragma unroll
+                for (int i = 1; i < 32; ++i) x[i] = x[i - 1] * *Gp(32 + i, ch);
+                named_bar(1, kPrepThreads);
+                const float carry = *Gp(31, ch);
+#pragma unroll
+                for (int i = 0; i < 32; ++i) {
+                    x[i] *= carry;
+                    *Gp(32 + i, ch) = x[i];
+                    gmin = fminf(gmin, x[i]);
+                }
+            }
+        } else {
+            {
+                float gacc = 1.f;
+                const int tb = half * 32;
 #pragma unroll 8
-            for (int t = tb; t < tb + 32; ++t) {
-                const bool active = t >= t_lo && t < t_hi;
-                float* gp = Gp(t, ch);
-                gacc = (!active || ((mask >> t) & 1ull)) ? 1.f : gacc * *gp;
-                *gp = gacc;
+                for (int t = tb; t < tb + 32; ++t) {
+                    const bool active = t >= t_lo && t < t_hi;
+                    float* gp = Gp(t, ch);
+                    gacc = (!active || ((mask >> t) & 1ull)) ? 1.f : gacc * *gp;
+                    *gp = gacc;
+                }
+            }
+            __syncthreads();
+            if (half == 1) {
+                // tokens 32.. up to the first cut in this half continue the first half's product
+                const uint64_t cuts = mask >> 32;
+                const int n_carry = cuts ? (__ffsll((long long)cuts) - 1) : 32;
+                const float carry = (31 >= t_lo && 31 < t_hi) ? *Gp(31, ch) : 1.f;
+                for (int t = 32; t < 32 + n_carry; ++t)
+                    if (t >= t_lo && t < t_hi) *Gp(t, ch) *= carry;
+            }
+            __syncthreads();
+            {
+                const int tb = half * 32;
+#pragma unroll 8
+                for (int t = tb; t < tb + 32; ++t) gmin = fminf(gmin, *Gp(t, ch));
             }
         }
-        __syncthreads();
-        if (half == 1) {
-            // tokens 32.. up to the first cut in this half continue the first half's product
-            const uint64_t cuts = mask >> 32;
-            const int n_carry = cuts ? (__ffsll((long long)cuts) - 1) : 32;
-            const float carry = (31 >= t_lo && 31 < t_hi) ? *Gp(31, ch) : 1.f;
-            for (int t = 32; t < 32 + n_carry; ++t)
-                if (t >= t_lo && t < t_hi) *Gp(t, ch) *= carry;
-        }
-        __syncthreads();
-        {
-            const int tb = half * 32;
-#pragma unroll 8
-            for (int t = tb; t < tb + 32; ++t) gmin = fminf(gmin, *Gp(t, ch));
 #pragma unroll
-            for (int o = 16; o > 0; o >>= 1) gmin = fminf(gmin, __shfl_xor_sync(0xffffffffu, gmin, o));
-            if (lane == 0) s_red[warp] = gmin;
-            __syncthreads();
-            gmin = fminf(fminf(fminf(s_red[0], s_red[1]), fminf(s_red[2], s_red[3])),
-                         fminf(fminf(s_red[4], s_red[5]), fminf(s_red[6], s_red[7])));
-        }
+        for (int o = 16; o > 0; o >>= 1) gmin = fminf(gmin, __shfl_xor_sync(0xffffffffu, gmin, o));
+        if (lane == 0) s_red[warp] = gmin;
+        __syncthreads();
+        gmin = fminf(fminf(fminf(s_red[0], s_red[1]), fminf(s_red[2], s_red[3])),
+                     fminf(fminf(s_red[4], s_red[5]), fminf(s_red[6], s_red[7])));
         if (!(gmin >= kMinGamma)) {
             // ---- slow path (rare): some channel decays below 2^-40 inside a sub-block.  The token that causes it starts
             //      a new sub-block; thread c < 128 follows channel c, the cuts are found one at a time.
@@ -379,6 +411,8 @@ kda_tc_prep_kernel(const __grid_constant__ PrepMaps maps, const KdaTcParams p) {
         ok = __syncthreads_and(mbar_wait(bKQ, in_phase, abort_flag));
         if (!ok) break;
         uint4 qt_h[4], qt_l[4];
+        float ee[8];                       // the decay products at the end of the sub-block, for this thread's channels
+        int e_have = -1;
 #pragma unroll
         for (int it = 0; it < 4; ++it) {
             const int idx = it * kPrepThreads + tid, t = idx >> 4, c8 = idx & 15, c0 = c8 * 8;
@@ -393,9 +427,12 @@ kda_tc_prep_kernel(const __grid_constant__ PrepMaps maps, const KdaTcParams p) {
                 const uint4 qraw = *reinterpret_cast<const uint4*>(sm + (2 + kh) * kSlab + sw);
                 const uint32_t rw[4] = {kraw.x, kraw.y, kraw.z, kraw.w}, rq[4] = {qraw.x, qraw.y, qraw.z, qraw.w};
                 const float4 g0 = *reinterpret_cast<const float4*>(Gp(t, c0)), g1 = *reinterpret_cast<const float4*>(Gp(t, c0 + 4));
-                const float4 e0 = *reinterpret_cast<const float4*>(Gp(e_t, c0)), e1 = *reinterpret_cast<const float4*>(Gp(e_t, c0 + 4));
+                if (e_t != e_have) {
+                    const float4 e0 = *reinterpret_cast<const float4*>(Gp(e_t, c0)), e1 = *reinterpret_cast<const float4*>(Gp(e_t, c0 + 4));
+                    ee[0] = e0.x; ee[1] = e0.y; ee[2] = e0.z; ee[3] = e0.w; ee[4] = e1.x; ee[5] = e1.y; ee[6] = e1.z; ee[7] = e1.w;
+                    e_have = e_t;
+                }
                 const float gg[8] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w};
-                const float ee[8] = {e0.x, e0.y, e0.z, e0.w, e1.x, e1.y, e1.z, e1.w};
                 uint32_t o[8][4];
 #pragma unroll
                 for (int w = 0; w < 4; ++w) {
@@ -482,7 +519,6 @@ kda_tc_prep_kernel(const __grid_constant__ PrepMaps maps, const KdaTcParams p) {
             tmem_wait_ld();
             if (qd < 2) {
                 const float bt = s_beta[t];
-                float* arow = Arow(t) + cb;
 #pragma unroll
                 for (int s4 = 0; s4 < 8; ++s4) {
                     float4 a;
@@ -490,7 +526,7 @@ kda_tc_prep_kernel(const __grid_constant__ PrepMaps maps, const KdaTcParams p) {
                     a.y = (active && cb + 4 * s4 + 1 >= s0 && cb + 4 * s4 + 1 < t) ? bt * x[4 * s4 + 1] : 0.f;
                     a.z = (active && cb + 4 * s4 + 2 >= s0 && cb + 4 * s4 + 2 < t) ? bt * x[4 * s4 + 2] : 0.f;
                     a.w = (active && cb + 4 * s4 + 3 >= s0 && cb + 4 * s4 + 3 < t) ? bt * x[4 * s4 + 3] : 0.f;
-                    *reinterpret_cast<float4*>(arow + 4 * s4) = a;
+                    *reinterpret_cast<float4*>(Ap(t, cb + 4 * s4)) = a;
                 }
             } else {
 #pragma unroll
@@ -517,70 +553,96 @@ kda_tc_prep_kernel(const __grid_constant__ PrepMaps maps, const KdaTcParams p) {
             tma_store_2d(&maps.m_l, a2 + kTileBytes, 0, row_ws);
             bulk_commit();
         }
-        // ---- T = (I + A)^-1 diag(beta).  The unit lower triangular 64 x 64 matrix L = I + A is inverted in 16 x 16
-        //      blocks: the four diagonal blocks by forward substitution (64 threads, one column each), then the blocks
-        //      below the diagonal, one block diagonal after the other, from X_ij = -X_ii sum_{j <= k < i} L_ik X_kj as
-        //      small products (one 1 x 4 patch of a 16 x 16 block per thread).  X lives in the upper half of R2, where
-        //      (and over the staging tiles of M) the T tiles go afterwards.
-        float* Xm = reinterpret_cast<float*>(r2 + 2 * kTileBytes);        // [64][64] fp32
+        // ---- T = (I + A)^-1 diag(beta).  The unit lower triangular 64 x 64 matrix L = I + A is inverted by halving: the
+        //      four 16 x 16 diagonal blocks by forward substitution (64 threads, one column each, while the others zero
+        //      the blocks above the diagonal), then twice [[X11, 0], [-X22 L21 X11, X22]]: for the two 32 x 32 diagonal
+        //      blocks (16 x 16 products) and for the whole matrix (32 x 32 products), each as two small products with
+        //      every thread busy.  X lives in the upper half of R2, where (and over the staging tiles of M) the T
+        //      tiles go afterwards.
+        auto Xp = [&](int r, int c) -> float* {                           // [64][64] fp32
+            return reinterpret_cast<float*>(r2 + 2 * kTileBytes) + r * kL + ((((c >> 2) ^ (r & 7)) << 2) | (c & 3));
+        };
         {
-            for (int i = tid; i < kL * kL; i += kPrepThreads) Xm[i] = 0.f;
-            __syncthreads();
             if (tid < kL) {
                 const int bi = tid >> 4, c = tid & 15;
                 float x[16];
 #pragma unroll
                 for (int r = 0; r < 16; ++r) {
                     float acc = (r == c) ? 1.f : 0.f;
-                    const float* arow = Arow(bi * 16 + r) + bi * 16;
 #pragma unroll
-                    for (int q = 0; q < r; ++q) acc = fmaf(-arow[q], x[q], acc);
+                    for (int q = 0; q < r; ++q) acc = fmaf(-*Ap(bi * 16 + r, bi * 16 + q), x[q], acc);
                     x[r] = acc;
-                    Xm[(bi * 16 + r) * kL + bi * 16 + c] = acc;
+                    *Xp(bi * 16 + r, bi * 16 + c) = acc;
+                }
+            } else {
+                for (int i = tid - kL; i < 6 * 64; i += kPrepThreads - kL) {
+                    const int b = i >> 6, r = (i & 63) >> 2, c4 = (i & 3) * 4;      // blocks (0,1) (0,2) (0,3) (1,2) (1,3) (2,3)
+                    const int bi = b < 3 ? 0 : (b < 5 ? 1 : 2), bj = b < 3 ? b + 1 : (b < 5 ? b - 1 : 3);
+                    *reinterpret_cast<float4*>(Xp(bi * 16 + r, bj * 16 + c4)) = make_float4(0.f, 0.f, 0.f, 0.f);
                 }
             }
             __syncthreads();
-            // a thread owns a 1 x 4 patch of one block of the current diagonal: thread -> (block slot, row, 4 columns)
-            const int bs = tid >> 6, er = (tid >> 2) & 15, ec = (tid & 3) * 4;
-#pragma unroll 1
-            for (int d = 1; d < 4; ++d) {
-                const int i = d + bs, j = bs;                             // block (i, j = i - d), for bs < 4 - d
-                // sums S_ij = sum_k L_ik X_kj
-                if (i < 4) {
-                    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-                    const float* arow = Arow(i * 16 + er);
-#pragma unroll 1
-                    for (int k = j; k < i; ++k) {
+            {
+                // blocks (1, 0) and (3, 2): thread -> (which, row, 2 columns)
+                const int pr = tid >> 7, er = (tid >> 3) & 15, ec = (tid & 7) * 2;
+                const int i = 2 * pr + 1, j = 2 * pr;
+                float2 acc = make_float2(0.f, 0.f);
 #pragma unroll
-                        for (int q4 = 0; q4 < 16; q4 += 4) {
-                            const float4 l = *reinterpret_cast<const float4*>(arow + k * 16 + q4);
-                            const float lq[4] = {l.x, l.y, l.z, l.w};
+                for (int q4 = 0; q4 < 16; q4 += 4) {
+                    const float4 l = *reinterpret_cast<const float4*>(Ap(i * 16 + er, j * 16 + q4));
+                    const float lq[4] = {l.x, l.y, l.z, l.w};
 #pragma unroll
-                            for (int q = 0; q < 4; ++q) {
-                                const float4 xv = *reinterpret_cast<const float4*>(Xm + (k * 16 + q4 + q) * kL + j * 16 + ec);
-                                acc.x = fmaf(lq[q], xv.x, acc.x); acc.y = fmaf(lq[q], xv.y, acc.y);
-                                acc.z = fmaf(lq[q], xv.z, acc.z); acc.w = fmaf(lq[q], xv.w, acc.w);
-                            }
-                        }
+                    for (int q = 0; q < 4; ++q) {
+                        const float2 xv = *reinterpret_cast<const float2*>(Xp(j * 16 + q4 + q, j * 16 + ec));
+                        acc.x = fmaf(lq[q], xv.x, acc.x); acc.y = fmaf(lq[q], xv.y, acc.y);
                     }
-                    *reinterpret_cast<float4*>(Tmp + bs * 256 + er * 16 + ec) = acc;
                 }
+                *reinterpret_cast<float2*>(Tmp + pr * 256 + er * 16 + ec) = acc;
                 __syncthreads();
-                if (i < 4) {
-                    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+                acc = make_float2(0.f, 0.f);
 #pragma unroll
-                    for (int q4 = 0; q4 < 16; q4 += 4) {
-                        const float4 x = *reinterpret_cast<const float4*>(Xm + (i * 16 + er) * kL + i * 16 + q4);
-                        const float xq[4] = {x.x, x.y, x.z, x.w};
+                for (int q4 = 0; q4 < 16; q4 += 4) {
+                    const float4 x = *reinterpret_cast<const float4*>(Xp(i * 16 + er, i * 16 + q4));
+                    const float xq[4] = {x.x, x.y, x.z, x.w};
 #pragma unroll
-                        for (int q = 0; q < 4; ++q) {
-                            const float4 tv = *reinterpret_cast<const float4*>(Tmp + bs * 256 + (q4 + q) * 16 + ec);
-                            acc.x = fmaf(xq[q], tv.x, acc.x); acc.y = fmaf(xq[q], tv.y, acc.y);
-                            acc.z = fmaf(xq[q], tv.z, acc.z); acc.w = fmaf(xq[q], tv.w, acc.w);
-                        }
+                    for (int q = 0; q < 4; ++q) {
+                        const float2 tv = *reinterpret_cast<const float2*>(Tmp + pr * 256 + (q4 + q) * 16 + ec);
+                        acc.x = fmaf(xq[q], tv.x, acc.x); acc.y = fmaf(xq[q], tv.y, acc.y);
                     }
-                    *reinterpret_cast<float4*>(Xm + (i * 16 + er) * kL + j * 16 + ec) = make_float4(-acc.x, -acc.y, -acc.z, -acc.w);
                 }
+                *reinterpret_cast<float2*>(Xp(i * 16 + er, j * 16 + ec)) = make_float2(-acc.x, -acc.y);
+                __syncthreads();
+            }
+            {
+                // rows 32..63, columns 0..31: thread -> (row, 4 columns)
+                const int er = tid >> 3, ec = (tid & 7) * 4;
+                float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 2
+                for (int q4 = 0; q4 < 32; q4 += 4) {
+                    const float4 l = *reinterpret_cast<const float4*>(Ap(32 + er, q4));
+                    const float lq[4] = {l.x, l.y, l.z, l.w};
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        const float4 xv = *reinterpret_cast<const float4*>(Xp(q4 + q, ec));
+                        acc.x = fmaf(lq[q], xv.x, acc.x); acc.y = fmaf(lq[q], xv.y, acc.y);
+                        acc.z = fmaf(lq[q], xv.z, acc.z); acc.w = fmaf(lq[q], xv.w, acc.w);
+                    }
+                }
+                *reinterpret_cast<float4*>(Tmp + er * 32 + ec) = acc;
+                __syncthreads();
+                acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 2
+                for (int q4 = 0; q4 < 32; q4 += 4) {
+                    const float4 x = *reinterpret_cast<const float4*>(Xp(32 + er, 32 + q4));
+                    const float xq[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        const float4 tv = *reinterpret_cast<const float4*>(Tmp + (q4 + q) * 32 + ec);
+                        acc.x = fmaf(xq[q], tv.x, acc.x); acc.y = fmaf(xq[q], tv.y, acc.y);
+                        acc.z = fmaf(xq[q], tv.z, acc.z); acc.w = fmaf(xq[q], tv.w, acc.w);
+                    }
+                }
+                *reinterpret_cast<float4*>(Xp(32 + er, ec)) = make_float4(-acc.x, -acc.y, -acc.z, -acc.w);
                 __syncthreads();
             }
             // T[t][c] = X[t][c] beta_c as hi/lo operand tiles, each stored twice: thread -> (row, 16 columns)
@@ -591,9 +653,12 @@ kda_tc_prep_kernel(const __grid_constant__ PrepMaps maps, const KdaTcParams p) {
                 for (int j8 = 0; j8 < 2; ++j8) {
                     uint32_t oh[4], ol[4];
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        const int c = cb + j8 * 8 + 2 * i;
-                        split2(Xm[t * kL + c] * s_beta[c], Xm[t * kL + c + 1] * s_beta[c + 1], oh[i], ol[i]);
+                    for (int i = 0; i < 2; ++i) {
+                        const int c = cb + j8 * 8 + 4 * i;
+                        const float4 x = *reinterpret_cast<const float4*>(Xp(t, c));
+                        const float4 b = *reinterpret_cast<const float4*>(s_beta + c);
+                        split2(x.x * b.x, x.y * b.y, oh[2 * i], ol[2 * i]);
+                        split2(x.z * b.z, x.w * b.w, oh[2 * i + 1], ol[2 * i + 1]);
                     }
                     th[j8] = make_uint4(oh[0], oh[1], oh[2], oh[3]);
                     tl[j8] = make_uint4(ol[0], ol[1], ol[2], ol[3]);
