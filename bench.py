@@ -40,9 +40,9 @@ DRAM_SOURCE = ("estimate: 607.6 DRAM bytes per 128x128 key step (dram__bytes_rea
 # Recurrent layer: dram read + write bytes of one wpp_kda_chunk launch on the default wave (8 x 2,048 tokens, 32 heads)
 # / its 524,288 (token, head) pairs; other wave shapes scale with the pairs (the state traffic per request is small).
 KDA_DRAM_BYTES_PER_TOKEN_HEAD = 1571.3
-# Chunk-parallel form: (686.6 MB + 1160.2 MB) of the preparation kernel + (1233.3 MB + 137.7 MB) of the chain kernel on
+# Chunk-parallel form: (673.3 MB + 1156.4 MB) of the preparation kernel + (1233.3 MB + 137.7 MB) of the chain kernel on
 # the same wave / 524,288 pairs.
-KDA_TC_DRAM_BYTES_PER_TOKEN_HEAD = 6137.6
+KDA_TC_DRAM_BYTES_PER_TOKEN_HEAD = 6104.9
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 

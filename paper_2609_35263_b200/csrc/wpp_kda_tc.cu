@@ -614,16 +614,19 @@ kda_tc_prep_kernel(const __grid_constant__ PrepMaps maps, const KdaTcParams p) {
                 __syncthreads();
             }
             {
-                // rows 32..63, columns 0..31: thread -> (row, 4 columns)
+                // rows 32..63, columns 0..31: thread -> (row, 4 columns).  Eight steps at a time: the swizzle of the rows
+                // walked then folds into constants.
                 const int er = tid >> 3, ec = (tid & 7) * 4;
                 float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll 2
-                for (int q4 = 0; q4 < 32; q4 += 4) {
-                    const float4 l = *reinterpret_cast<const float4*>(Ap(32 + er, q4));
-                    const float lq[4] = {l.x, l.y, l.z, l.w};
+#pragma unroll 1
+                for (int k8 = 0; k8 < 32; k8 += 8) {
+                    const float4 l0 = *reinterpret_cast<const float4*>(Ap(32 + er, k8));
+                    const float4 l1 = *reinterpret_cast<const float4*>(Ap(32 + er, k8 + 4));
+                    const float lq[8] = {l0.x, l0.y, l0.z, l0.w, l1.x, l1.y, l1.z, l1.w};
+                    const float* xrow = reinterpret_cast<const float*>(r2 + 2 * kTileBytes) + k8 * kL + (ec & 3);
 #pragma unroll
-                    for (int q = 0; q < 4; ++q) {
-                        const float4 xv = *reinterpret_cast<const float4*>(Xp(q4 + q, ec));
+                    for (int q = 0; q < 8; ++q) {
+                        const float4 xv = *reinterpret_cast<const float4*>(xrow + q * kL + (((ec >> 2) ^ q) << 2));
                         acc.x = fmaf(lq[q], xv.x, acc.x); acc.y = fmaf(lq[q], xv.y, acc.y);
                         acc.z = fmaf(lq[q], xv.z, acc.z); acc.w = fmaf(lq[q], xv.w, acc.w);
                     }
@@ -631,13 +634,14 @@ kda_tc_prep_kernel(const __grid_constant__ PrepMaps maps, const KdaTcParams p) {
                 *reinterpret_cast<float4*>(Tmp + er * 32 + ec) = acc;
                 __syncthreads();
                 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll 2
-                for (int q4 = 0; q4 < 32; q4 += 4) {
-                    const float4 x = *reinterpret_cast<const float4*>(Xp(32 + er, 32 + q4));
-                    const float xq[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll 1
+                for (int k8 = 0; k8 < 32; k8 += 8) {
+                    const float4 x0 = *reinterpret_cast<const float4*>(Xp(32 + er, 32 + k8));
+                    const float4 x1 = *reinterpret_cast<const float4*>(Xp(32 + er, 32 + k8 + 4));
+                    const float xq[8] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w};
 #pragma unroll
-                    for (int q = 0; q < 4; ++q) {
-                        const float4 tv = *reinterpret_cast<const float4*>(Tmp + (q4 + q) * 32 + ec);
+                    for (int q = 0; q < 8; ++q) {
+                        const float4 tv = *reinterpret_cast<const float4*>(Tmp + (k8 + q) * 32 + ec);
                         acc.x = fmaf(xq[q], tv.x, acc.x); acc.y = fmaf(xq[q], tv.y, acc.y);
                         acc.z = fmaf(xq[q], tv.z, acc.z); acc.w = fmaf(xq[q], tv.w, acc.w);
                     }
