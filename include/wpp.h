@@ -101,7 +101,9 @@ typedef struct {
     int32_t tile_m;           /* query rows per work tile: 128 or 256 (default 256: two 128-row halves) */
     int32_t tile_n;           /* keys per inner step: 128 */
     int32_t force_kv_splits;  /* >= 2: split every tile's key range into this many parts (when it has that many
-                                 key steps); 1: never split; 0: library decides */
+                                 key steps); 1: never split; 0: library decides (all tiles when there are fewer of
+                                 them than CTAs; the tiles of a partly filled last round when the tiles are long and
+                                 the rounds few; wpp_plan_info.workspace_bytes says what the partials need) */
     int32_t max_ctas;         /* persistent CTAs to launch (default: SM count of the context, 148 without one) */
     int32_t order;            /* order in which the persistent CTAs take the tiles at run time.  0: stream order -
                                  tiles that read the same (request, KV head) pages are neighbours and so run at the

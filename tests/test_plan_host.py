@@ -194,6 +194,30 @@ def test_few_tiles_fall_back_to_128_row_tiles_and_split_keys():
     assert pl2["slots"] > 0 and len(pl2["units"]) > 100                          # long prefix, two tiles: split along keys
 
 
+def test_a_partly_filled_last_round_of_long_tiles_is_cut_along_the_keys():
+    """32 requests of 64 new tokens over a 32,768-token prefix, 64/8 heads: 512 tiles of 257 key steps per half on 148
+    CTAs are three full rounds and 68 tiles; those 68 are cut in two so that the last round takes half a tile's time.
+    Nothing is cut when the rounds divide evenly, when the tiles are short, or when the caller says 1 (never)."""
+    R, P, C = 32, 32768, 64
+    d = desc(R, 64, 8, 128, 64, 520, pages=20000)
+    pl = parse_plan(wpp.wpp_plan_tiles(None, d, [P] * R, [C] * R, opts=wpp.PlanOpts(0, 0, 0, 148), pin=False))
+    units = pl["units"]
+    whole = [u for u in units if u["split_slot"] < 0]
+    cut = [u for u in units if u["split_slot"] >= 0]
+    assert len(whole) == 512 - 68 and len(cut) == 2 * 68 and pl["slots"] == 2 * 68
+    assert all(u["split_slot"] >= 0 for u in units[len(whole):])              # the cut tiles are the last in the order
+    assert sorted(u["kv_end"] - u["kv_begin"] for u in cut[:2]) == [128, 129] and cut[0]["kv_end"] == cut[1]["kv_begin"]
+    assert sum(u["cost"] for u in units) == pl["key_steps"] == 512 * 2 * 257
+    finish = _greedy_finish_times([u["cost"] + 3 for u in units], 148)
+    assert max(finish) <= 3.6 * (514 + 3)                                      # against 4 rounds uncut
+    never = parse_plan(wpp.wpp_plan_tiles(None, d, [P] * R, [C] * R, opts=wpp.PlanOpts(0, 0, 1, 148), pin=False))
+    assert never["slots"] == 0 and len(never["units"]) == 512
+    even = parse_plan(wpp.wpp_plan_tiles(None, d, [P] * R, [C] * R, opts=wpp.PlanOpts(0, 0, 0, 128), pin=False))
+    assert even["slots"] == 0                                                  # 512 tiles on 128 CTAs: four full rounds
+    short = parse_plan(wpp.wpp_plan_tiles(None, d, [4096] * R, [C] * R, opts=wpp.PlanOpts(0, 0, 0, 148), pin=False))
+    assert short["slots"] == 0                                                 # 33 key steps per half: not worth a cut
+
+
 def _status(fn, *a, **k):
     try:
         fn(*a, **k)
