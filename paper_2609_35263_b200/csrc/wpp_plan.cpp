@@ -148,55 +148,70 @@ int wpp_plan_tiles(const wpp_ctx* ctx, const wpp_batch_desc* desc, const int32_t
     if (T > 0x7fffffff) return WPP_ERR_INVALID_ARG;
     if (plan_host_bytes < plan_bytes_bound(&d, &o, T)) return WPP_ERR_PLAN_MISMATCH;
 
-    // ---- base tiles in natural order (request, row block, head): the heads of one KV group and the row
-    //      blocks of one request stay next to each other, so tiles that run at the same time share K/V in L2.
-    struct Base { int32_t request, row0[2], rows[2], head[2], steps, pack; };
+    // ---- row blocks of every request.  A tile is a row block times the heads it takes (one head, or 2..16 heads of
+    //      one KV group for short blocks), so everything but the heads is worked out once per row block.
+    struct RowBlock {
+        int32_t request, r0, rows[2], row0_b, head_b, pack, per_tile, steps, end[2];   // head_b: second half's first head
+                                                                                        // minus the first's; end[h]: key steps half h can see
+        int32_t cost() const { return end[0] + end[1]; }                       // 128x128 steps over both halves
+    };
     const int G = Hq / d.num_kv_heads;
     auto steps_for = [](int64_t last_visible_plus1) { return (int32_t)((last_visible_plus1 + WPP_TILE_N - 1) / WPP_TILE_N); };
-    auto build_base = [&](int tile_m, std::vector<Base>& base) {
-        base.clear();
+    std::vector<RowBlock> rbs;
+    std::vector<int32_t> rb_first((size_t)R + 1);
+    auto build_rows = [&](int tile_m) -> int64_t {
+        rbs.clear();
+        int64_t n_tiles = 0;
         for (int i = 0; i < R; ++i) {
+            rb_first[(size_t)i] = (int32_t)rbs.size();
             const int64_t P = prefix_lens[i], C = chunk_lens[i];
             for (int64_t r0 = 0; r0 < C; r0 += tile_m) {
                 const int32_t rows = (int32_t)std::min<int64_t>(tile_m, C - r0);
+                RowBlock rb;
+                rb.request = i;
+                rb.r0 = (int32_t)r0;
+                rb.steps = steps_for(P + r0 + rows);
                 if (rows <= WPP_HALF_M) {
                     // short block: each half takes `pack` heads of one KV group over the same rows (pack is the
                     // largest power of two that divides the group size and leaves 128/pack >= rows tensor rows
                     // per head); with 256-row tiles the second half takes the next heads of the group
                     int pack = 1;
                     while (pack < 8 && G % (2 * pack) == 0 && WPP_HALF_M / (2 * pack) >= rows) pack *= 2;
-                    const int per_tile = (tile_m == 256 && G % (2 * pack) == 0) ? 2 * pack : pack;
-                    for (int h = 0; h < Hq; h += per_tile) {
-                        const int32_t rows_b = per_tile == 2 * pack ? rows : 0;
-                        base.push_back({i, {(int32_t)r0, (int32_t)r0}, {rows, rows_b}, {h, h + pack},
-                                        steps_for(P + r0 + rows), pack});
-                    }
+                    rb.pack = pack;
+                    rb.per_tile = (tile_m == 256 && G % (2 * pack) == 0) ? 2 * pack : pack;
+                    rb.rows[0] = rows;
+                    rb.rows[1] = rb.per_tile == 2 * pack ? rows : 0;
+                    rb.row0_b = (int32_t)r0;
+                    rb.head_b = pack;
+                    rb.end[0] = rb.steps;
+                    rb.end[1] = rb.rows[1] > 0 ? rb.steps : 0;
                 } else {
-                    const int32_t ra = WPP_HALF_M, rb = rows - ra;
-                    for (int h = 0; h < Hq; ++h)
-                        base.push_back({i, {(int32_t)r0, (int32_t)r0 + WPP_HALF_M}, {ra, rb}, {h, h},
-                                        steps_for(P + r0 + rows), 1});
+                    rb.pack = 1;
+                    rb.per_tile = 1;
+                    rb.rows[0] = WPP_HALF_M;
+                    rb.rows[1] = rows - WPP_HALF_M;
+                    rb.row0_b = (int32_t)r0 + WPP_HALF_M;
+                    rb.head_b = 0;
+                    rb.end[0] = steps_for(P + r0 + WPP_HALF_M);
+                    rb.end[1] = rb.steps;
                 }
+                n_tiles += Hq / rb.per_tile;
+                rbs.push_back(rb);
             }
         }
+        rb_first[(size_t)R] = (int32_t)rbs.size();
+        return n_tiles;
     };
-    std::vector<Base> base;
     int TM = o.tile_m;
-    build_base(TM, base);
-    if (auto_tile_m && TM == 256 && (int64_t)base.size() < o.max_ctas) {   // few tiles: prefer more, smaller ones
+    int64_t n_base = build_rows(TM);
+    if (auto_tile_m && TM == 256 && n_base < o.max_ctas) {   // few tiles: prefer more, smaller ones
         TM = 128;
-        build_base(TM, base);
+        n_base = build_rows(TM);
     }
-    const int64_t n_base = (int64_t)base.size();
-
+    if (n_base > 0x3fffffff) return WPP_ERR_INVALID_ARG;
     // cost of key steps [a, b) of a tile = 128x128 steps over its halves, each cut at its own causal end
-    auto half_end = [&](const Base& t, int h) -> int32_t {
-        return t.rows[h] > 0 ? steps_for((int64_t)prefix_lens[t.request] + t.row0[h] + t.rows[h]) : 0;
-    };
-    auto cost_of = [&](const Base& t, int32_t a, int32_t b) -> int32_t {
-        int32_t c = 0;
-        for (int h = 0; h < 2; ++h) c += std::max(0, std::min(b, half_end(t, h)) - a);
-        return c;
+    auto cost_of = [](const RowBlock& t, int32_t a, int32_t b) -> int32_t {
+        return std::max(0, std::min(b, t.end[0]) - a) + std::max(0, std::min(b, t.end[1]) - a);
     };
 
     // ---- order of execution.  The persistent CTAs take tiles in this order at run time (a counter in the
@@ -206,42 +221,35 @@ int wpp_plan_tiles(const wpp_ctx* ctx, const wpp_batch_desc* desc, const int32_t
     //      so a page comes from DRAM once and is then hit in L2 by the other tiles; a prefix shared by many
     //      requests stays L2-resident while its KV head is being worked on.
     //      order 1: longest tile first (best balance, no regard for which tiles run together).
-    std::vector<int32_t> order((size_t)n_base);
-    for (int64_t u = 0; u < n_base; ++u) order[(size_t)u] = (int32_t)u;
+    struct Tile { int32_t rb, head; };          // row block and first head
+    std::vector<Tile> tiles;
+    tiles.reserve((size_t)n_base);
     if (o.order == 1) {
-        std::stable_sort(order.begin(), order.end(), [&](int32_t a, int32_t b) {
-            return cost_of(base[(size_t)a], 0, base[(size_t)a].steps) > cost_of(base[(size_t)b], 0, base[(size_t)b].steps);
-        });
+        for (int32_t k = 0; k < (int32_t)rbs.size(); ++k)
+            for (int h = 0; h < Hq; h += rbs[(size_t)k].per_tile) tiles.push_back({k, h});
+        std::stable_sort(tiles.begin(), tiles.end(),
+                         [&](const Tile& a, const Tile& b) { return rbs[(size_t)a.rb].cost() > rbs[(size_t)b.rb].cost(); });
     } else {
         std::vector<int64_t> req_cost((size_t)std::max(R, 1), 0);
-        for (const Base& t : base) req_cost[(size_t)t.request] += cost_of(t, 0, t.steps);
-        std::vector<int32_t> req_rank((size_t)std::max(R, 1));
-        {
-            std::vector<int32_t> by_cost((size_t)R);
-            for (int i = 0; i < R; ++i) by_cost[(size_t)i] = i;
-            std::stable_sort(by_cost.begin(), by_cost.end(),
-                             [&](int32_t a, int32_t b) { return req_cost[(size_t)a] > req_cost[(size_t)b]; });
-            for (int i = 0; i < R; ++i) req_rank[(size_t)by_cost[(size_t)i]] = i;
-        }
-        std::stable_sort(order.begin(), order.end(), [&](int32_t a, int32_t b) {
-            const Base& ua = base[(size_t)a];
-            const Base& ub = base[(size_t)b];
-            const int ka = ua.head[0] / G, kb = ub.head[0] / G;
-            if (ka != kb) return ka < kb;
-            return req_rank[(size_t)ua.request] < req_rank[(size_t)ub.request];
-        });
+        for (const RowBlock& rb : rbs) req_cost[(size_t)rb.request] += (int64_t)rb.cost() * (Hq / rb.per_tile);
+        std::vector<int32_t> by_cost((size_t)R);
+        for (int i = 0; i < R; ++i) by_cost[(size_t)i] = i;
+        std::stable_sort(by_cost.begin(), by_cost.end(),
+                         [&](int32_t a, int32_t b) { return req_cost[(size_t)a] > req_cost[(size_t)b]; });
+        for (int kvh = 0; kvh < d.num_kv_heads; ++kvh)
+            for (int rank = 0; rank < R; ++rank) {
+                const int i = by_cost[(size_t)rank];
+                for (int32_t k = rb_first[(size_t)i]; k < rb_first[(size_t)i + 1]; ++k)
+                    for (int h = kvh * G; h < (kvh + 1) * G; h += rbs[(size_t)k].per_tile) tiles.push_back({k, h});
+            }
     }
 
     // ---- split decision: into how many key ranges each tile is cut (1 = not at all)
-    std::vector<int32_t> parts_of((size_t)n_base, 1);
-    if (o.force_kv_splits >= 2) {
-        for (int64_t k = 0; k < n_base; ++k)
-            parts_of[(size_t)k] = std::max(1, std::min(o.force_kv_splits, base[(size_t)k].steps));
-    } else if (o.force_kv_splits == 0 && n_base > 0 && n_base < o.max_ctas) {
-        // fewer tiles than CTAs: every tile is cut so that all CTAs have work (>= 2 steps per part)
-        const int32_t want = (int32_t)((o.max_ctas + n_base - 1) / n_base);
-        for (int64_t k = 0; k < n_base; ++k)
-            parts_of[(size_t)k] = std::max(1, std::min(want, base[(size_t)k].steps / 2));
+    int32_t few_want = 0;          // fewer tiles than CTAs: every tile is cut so that all CTAs have work (>= 2 steps per part)
+    int64_t tail = 0;              // tiles of a partly filled last round ...
+    int32_t tail_parts = 1;        // ... and the number of key ranges each of them is cut into
+    if (o.force_kv_splits == 0 && n_base > 0 && n_base < o.max_ctas) {
+        few_want = (int32_t)((o.max_ctas + n_base - 1) / n_base);
     } else if (o.force_kv_splits == 0 && n_base % o.max_ctas != 0 && n_base < kTailSplitMaxRounds * (int64_t)o.max_ctas) {
         // A few rounds of long tiles: the last, partly filled round leaves CTAs idle for a whole tile.  Cutting the
         // tiles of that round into p key ranges each fills it.  The candidates are compared on a model of the run
@@ -249,94 +257,114 @@ int wpp_plan_tiles(const wpp_ctx* ctx, const wpp_batch_desc* desc, const int32_t
         // and end, a part a little more, the combine pass a constant).  The model flatters the cut: SMs of a partly
         // filled round run faster than those of a full one (more of the power budget and of L2 each), so that a
         // modelled gain of 12 % measured as 5-6 % and one of 8 % as a small loss; a cut is made from 10 % up.
-        const int64_t tail = n_base % o.max_ctas;
+        const int64_t n_tail = n_base % o.max_ctas;
         int32_t min_steps = 0x7fffffff;
-        for (int64_t k = n_base - tail; k < n_base; ++k) min_steps = std::min(min_steps, base[(size_t)order[(size_t)k]].steps);
-        using MinHeap = std::priority_queue<int64_t, std::vector<int64_t>, std::greater<int64_t>>;
-        MinHeap before_tail;                 // when each CTA is free once the full rounds have been handed out
-        for (int c = 0; c < o.max_ctas; ++c) before_tail.push(0);
-        int64_t end_before = 0;
-        for (int64_t k = 0; k < n_base - tail; ++k) {
-            const Base& t = base[(size_t)order[(size_t)k]];
-            const int64_t done = before_tail.top() + cost_of(t, 0, t.steps) + kTileFixedCost;
-            before_tail.pop();
-            before_tail.push(done);
-            end_before = std::max(end_before, done);
-        }
-        auto makespan = [&](int32_t p) -> int64_t {
-            MinHeap free_at = before_tail;
-            int64_t end = end_before;
-            for (int64_t k = n_base - tail; k < n_base; ++k) {
-                const Base& t = base[(size_t)order[(size_t)k]];
-                for (int32_t q = 0; q < p; ++q) {
-                    const int32_t a = (int32_t)((int64_t)t.steps * q / p), b = (int32_t)((int64_t)t.steps * (q + 1) / p);
-                    const int64_t done = free_at.top() + cost_of(t, a, b) + kTileFixedCost + (p > 1 ? kPartExtraCost : 0);
-                    free_at.pop();
-                    free_at.push(done);
-                    end = std::max(end, done);
-                }
+        for (int64_t k = n_base - n_tail; k < n_base; ++k) min_steps = std::min(min_steps, rbs[(size_t)tiles[(size_t)k].rb].steps);
+        if (min_steps >= 2 * kTailSplitMinSteps) {
+            using MinHeap = std::priority_queue<int64_t, std::vector<int64_t>, std::greater<int64_t>>;
+            MinHeap before_tail;                 // when each CTA is free once the full rounds have been handed out
+            for (int c = 0; c < o.max_ctas; ++c) before_tail.push(0);
+            int64_t end_before = 0;
+            for (int64_t k = 0; k < n_base - n_tail; ++k) {
+                const int64_t done = before_tail.top() + rbs[(size_t)tiles[(size_t)k].rb].cost() + kTileFixedCost;
+                before_tail.pop();
+                before_tail.push(done);
+                end_before = std::max(end_before, done);
             }
-            return end + (p > 1 ? kCombineCost : 0);
-        };
-        const int64_t whole = makespan(1);
-        int64_t best = whole;
-        int32_t best_p = 1;
-        for (int32_t p = 2; p <= kTailSplitMaxParts && min_steps >= p * kTailSplitMinSteps; ++p) {
-            const int64_t m = makespan(p);
-            if (m < best) { best = m; best_p = p; }
+            auto makespan = [&](int32_t p) -> int64_t {
+                MinHeap free_at = before_tail;
+                int64_t end = end_before;
+                for (int64_t k = n_base - n_tail; k < n_base; ++k) {
+                    const RowBlock& t = rbs[(size_t)tiles[(size_t)k].rb];
+                    for (int32_t q = 0; q < p; ++q) {
+                        const int32_t a = (int32_t)((int64_t)t.steps * q / p), b = (int32_t)((int64_t)t.steps * (q + 1) / p);
+                        const int64_t done = free_at.top() + cost_of(t, a, b) + kTileFixedCost + (p > 1 ? kPartExtraCost : 0);
+                        free_at.pop();
+                        free_at.push(done);
+                        end = std::max(end, done);
+                    }
+                }
+                return end + (p > 1 ? kCombineCost : 0);
+            };
+            const int64_t whole = makespan(1);
+            int64_t best = whole;
+            for (int32_t p = 2; p <= kTailSplitMaxParts && min_steps >= p * kTailSplitMinSteps; ++p) {
+                const int64_t m = makespan(p);
+                if (m < best) { best = m; tail_parts = p; }
+            }
+            if (tail_parts > 1 && best * 100 <= whole * (100 - kTailSplitMinGainPct)) tail = n_tail;
+            else tail_parts = 1;
         }
-        if (best_p > 1 && best * 100 <= whole * (100 - kTailSplitMinGainPct))
-            for (int64_t k = n_base - tail; k < n_base; ++k) parts_of[(size_t)order[(size_t)k]] = best_p;
     }
 
-    std::vector<WppUnit> units;
+    // ---- the plan: header, row offsets, the spans the plan is made for, units, combine records
+    WppPlanHeader hd;
+    std::memset(&hd, 0, sizeof(hd));
+    size_t off = sizeof(WppPlanHeader);
+    hd.off_q_offsets = (uint32_t)off;
+    off += align_up(sizeof(int32_t) * (size_t)(R + 1), 16);
+    hd.off_prefix = (uint32_t)off;
+    off += align_up(sizeof(int32_t) * (size_t)(R + 1), 16);
+    hd.off_units = (uint32_t)off;
+    char* p = static_cast<char*>(plan_host);
+    std::memset(p, 0, off);
+    const int64_t unit_cap = ((int64_t)plan_host_bytes - (int64_t)off) / (int64_t)sizeof(WppUnit);
+    WppUnit* us = reinterpret_cast<WppUnit*>(p + hd.off_units);
     std::vector<WppCombine> combines;
-    units.reserve((size_t)n_base);
     int32_t slots = 0;
-    int64_t key_steps = 0, n_split_units = 0;
+    int64_t n_units = 0, key_steps = 0, n_split_units = 0, nonempty_halves = 0;
     for (int64_t k = 0; k < n_base; ++k) {
-        const Base& t = base[(size_t)order[(size_t)k]];
-        const int32_t parts = parts_of[(size_t)order[(size_t)k]];
+        const RowBlock& t = rbs[(size_t)tiles[(size_t)k].rb];
+        const int32_t h = tiles[(size_t)k].head;
+        int32_t parts = 1;
+        if (o.force_kv_splits >= 2) parts = std::max(1, std::min(o.force_kv_splits, t.steps));
+        else if (few_want > 1) parts = std::max(1, std::min(few_want, t.steps / 2));
+        else if (k >= n_base - tail) parts = tail_parts;
+        if (n_units + parts > unit_cap) return WPP_ERR_PLAN_MISMATCH;
         WppUnit u;
-        std::memset(&u, 0, sizeof(u));
         u.request = t.request;
-        for (int h = 0; h < 2; ++h) { u.row0[h] = t.row0[h]; u.rows[h] = t.rows[h]; u.head[h] = t.head[h]; }
+        u.row0[0] = t.r0; u.row0[1] = t.row0_b;
+        u.rows[0] = t.rows[0]; u.rows[1] = t.rows[1];
+        u.head[0] = h; u.head[1] = h + t.head_b;
         u.pack = t.pack;
+        nonempty_halves += (int64_t)parts * ((t.rows[0] > 0) + (t.rows[1] > 0));
         if (parts == 1) {
-            u.kv_begin = 0; u.kv_end = t.steps; u.split_slot = -1; u.cost = cost_of(t, 0, t.steps);
-            units.push_back(u);
+            u.kv_begin = 0; u.kv_end = t.steps; u.split_slot = -1; u.cost = t.cost();
+            us[n_units++] = u;
             key_steps += u.cost;
         } else {
-            for (int h = 0; h < 2; ++h)
-                for (int kk = 0; kk < t.pack && t.rows[h] > 0; ++kk)
-                    combines.push_back({t.request, t.row0[h], t.rows[h], t.head[h] + kk, slots, parts, h,
+            for (int hf = 0; hf < 2; ++hf)
+                for (int kk = 0; kk < t.pack && t.rows[hf] > 0; ++kk)
+                    combines.push_back({t.request, u.row0[hf], t.rows[hf], u.head[hf] + kk, slots, parts, hf,
                                         kk * (WPP_HALF_M / t.pack)});
-            for (int32_t p = 0; p < parts; ++p) {
-                u.kv_begin = (int32_t)((int64_t)t.steps * p / parts);
-                u.kv_end = (int32_t)((int64_t)t.steps * (p + 1) / parts);
-                u.split_slot = slots + p;
+            for (int32_t q = 0; q < parts; ++q) {
+                u.kv_begin = (int32_t)((int64_t)t.steps * q / parts);
+                u.kv_end = (int32_t)((int64_t)t.steps * (q + 1) / parts);
+                u.split_slot = slots + q;
                 u.cost = cost_of(t, u.kv_begin, u.kv_end);
-                units.push_back(u);
+                us[n_units++] = u;
                 key_steps += u.cost;
                 ++n_split_units;
             }
             slots += parts;
         }
     }
-    const int64_t n_units = (int64_t)units.size();
     if (n_units > 0x3fffffff) return WPP_ERR_INVALID_ARG;
     // ---- kernel shape: short tiles (few key steps per half) go to the small CTAs, two per SM, where the start and end of
     //      one tile hide under the other CTA's steps; long tiles to the SM-wide CTA whose two halves overlap each other
-    int64_t nonempty_halves = 0;
-    for (const WppUnit& u : units)
-        for (int h = 0; h < 2; ++h) nonempty_halves += u.rows[h] > 0;
     int shape = o.shape;
     if (shape == 0) shape = (key_steps <= WPP_SMALL_SHAPE_MAX_STEPS * nonempty_halves) ? 2 : 1;
     const int num_ctas = shape == 2 ? (int)std::max<int64_t>(1, std::min<int64_t>(2 * (int64_t)o.max_ctas, 2 * n_units))
                                     : (int)std::max<int64_t>(1, std::min<int64_t>(o.max_ctas, n_units));
-    // ---- serialise
-    WppPlanHeader hd;
-    std::memset(&hd, 0, sizeof(hd));
+    off += sizeof(WppUnit) * (size_t)n_units;
+    hd.off_combine = (uint32_t)off;
+    off += sizeof(WppCombine) * combines.size();
+    hd.plan_bytes = align_up(off, 16);
+    if (hd.plan_bytes > plan_host_bytes) return WPP_ERR_PLAN_MISMATCH;
+    if (!combines.empty())
+        std::memcpy(p + hd.off_combine, combines.data(), sizeof(WppCombine) * combines.size());
+    std::memset(p + off, 0, hd.plan_bytes - off);
+
     hd.magic = WPP_PLAN_MAGIC;
     hd.version = WPP_PLAN_VERSION;
     hd.desc_hash = wpp_desc_hash(&d);
@@ -354,30 +382,12 @@ int wpp_plan_tiles(const wpp_ctx* ctx, const wpp_batch_desc* desc, const int32_t
     hd.key_steps = key_steps;
     hd.flops = 4 * (int64_t)d.head_dim * Hq * pairs;
     hd.workspace_bytes = WPP_WS_HEADER_BYTES + align_up((size_t)slots * 2 * WPP_HALF_M * (d.head_dim + 1) * sizeof(float), 256);
-    size_t off = sizeof(WppPlanHeader);
-    hd.off_q_offsets = (uint32_t)off;
-    off += align_up(sizeof(int32_t) * (size_t)(R + 1), 16);
-    hd.off_prefix = (uint32_t)off;
-    off += align_up(sizeof(int32_t) * (size_t)(R + 1), 16);
-    hd.off_units = (uint32_t)off;
-    off += sizeof(WppUnit) * (size_t)n_units;
-    hd.off_combine = (uint32_t)off;
-    off += sizeof(WppCombine) * combines.size();
-    hd.plan_bytes = align_up(off, 16);
-    if (hd.plan_bytes > plan_host_bytes) return WPP_ERR_PLAN_MISMATCH;
-
-    char* p = static_cast<char*>(plan_host);
-    std::memset(p, 0, hd.plan_bytes);
     std::memcpy(p, &hd, sizeof(hd));
     int32_t* qo = reinterpret_cast<int32_t*>(p + hd.off_q_offsets);
     qo[0] = 0;
     for (int i = 0; i < R; ++i) qo[i + 1] = qo[i] + chunk_lens[i];
     int32_t* pp = reinterpret_cast<int32_t*>(p + hd.off_prefix);
     for (int i = 0; i < R; ++i) pp[i] = prefix_lens[i];
-    WppUnit* us = reinterpret_cast<WppUnit*>(p + hd.off_units);
-    for (int64_t k = 0; k < n_units; ++k) us[k] = units[(size_t)k];
-    if (!combines.empty())
-        std::memcpy(p + hd.off_combine, combines.data(), sizeof(WppCombine) * combines.size());
 
     info->num_tiles = n_units;
     info->num_split_tiles = n_split_units;
