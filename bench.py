@@ -713,7 +713,8 @@ def main():
         ms_step = statistics.mean(a0.elapsed_time(b) for _, b, a0, _ in attn_events)
     ms_step = max_over_ranks(ms_step)
     attn_ms = statistics.mean(a.elapsed_time(b) for a, b, _, _ in attn_events)
-    phases = {"plan_host_ms": 1e3 * statistics.mean(t for _, _, _, t in attn_events),
+    phases = {"plan_host_ms": 1e3 * statistics.median(t for _, _, _, t in attn_events),
+              "plan_host_ms_max": 1e3 * max(t for _, _, _, t in attn_events),
               "append_ms": statistics.mean(a0.elapsed_time(a) for a, _, a0, _ in attn_events),
               "attention_ms": attn_ms,
               "note": "the host plans the next wave while the GPU runs the current one; append and attention are "
