@@ -116,6 +116,15 @@ def test_forced_kv_splits_and_combine(splits, tile_m):
     assert res["plan"].info.num_combine_tiles > 0 and res["plan"].info.workspace_bytes > 0
 
 
+def test_tail_round_cut_along_the_keys_by_the_planner():
+    """Eight long tiles on six CTAs: the planner cuts the two tiles of the second round in three (nobody asked for
+    splits: six parts fill the six CTAs); partials and the combine pass must give the same rows as whole tiles."""
+    w = W.custom_workload([16000, 16100, 15900, 16200], [64, 64, 64, 64], 4, 2, 128, 64, seed=31, spare_pages=4)
+    res, _ = _full_parity(w, opts=wpp.PlanOpts(0, 0, 0, 6))
+    info = res["plan"].info
+    assert info.num_tiles == 6 + 2 * 3 and info.num_split_tiles == 6 and info.workspace_bytes > 256
+
+
 def test_explicit_scale():
     w = W.custom_workload([70], [150], 2, 1, 128, 64, seed=10)
     _full_parity(w, sm_scale=0.05)
