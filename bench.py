@@ -44,6 +44,7 @@ KDA_DRAM_BYTES_PER_TOKEN_HEAD = 1571.3
 # the same wave / 524,288 pairs.
 KDA_TC_DRAM_BYTES_PER_TOKEN_HEAD = 6104.9
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+NOMINAL_BF16_TFLOPS = 2250.0        # dense bf16 of the data sheet (context only: no kernel reaches it under the power cap)
 
 
 def load_peaks():
@@ -130,6 +131,42 @@ def measure_other_config(name, ctx, dev, peaks, steps=3, warmup=3):
 
 
 OTHER_CONFIGS = ("cfg2", "cfg4_alt", "cfg5_C256_P0", "cfg5_C1024_P4096", "cfg5_C4096_P32768")
+
+
+def measure_yardsticks(dev):
+    """The two library kernels the roofline denominators were measured with, timed again in this run on this GPU
+    (boxes of the pool differ by a few percent): a bf16 8192^3 torch.matmul, best of 10, and a 2 GiB copy, best of 5.
+    Measurement only: the denominators of `roofline` stay the recorded ones."""
+    import torch
+    a = torch.randn(8192, 8192, device=dev, dtype=torch.bfloat16)
+    b = torch.randn(8192, 8192, device=dev, dtype=torch.bfloat16)
+    c = torch.empty(8192, 8192, device=dev, dtype=torch.bfloat16)
+    best = float("inf")
+    for i in range(13):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        torch.matmul(a, b, out=c)
+        e1.record()
+        e1.synchronize()
+        if i >= 3:
+            best = min(best, e0.elapsed_time(e1))
+    tflops = 2 * 8192 ** 3 / (best * 1e-3) / 1e12
+    del a, b, c
+    src = torch.empty(1 << 30, device=dev, dtype=torch.bfloat16)
+    dst = torch.empty_like(src)
+    best_c = float("inf")
+    for i in range(7):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        dst.copy_(src)
+        e1.record()
+        e1.synchronize()
+        if i >= 2:
+            best_c = min(best_c, e0.elapsed_time(e1))
+    gbs = 2 * src.numel() * 2 / (best_c * 1e-3) / 1e9
+    del src, dst
+    return {"bf16_matmul_8192_tflops_best": tflops, "copy_1gi_bf16_gbs_best": gbs,
+            "how": "torch.matmul and Tensor.copy_ (library kernels, yardsticks only), CUDA events"}
 
 
 class ClockSampler:
@@ -586,6 +623,7 @@ def main():
     ap.add_argument("--impl", default="native", choices=["native", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-yardsticks", action="store_true", help="skip the in-run matmul and copy timings")
     ap.add_argument("--no-other-configs", action="store_true",
                     help="skip the short runs of further workloads reported under other_configs")
     ap.add_argument("--force-kv-splits", type=int, default=0)
@@ -737,6 +775,10 @@ def main():
                 "traffic": traffic, "traffic_source": DRAM_SOURCE, "compulsory_bytes": kv_bytes + qo_bytes,
                 "flops_per_launch": flops, "kernel_ms": attn_ms,
                 "roofline_ms": max(t_flops, t_bytes), "frac_of_roofline_time": max(t_flops, t_bytes) / attn_ms}
+
+    roofline["frac_of_nominal"] = achieved / NOMINAL_BF16_TFLOPS
+    if not args.no_yardsticks:
+        roofline["yardsticks_this_run"] = measure_yardsticks(dev)
 
     # the append alone, back to back (the per-step bracket above includes the gap to the previous kernel)
     n_app = 20
