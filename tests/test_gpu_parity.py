@@ -125,6 +125,46 @@ def test_tail_round_cut_along_the_keys_by_the_planner():
     assert info.num_tiles == 6 + 2 * 3 and info.num_split_tiles == 6 and info.workspace_bytes > 256
 
 
+def test_a_wave_captured_in_a_cuda_graph_replays_bit_identically():
+    """Both calls only enqueue work on the stream they are given (a memset node and kernels): a wave whose plan stays
+    the same can be captured once and replayed, which for the smallest waves halves the time per wave."""
+    w = W.cfg1()
+    inp = cpu_inputs(w)
+    _, _, ref, _ = run_oracle(w, inp)
+    dev_inp = H.device_inputs(w, inp)
+    c, d = H.ctx(), H.desc_of(w)
+    plan = wpp.wpp_plan_tiles(c, d, w.prefix_lens, w.chunk_lens).to_device()
+    dev = torch.device("cuda")
+    bt = torch.from_numpy(w.block_tables).to(dev)
+    P = torch.from_numpy(np.asarray(w.prefix_lens, dtype=np.int32)).to(dev)
+    C = torch.from_numpy(np.asarray(w.chunk_lens, dtype=np.int32)).to(dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    out = torch.empty(w.total_new_tokens, w.num_q_heads, w.head_dim, dtype=torch.bfloat16, device=dev)
+    ws = torch.empty(max(256, int(plan.info.workspace_bytes)), dtype=torch.uint8, device=dev)
+
+    def wave():
+        wpp.wpp_kv_append(c, d, dev_inp["k_new"], dev_inp["v_new"], dev_inp["k_pool"], dev_inp["v_pool"], bt, P, C, plan,
+                          status=status)
+        wpp.wpp_prefill_attention_varlen(c, d, dev_inp["q"], out, None, dev_inp["k_pool"], dev_inp["v_pool"], bt, P, C,
+                                         plan, workspace=ws, status=status)
+
+    s = torch.cuda.Stream()
+    with torch.cuda.stream(s):
+        wave()                                           # first call outside the capture (one-time function attributes)
+        s.synchronize()
+        direct = out.clone()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=s):
+            wave()
+        for _ in range(3):
+            out.view(torch.int16).fill_(0x7FC0)
+            g.replay()
+            s.synchronize()
+            assert int(status.item()) == 0
+            assert torch.equal(out.view(torch.int16), direct.view(torch.int16))
+    H.assert_close(f64(out), ref, "replayed wave")
+
+
 def test_explicit_scale():
     w = W.custom_workload([70], [150], 2, 1, 128, 64, seed=10)
     _full_parity(w, sm_scale=0.05)
