@@ -624,6 +624,9 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-yardsticks", action="store_true", help="skip the in-run matmul and copy timings")
+    ap.add_argument("--rescale-mode", type=int, default=2, choices=[0, 1, 2],
+                    help="where a moved row reference rescales the accumulator: 0 before the exponentials (the "
+                         "library's default), 1 after them, 2 the library chooses from what its kernels counted")
     ap.add_argument("--no-other-configs", action="store_true",
                     help="skip the short runs of further workloads reported under other_configs")
     ap.add_argument("--force-kv-splits", type=int, default=0)
@@ -672,6 +675,7 @@ def main():
     peaks, peak_kind = load_peaks()
     w = build_workload(args.config)
     ctx = wpp.Context(local_rank)
+    ctx.set_rescale_mode(args.rescale_mode)
     desc = wpp.make_desc(w.num_requests, w.num_q_heads, w.num_kv_heads, w.head_dim, w.page_size,
                          w.max_blocks_per_req, w.num_pages)
     opts = wpp.PlanOpts(0, 0, args.force_kv_splits, args.max_ctas, args.plan_order, args.shape)
@@ -762,6 +766,10 @@ def main():
     info = plan.info
     flops = float(info.flops)
     tokens_per_s = world * T / (ms_step * 1e-3)
+    r_steps, r_moves, r_late = ctx.rescale_stats()
+    rescale_note = {"mode": ["before the exponentials", "after the exponentials", "chosen from the kernels' counters"][args.rescale_mode],
+                    "in_use": "after" if r_late else "before",
+                    "share_of_key_steps_that_rescaled": (r_moves / r_steps) if r_steps else None}
 
     roof_peak = float(peaks.get("bf16_tflops", FALLBACK_PEAKS["bf16_tflops"]))
     roof_sus = float(peaks.get("bf16_tflops_sustained", FALLBACK_PEAKS["bf16_tflops_sustained"]))
@@ -904,7 +912,7 @@ def main():
                               "between steps; ms_per_step is the sum of append and attention event times"),
                            step="wpp_plan_tiles + plan H2D + wpp_kv_append + wpp_prefill_attention_varlen",
                            tiles=int(info.num_tiles), ctas=int(info.num_ctas), key_steps=int(info.key_steps),
-                           kernel_shape=int(info.shape)),
+                           kernel_shape=int(info.shape), rescale=rescale_note),
             "tflops": flops / (ms_step * 1e-3) / 1e12 * world,
             "served_tokens_per_s": world * float((w.prefix_lens.astype(np.int64) + w.chunk_lens).sum()) / (ms_step * 1e-3),
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline, "cpu_baseline": cpu,

@@ -239,6 +239,21 @@ int wpp_selftest_bounded_wait(const wpp_ctx* ctx, int64_t limit_cycles, int32_t*
 /* Number of kernels the library has launched through this context so far (for launch accounting). */
 int64_t wpp_launch_count(const wpp_ctx* ctx);
 
+/* The attention kernel keeps a reference per query row for its exponentials and rescales the row's accumulator when
+ * the reference has to move.  It exists in two orders of work: rescale before the step's exponentials (best when
+ * references move now and then: every workload whose scores do not keep growing along the sequence) or after them
+ * (best when most steps move a reference).  Both are within the tolerance; they differ in rounding order.
+ *   wpp_set_rescale_mode : 0 = always before (default: outputs are bit-reproducible from call to call),
+ *                          1 = always after,
+ *                          2 = chosen per call from what the kernels of earlier launches on this context counted -
+ *                              their key steps and the steps that rescaled, added up in two words of pinned host
+ *                              memory that wpp_create maps for the device and that the call reads without
+ *                              synchronising: at least 30 % of the steps rescaling: after; under 15 %: before; in
+ *                              between: as it was.  Outputs may then differ in the last bit from call to call.
+ *   wpp_rescale_stats    : the counters so far (either pointer may be null) and the order the next call would use. */
+int wpp_set_rescale_mode(wpp_ctx* ctx, int mode);
+int wpp_rescale_stats(const wpp_ctx* ctx, uint64_t* key_steps, uint64_t* rescaling_steps, int* late);
+
 /* ---------------------------------------------------------------------------------------------------------
  * Wave-budget planner (Section 4.5, "Pipeline Scheduling": Maximum Pipeline Utilization).  Host only, integer
  * arithmetic only, no CUDA call; it produces the chunk_lens the calls above consume: the step directly upstream of

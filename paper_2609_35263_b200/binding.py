@@ -85,7 +85,8 @@ WAVE_RING_BUSY, WAVE_ADMISSION_PENDING, WAVE_ALREADY_DEFERRED = 1, 2, 4
 
 EXPORTS = ["wpp_create", "wpp_destroy", "wpp_status_string", "wpp_last_cuda_error", "wpp_plan_bytes",
            "wpp_plan_tiles", "wpp_validate_batch", "wpp_kv_append", "wpp_prefill_attention_varlen",
-           "wpp_launch_count", "wpp_prefill_attention_varlen_static", "wpp_static_scratch_bytes",
+           "wpp_launch_count", "wpp_set_rescale_mode", "wpp_rescale_stats", "wpp_prefill_attention_varlen_static",
+           "wpp_static_scratch_bytes",
            "wpp_selftest_bounded_wait", "wpp_wave_ladder", "wpp_plan_waves",
            "wpp_hash_blocks", "wpp_hash_blocks_host", "wpp_hint_index_create", "wpp_hint_index_destroy",
            "wpp_hint_index_add", "wpp_hint_index_remove", "wpp_hint_index_size", "wpp_hint_probe",
@@ -110,6 +111,9 @@ def load_library() -> ctypes.CDLL:
         lib.wpp_last_cuda_error.argtypes = [vp]
         lib.wpp_launch_count.argtypes = [vp]
         lib.wpp_launch_count.restype = ctypes.c_int64
+        lib.wpp_set_rescale_mode.argtypes = [vp, ctypes.c_int]
+        lib.wpp_rescale_stats.argtypes = [vp, ctypes.POINTER(ctypes.c_uint64), ctypes.POINTER(ctypes.c_uint64),
+                                          ctypes.POINTER(ctypes.c_int)]
         lib.wpp_plan_bytes.restype = ctypes.c_size_t
         lib.wpp_plan_bytes.argtypes = [vp, ctypes.POINTER(BatchDesc), ctypes.c_int64, ctypes.POINTER(PlanOpts)]
         lib.wpp_plan_tiles.argtypes = [vp, ctypes.POINTER(BatchDesc), i32p, i32p, i32p, ctypes.POINTER(PlanOpts),
@@ -167,6 +171,17 @@ class Context:
 
     def launch_count(self) -> int:
         return int(load_library().wpp_launch_count(self._h))
+
+    def set_rescale_mode(self, mode: int) -> None:
+        """0: rescale before the exponentials (default); 1: after; 2: the library chooses from what its kernels counted."""
+        _check(load_library().wpp_set_rescale_mode(self._h, int(mode)), "wpp_set_rescale_mode")
+
+    def rescale_stats(self):
+        """(key steps, steps that rescaled an accumulator, whether the next call rescales after the exponentials)."""
+        s, m, late = ctypes.c_uint64(0), ctypes.c_uint64(0), ctypes.c_int(0)
+        _check(load_library().wpp_rescale_stats(self._h, ctypes.byref(s), ctypes.byref(m), ctypes.byref(late)),
+               "wpp_rescale_stats")
+        return int(s.value), int(m.value), bool(late.value)
 
     def last_cuda_error(self) -> int:
         return int(load_library().wpp_last_cuda_error(self._h))

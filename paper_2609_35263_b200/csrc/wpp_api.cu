@@ -33,6 +33,7 @@ struct MapEntry {
     uint64_t used;      // 0 = empty; else the tick of the last use (least recently used entry is replaced)
 };
 constexpr int kMapCacheEntries = 32;
+constexpr int kLateRescaleOnPct = 30, kLateRescaleOffPct = 15;   // share of key steps that rescale O (see choose_late_rescale)
 
 struct wpp_ctx {
     int device;
@@ -42,6 +43,13 @@ struct wpp_ctx {
     int64_t launches;
     EncodeTiledFn encode_tiled;
     void* static_scratch;           // device address of the built-in scratch array on this context's device
+    // Where a moved row reference rescales O (see the attention kernel's kLate) is chosen per launch from what the
+    // kernels of earlier launches counted: key steps and steps that rescaled, added up in mapped host memory.
+    unsigned long long* stats_host; // [0] key steps, [1] rescaling steps (pinned, mapped; the kernels add to it)
+    unsigned long long* stats_dev;  // the same two words as the device sees them
+    unsigned long long seen_steps, seen_moves;   // the counters when the choice was last looked at
+    int rescale_mode;               // 0: always before the exponentials (default), 1: always after, 2: chosen from the counters
+    int late_rescale;               // the current choice
     std::mutex* map_lock;
     uint64_t map_tick;
     MapEntry maps[kMapCacheEntries];
@@ -120,14 +128,66 @@ extern "C" int wpp_create(wpp_ctx** out, int cuda_device) {
         free(c);
         return WPP_ERR_INVALID_ARG;
     }
+    // two counters the attention kernels add to and the next call reads without synchronising (a missing mapping
+    // only means that the choice they feed stays at its default)
+    void* hp = nullptr;
+    if (cudaHostAlloc(&hp, 64, cudaHostAllocMapped | cudaHostAllocPortable) == cudaSuccess) {
+        memset(hp, 0, 64);
+        void* dp = nullptr;
+        if (cudaHostGetDevicePointer(&dp, hp, 0) == cudaSuccess) {
+            c->stats_host = static_cast<unsigned long long*>(hp);
+            c->stats_dev = static_cast<unsigned long long*>(dp);
+        } else {
+            cudaFreeHost(hp);
+        }
+    }
+    (void)cudaGetLastError();
     *out = c;
     return WPP_OK;
 }
 
 extern "C" int wpp_destroy(wpp_ctx* ctx) {
-    if (ctx) delete ctx->map_lock;
+    if (ctx) {
+        delete ctx->map_lock;
+        if (ctx->stats_host) cudaFreeHost(ctx->stats_host);
+    }
     free(ctx);
     return WPP_OK;
+}
+
+extern "C" int wpp_set_rescale_mode(wpp_ctx* ctx, int mode) {
+    if (!ctx || mode < 0 || mode > 2) return WPP_ERR_INVALID_ARG;
+    std::lock_guard<std::mutex> guard(*ctx->map_lock);
+    ctx->rescale_mode = mode;
+    return WPP_OK;
+}
+
+extern "C" int wpp_rescale_stats(const wpp_ctx* ctx, uint64_t* key_steps, uint64_t* rescaling_steps, int* late) {
+    if (!ctx) return WPP_ERR_INVALID_ARG;
+    volatile unsigned long long* s = ctx->stats_host;
+    if (key_steps) *key_steps = s ? s[0] : 0;
+    if (rescaling_steps) *rescaling_steps = s ? s[1] : 0;
+    if (late) *late = ctx->rescale_mode == 1 || (ctx->rescale_mode == 2 && ctx->late_rescale);
+    return WPP_OK;
+}
+
+// The choice for the next launch: with the counters' increase since the last look, once there are enough steps to
+// judge by; between the two thresholds the choice stays what it was.
+static int choose_late_rescale(const wpp_ctx* cctx) {
+    wpp_ctx* c = const_cast<wpp_ctx*>(cctx);
+    std::lock_guard<std::mutex> guard(*c->map_lock);
+    if (c->rescale_mode != 2) return c->rescale_mode == 1;
+    if (!c->stats_host) return 0;
+    volatile unsigned long long* s = c->stats_host;
+    const unsigned long long steps = s[0], moves = s[1];
+    const unsigned long long ds = steps - c->seen_steps, dm = moves - c->seen_moves;
+    if (ds >= 4096) {
+        if (dm * 100 >= ds * kLateRescaleOnPct) c->late_rescale = 1;
+        else if (dm * 100 < ds * kLateRescaleOffPct) c->late_rescale = 0;
+        c->seen_steps = steps;
+        c->seen_moves = moves;
+    }
+    return c->late_rescale;
 }
 
 // Every launching entry point runs with the context's device current: a call made with another device current
@@ -308,8 +368,10 @@ extern "C" int wpp_prefill_attention_varlen(const wpp_ctx* ctx, const wpp_batch_
     // the counter the CTAs take their tiles from starts at zero (a memset node on the caller's stream)
     int e = (int)cudaMemsetAsync(workspace, 0, WPP_WS_HEADER_BYTES, (cudaStream_t)cuda_stream);
     if (e != 0) return cuda_fail(ctx, e);
+    p.stats = ctx->stats_dev;
     e = hd->shape == 2 ? wpp_launch_attention_small(d.head_dim, tq, &tk, &tv, &p, hd->num_ctas, cuda_stream)
-                       : wpp_launch_attention(d.head_dim, tq, &tk, &tv, &p, hd->num_ctas, cuda_stream);
+                       : wpp_launch_attention(d.head_dim, tq, &tk, &tv, &p, hd->num_ctas, choose_late_rescale(ctx),
+                                              cuda_stream);
     if (e != 0) return cuda_fail(ctx, e);
     const_cast<wpp_ctx*>(ctx)->launches += 1;
     if (hd->num_combine > 0) {

@@ -105,7 +105,12 @@ __device__ __forceinline__ UnitView view_of(const WppUnit& un, const AttnParams&
     return v;
 }
 
-template <int D>
+// kLate: where a moved reference rescales O.  false: before the step's exponentials (they then start from a settled
+// O and the wait for the previous product is usually over by the time P is ready): the choice for workloads whose
+// references move now and then.  true: after the exponentials, which do not depend on O and so run while the
+// previous O += P V is still on the tensor pipe: better when most steps move a reference (scores that keep growing
+// along the sequence), a little worse otherwise.  The kernel counts its steps and its moves for the caller to choose.
+template <int D, bool kLate>
 __global__ void __launch_bounds__(kThreads, 1)
 wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_q64,
                 const __grid_constant__ CUtensorMap tm_q32, const __grid_constant__ CUtensorMap tm_q16,
@@ -479,6 +484,7 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         const float c = p.scale_log2;
         const uint64_t c2 = pack2(c, c);
         bool dead = false;
+        uint32_t n_steps_seen = 0, n_moves_seen = 0;      // this warp's key steps, and those that rescaled O
         while (!dead) {
             const int u = next_tile();
             if (!__all_sync(0xffffffffu, u != -2) || u < 0) break;
@@ -486,6 +492,7 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             const UnitView v = view_of(un, p, q_offsets, plan_prefix);
             const int n = v.n[hf];
             if (n == 0) continue;
+            n_steps_seen += (uint32_t)n;
             const int first_pos = v.P + un.row0[hf];          // last key visible to row 0 of this half
             // last key this thread's row may see: its own position (rows of packed heads repeat every 128/pack
             // tensor rows), never past the end of the sequence
@@ -533,15 +540,18 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 // overflow and small terms keep 8 bits below that.  Otherwise (or when the row has no reference
                 // yet) the warp moves its references to the running maxima and rescales O and l.
                 const bool move = (m_ref == -INFINITY) || !(fmaf(mxx, c, nmc) <= kRefSlack);
-                if (__any_sync(0xffffffffu, move)) {
+                const bool warp_moves = __any_sync(0xffffffffu, move);
+                float alpha = 1.f;
+                if (warp_moves) {
                     const float m_new = fmaxf(m_ref, mxx);
                     const float m_safe = (m_new == -INFINITY) ? 0.f : m_new;
                     const float nmc_new = -m_safe * c;
-                    const float alpha = (m_ref == -INFINITY) ? 0.f : fast_exp2(nmc_new - nmc);
+                    alpha = (m_ref == -INFINITY) ? 0.f : fast_exp2(nmc_new - nmc);
                     nmc = nmc_new;
                     m_ref = m_new;
                     l_run *= alpha;
-                    if (j > 0) {
+                    n_moves_seen += (j > 0);
+                    if (!kLate && j > 0) {
                         // O may only be touched once the O += P V of step j-1 has landed
                         const bool okp = mbar_wait(bPFree(hf), pf_phase ^ 1u, abort_flag);
                         if (!__all_sync(0xffffffffu, okp)) { dead = true; break; }
@@ -607,6 +617,21 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     pf_phase ^= 1u;
                     tc_fence_after();
                 }
+                if (kLate && warp_moves && j > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
+#pragma unroll 1
+                    for (int q0 = 0; q0 < D; q0 += kRescaleCols) {
+                        float o[kRescaleCols];
+#pragma unroll
+                        for (int c8 = 0; c8 < kRescaleCols; c8 += 8)
+                            tmem_ld8(lane_addr + col_o(hf) + q0 + c8, reinterpret_cast<uint32_t*>(o) + c8);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int i = 0; i < kRescaleCols; ++i) o[i] *= alpha;
+#pragma unroll
+                        for (int c8 = 0; c8 < kRescaleCols; c8 += 8)
+                            tmem_st8(lane_addr + col_o(hf) + q0 + c8, reinterpret_cast<uint32_t*>(o) + c8);
+                    }
+                }
                 // eight stores of eight columns rather than two of 32: the narrow form only needs eight consecutive
                 // registers at a time, which leaves the register allocator free in the loop above (+0.7 % measured)
 #pragma unroll
@@ -626,6 +651,12 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             s_final[hf * 128 + r] = make_float2(-nmc, l_run);
             mbar_arrive(bFinalReady(hf));
         }
+        // the launch's counters live behind the tile counter in the workspace header (zeroed with it)
+        if (p.stats && lane == 0 && n_steps_seen) {
+            unsigned long long* ws_stats = reinterpret_cast<unsigned long long*>(p.tile_counter) + 1;
+            atomicAdd(ws_stats, (unsigned long long)n_steps_seen);
+            atomicAdd(ws_stats + 1, (unsigned long long)n_moves_seen);
+        }
     }
 
     // ---- teardown: every loop above is bounded, so every thread gets here.  The abort flag is read after the
@@ -642,30 +673,47 @@ wpp_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         tc_fence_after();
         tmem_dealloc(tmem, kTmemCols);
     }
+    // the last CTA to get here hands the launch's two counters to the caller's words (mapped host memory: two
+    // transactions per launch, where one per warp would cost milliseconds)
+    if (p.stats && threadIdx.x == 0) {
+        unsigned long long* ws_stats = reinterpret_cast<unsigned long long*>(p.tile_counter) + 1;
+        __threadfence();
+        if (atomicAdd(reinterpret_cast<unsigned int*>(ws_stats + 2), 1u) == gridDim.x - 1) {
+            __threadfence();
+            atomicAdd_system(p.stats, atomicAdd(ws_stats, 0ull));
+            atomicAdd_system(p.stats + 1, atomicAdd(ws_stats + 1, 0ull));
+        }
+    }
 }
 
-template <int D>
+template <int D, bool kLate>
 static cudaError_t launch(const CUtensorMap* tq, const CUtensorMap& tk, const CUtensorMap& tv, const AttnParams& p,
                           int num_ctas, cudaStream_t stream) {
     static bool attr_set[64] = {};
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev >= 0 && dev < 64 && !attr_set[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(wpp_attn_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        cudaError_t e = cudaFuncSetAttribute(wpp_attn_kernel<D, kLate>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              Cfg<D>::kSmemBytes);
         if (e != cudaSuccess) return e;
         attr_set[dev] = true;
     }
-    wpp_attn_kernel<D><<<num_ctas, kThreads, Cfg<D>::kSmemBytes, stream>>>(tq[0], tq[1], tq[2], tq[3], tk, tv, p);
+    wpp_attn_kernel<D, kLate><<<num_ctas, kThreads, Cfg<D>::kSmemBytes, stream>>>(tq[0], tq[1], tq[2], tq[3], tk, tv, p);
     return cudaGetLastError();
 }
 
 }  // namespace wpp
 
 // tq: four maps of q with boxes of 128, 64, 32 and 16 rows
+// late_rescale: see the kernel's kLate
 extern "C" int wpp_launch_attention(int head_dim, const CUtensorMap* tq, const CUtensorMap* tk, const CUtensorMap* tv,
-                                    const wpp::AttnParams* p, int num_ctas, void* stream) {
-    if (head_dim == 128) return (int)wpp::launch<128>(tq, *tk, *tv, *p, num_ctas, (cudaStream_t)stream);
-    if (head_dim == 64) return (int)wpp::launch<64>(tq, *tk, *tv, *p, num_ctas, (cudaStream_t)stream);
+                                    const wpp::AttnParams* p, int num_ctas, int late_rescale, void* stream) {
+    cudaStream_t st = (cudaStream_t)stream;
+    if (head_dim == 128)
+        return (int)(late_rescale ? wpp::launch<128, true>(tq, *tk, *tv, *p, num_ctas, st)
+                                  : wpp::launch<128, false>(tq, *tk, *tv, *p, num_ctas, st));
+    if (head_dim == 64)
+        return (int)(late_rescale ? wpp::launch<64, true>(tq, *tk, *tv, *p, num_ctas, st)
+                                  : wpp::launch<64, false>(tq, *tk, *tv, *p, num_ctas, st));
     return (int)cudaErrorInvalidValue;
 }

@@ -19,6 +19,7 @@ struct AttnParams {
     float* ws_lse;                   // [slots][2][128], log2 units
     int32_t* status;                 // sticky device status word or null
     uint32_t* tile_counter;          // zeroed before the launch: index of the next tile nobody has taken yet
+    unsigned long long* stats;       // or null: [0] += key steps of the softmax warps, [1] += those that rescaled O
     int64_t o_token_stride, o_head_stride;
     int32_t num_q_heads, group, page_size, max_blocks, num_pages;
     float scale_log2;                // sm_scale * log2(e)
@@ -98,7 +99,7 @@ extern "C" {
 // maps: 0..5 the operand arrays W0, Qt, Kb (hi, lo each), 6..7 M (hi, lo), 8 U0, 9..12 q, k, v, alpha
 int wpp_launch_kda_tc(const wpp::KdaTcParams* p, const CUtensorMap* maps, int max_blocks, int num_sms, void* stream);
 int wpp_launch_attention(int head_dim, const CUtensorMap* tq, const CUtensorMap* tk, const CUtensorMap* tv,
-                         const wpp::AttnParams* p, int num_ctas, void* stream);
+                         const wpp::AttnParams* p, int num_ctas, int late_rescale, void* stream);
 int wpp_launch_attention_small(int head_dim, const CUtensorMap* tq, const CUtensorMap* tk, const CUtensorMap* tv,
                                const wpp::AttnParams* p, int num_ctas, void* stream);
 int wpp_launch_append(const wpp::AppendParams* p, int num_sms, void* stream);

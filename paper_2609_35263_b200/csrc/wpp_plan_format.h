@@ -51,7 +51,9 @@ struct WppCombine {
     int32_t lane0;                  // first tensor row of this head inside the half (packed heads)
 };
 
-// Workspace layout: WPP_WS_HEADER_BYTES of header (a uint32 counter: the next tile of the order nobody has taken
-// yet; the attention call zeroes it on the stream before the launch), then fp32
+// Workspace layout: WPP_WS_HEADER_BYTES of header (byte 0: a uint32 counter, the next tile of the order nobody has
+// taken yet; bytes 8 and 16: two uint64 counters of the SM-wide kernel, key steps and steps that rescaled an
+// accumulator; byte 24: a uint32 count of CTAs that have finished - the attention call zeroes the header on the
+// stream before the launch), then fp32
 // O_part[num_split_slots][2][128][head_dim] followed by fp32 lse_part[num_split_slots][2][128] (log2 units of the
 // scaled scores; -inf marks a row with no visible key in that part).

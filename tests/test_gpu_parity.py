@@ -165,6 +165,40 @@ def test_a_wave_captured_in_a_cuda_graph_replays_bit_identically():
     H.assert_close(f64(out), ref, "replayed wave")
 
 
+def test_rescale_before_and_after_the_exponentials_and_the_library_choosing():
+    """Scores that keep growing along the sequence (K scaled by 2^floor(pos / 4096)) move the row references on most
+    key steps.  Both orders of work stay within the tolerance; with the choice left to the library it goes to
+    "after" once its kernels have counted enough such steps, and back once a wave without them has run."""
+    c = H.ctx()
+    grow = W.custom_workload([45056], [256], 2, 1, 128, 64, seed=41, spare_pages=4, k_scale="cumulative")
+    calm = W.custom_workload([45056], [256], 2, 1, 128, 64, seed=42, spare_pages=4)
+    inp_g, inp_c = cpu_inputs(grow), cpu_inputs(calm)
+    _, _, ref_g, _ = run_oracle(grow, inp_g)
+    _, _, ref_c, _ = run_oracle(calm, inp_c)
+    opts = wpp.PlanOpts(256, 0, 1, 0, 0, 1)              # whole 256-row tiles on the SM-wide kernel
+    try:
+        for mode in (0, 1):
+            c.set_rescale_mode(mode)
+            for w, inp, ref in ((grow, inp_g, ref_g), (calm, inp_c, ref_c)):
+                res = H.run_wave(w, H.device_inputs(w, inp), opts=opts)
+                assert res["status"] == 0
+                H.assert_close(f64(res["out"]), ref, f"{w.name} rescale mode {mode}")
+        c.set_rescale_mode(2)
+        s0, m0, _ = c.rescale_stats()
+        for _ in range(2):                               # per wave: 2 tiles x 4 warps x (353 + 354) key steps of the halves
+            res = H.run_wave(grow, H.device_inputs(grow, inp_g), opts=opts)
+            H.assert_close(f64(res["out"]), ref_g, "growing scores, library's choice")
+        s1, m1, late = c.rescale_stats()
+        assert s1 - s0 == 2 * 2 * 4 * (353 + 354) and (m1 - m0) * 10 >= (s1 - s0) * 3 and late
+        for _ in range(2):
+            res = H.run_wave(calm, H.device_inputs(calm, inp_c), opts=opts)
+            H.assert_close(f64(res["out"]), ref_c, "calm scores, library's choice")
+        s2, m2, late = c.rescale_stats()
+        assert (m2 - m1) * 20 < (s2 - s1) * 3 and not late
+    finally:
+        c.set_rescale_mode(0)
+
+
 def test_explicit_scale():
     w = W.custom_workload([70], [150], 2, 1, 128, 64, seed=10)
     _full_parity(w, sm_scale=0.05)
