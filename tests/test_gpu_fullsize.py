@@ -127,13 +127,18 @@ def test_cfg4_long_context_alternating_scale(splits):
     print("cfg4_alt", splits, e)
 
 
-@pytest.mark.parametrize("splits", [0, 8])
-def test_cfg4_long_context_cumulative_scale(splits):
-    """K doubles every 4096 positions (up to 2^25): the running reference jumps 26 times per row."""
+@pytest.mark.parametrize("splits,rescale_mode", [(0, 0), (8, 0), (0, 1)])
+def test_cfg4_long_context_cumulative_scale(splits, rescale_mode):
+    """K doubles every 4096 positions (up to 2^25): the running reference jumps 26 times per row.  Both orders of
+    work of the kernel (accumulator rescaled before or after the step's exponentials) are checked."""
     w = W.cfg4("cumulative")
-    e = run_and_check_whole(w, sample_units(w, 3000, seed=405, max_boundary_requests=3),
-                            opts=wpp.PlanOpts(0, 0, splits, 0), screen_ill_conditioned=True)
-    print("cfg4", splits, e)
+    H.ctx().set_rescale_mode(rescale_mode)
+    try:
+        e = run_and_check_whole(w, sample_units(w, 3000, seed=405, max_boundary_requests=3),
+                                opts=wpp.PlanOpts(0, 0, splits, 0), screen_ill_conditioned=True)
+    finally:
+        H.ctx().set_rescale_mode(0)
+    print("cfg4", splits, rescale_mode, e)
 
 
 CHUNKS = (64, 256, 1024, 4096, 8192)
