@@ -130,7 +130,7 @@ def measure_other_config(name, ctx, dev, peaks, steps=3, warmup=3):
             "l2": "flushed between steps" if flush is not None else "inputs larger than L2"}
 
 
-OTHER_CONFIGS = ("cfg2", "cfg4_alt", "cfg5_C256_P0", "cfg5_C1024_P4096", "cfg5_C4096_P32768")
+OTHER_CONFIGS = ("cfg2", "cfg4", "cfg4_alt", "cfg5_C256_P0", "cfg5_C1024_P4096", "cfg5_C4096_P32768")
 
 
 def measure_yardsticks(dev):
