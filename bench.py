@@ -109,6 +109,9 @@ def measure_other_config(name, ctx, dev, peaks, steps=3, warmup=3):
     stream = torch.cuda.current_stream()
     times = []
     for i in range(warmup + steps):
+        if i == warmup:
+            torch.cuda.synchronize()         # the timed steps start from an idle device (and the library has seen
+                                             # what its kernels counted during the warm-up)
         if flush is not None:
             flush.fill_(i & 0xFF)
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -127,7 +130,8 @@ def measure_other_config(name, ctx, dev, peaks, steps=3, warmup=3):
             "tokens_per_s": w.total_new_tokens / (ms * 1e-3), "tflops": flops / (ms * 1e-3) / 1e12,
             "bound": "tensor" if t_flops >= t_bytes else "hbm", "roofline_ms": max(t_flops, t_bytes),
             "frac_of_roofline_time": max(t_flops, t_bytes) / ms,
-            "l2": "flushed between steps" if flush is not None else "inputs larger than L2"}
+            "l2": "flushed between steps" if flush is not None else "inputs larger than L2",
+            "rescale_in_use": "after" if ctx.rescale_stats()[2] else "before"}
 
 
 OTHER_CONFIGS = ("cfg2", "cfg4", "cfg4_alt", "cfg5_C256_P0", "cfg5_C1024_P4096", "cfg5_C4096_P32768")
