@@ -67,7 +67,9 @@ typedef struct wpp_ctx wpp_ctx;
  * the KV pool is sized from the free memory.  WPP_ERR_CUDA if the device or driver is unusable (there is no CPU
  * fallback).  *out is host memory owned by the library until wpp_destroy.  Every launching entry point must be
  * called with the context's device current (WPP_ERR_INVALID_ARG otherwise).  The context caches the tensor maps
- * it encodes, keyed by (pointer, extents, strides); it may be used from several host threads. */
+ * it encodes, keyed by (pointer, extents, strides); it may be used from several host threads.  It also owns 64
+ * bytes of pinned host memory mapped for the device, to which the attention kernels add two counters (see
+ * wpp_set_rescale_mode): everything enqueued through the context must have completed before wpp_destroy. */
 int wpp_create(wpp_ctx** out, int cuda_device);
 int wpp_destroy(wpp_ctx* ctx);
 const char* wpp_status_string(int status);
